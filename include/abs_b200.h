@@ -1,0 +1,146 @@
+/*
+ * abs_b200.h -- C ABI of the B200 (sm_100a) quantize / dequantize library for the
+ * Adaptive Block-Scaled (IF) data types: IF4, IF3, IF6 and plain NVFP4.
+ *
+ * Data model (paper Sec. 3, Eq. 1-2, Fig. 3a; Sec. 5.1 for the other widths):
+ *   - a row-major bf16 matrix [rows, cols], cols a multiple of 16;
+ *   - one FP32 tensor scale alpha = max|X| / (M_FP * 448)                      (Eq. 1);
+ *   - one E4M3 byte per 16 consecutive row elements, Delta = E4M3(gmax/(alpha*M_FP)) (Eq. 2);
+ *     bit 7 of that byte is the type flag: 1 = the group is stored as scaled integers
+ *     (pre-scaled by M_INT/M_FP, de-scaled by M_FP/M_INT on the way back), 0 = as the
+ *     format's minifloat, in which case an IF4 group is exactly an NVFP4 group   (Sec. 3);
+ *   - 16 b-bit codes per group, packed as a little-endian bitstream: code j occupies bits
+ *     [b*j, b*j+b) of the group's 2*b bytes (IF4/NVFP4: element 2j in the low nibble of
+ *     byte j).  FP codes are sign|exponent|mantissa, integer codes two's complement.
+ *
+ * Unless a function says otherwise every data pointer is a DEVICE pointer owned by the
+ * caller; the library neither frees nor keeps it.  Calls validate on the host, enqueue
+ * their kernels on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ * return without synchronising; execution errors surface at the caller's next sync.
+ * Inputs must be finite and the tensor maximum either 0 or at least 2^-100; input and
+ * output buffers must not overlap.  All device pointers must be 16-byte aligned.
+ * The library keeps a small per-device scratch ring (allocated on the first quantize call
+ * on a device, or by abs_init); make that first call outside any stream capture.  At most
+ * ABS_MAX_INFLIGHT quantize calls may be in flight on one device at a time.
+ * There is no CPU fallback: without a CUDA device every compute call returns ABS_ERR_CUDA.
+ */
+#ifndef ABS_B200_H
+#define ABS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ABS_API __attribute__((visibility("default")))
+#else
+#define ABS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Formats.  (M_FP, M_INT, bits): NVFP4 (6, -, 4); IF4 (6, 7, 4) Sec. 3; IF3 (4, 3, 3),
+ * IF6_E2M3 (7.5, 31, 6), IF6_E3M2 (28, 31, 6) Sec. 5.1 footnote and Table 5. */
+typedef enum {
+    ABS_FMT_NVFP4 = 0,
+    ABS_FMT_IF4 = 1,
+    ABS_FMT_IF3 = 2,
+    ABS_FMT_IF6_E2M3 = 3,
+    ABS_FMT_IF6_E3M2 = 4
+} abs_fmt_t;
+
+typedef enum {
+    ABS_OK = 0,
+    ABS_ERR_NULL = 1,   /* a required pointer is NULL                         */
+    ABS_ERR_SHAPE = 2,  /* negative size, or cols not a multiple of 16        */
+    ABS_ERR_ALIGN = 3,  /* a device pointer is not 16-byte aligned            */
+    ABS_ERR_FMT = 4,    /* unknown format                                     */
+    ABS_ERR_FLAGS = 5,  /* unknown flag bit, or a flag the call cannot honour */
+    ABS_ERR_CUDA = 6,   /* a CUDA runtime call or a launch failed             */
+    ABS_ERR_SIZE = 7    /* workspace too small / size beyond a stated maximum */
+} abs_status_t;
+
+enum {
+    ABS_F_HADAMARD16 = 1u << 0,     /* quantize: 16-point blockwise random Hadamard transform of every
+                                       group before the amax pass and the encoding (Sec. 4.1)            */
+    ABS_F_STOCHASTIC = 1u << 1,     /* quantize: stochastic rounding of both candidates from
+                                       Philox4x32-10(sr_seed, element index) (Sec. 4.1, App. B)          */
+    ABS_F_SR_SCALE_17_16 = 1u << 2, /* quantize: group scale target times 17/16 before E4M3 rounding,
+                                       the 16/17 factor of Sec. 4.1, so stochastic values never clip     */
+    ABS_F_ALPHA_GIVEN = 1u << 3,    /* quantize: *tensor_scale_f32 is an input; the amax pass is skipped */
+    ABS_F_OUT_FP32 = 1u << 4        /* dequantize: write the FP32 products instead of bf16               */
+};
+
+#define ABS_MAX_INFLIGHT 1024
+
+typedef struct {
+    uint32_t flags;         /* OR of ABS_F_*                                                     */
+    uint16_t had_sign_mask; /* Hadamard option: bit i = 1 multiplies element i of each group by -1 */
+    uint16_t _pad;          /* must be 0                                                          */
+    uint64_t sr_seed;       /* stochastic rounding: Philox key                                    */
+} abs_opts_t;
+
+/* Sizes of the outputs of abs_quantize: rows*cols*b/8 and rows*cols/16 bytes (0 on bad arguments). */
+ABS_API size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
+ABS_API size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
+ABS_API const char* abs_status_string(abs_status_t status);
+
+/* Allocates the per-device scratch ring of `device` now (synchronous).  Optional: the first
+ * quantize call on a device does the same. */
+ABS_API abs_status_t abs_init(int device);
+
+/* Quantize (Eq. 1-2, Fig. 3a steps 1-10, Sec. 3 "6/7 method" and sign-bit flag).
+ *   in_bf16          [rows, cols] bf16, row-major, leading dimension = cols
+ *   codes_u8         out, abs_codes_bytes() bytes, group g at byte offset g*2*b
+ *   scales_e4m3      out, abs_scales_bytes() bytes, row-major [rows, cols/16]
+ *   tensor_scale_f32 device pointer to one float: out (alpha), or in with ABS_F_ALPHA_GIVEN
+ * Launches a grid-wide amax reduction that also writes alpha, then the group-quantize kernel.
+ * rows*cols == 0 is ABS_OK and enqueues nothing.  abs_quantize == abs_quantize_ex with no options. */
+ABS_API abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
+                          void* scales_e4m3, float* tensor_scale_f32, void* stream);
+ABS_API abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
+                             void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream);
+
+/* Dequantize (Sec. 3: de-scale integer groups by M_FP/M_INT; Sec. 4.1: product in FP32, then
+ * bf16 round-to-nearest-even).  out is bf16 [rows, cols], or float with ABS_F_OUT_FP32 (the only
+ * flag accepted).  The Hadamard option is not inverted here. */
+ABS_API abs_status_t abs_dequantize(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
+                            const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out_bf16,
+                            void* stream);
+ABS_API abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
+                               const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out,
+                               const abs_opts_t* opts, void* stream);
+
+/* Eq. 1 alone: the grid-wide amax pass.  Writes max|X| (after the Hadamard option when asked) to
+ * *amax_f32 (device).  With it a row-sharded tensor can be quantized on several GPUs: each rank
+ * reduces its rows, the ranks exchange one float (max), and each rank calls abs_quantize_ex with
+ * ABS_F_ALPHA_GIVEN and alpha = abs_alpha_from_amax(fmt, global max). */
+ABS_API abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs_opts_t* opts, float* amax_f32,
+                      void* stream);
+/* Host arithmetic of Eq. 1: amax / (M_FP * 448) in IEEE single precision; 1.0f when amax == 0. */
+ABS_API float abs_alpha_from_amax(abs_fmt_t fmt, float amax);
+
+/* Host-buffer variants: `*_host` pointers are HOST memory (pinned memory makes the copies
+ * asynchronous), `d_workspace` is a device buffer of at least abs_host_workspace_bytes() bytes.
+ * Each call copies its inputs to the device, runs the same kernels as above, copies the results
+ * back and returns after synchronising `stream`. */
+ABS_API size_t abs_host_workspace_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
+ABS_API abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t rows, int64_t cols,
+                               void* codes_u8_host, void* scales_e4m3_host, float* tensor_scale_f32_host,
+                               const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream);
+ABS_API abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const void* scales_e4m3_host,
+                                 const float* tensor_scale_f32_host, int64_t rows, int64_t cols, void* out_host,
+                                 const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream);
+
+/* Self-test hook: applies one of the device conversions the kernels use to n FP32 values.
+ *   kind 0: E4M3 scale byte (Fig. 3a step 2)   kind 1..4: FP element code of NVFP4/IF4 (E2M1),
+ *   IF3 (E2M0), IF6_E2M3, IF6_E3M2 (step 4)    kind 5: integer candidate rint(z) & 0xFF (step 7)
+ * out_u8[i] = conversion(in_f32[i]).  kind 16 + k (k = 0..4): decode, in_f32[i] holds a code in its
+ * low byte as an integer-valued float and out is float: value of E4M3 byte / FP element code. */
+ABS_API abs_status_t abs_selftest_convert(int kind, const float* in_f32, int64_t n, void* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ABS_B200_H */

@@ -1,0 +1,215 @@
+"""Thin ctypes binding of ``libabs_b200.so`` (the C ABI declared in ``include/abs_b200.h``).
+
+Argument marshalling only: every step of quantize / dequantize runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  There is no CPU fallback -- if the
+library cannot be loaded, or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import threading
+
+from . import build as _build
+
+ABS_FMT_NVFP4, ABS_FMT_IF4, ABS_FMT_IF3, ABS_FMT_IF6_E2M3, ABS_FMT_IF6_E3M2 = range(5)
+FMT_NAMES = {"nvfp4": 0, "if4": 1, "if3": 2, "if6_e2m3": 3, "if6_e3m2": 4}
+FMT_BITS = {0: 4, 1: 4, 2: 3, 3: 6, 4: 6}
+
+ABS_F_HADAMARD16 = 1 << 0
+ABS_F_STOCHASTIC = 1 << 1
+ABS_F_SR_SCALE_17_16 = 1 << 2
+ABS_F_ALPHA_GIVEN = 1 << 3
+ABS_F_OUT_FP32 = 1 << 4
+
+ABS_OK = 0
+
+EXPORTS = [
+    "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
+    "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
+    "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert",
+]
+
+
+class AbsOpts(C.Structure):
+    _fields_ = [("flags", C.c_uint32), ("had_sign_mask", C.c_uint16), ("_pad", C.c_uint16), ("sr_seed", C.c_uint64)]
+
+
+class AbsError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+        self.status = status
+
+
+_lock = threading.Lock()
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib():
+    """Loads (building first if the sources are newer) the CUDA library. Raises if unavailable."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            path = _build.LIB_PATH
+            if not os.path.exists(path) or _build.needs_build():
+                path = _build.build()
+            L = C.CDLL(path)
+            vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+            op = C.POINTER(AbsOpts)
+            L.abs_codes_bytes.restype = sz
+            L.abs_codes_bytes.argtypes = [C.c_int, i64, i64]
+            L.abs_scales_bytes.restype = sz
+            L.abs_scales_bytes.argtypes = [C.c_int, i64, i64]
+            L.abs_status_string.restype = C.c_char_p
+            L.abs_status_string.argtypes = [C.c_int]
+            L.abs_init.restype = C.c_int
+            L.abs_init.argtypes = [C.c_int]
+            L.abs_quantize.restype = C.c_int
+            L.abs_quantize.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
+            L.abs_quantize_ex.restype = C.c_int
+            L.abs_quantize_ex.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
+            L.abs_dequantize.restype = C.c_int
+            L.abs_dequantize.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, vp]
+            L.abs_dequantize_ex.restype = C.c_int
+            L.abs_dequantize_ex.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, op, vp]
+            L.abs_amax.restype = C.c_int
+            L.abs_amax.argtypes = [vp, i64, i64, op, vp, vp]
+            L.abs_alpha_from_amax.restype = C.c_float
+            L.abs_alpha_from_amax.argtypes = [C.c_int, C.c_float]
+            L.abs_host_workspace_bytes.restype = sz
+            L.abs_host_workspace_bytes.argtypes = [C.c_int, i64, i64]
+            L.abs_quantize_host.restype = C.c_int
+            L.abs_quantize_host.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp, sz, vp]
+            L.abs_dequantize_host.restype = C.c_int
+            L.abs_dequantize_host.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, op, vp, sz, vp]
+            L.abs_selftest_convert.restype = C.c_int
+            L.abs_selftest_convert.argtypes = [C.c_int, vp, i64, vp, vp]
+            _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().abs_status_string(status).decode()
+
+
+def _check(status: int, what: str):
+    if status != ABS_OK:
+        raise AbsError(status, what)
+
+
+def make_opts(flags: int = 0, had_sign_mask: int = 0, sr_seed: int = 0) -> AbsOpts:
+    return AbsOpts(flags, had_sign_mask, 0, sr_seed)
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def abs_codes_bytes(fmt: int, rows: int, cols: int) -> int:
+    return lib().abs_codes_bytes(fmt, rows, cols)
+
+
+def abs_scales_bytes(fmt: int, rows: int, cols: int) -> int:
+    return lib().abs_scales_bytes(fmt, rows, cols)
+
+
+def abs_alpha_from_amax(fmt: int, amax: float) -> float:
+    return lib().abs_alpha_from_amax(fmt, amax)
+
+
+def abs_init(device: int = 0):
+    _check(lib().abs_init(device), "abs_init")
+
+
+def abs_quantize(fmt: int, x, codes=None, scales=None, tensor_scale=None, opts: AbsOpts | None = None, stream=None):
+    """Quantize a CUDA bf16 matrix ``x`` [rows, cols] (contiguous).
+
+    Output buffers are allocated with torch when not given.  Returns (codes u8, scales u8,
+    tensor_scale f32[1]); with ABS_F_ALPHA_GIVEN ``tensor_scale`` is the input alpha."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    rows, cols = x.shape
+    L = lib()
+    if codes is None:
+        codes = torch.empty(max(L.abs_codes_bytes(fmt, rows, cols), 1) if cols % 16 == 0 else 1, dtype=torch.uint8,
+                            device=x.device)
+    if scales is None:
+        scales = torch.empty(max(rows * cols // 16, 1), dtype=torch.uint8, device=x.device)
+    if tensor_scale is None:
+        tensor_scale = torch.zeros(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        rc = L.abs_quantize_ex(fmt, x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(),
+                               tensor_scale.data_ptr(), C.byref(opts) if opts is not None else None,
+                               _stream_ptr(stream))
+    _check(rc, "abs_quantize")
+    return codes, scales, tensor_scale
+
+
+def abs_dequantize(fmt: int, codes, scales, tensor_scale, rows: int, cols: int, out=None,
+                   opts: AbsOpts | None = None, stream=None):
+    """Dequantize to a CUDA bf16 matrix (float32 with ABS_F_OUT_FP32)."""
+    import torch
+    fp32 = bool(opts is not None and (opts.flags & ABS_F_OUT_FP32))
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.float32 if fp32 else torch.bfloat16, device=codes.device)
+    with torch.cuda.device(codes.device):
+        rc = lib().abs_dequantize_ex(fmt, codes.data_ptr(), scales.data_ptr(), tensor_scale.data_ptr(), rows, cols,
+                                     out.data_ptr(), C.byref(opts) if opts is not None else None, _stream_ptr(stream))
+    _check(rc, "abs_dequantize")
+    return out
+
+
+def abs_amax(x, opts: AbsOpts | None = None, out=None, stream=None):
+    """Grid-wide max |x| (after the Hadamard option when asked) into a CUDA float32[1]."""
+    import torch
+    rows, cols = x.shape
+    if out is None:
+        out = torch.zeros(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        rc = lib().abs_amax(x.data_ptr(), rows, cols, C.byref(opts) if opts is not None else None, out.data_ptr(),
+                            _stream_ptr(stream))
+    _check(rc, "abs_amax")
+    return out
+
+
+def abs_host_workspace_bytes(fmt: int, rows: int, cols: int) -> int:
+    return lib().abs_host_workspace_bytes(fmt, rows, cols)
+
+
+def abs_quantize_host(fmt: int, x_host, codes_host, scales_host, alpha_host, workspace, opts: AbsOpts | None = None,
+                      stream=None):
+    """Host-buffer variant: ``*_host`` are CPU tensors (pinned for speed), ``workspace`` a CUDA u8 tensor."""
+    rows, cols = x_host.shape
+    import torch
+    with torch.cuda.device(workspace.device):
+        rc = lib().abs_quantize_host(fmt, x_host.data_ptr(), rows, cols, codes_host.data_ptr(), scales_host.data_ptr(),
+                                     alpha_host.data_ptr(), C.byref(opts) if opts is not None else None,
+                                     workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "abs_quantize_host")
+
+
+def abs_dequantize_host(fmt: int, codes_host, scales_host, alpha_host, rows: int, cols: int, out_host, workspace,
+                        opts: AbsOpts | None = None, stream=None):
+    import torch
+    with torch.cuda.device(workspace.device):
+        rc = lib().abs_dequantize_host(fmt, codes_host.data_ptr(), scales_host.data_ptr(), alpha_host.data_ptr(), rows,
+                                       cols, out_host.data_ptr(), C.byref(opts) if opts is not None else None,
+                                       workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "abs_dequantize_host")
+
+
+def abs_selftest_convert(kind: int, x_f32, out=None, stream=None):
+    import torch
+    n = x_f32.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.uint8 if kind < 16 else torch.float32, device=x_f32.device)
+    with torch.cuda.device(x_f32.device):
+        rc = lib().abs_selftest_convert(kind, x_f32.data_ptr(), n, out.data_ptr(), _stream_ptr(stream))
+    _check(rc, "abs_selftest_convert")
+    return out

@@ -1,0 +1,592 @@
+// Kernels and C ABI of the B200 IF4 / IF3 / IF6 / NVFP4 quantize-dequantize library.
+//
+// Path (paper Sec. 3): amax_kernel (Eq. 1, grid-wide max -> alpha) -> quantize_kernel (Eq. 2 and
+// Fig. 3a steps 1-10 per 16-value group, flag in the scale's sign bit, packed codes);
+// dequantize_kernel is the inverse (Sec. 3, Sec. 4.1).  One thread owns one group of 16
+// consecutive row elements: 32 bytes in, 2*b + 1 bytes out.
+#include "../../include/abs_b200.h"
+#include "abs_device.cuh"
+
+#include <atomic>
+#include <mutex>
+
+using namespace absq;
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxDevices = 64;
+
+// ------------------------------------------------------------------------------------------ amax
+
+// Eq. 1, numerator: grid-wide max |x|.  Each block reduces its share and publishes it with one
+// atomicMax on the bit pattern (non-negative floats order like unsigned integers); the last block
+// to finish (ticket counter) turns the maximum into alpha (or returns the raw maximum), writes it
+// to the caller's slot and re-arms the scratch slot for the next call.
+//   slot[0] = running max bits, slot[1] = ticket counter; both are 0 between calls.
+template <bool RHT>
+__global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t ngroups,
+                                                        uint32_t sign_mask, uint32_t* __restrict__ slot,
+                                                        float* __restrict__ result, float denom) {
+    uint32_t local = 0u;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    if constexpr (!RHT) {
+        // |x| and max on packed bf16 pairs; 8 elements per 128-bit load.
+        const int64_t nvec = ngroups * 2;
+        uint32_t m0 = 0u, m1 = 0u;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+            uint4 v = __ldg(in + i);
+            uint32_t a = v.x & 0x7FFF7FFFu, b = v.y & 0x7FFF7FFFu, c = v.z & 0x7FFF7FFFu, d = v.w & 0x7FFF7FFFu;
+            m0 = __vmaxu2(m0, __vmaxu2(a, b));
+            m1 = __vmaxu2(m1, __vmaxu2(c, d));
+        }
+        uint32_t m = __vmaxu2(m0, m1);
+        local = max(m & 0xFFFFu, m >> 16) << 16;   // bf16 bits -> FP32 bits
+    } else {
+        for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+            float x[16];
+            unpack_bf16x8(__ldg(in + 2 * g), x);
+            unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
+            hadamard16(x, sign_mask);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) local = max(local, __float_as_uint(x[i]) & 0x7FFFFFFFu);
+        }
+    }
+    local = __reduce_max_sync(0xFFFFFFFFu, local);
+    __shared__ uint32_t warp_max[kThreads / 32];
+    __shared__ bool is_last;
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t m = 0u;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) m = max(m, warp_max[w]);
+        atomicMax(&slot[0], m);
+        __threadfence();
+        uint32_t ticket = atomicAdd(&slot[1], 1u);
+        is_last = (ticket == gridDim.x - 1);
+        if (is_last) {
+            __threadfence();
+            float A = __uint_as_float(atomicMax(&slot[0], 0u));
+            float out = A;
+            if (denom != 0.0f) out = (A == 0.0f) ? 1.0f : __fdiv_rn(A, denom);   // Eq. 1
+            *result = out;
+            slot[0] = 0u;
+            slot[1] = 0u;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ quantize
+
+template <int FMT, bool RHT, bool SR>
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
+                                                            uint8_t* __restrict__ scales,
+                                                            const float* __restrict__ alpha_p, int64_t ngroups,
+                                                            float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
+                                                            uint32_t seed_hi) {
+    using F = Fmt<FMT>;
+    constexpr int B = F::BITS;
+    const float alpha = __ldg(alpha_p);
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));                      // T3
+    const float c_pre = F::HAS_INT ? __fdiv_rn(F::M_INT, F::M_FP) : 0.0f;
+    const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+        float x[16];
+        unpack_bf16x8(__ldg(in + 2 * g), x);
+        unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
+        if constexpr (RHT) hadamard16(x, sign_mask);
+
+        // G1-G3 (Eq. 2, steps 1-2).
+        float gmax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) gmax = fmaxf(gmax, fabsf(x[i]));
+        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
+        const uint32_t sb = e4m3_encode(t);
+
+        uint32_t w[3] = {0u, 0u, 0u};
+        uint32_t sbyte = 0u;
+        if (sb != 0u) {                                                               // G4
+            const float d = __fmul_rn(e4m3_value(sb), alpha);                         // G5
+            const float r = __frcp_rn(d);
+            const float d_int = __fmul_rn(d, c_post);
+
+            uint32_t rnd[8];
+            if constexpr (SR) {
+                const uint64_t i8 = (uint64_t)g * 2u;
+                uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
+                uint4 p1 = philox4x32_10((uint32_t)(i8 + 1), (uint32_t)((i8 + 1) >> 32), seed_lo, seed_hi);
+                rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;
+                rnd[4] = p1.x; rnd[5] = p1.y; rnd[6] = p1.z; rnd[7] = p1.w;
+            }
+
+            uint32_t q_fp[16], q_int[16];
+            float s_fp[4] = {0.f, 0.f, 0.f, 0.f}, s_int[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+                const float x0 = x[i], x1 = x[i + 1];
+                float y0 = __fmul_rn(x0, r), y1 = __fmul_rn(x1, r);                    // E1 (step 3)
+                float u0 = 0.f, u1 = 0.f;
+                float yq0 = y0, yq1 = y1;
+                if constexpr (SR) {
+                    u0 = __fmul_rn(__fadd_rn((float)(rnd[i >> 1] & 0xFFFFu), 0.5f), 1.0f / 65536.0f);
+                    u1 = __fmul_rn(__fadd_rn((float)(rnd[i >> 1] >> 16), 0.5f), 1.0f / 65536.0f);
+                    yq0 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y0), F::M_FP, u0), y0);
+                    yq1 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y1), F::M_FP, u1), y1);
+                }
+                float v0, v1;
+                fp_encode_pair<F::EK>(yq0, yq1, q_fp[i], q_fp[i + 1], v0, v1);         // E2 (step 4)
+                const int chain = ((i >> 3) << 1);                                     // elements 0-7 -> S0,S1; 8-15 -> S2,S3
+                if constexpr (F::HAS_INT) {
+                    const float e0 = __fmaf_rn(v0, d, -x0), e1 = __fmaf_rn(v1, d, -x1);   // E3 (steps 5-6)
+                    s_fp[chain] = __fmaf_rn(e0, e0, s_fp[chain]);
+                    s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
+                    const float z0 = __fmul_rn(y0, c_pre), z1 = __fmul_rn(y1, c_pre);     // E4 (step 7)
+                    float k0, k1;
+                    if constexpr (SR) {
+                        k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
+                        k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
+                    } else {
+                        k0 = fminf(fmaxf(rintf(z0), -F::M_INT), F::M_INT);
+                        k1 = fminf(fmaxf(rintf(z1), -F::M_INT), F::M_INT);
+                    }
+                    const float f0 = __fmaf_rn(k0, d_int, -x0), f1 = __fmaf_rn(k1, d_int, -x1);   // E5 (steps 8-9)
+                    s_int[chain] = __fmaf_rn(f0, f0, s_int[chain]);
+                    s_int[chain + 1] = __fmaf_rn(f1, f1, s_int[chain + 1]);
+                    q_int[i] = (uint32_t)__float2int_rn(k0) & ((1u << B) - 1u);
+                    q_int[i + 1] = (uint32_t)__float2int_rn(k1) & ((1u << B) - 1u);
+                }
+            }
+            uint32_t flag = 0u;
+            if constexpr (F::HAS_INT) {                                                // S1-S2 (step 10)
+                const float E_fp = __fadd_rn(__fadd_rn(s_fp[0], s_fp[1]), __fadd_rn(s_fp[2], s_fp[3]));
+                const float E_int = __fadd_rn(__fadd_rn(s_int[0], s_int[1]), __fadd_rn(s_int[2], s_int[3]));
+                flag = (E_int < E_fp) ? 1u : 0u;
+                if (flag) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) q_fp[i] = q_int[i];
+                }
+            }
+            sbyte = sb | (flag << 7);                                                 // S3
+            pack_codes<B>(q_fp, w);                                                   // S4
+        }
+        scales[g] = (uint8_t)sbyte;
+        if constexpr (B == 4) {
+            *reinterpret_cast<uint2*>(codes + g * 8) = make_uint2(w[0], w[1]);
+        } else if constexpr (B == 6) {
+            uint32_t* p = reinterpret_cast<uint32_t*>(codes + g * 12);
+            p[0] = w[0]; p[1] = w[1]; p[2] = w[2];
+        } else {
+            uint16_t* p = reinterpret_cast<uint16_t*>(codes + g * 6);
+            p[0] = (uint16_t)w[0]; p[1] = (uint16_t)(w[0] >> 16); p[2] = (uint16_t)w[1];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ dequantize
+
+template <int FMT, bool OUT_FP32>
+__global__ void __launch_bounds__(kThreads) dequantize_kernel(const uint8_t* __restrict__ codes,
+                                                              const uint8_t* __restrict__ scales,
+                                                              const float* __restrict__ alpha_p, int64_t ngroups,
+                                                              void* __restrict__ out) {
+    using F = Fmt<FMT>;
+    constexpr int B = F::BITS;
+    const float alpha = __ldg(alpha_p);
+    const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+        uint32_t w[3] = {0u, 0u, 0u};
+        if constexpr (B == 4) {
+            uint2 v = __ldg(reinterpret_cast<const uint2*>(codes + g * 8));
+            w[0] = v.x; w[1] = v.y;
+        } else if constexpr (B == 6) {
+            const uint32_t* p = reinterpret_cast<const uint32_t*>(codes + g * 12);
+            w[0] = __ldg(p); w[1] = __ldg(p + 1); w[2] = __ldg(p + 2);
+        } else {
+            const uint16_t* p = reinterpret_cast<const uint16_t*>(codes + g * 6);
+            w[0] = (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 16); w[1] = (uint32_t)__ldg(p + 2);
+        }
+        const uint32_t sbyte = __ldg(scales + g);
+        const uint32_t flag = sbyte >> 7, mag = sbyte & 0x7Fu;
+        float Delta = e4m3_value(mag);
+        if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
+        float d = __fmul_rn(Delta, alpha);
+        if (F::HAS_INT && flag) d = __fmul_rn(d, c_post);              // de-scale integer groups (Sec. 3)
+        float o[16];
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+            const uint32_t c0 = extract_code<B>(w, i), c1 = extract_code<B>(w, i + 1);
+            float v0, v1;
+            if (F::HAS_INT && flag) {
+                v0 = (float)((int32_t)(c0 << (32 - B)) >> (32 - B));   // sign-extend b bits
+                v1 = (float)((int32_t)(c1 << (32 - B)) >> (32 - B));
+            } else {
+                float2 v = fp_decode_pair<F::EK>(c0, c1);
+                v0 = v.x; v1 = v.y;
+            }
+            o[i] = __fmul_rn(v0, d);
+            o[i + 1] = __fmul_rn(v1, d);
+        }
+        if constexpr (OUT_FP32) {
+            float4* p = reinterpret_cast<float4*>(out) + g * 4;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) p[k] = make_float4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
+        } else {
+            uint32_t pk[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);   // FP32 -> bf16, nearest even
+                pk[k] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            uint4* p = reinterpret_cast<uint4*>(out) + g * 2;
+            p[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            p[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ self-test hook
+
+__global__ void selftest_kernel(int kind, const float* __restrict__ in, int64_t n, void* __restrict__ out) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const float v = in[i];
+        uint32_t c0 = 0, c1 = 0;
+        float v0, v1;
+        if (kind < 16) {
+            uint32_t r = 0;
+            switch (kind) {
+                case 0: r = e4m3_encode(v); break;
+                case 1: fp_encode_pair<EK_E2M1>(v, 0.f, c0, c1, v0, v1); r = c0; break;
+                case 2: fp_encode_pair<EK_E2M0>(v, 0.f, c0, c1, v0, v1); r = c0; break;
+                case 3: fp_encode_pair<EK_E2M3>(v, 0.f, c0, c1, v0, v1); r = c0; break;
+                case 4: fp_encode_pair<EK_E3M2>(v, 0.f, c0, c1, v0, v1); r = c0; break;
+                default: r = (uint32_t)__float2int_rn(rintf(v)) & 0xFFu; break;
+            }
+            reinterpret_cast<uint8_t*>(out)[i] = (uint8_t)r;
+        } else {
+            const uint32_t code = (uint32_t)v;
+            float r;
+            switch (kind - 16) {
+                case 0: r = e4m3_value(code & 0x7Fu); break;
+                case 1: r = fp_decode_pair<EK_E2M1>(code, 0u).x; break;
+                case 2: r = fp_decode_pair<EK_E2M0>(code, 0u).x; break;
+                case 3: r = fp_decode_pair<EK_E2M3>(code, 0u).x; break;
+                default: r = fp_decode_pair<EK_E3M2>(code, 0u).x; break;
+            }
+            reinterpret_cast<float*>(out)[i] = r;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host state
+
+struct DeviceState {
+    std::once_flag once;
+    cudaError_t init_err = cudaSuccess;
+    uint32_t* ring = nullptr;          // ABS_MAX_INFLIGHT slots of 4 words (amax bits, ticket, pad, pad)
+    float* amax_alpha = nullptr;       // unused spare floats, one per slot (alpha hand-off for abs_amax)
+    std::atomic<uint32_t> next{0};
+    int sm_count = 148;
+};
+DeviceState g_dev[kMaxDevices];
+
+abs_status_t device_state(DeviceState** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ABS_ERR_CUDA;
+    DeviceState& st = g_dev[dev];
+    std::call_once(st.once, [&]() {
+        st.init_err = cudaMalloc(&st.ring, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t));
+        if (st.init_err == cudaSuccess) st.init_err = cudaMemset(st.ring, 0, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t));
+        int sms = 0;
+        if (st.init_err == cudaSuccess) st.init_err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms > 0) st.sm_count = sms;
+    });
+    if (st.init_err != cudaSuccess) return ABS_ERR_CUDA;
+    *out = &st;
+    return ABS_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int fmt_bits(int fmt) {
+    switch (fmt) {
+        case ABS_FMT_NVFP4: case ABS_FMT_IF4: return 4;
+        case ABS_FMT_IF3: return 3;
+        case ABS_FMT_IF6_E2M3: case ABS_FMT_IF6_E3M2: return 6;
+        default: return 0;
+    }
+}
+float fmt_mfp(int fmt) {
+    switch (fmt) {
+        case ABS_FMT_NVFP4: case ABS_FMT_IF4: return 6.0f;
+        case ABS_FMT_IF3: return 4.0f;
+        case ABS_FMT_IF6_E2M3: return 7.5f;
+        default: return 28.0f;
+    }
+}
+
+constexpr uint32_t kQuantFlags = ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN;
+
+int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
+    int64_t want = (work_items + kThreads - 1) / kThreads;
+    int64_t cap = (int64_t)st.sm_count * blocks_per_sm;
+    return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+}
+
+abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const abs_opts_t& o, float* result,
+                         float denom, cudaStream_t s) {
+    uint32_t* slot = st.ring + 4 * (st.next.fetch_add(1) % ABS_MAX_INFLIGHT);
+    const bool rht = o.flags & ABS_F_HADAMARD16;
+    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, 8);
+    if (rht)
+        amax_kernel<true><<<grid, kThreads, 0, s>>>((const uint4*)in, ngroups, o.had_sign_mask, slot, result, denom);
+    else
+        amax_kernel<false><<<grid, kThreads, 0, s>>>((const uint4*)in, ngroups, o.had_sign_mask, slot, result, denom);
+    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+template <int FMT>
+abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
+                                 const float* alpha, const abs_opts_t& o, cudaStream_t s) {
+    const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
+    const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
+    const int grid = grid_for(st, ngroups, 64);
+    const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
+#define ABS_LAUNCH_Q(R, S)                                                                                      \
+    quantize_kernel<FMT, R, S><<<grid, kThreads, 0, s>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales,   \
+                                                         alpha, ngroups, mul, o.had_sign_mask, k0, k1)
+    if (rht && sr) ABS_LAUNCH_Q(true, true);
+    else if (rht) ABS_LAUNCH_Q(true, false);
+    else if (sr) ABS_LAUNCH_Q(false, true);
+    else ABS_LAUNCH_Q(false, false);
+#undef ABS_LAUNCH_Q
+    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+template <int FMT>
+abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
+                                   int64_t ngroups, void* out, bool fp32, cudaStream_t s) {
+    const int grid = grid_for(st, ngroups, 64);
+    if (fp32)
+        dequantize_kernel<FMT, true><<<grid, kThreads, 0, s>>>((const uint8_t*)codes, (const uint8_t*)scales, alpha,
+                                                               ngroups, out);
+    else
+        dequantize_kernel<FMT, false><<<grid, kThreads, 0, s>>>((const uint8_t*)codes, (const uint8_t*)scales, alpha,
+                                                                ngroups, out);
+    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+abs_status_t check_shape(abs_fmt_t fmt, int64_t rows, int64_t cols) {
+    if (fmt_bits((int)fmt) == 0) return ABS_ERR_FMT;
+    if (rows < 0 || cols < 0 || (cols % 16) != 0) return ABS_ERR_SHAPE;
+    return ABS_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------ C ABI
+
+extern "C" {
+
+size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
+    if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
+    return (size_t)rows * (size_t)cols / 16 * (size_t)(2 * fmt_bits((int)fmt));
+}
+
+size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
+    if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
+    return (size_t)rows * (size_t)cols / 16;
+}
+
+const char* abs_status_string(abs_status_t status) {
+    switch (status) {
+        case ABS_OK: return "ok";
+        case ABS_ERR_NULL: return "null pointer";
+        case ABS_ERR_SHAPE: return "bad shape (negative size or cols not a multiple of 16)";
+        case ABS_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case ABS_ERR_FMT: return "unknown format";
+        case ABS_ERR_FLAGS: return "unknown or unsupported flag";
+        case ABS_ERR_CUDA: return "CUDA error";
+        case ABS_ERR_SIZE: return "size beyond the supported maximum or workspace too small";
+        default: return "unknown status";
+    }
+}
+
+abs_status_t abs_init(int device) {
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) return ABS_ERR_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return ABS_ERR_CUDA;
+    DeviceState* st = nullptr;
+    abs_status_t rc = device_state(&st);
+    cudaSetDevice(prev);
+    return rc;
+}
+
+float abs_alpha_from_amax(abs_fmt_t fmt, float amax) {
+    if (fmt_bits((int)fmt) == 0) return 0.0f;
+    volatile float den = fmt_mfp((int)fmt) * 448.0f;
+    volatile float a = amax;
+    return (a == 0.0f) ? 1.0f : a / den;
+}
+
+abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs_opts_t* opts, float* amax_f32,
+                      void* stream) {
+    abs_opts_t o = {0, 0, 0, 0};
+    if (opts) o = *opts;
+    if (rows < 0 || cols < 0 || (cols % 16) != 0) return ABS_ERR_SHAPE;
+    if ((o.flags & ~(uint32_t)ABS_F_HADAMARD16) || o._pad) return ABS_ERR_FLAGS;
+    if (!amax_f32) return ABS_ERR_NULL;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (rows * cols == 0) return cudaMemsetAsync(amax_f32, 0, sizeof(float), s) == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+    if (!in_bf16) return ABS_ERR_NULL;
+    if (!aligned16(in_bf16)) return ABS_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
+    return launch_amax(*st, in_bf16, rows * cols / 16, o, amax_f32, 0.0f, s);
+}
+
+abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
+                             void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream) {
+    abs_opts_t o = {0, 0, 0, 0};
+    if (opts) o = *opts;
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if ((o.flags & ~kQuantFlags) || o._pad) return ABS_ERR_FLAGS;
+    if (rows * cols == 0) return ABS_OK;
+    if (!in_bf16 || !codes_u8 || !scales_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
+    if (!aligned16(in_bf16) || !aligned16(codes_u8) || !aligned16(scales_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
+        return ABS_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t ngroups = rows * cols / 16;
+    if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
+        rc = launch_amax(*st, in_bf16, ngroups, o, tensor_scale_f32, fmt_mfp((int)fmt) * 448.0f, s);
+        if (rc != ABS_OK) return rc;
+    }
+    switch (fmt) {
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        default: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+    }
+}
+
+abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
+                          void* scales_e4m3, float* tensor_scale_f32, void* stream) {
+    return abs_quantize_ex(fmt, in_bf16, rows, cols, codes_u8, scales_e4m3, tensor_scale_f32, nullptr, stream);
+}
+
+abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
+                               const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out,
+                               const abs_opts_t* opts, void* stream) {
+    abs_opts_t o = {0, 0, 0, 0};
+    if (opts) o = *opts;
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if ((o.flags & ~(uint32_t)ABS_F_OUT_FP32) || o._pad) return ABS_ERR_FLAGS;
+    if (rows * cols == 0) return ABS_OK;
+    if (!codes_u8 || !scales_e4m3 || !tensor_scale_f32 || !out) return ABS_ERR_NULL;
+    if (!aligned16(codes_u8) || !aligned16(scales_e4m3) || !aligned16(out) || ((uintptr_t)tensor_scale_f32 & 3u))
+        return ABS_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t ngroups = rows * cols / 16;
+    const bool fp32 = o.flags & ABS_F_OUT_FP32;
+    switch (fmt) {
+        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+        case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+        case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+        default: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+    }
+}
+
+abs_status_t abs_dequantize(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
+                            const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out_bf16, void* stream) {
+    return abs_dequantize_ex(fmt, codes_u8, scales_e4m3, tensor_scale_f32, rows, cols, out_bf16, nullptr, stream);
+}
+
+// Workspace layout of the host-buffer variants: [input bf16 | codes | scales | alpha], each
+// section rounded up to 256 bytes; the dequantize variant reuses the first section for its output.
+static size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+size_t abs_host_workspace_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
+    if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
+    const size_t n = (size_t)rows * (size_t)cols;
+    return round256(n * 4) + round256(abs_codes_bytes(fmt, rows, cols)) + round256(n / 16) + 256;
+}
+
+abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t rows, int64_t cols,
+                               void* codes_u8_host, void* scales_e4m3_host, float* tensor_scale_f32_host,
+                               const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream) {
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if (rows * cols == 0) return ABS_OK;
+    if (!in_bf16_host || !codes_u8_host || !scales_e4m3_host || !tensor_scale_f32_host || !d_workspace) return ABS_ERR_NULL;
+    if (!aligned16(d_workspace)) return ABS_ERR_ALIGN;
+    if (workspace_bytes < abs_host_workspace_bytes(fmt, rows, cols)) return ABS_ERR_SIZE;
+    const size_t n = (size_t)rows * (size_t)cols;
+    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = n / 16;
+    uint8_t* base = (uint8_t*)d_workspace;
+    uint8_t* d_in = base;
+    uint8_t* d_codes = d_in + round256(n * 4);
+    uint8_t* d_scales = d_codes + round256(cb);
+    float* d_alpha = (float*)(d_scales + round256(sb));
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(d_in, in_bf16_host, n * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+    if (opts && (opts->flags & ABS_F_ALPHA_GIVEN))
+        if (cudaMemcpyAsync(d_alpha, tensor_scale_f32_host, 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+    rc = abs_quantize_ex(fmt, d_in, rows, cols, d_codes, d_scales, d_alpha, opts, stream);
+    if (rc != ABS_OK) return rc;
+    if (cudaMemcpyAsync(codes_u8_host, d_codes, cb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ABS_ERR_CUDA;
+    if (cudaMemcpyAsync(scales_e4m3_host, d_scales, sb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ABS_ERR_CUDA;
+    if (cudaMemcpyAsync(tensor_scale_f32_host, d_alpha, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ABS_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const void* scales_e4m3_host,
+                                 const float* tensor_scale_f32_host, int64_t rows, int64_t cols, void* out_host,
+                                 const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream) {
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if (rows * cols == 0) return ABS_OK;
+    if (!codes_u8_host || !scales_e4m3_host || !tensor_scale_f32_host || !out_host || !d_workspace) return ABS_ERR_NULL;
+    if (!aligned16(d_workspace)) return ABS_ERR_ALIGN;
+    if (workspace_bytes < abs_host_workspace_bytes(fmt, rows, cols)) return ABS_ERR_SIZE;
+    const size_t n = (size_t)rows * (size_t)cols;
+    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = n / 16;
+    const bool fp32 = opts && (opts->flags & ABS_F_OUT_FP32);
+    uint8_t* base = (uint8_t*)d_workspace;
+    uint8_t* d_out = base;
+    uint8_t* d_codes = d_out + round256(n * 4);
+    uint8_t* d_scales = d_codes + round256(cb);
+    float* d_alpha = (float*)(d_scales + round256(sb));
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(d_codes, codes_u8_host, cb, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+    if (cudaMemcpyAsync(d_scales, scales_e4m3_host, sb, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+    if (cudaMemcpyAsync(d_alpha, tensor_scale_f32_host, 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+    rc = abs_dequantize_ex(fmt, d_codes, d_scales, d_alpha, rows, cols, d_out, opts, stream);
+    if (rc != ABS_OK) return rc;
+    if (cudaMemcpyAsync(out_host, d_out, n * (fp32 ? 4 : 2), cudaMemcpyDeviceToHost, s) != cudaSuccess) return ABS_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+abs_status_t abs_selftest_convert(int kind, const float* in_f32, int64_t n, void* out, void* stream) {
+    if (!((kind >= 0 && kind <= 5) || (kind >= 16 && kind <= 20))) return ABS_ERR_FLAGS;
+    if (n < 0) return ABS_ERR_SHAPE;
+    if (n == 0) return ABS_OK;
+    if (!in_f32 || !out) return ABS_ERR_NULL;
+    int64_t blocks = (n + kThreads - 1) / kThreads;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    selftest_kernel<<<(int)blocks, kThreads, 0, (cudaStream_t)stream>>>(kind, in_f32, n, out);
+    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+}  // extern "C"

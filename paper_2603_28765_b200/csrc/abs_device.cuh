@@ -1,0 +1,221 @@
+// Device-side building blocks of the IF quantize / dequantize kernels (sm_100a only).
+//
+// Every floating-point operation that decides a stored bit is written with an explicit
+// rounding intrinsic (__fmul_rn, __fmaf_rn, ...), so the compiler never contracts or
+// reorders it; the file is compiled with -fmad=false as a second line of defence.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace absq {
+
+enum ElemKind { EK_E2M1 = 0, EK_E2M0 = 1, EK_E2M3 = 2, EK_E3M2 = 3 };
+
+// Format traits: (M_FP, M_INT, bits) per Sec. 3 (IF4) and the Sec. 5.1 footnote (IF3, IF6).
+template <int FMT> struct Fmt;
+template <> struct Fmt<0> {  // NVFP4: Fig. 3a stops after step 4
+    static constexpr int BITS = 4; static constexpr bool HAS_INT = false; static constexpr ElemKind EK = EK_E2M1;
+    static constexpr float M_FP = 6.0f, M_INT = 0.0f; static constexpr int EMIN = 0, MBITS = 1;
+};
+template <> struct Fmt<1> {  // IF4
+    static constexpr int BITS = 4; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M1;
+    static constexpr float M_FP = 6.0f, M_INT = 7.0f; static constexpr int EMIN = 0, MBITS = 1;
+};
+template <> struct Fmt<2> {  // IF3: E2M0 or INT3
+    static constexpr int BITS = 3; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M0;
+    static constexpr float M_FP = 4.0f, M_INT = 3.0f; static constexpr int EMIN = 0, MBITS = 0;
+};
+template <> struct Fmt<3> {  // IF6-E2M3
+    static constexpr int BITS = 6; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M3;
+    static constexpr float M_FP = 7.5f, M_INT = 31.0f; static constexpr int EMIN = 0, MBITS = 3;
+};
+template <> struct Fmt<4> {  // IF6-E3M2
+    static constexpr int BITS = 6; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E3M2;
+    static constexpr float M_FP = 28.0f, M_INT = 31.0f; static constexpr int EMIN = -2, MBITS = 2;
+};
+
+// ----------------------------------------------------------------------------- conversions
+
+// Fig. 3a step 2: FP32 -> E4M3 byte, nearest-even, saturating at 448 (hardware convert).
+__device__ __forceinline__ uint32_t e4m3_encode(float t) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.0f), "f"(t));
+    return (uint32_t)r & 0xFFu;
+}
+
+// Value of an E4M3 magnitude byte 0x00..0x7E: the byte placed in FP32's exponent/mantissa top
+// bits is (1+m/8)*2^(e-127) (or m*2^-129 for e = 0, an FP32 subnormal); times 2^120 it is exact.
+__device__ __forceinline__ float e4m3_value(uint32_t mag7) {
+    return __fmul_rn(__uint_as_float(mag7 << 20), 1.329227995784916e36f /* 2^120 */);
+}
+
+// Step 4 for E2M1, two values at once: returns (code(y1) << 4) | code(y0).
+__device__ __forceinline__ uint32_t e2m1x2_encode(float y0, float y1) {
+    uint16_t r;
+    asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; cvt.u16.u8 %0, t; }" : "=h"(r) : "f"(y1), "f"(y0));
+    return (uint32_t)r;
+}
+// Values of the two E2M1 codes of a byte as a half2 (low nibble in the low half).
+__device__ __forceinline__ __half2 e2m1x2_decode(uint32_t byte) {
+    uint32_t h2;
+    asm("{ .reg .b8 t; cvt.u8.u16 t, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "h"((uint16_t)byte));
+    return *reinterpret_cast<__half2*>(&h2);
+}
+// E2M3 / E3M2: two 6-bit codes in the two bytes of a 16-bit container (y0 in the low byte).
+__device__ __forceinline__ uint32_t e2m3x2_encode(float y0, float y1) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e2m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(y1), "f"(y0));
+    return (uint32_t)r;
+}
+__device__ __forceinline__ uint32_t e3m2x2_encode(float y0, float y1) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e3m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(y1), "f"(y0));
+    return (uint32_t)r;
+}
+__device__ __forceinline__ __half2 e2m3x2_decode(uint32_t two_bytes) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e2m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)two_bytes));
+    return *reinterpret_cast<__half2*>(&h2);
+}
+__device__ __forceinline__ __half2 e3m2x2_decode(uint32_t two_bytes) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e3m2x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)two_bytes));
+    return *reinterpret_cast<__half2*>(&h2);
+}
+
+// E2M0 has no hardware convert: magnitudes {0,1,2,4}, ties to the even code
+// (0.5 -> 0, 1.5 -> 2, 3 -> 2), saturating at 4.  Returns the 3-bit code s|ee.
+__device__ __forceinline__ uint32_t e2m0_encode(float y) {
+    float a = fabsf(y);
+    uint32_t idx = (a > 0.5f ? 1u : 0u) + (a >= 1.5f ? 1u : 0u) + (a > 3.0f ? 1u : 0u);
+    return idx | ((__float_as_uint(y) >> 31) << 2);
+}
+__device__ __forceinline__ float e2m0_value(uint32_t code) {
+    uint32_t idx = code & 3u;
+    float v = (idx == 3u) ? 4.0f : (float)idx;
+    return (code & 4u) ? -v : v;
+}
+
+// FP element codes and their values for a pair of scaled inputs (steps 4-5).
+template <ElemKind EK>
+__device__ __forceinline__ void fp_encode_pair(float y0, float y1, uint32_t& c0, uint32_t& c1, float& v0, float& v1) {
+    if constexpr (EK == EK_E2M1) {
+        uint32_t byte = e2m1x2_encode(y0, y1);
+        c0 = byte & 0xFu; c1 = byte >> 4;
+        float2 v = __half22float2(e2m1x2_decode(byte));
+        v0 = v.x; v1 = v.y;
+    } else if constexpr (EK == EK_E2M3) {
+        uint32_t w = e2m3x2_encode(y0, y1);
+        c0 = w & 0x3Fu; c1 = (w >> 8) & 0x3Fu;
+        float2 v = __half22float2(e2m3x2_decode(w));
+        v0 = v.x; v1 = v.y;
+    } else if constexpr (EK == EK_E3M2) {
+        uint32_t w = e3m2x2_encode(y0, y1);
+        c0 = w & 0x3Fu; c1 = (w >> 8) & 0x3Fu;
+        float2 v = __half22float2(e3m2x2_decode(w));
+        v0 = v.x; v1 = v.y;
+    } else {
+        c0 = e2m0_encode(y0); c1 = e2m0_encode(y1);
+        v0 = e2m0_value(c0); v1 = e2m0_value(c1);
+    }
+}
+
+// Value of one FP element code (dequantize path).
+template <ElemKind EK>
+__device__ __forceinline__ float2 fp_decode_pair(uint32_t c0, uint32_t c1) {
+    if constexpr (EK == EK_E2M1) return __half22float2(e2m1x2_decode((c0 & 0xFu) | ((c1 & 0xFu) << 4)));
+    else if constexpr (EK == EK_E2M3) return __half22float2(e2m3x2_decode((c0 & 0x3Fu) | ((c1 & 0x3Fu) << 8)));
+    else if constexpr (EK == EK_E3M2) return __half22float2(e3m2x2_decode((c0 & 0x3Fu) | ((c1 & 0x3Fu) << 8)));
+    else return make_float2(e2m0_value(c0), e2m0_value(c1));
+}
+
+// ----------------------------------------------------------------------------- stochastic rounding
+
+// Philox4x32-10 (Salmon et al.): counter (c0,c1,0,0), key (k0,k1).
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1) {
+    uint32_t c2 = 0u, c3 = 0u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Stochastic rounding of a magnitude onto a minifloat grid with MBITS mantissa bits and smallest
+// normal exponent EMIN: clamp to the top; step s = 2^(max(exponent, EMIN) - MBITS); lo = floor to
+// the step; round up iff u < (a - lo) / s.  All operations are exact in FP32.
+template <int EMIN, int MBITS>
+__device__ __forceinline__ float sr_round_fp(float a, float top, float u) {
+    a = fminf(a, top);
+    int e = (int)(__float_as_uint(a) >> 23) - 127;
+    e = max(e, EMIN);
+    float s = __uint_as_float((uint32_t)(e - MBITS + 127) << 23);
+    float inv_s = __uint_as_float((uint32_t)(MBITS - e + 127) << 23);
+    float lo = __fmul_rn(floorf(__fmul_rn(a, inv_s)), s);
+    float p = __fmul_rn(__fsub_rn(a, lo), inv_s);
+    return (u < p) ? __fadd_rn(lo, s) : lo;
+}
+__device__ __forceinline__ float sr_round_int(float a, float top, float u) {
+    a = fminf(a, top);
+    float lo = floorf(a);
+    float p = __fsub_rn(a, lo);
+    return (u < p) ? __fadd_rn(lo, 1.0f) : lo;
+}
+
+// ----------------------------------------------------------------------------- Hadamard option
+
+// 16-point transform of one group held in registers: sign flips from the mask, natural-order
+// Sylvester butterflies h = 1,2,4,8 with every add/sub rounded to FP32, then times 1/4.
+__device__ __forceinline__ void hadamard16(float (&a)[16], uint32_t sign_mask) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(__float_as_uint(a[i]) ^ (((sign_mask >> i) & 1u) << 31));
+#pragma unroll
+    for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+        for (int base = 0; base < 16; base += 2 * h) {
+#pragma unroll
+            for (int j = base; j < base + h; ++j) {
+                float p = a[j], q = a[j + h];
+                a[j] = __fadd_rn(p, q);
+                a[j + h] = __fsub_rn(p, q);
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = __fmul_rn(a[i], 0.25f);
+}
+
+// ----------------------------------------------------------------------------- loads / unpack
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& v, float* x) {
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
+    x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
+}
+
+// Pack 16 b-bit codes into the little-endian bitstream (code j at bits [b*j, b*j+b)).
+template <int BITS>
+__device__ __forceinline__ void pack_codes(const uint32_t (&c)[16], uint32_t (&w)[3]) {
+    w[0] = w[1] = w[2] = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int pos = BITS * j, word = pos >> 5, sh = pos & 31;
+        w[word] |= c[j] << sh;
+        if (sh + BITS > 32) w[word + 1] |= c[j] >> (32 - sh);
+    }
+}
+template <int BITS>
+__device__ __forceinline__ uint32_t extract_code(const uint32_t (&w)[3], int j) {
+    const int pos = BITS * j, word = pos >> 5, sh = pos & 31;
+    uint32_t v = w[word] >> sh;
+    if (sh + BITS > 32) v |= w[word + 1] << (32 - sh);
+    return v & ((1u << BITS) - 1u);
+}
+
+}  // namespace absq

@@ -1,0 +1,317 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit.
+
+Codes, scale bytes (selection bit included), alpha and dequantized outputs must be identical
+on the same seeded inputs: integer / byte work is compared exactly, and the floating-point
+outputs (alpha, dequantized bf16 / fp32) are compared by bit pattern too, because both sides
+fix the same FP32 operation order.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2603_28765_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+THREADS = max(1, min(32, os.cpu_count() or 1))
+ALL_FMTS = [0, 1, 2, 3, 4]
+
+
+@pytest.fixture(scope="module")
+def B():
+    assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
+    from paper_2603_28765_b200 import binding
+    binding.lib()          # raises if the CUDA library is missing: there is no fallback
+    return binding
+
+
+def to_dev(xb: np.ndarray):
+    return torch.from_numpy(xb.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def gpu_quantize(B, fmt, xb, flags=0, mask=0, seed=0, alpha=None):
+    x = to_dev(xb)
+    opts = B.make_opts(flags, mask, seed)
+    ts = None
+    if flags & B.ABS_F_ALPHA_GIVEN:
+        ts = torch.tensor([alpha], dtype=torch.float32, device="cuda")
+    codes, scales, ts = B.abs_quantize(fmt, x, tensor_scale=ts, opts=opts)
+    torch.cuda.synchronize()
+    rows, cols = xb.shape
+    nb = rows * cols * B.FMT_BITS[fmt] // 8
+    return (codes[:nb].cpu().numpy().reshape(rows, -1) if nb else np.zeros((rows, 0), np.uint8),
+            scales[:rows * cols // 16].cpu().numpy().reshape(rows, -1) if nb else np.zeros((rows, 0), np.uint8),
+            np.float32(ts.item()), (codes, scales, ts))
+
+
+def assert_same(name, got, want):
+    got = np.asarray(got)
+    want = np.asarray(want)
+    assert got.shape == want.shape, (name, got.shape, want.shape)
+    if not np.array_equal(got, want):
+        bad = np.argwhere(got != want)
+        raise AssertionError(f"{name}: {len(bad)} of {got.size} differ; first at {bad[:5].tolist()} "
+                             f"got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}")
+
+
+def check_case(B, oracle, fmt, xb, flags=0, mask=0, seed=0, alpha=None, dequant=True):
+    rows, cols = xb.shape
+    c, s, a, dev = gpu_quantize(B, fmt, xb, flags, mask, seed, alpha)
+    oc, osc, oa = oracle.quantize(fmt, xb, flags=flags, sign_mask=mask, sr_seed=seed, alpha=alpha, threads=THREADS)
+    assert np.float32(a).view(np.uint32) == np.float32(oa).view(np.uint32), ("alpha", a, oa)
+    assert_same("scales", s, osc)
+    assert_same("codes", c, oc)
+    if dequant and rows * cols:
+        out = B.abs_dequantize(fmt, dev[0], dev[1], dev[2], rows, cols)
+        want = oracle.dequantize(fmt, oc, osc, oa, rows, cols, threads=THREADS)
+        assert_same("dequant bf16", out.view(torch.int16).cpu().numpy().view(np.uint16), want)
+        out32 = B.abs_dequantize(fmt, dev[0], dev[1], dev[2], rows, cols, opts=B.make_opts(B.ABS_F_OUT_FP32))
+        want32 = oracle.dequantize(fmt, oc, osc, oa, rows, cols, out_fp32=True, threads=THREADS)
+        assert_same("dequant fp32", out32.cpu().numpy().view(np.uint32), want32.view(np.uint32))
+    return s
+
+
+# ------------------------------------------------------------------ the converts the kernels rely on
+
+@pytest.mark.parametrize("kind,fmt", [(0, None), (1, 1), (2, 2), (3, 3), (4, 4)])
+def test_hardware_converts_match_oracle_exhaustively(B, oracle, kind, fmt):
+    """All 2^32 FP32 inputs go through the device convert; the output is checked to be monotone in
+    |x| on the device, and every change point (plus its neighbour) is compared with the oracle, which
+    is monotone by construction -- together that is equality on every finite input."""
+    enc = (lambda v: oracle.e4m3_encode(v)) if kind == 0 else (lambda v: oracle.fp_encode(fmt, v))
+    chunk = 1 << 28
+    top_finite = 0x7F800000
+    for sign in (0, 1):
+        if kind == 0 and sign == 1:
+            continue          # scale inputs are non-negative
+        prev_last = None
+        changes = []
+        for start in range(0, top_finite, chunk):
+            n = min(chunk, top_finite - start)
+            bits = torch.arange(start, start + n, dtype=torch.int32, device="cuda")
+            if sign:
+                bits = bits + (-2 ** 31)          # sets the sign bit of the pattern
+            f = bits.view(torch.float32)
+            out = B.abs_selftest_convert(kind, f)
+            o = out.to(torch.int16)
+            d = o[1:] - o[:-1]
+            assert int(d.min()) >= 0, "device convert is not monotone in |x|"
+            idx = torch.nonzero(d).flatten().cpu().numpy()
+            ocpu = out[idx + 1].cpu().numpy() if len(idx) else np.zeros(0, np.uint8)
+            for i, code in zip(idx, ocpu):
+                changes.append((start + int(i) + 1, int(code)))
+            first, last = int(out[0]), int(out[-1])
+            if prev_last is not None and first != prev_last:
+                assert first > prev_last
+                changes.append((start, first))
+            elif prev_last is None:
+                changes.append((start, first))
+            prev_last = last
+            del bits, f, out, o, d
+        assert len(changes) >= 4
+        for pos, code in changes:
+            v = np.array([pos | (sign << 31)], dtype=np.uint32).view(np.float32)[0]
+            assert enc(v) == code, (kind, hex(pos), code, enc(v))
+            if pos > 0:
+                vm = np.array([(pos - 1) | (sign << 31)], dtype=np.uint32).view(np.float32)[0]
+                assert enc(vm) < code
+        # +-inf saturate like the largest finite input
+        vinf = torch.tensor([np.inf if sign == 0 else -np.inf], dtype=torch.float32, device="cuda")
+        assert int(B.abs_selftest_convert(kind, vinf)[0]) == enc(np.float32(np.inf if sign == 0 else -np.inf))
+
+
+@pytest.mark.parametrize("k,fmt", [(0, None), (1, 1), (2, 2), (3, 3), (4, 4)])
+def test_device_decode_tables(B, oracle, k, fmt):
+    n = 127 if k == 0 else (1 << B.FMT_BITS[fmt])
+    codes = torch.arange(n, dtype=torch.float32, device="cuda")
+    got = B.abs_selftest_convert(16 + k, codes).cpu().numpy()
+    want = np.array([oracle.e4m3_value(c) if k == 0 else oracle.fp_value(fmt, c) for c in range(n)], dtype=np.float32)
+    assert_same("decode", got.view(np.uint32), want.view(np.uint32))
+
+
+def test_device_rint_is_ties_even(B):
+    v = torch.tensor([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 6.5, 7.4999995, -7.5, 30.5, 31.5], dtype=torch.float32,
+                     device="cuda")
+    got = B.abs_selftest_convert(5, v).cpu().numpy().astype(np.int8)
+    assert list(got) == [0, 2, 2, 0, -2, -2, 6, 7, -8, 30, 32]
+
+
+# ------------------------------------------------------------------ parity on the configurations
+
+SMALL = {
+    "cfg1": ("cfg1", 256, 1024),            # the full first configuration
+    "cfg2": ("cfg2", 300, 4096),            # several tiles and a ragged tail (300 rows)
+    "cfg3a": ("cfg3a", 64, 14336),
+    "cfg3b": ("cfg3b", 515, 4096),
+    "cfg4": ("cfg4", 384, 8192),
+    "cfg5": ("cfg5", 257, 8192),
+}
+
+
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+@pytest.mark.parametrize("case", sorted(SMALL))
+def test_rtn_parity_small(B, oracle, fmt, case):
+    name, rows, cols = SMALL[case]
+    check_case(B, oracle, fmt, I.generate(name, rows, cols))
+
+
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+@pytest.mark.parametrize("case", sorted(I.edge_tensors()))
+def test_edge_tensor_parity(B, oracle, fmt, case):
+    check_case(B, oracle, fmt, I.edge_tensors()[case])
+
+
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+@pytest.mark.parametrize("flags", ["H", "S", "S17", "HS", "HS17"])
+def test_option_parity(B, oracle, fmt, flags):
+    f = (B.ABS_F_HADAMARD16 if "H" in flags else 0) | (B.ABS_F_STOCHASTIC if "S" in flags else 0) \
+        | (B.ABS_F_SR_SCALE_17_16 if "17" in flags else 0)
+    mask = oracle.hadamard_sign_mask(2024)
+    for name, rows, cols in (("cfg4", 200, 2048), ("cfg2", 96, 1024), ("cfg1", 64, 256)):
+        check_case(B, oracle, fmt, I.generate(name, rows, cols), flags=f, mask=mask, seed=0xDEADBEEF12345678)
+    for case in ("tiny_row", "wide_dynamic_range", "signed_zeros", "zeros_3x48", "ragged_37x208"):
+        check_case(B, oracle, fmt, I.edge_tensors()[case], flags=f, mask=mask, seed=99)
+
+
+def test_sr_element_index_beyond_32_bits_of_groups(B, oracle):
+    """Different seeds and row offsets give different streams; the same seed repeats exactly."""
+    xb = I.generate("cfg1", 64, 256)
+    a = gpu_quantize(B, 1, xb, B.ABS_F_STOCHASTIC, 0, 5)
+    b = gpu_quantize(B, 1, xb, B.ABS_F_STOCHASTIC, 0, 5)
+    c = gpu_quantize(B, 1, xb, B.ABS_F_STOCHASTIC, 0, 6)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert not np.array_equal(a[0], c[0])
+
+
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+def test_alpha_given_and_worked_example(B, oracle, fmt):
+    x = np.zeros((1, 16), np.float32)
+    x[0, :4] = [6, 18, 36, 42]
+    xb = I.f32_to_bf16_bits(x)
+    check_case(B, oracle, fmt, xb, flags=B.ABS_F_ALPHA_GIVEN, alpha=1.0)
+    check_case(B, oracle, fmt, xb)
+    check_case(B, oracle, fmt, I.generate("cfg5", 64, 512), flags=B.ABS_F_ALPHA_GIVEN, alpha=0.01)
+    if fmt == 1:    # Fig. 3a: integer candidate selected, bytes 31 76, scale 0xFE with Eq. 1's alpha
+        c, s, a, _ = gpu_quantize(B, 1, xb)
+        assert c[0].tobytes() == bytes([0x31, 0x76, 0, 0, 0, 0, 0, 0]) and s[0, 0] == 0xFE and a == np.float32(2 ** -6)
+
+
+def test_amax_entry_point(B, oracle):
+    xb = I.generate("cfg2", 123, 2048)
+    mask = 0x5A3C
+    for flags in (0, B.ABS_F_HADAMARD16):
+        got = B.abs_amax(to_dev(xb), opts=B.make_opts(flags, mask)).item()
+        want = oracle.amax(xb, flags=flags, sign_mask=mask, threads=THREADS)
+        assert np.float32(got).view(np.uint32) == np.float32(want).view(np.uint32)
+        for fmt in ALL_FMTS:
+            a = np.float32(B.abs_alpha_from_amax(fmt, float(want)))
+            assert a.view(np.uint32) == np.float32(oracle.alpha_from_amax(fmt, want)).view(np.uint32)
+
+
+def test_back_to_back_calls_reuse_scratch(B, oracle):
+    """The amax scratch slot re-arms itself: many calls in a row, on two streams, stay exact."""
+    xs = [I.generate("cfg1", 64, 256, seed=s) for s in range(4)]
+    want = [oracle.quantize(1, x) for x in xs]
+    devs = [to_dev(x) for x in xs]
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs = []
+    for rep in range(600):      # wraps the scratch ring more than once across both streams
+        k = rep % 4
+        outs.append((k, B.abs_quantize(1, devs[k], stream=(s1 if rep % 2 else s2))))
+    torch.cuda.synchronize()
+    for k, (c, s, a) in outs[-16:]:
+        assert np.float32(a.item()) == want[k][2]
+        assert np.array_equal(c.cpu().numpy().reshape(64, -1), want[k][0])
+        assert np.array_equal(s.cpu().numpy().reshape(64, -1), want[k][1])
+
+
+def test_host_buffer_entry_points(B, oracle):
+    xb = I.generate("cfg5", 96, 1024)
+    rows, cols = xb.shape
+    for fmt in (1, 3):
+        ws = torch.empty(B.abs_host_workspace_bytes(fmt, rows, cols), dtype=torch.uint8, device="cuda")
+        xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
+        ch = torch.empty(B.abs_codes_bytes(fmt, rows, cols), dtype=torch.uint8).pin_memory()
+        sh = torch.empty(B.abs_scales_bytes(fmt, rows, cols), dtype=torch.uint8).pin_memory()
+        ah = torch.zeros(1, dtype=torch.float32).pin_memory()
+        B.abs_quantize_host(fmt, xh, ch, sh, ah, ws)
+        oc, osc, oa = oracle.quantize(fmt, xb)
+        assert np.float32(ah.item()) == oa
+        assert_same("codes", ch.numpy().reshape(rows, -1), oc)
+        assert_same("scales", sh.numpy().reshape(rows, -1), osc)
+        oh = torch.empty((rows, cols), dtype=torch.int16).pin_memory()
+        B.abs_dequantize_host(fmt, ch, sh, ah, rows, cols, oh, ws)
+        assert_same("dequant", oh.numpy().view(np.uint16), oracle.dequantize(fmt, oc, osc, oa, rows, cols))
+
+
+def test_argument_validation_on_device(B):
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    L = B.lib()
+    codes = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    ts = torch.zeros(4, dtype=torch.float32, device="cuda")
+    q = lambda fmt, xp, r, c, cp, sp, tp, o=None: L.abs_quantize_ex(fmt, xp, r, c, cp, sp, tp, o, None)
+    assert q(9, x.data_ptr(), 4, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 4
+    assert q(1, x.data_ptr(), 4, 60, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 2
+    assert q(1, x.data_ptr(), -1, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 2
+    assert q(1, None, 4, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 1
+    assert q(1, x.data_ptr() + 2, 4, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 3
+    import ctypes
+    bad = B.make_opts(1 << 9)
+    assert q(1, x.data_ptr(), 4, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr(), ctypes.byref(bad)) == 5
+    assert q(1, x.data_ptr(), 0, 64, codes.data_ptr(), scales.data_ptr(), ts.data_ptr()) == 0
+    sr = B.make_opts(B.ABS_F_STOCHASTIC)
+    assert L.abs_dequantize_ex(1, codes.data_ptr(), scales.data_ptr(), ts.data_ptr(), 4, 64, x.data_ptr(),
+                               ctypes.byref(sr), None) == 5
+    torch.cuda.synchronize()
+
+
+def test_guard_bands_stay_untouched(B, oracle):
+    """Outputs are written inside their buffers only: sentinel bytes around them survive."""
+    for fmt in ALL_FMTS:
+        xb = I.generate("cfg1", 37, 208)
+        rows, cols = xb.shape
+        nb, ns = B.abs_codes_bytes(fmt, rows, cols), rows * cols // 16
+        pad = 256
+        cbuf = torch.full((nb + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        sbuf = torch.full((ns + 2 * pad + 15,), 0xA5, dtype=torch.uint8, device="cuda")
+        obuf = torch.full((rows * cols * 2 + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        codes, scales, out = cbuf[pad:pad + nb], sbuf[pad:pad + ns], obuf[pad:pad + rows * cols * 2]
+        ts = torch.zeros(1, dtype=torch.float32, device="cuda")
+        B.abs_quantize(fmt, to_dev(xb), codes=codes, scales=scales, tensor_scale=ts)
+        B.abs_dequantize(fmt, codes, scales, ts, rows, cols, out=out.view(torch.bfloat16).view(rows, cols))
+        torch.cuda.synchronize()
+        for buf, n in ((cbuf, nb), (sbuf, ns), (obuf, rows * cols * 2)):
+            assert bool((buf[:pad] == 0xA5).all()) and bool((buf[pad + n:] == 0xA5).all())
+
+
+# ------------------------------------------------------------------ full-size configurations
+
+FULL = [
+    ("cfg2", [1], 0),
+    ("cfg3a", [0, 1], 0),
+    ("cfg3b", [0, 1], 0),
+    ("cfg5", [0, 1, 2, 3, 4], 0),
+    ("cfg4", [1], "HS17"),
+]
+
+
+@pytest.mark.parametrize("name,fmts,opt", FULL, ids=[f[0] for f in FULL])
+def test_full_size_parity(B, oracle, name, fmts, opt):
+    """Element-by-element comparison at the benchmark's full sizes (the oracle, threaded over rows,
+    still finishes in seconds per format)."""
+    xb = I.generate(name)
+    flags, mask, seed = 0, 0, 0
+    if opt == "HS17":
+        flags = B.ABS_F_HADAMARD16 | B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16
+        mask, seed = oracle.hadamard_sign_mask(5), 5
+    for fmt in fmts:
+        s = check_case(B, oracle, fmt, xb, flags=flags, mask=mask, seed=seed)
+        if fmt:
+            frac = float((s >> 7).mean())
+            assert 0.05 < frac < 0.999, (name, fmt, frac)
+    if opt == "HS17":       # the extra row of the gradient configuration: 17/16 option off
+        check_case(B, oracle, 1, xb, flags=flags & ~B.ABS_F_SR_SCALE_17_16, mask=mask, seed=seed, dequant=False)
