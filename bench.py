@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the IF4 quantize + dequantize hot path on B200.
+
+A step is one pass of the whole path over one tensor of the LLM-activation-like workload
+(bf16 8192 x 4096, 0.5*Student-t(3) with 0.5 % outlier columns x50): ``abs_quantize`` (grid-wide
+amax -> alpha, then the group-quantize kernel) followed by ``abs_dequantize`` -- three kernel
+launches.  The metric is GB/s of algorithmic bytes in + out per step:
+    quantize   2N (bf16 in) + N/2 (codes) + N/16 (scales)
+    dequantize N/2 + N/16 in, 2N (bf16 out)                    => 5.125 N bytes per step.
+Steps rotate over enough tensor sets to exceed 4x the L2 capacity, so every step starts cold.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]          CUDA path, one JSON line
+  python bench.py --impl reference ...                         the CPU oracle timed on host cores
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same step on its own tensors:
+independent problems, no data-path collective, weak scaling; time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_28765_b200 import inputs as I  # noqa: E402
+
+WORKLOAD = "cfg2"
+FMT_IF4 = 1
+METRIC = "IF4 quantize+dequantize GB/s (algorithmic bytes in+out)"
+UNIT = "GB/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the group-quantize kernel per element, from the ncu capture summarised in
+# profiles/quantize_if4_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch / N).
+NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = None
+
+
+def step_bytes(n_elems: int) -> float:
+    return 2.0 * (2.0 * n_elems + n_elems / 2.0 + n_elems / 16.0)
+
+
+def quant_kernel_bytes(n_elems: int) -> float:
+    return 2.0 * n_elems + n_elems / 2.0 + n_elems / 16.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, torch_device_index: int):
+        self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except TypeError:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # NVML missing: report that rather than guess
+            self.err = repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.ok:
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self, note=""):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable: " + getattr(self, "err", "")}
+        out = {"sm_mhz": int(statistics.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+               "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if note:
+            out["note"] = note
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_rate(xb: np.ndarray, repeats: int, threads: int):
+    """Times the oracle (quantize + dequantize, as it stands) on host cores; returns best GB/s and seconds."""
+    from oracle import abs_oracle as O
+    rows, cols = xb.shape
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        c, s, a = O.quantize(FMT_IF4, xb, threads=threads)
+        O.dequantize(FMT_IF4, c, s, a, rows, cols, threads=threads)
+        best = min(best, time.perf_counter() - t0)
+    return step_bytes(rows * cols) / best / 1e9, best
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the same workload, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = I.CONFIGS[WORKLOAD]
+    threads = os.cpu_count() or 1
+    total = args.steps + args.warmup
+    probe = I.generate(WORKLOAD, 256, cfg.cols)
+    _, t_probe = oracle_rate(probe, 1, threads)
+    budget_s = 120.0
+    rows = int(min(cfg.rows, max(256, (budget_s / max(total, 1)) / (t_probe / 256))))
+    rows -= rows % 64
+    xb = I.generate(WORKLOAD, rows, cfg.cols)
+    from oracle import abs_oracle as O
+    times = []
+    for i in range(total):
+        t0 = time.perf_counter()
+        c, s, a = O.quantize(FMT_IF4, xb, threads=threads)
+        O.dequantize(FMT_IF4, c, s, a, rows, cfg.cols, threads=threads)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    mean_s = sum(times) / len(times)
+    value = step_bytes(rows * cfg.cols) / mean_s / 1e9
+    sample = f"first {rows} of {cfg.rows} rows of the {cfg.rows}x{cfg.cols} tensor per step, {threads} threads over rows"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(mean_s * 1e3, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: IF4 quantize+dequantize, bf16 {cfg.rows}x{cfg.cols}, {cfg.note}",
+                   "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+# ----------------------------------------------------------------------------- CUDA path
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_28765_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    L = B.lib()                       # raises if the CUDA library is missing
+    B.abs_init(local)
+
+    cfg = I.CONFIGS[WORKLOAD]
+    rows, cols = cfg.rows, cfg.cols
+    n = rows * cols
+    nb_codes, nb_scales = B.abs_codes_bytes(FMT_IF4, rows, cols), B.abs_scales_bytes(FMT_IF4, rows, cols)
+    set_bytes = 2 * n + nb_codes + nb_scales + 2 * n
+    n_sets = max(2, -(-4 * L2_BYTES // set_bytes))          # rotate over > 4x L2 of distinct buffers
+
+    # Synthetic inputs: one host tensor per rank from the seeded recipe; the other sets are row
+    # rotations of it (same distribution, different addresses and group contents).
+    xb = I.generate(WORKLOAD, seed=cfg.seed + 1000 * rank)
+    x0 = torch.from_numpy(xb.view(np.int16)).to(dev).view(torch.bfloat16)
+    xs = [x0] + [torch.roll(x0, shifts=17 * k, dims=0).contiguous() for k in range(1, n_sets)]
+    codes = [torch.empty(nb_codes, dtype=torch.uint8, device=dev) for _ in range(n_sets)]
+    scales = [torch.empty(nb_scales, dtype=torch.uint8, device=dev) for _ in range(n_sets)]
+    alphas = [torch.zeros(1, dtype=torch.float32, device=dev) for _ in range(n_sets)]
+    outs = [torch.empty((rows, cols), dtype=torch.bfloat16, device=dev) for _ in range(n_sets)]
+    stream = torch.cuda.current_stream()
+    sp = C.c_void_p(stream.cuda_stream)
+    qargs = [(FMT_IF4, xs[k].data_ptr(), rows, cols, codes[k].data_ptr(), scales[k].data_ptr(), alphas[k].data_ptr(), sp)
+             for k in range(n_sets)]
+    dargs = [(FMT_IF4, codes[k].data_ptr(), scales[k].data_ptr(), alphas[k].data_ptr(), rows, cols, outs[k].data_ptr(), sp)
+             for k in range(n_sets)]
+
+    def step(i):
+        k = i % n_sets
+        rc = L.abs_quantize(*qargs[k])
+        rc |= L.abs_dequantize(*dargs[k])
+        if rc:
+            raise RuntimeError(f"C-ABI call failed with status {rc}")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    # ---- timed region: exactly K steps; the quantize kernel is also timed on its own on every
+    # 8th step through the library's event hook (events on the launching stream).
+    sampler = ClockSampler(local)
+    n_probe = min(64, max(1, args.steps // 8))
+    probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_probe)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for a, b in probes:        # torch creates the CUDA event on first record; the library re-records it later
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record(stream)
+    pi = 0
+    for i in range(args.steps):
+        if i % 8 == 7 and pi < n_probe:
+            B.abs_profile_events(*probes[pi])
+            step(i)
+            B.abs_profile_events()
+            pi += 1
+        else:
+            step(i)
+    end.record(stream)
+    barrier()
+    sampler.stop()
+    ms_total = start.elapsed_time(end)
+    clock_note = ""
+    if sampler.ok and len(sampler.samples) < 5:
+        # the timed region was shorter than a few NVML periods: sample an identical untimed loop too
+        sampler.start()
+        t_end = time.perf_counter() + 0.3
+        i = 0
+        while time.perf_counter() < t_end:
+            step(i)
+            i += 1
+        torch.cuda.synchronize()
+        sampler.stop()
+        clock_note = "timed region shorter than the sampling period; samples extended over an identical untimed loop"
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * step_bytes(n) / (ms_per_step * 1e-3) / 1e9
+
+    quant_ms = [a.elapsed_time(b) for a, b in probes[:pi]]
+    if not quant_ms:     # fewer than 8 steps: time the kernel on one extra step
+        B.abs_profile_events(*probes[0])
+        step(0)
+        B.abs_profile_events()
+        torch.cuda.synchronize()
+        quant_ms = [probes[0][0].elapsed_time(probes[0][1])]
+    q_ms = sum(quant_ms) / len(quant_ms)
+    peak, peak_src = measured_peak()
+    achieved = quant_kernel_bytes(n) / (q_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "quantize_kernel<IF4> (group-quantize, Fig. 3a steps 1-10)",
+                "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "peak_source": peak_src, "us_per_launch": round(q_ms * 1e3, 2),
+                "algorithmic_bytes_per_launch": quant_kernel_bytes(n),
+                "traffic": (NCU_QUANT_TRAFFIC_BYTES_PER_ELEM * n) if NCU_QUANT_TRAFFIC_BYTES_PER_ELEM else None}
+
+    # ---- end to end through the host-buffer C-ABI calls (pinned host memory, copies in the timed region)
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
+    ws = torch.empty(B.abs_host_workspace_bytes(FMT_IF4, rows, cols), dtype=torch.uint8, device=dev)
+    xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
+    ch = torch.empty(nb_codes, dtype=torch.uint8).pin_memory()
+    sh = torch.empty(nb_scales, dtype=torch.uint8).pin_memory()
+    ah = torch.zeros(1, dtype=torch.float32).pin_memory()
+    oh = torch.empty((rows, cols), dtype=torch.int16).pin_memory()
+
+    def e2e_step():
+        B.abs_quantize_host(FMT_IF4, xh, ch, sh, ah, ws)
+        B.abs_dequantize_host(FMT_IF4, ch, sh, ah, rows, cols, oh, ws)
+
+    for _ in range(3 if e2e_steps else 0):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / max(e2e_steps, 1)
+    t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_s = float(t.item())
+    e2e = {"value": round(world * step_bytes(n) / e2e_s / 1e9, 2) if e2e_steps else None, "unit": UNIT,
+           "h2d_bytes_per_step": 2 * n + nb_codes + nb_scales + 4, "d2h_bytes_per_step": nb_codes + nb_scales + 4 + 2 * n,
+           "ms_per_step": round(e2e_s * 1e3, 3), "steps": e2e_steps,
+           "api": "abs_quantize_host + abs_dequantize_host (pinned host buffers)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{WORKLOAD}: IF4 quantize+dequantize, bf16 {rows}x{cols}, {cfg.note}",
+                       "bytes_per_step": step_bytes(n), "elements_per_s": round(world * n / (ms_per_step * 1e-3), 0),
+                       "l2": f"cold: steps rotate over {n_sets} buffer sets ({n_sets * set_bytes >> 20} MiB > 4x L2)",
+                       "sharding": "one independent tensor per rank, no collective"},
+            "roofline": roofline, "e2e": e2e, "gpu_launches": 3 * args.steps,
+            "clocks": sampler.summary(clock_note),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            threads = os.cpu_count() or 1
+            gbs, best = oracle_rate(xb, 3, threads)
+            line["cpu_baseline"] = {"value": round(gbs, 4), "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": f"the whole {rows}x{cols} tensor, quantize+dequantize, best of 3 "
+                                              f"({best:.3f} s), {threads} threads over rows"}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,12 @@ ABS_API abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_hos
                                  const float* tensor_scale_f32_host, int64_t rows, int64_t cols, void* out_host,
                                  const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream);
 
+/* Profiling hook (no counterpart in the paper): while both handles (cudaEvent_t as void*) are set,
+ * every quantize call records them on its stream immediately before and after the group-quantize
+ * kernel, so a caller can time that kernel inside a longer stream of work.  Pass NULLs to switch it
+ * off.  Process-wide and not thread-safe: set it only while no other thread is calling the library. */
+ABS_API void abs_profile_events(void* quantize_begin, void* quantize_end);
+
 /* Self-test hook: applies one of the device conversions the kernels use to n FP32 values.
  *   kind 0: E4M3 scale byte (Fig. 3a step 2)   kind 1..4: FP element code of NVFP4/IF4 (E2M1),
  *   IF3 (E2M0), IF6_E2M3, IF6_E3M2 (step 4)    kind 5: integer candidate rint(z) & 0xFF (step 7)

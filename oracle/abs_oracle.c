@@ -359,13 +359,15 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
                 e_fp[i] = fmaf(vfp, d, -xi);
                 if (!F->has_int) continue;
                 /* E4 (step 7): integer candidate of y * M_INT / M_FP, clamped to +-M_INT. */
-                const float z = y * c_pre;
                 float kf;
                 if (flags & F_STOCHASTIC) {
+                    const float z = y * c_pre;   /* the stochastic draw needs the FP32 value itself */
                     kf = (float)grid_round_sr(intg, m_int + 1, fabsf(z), u);
                     if (f32_to_bits(z) >> 31) kf = -kf;
                 } else {
-                    kf = nearbyintf(z); /* default rounding mode: nearest, ties to even */
+                    /* int(.) of step 7 rounds the real product y * M_INT/M_FP once: the product of
+                     * two floats is exact in double, then nearest-integer, ties to even. */
+                    kf = (float)nearbyint((double)y * (double)c_pre);
                     if (kf > F->m_int) kf = F->m_int;
                     if (kf < -F->m_int) kf = -F->m_int;
                 }

@@ -27,7 +27,7 @@ ABS_OK = 0
 EXPORTS = [
     "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
-    "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert",
+    "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
 ]
 
 
@@ -86,6 +86,8 @@ def lib():
             L.abs_quantize_host.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp, sz, vp]
             L.abs_dequantize_host.restype = C.c_int
             L.abs_dequantize_host.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, op, vp, sz, vp]
+            L.abs_profile_events.restype = None
+            L.abs_profile_events.argtypes = [vp, vp]
             L.abs_selftest_convert.restype = C.c_int
             L.abs_selftest_convert.argtypes = [C.c_int, vp, i64, vp, vp]
             _lib = L
@@ -202,6 +204,13 @@ def abs_dequantize_host(fmt: int, codes_host, scales_host, alpha_host, rows: int
                                        cols, out_host.data_ptr(), C.byref(opts) if opts is not None else None,
                                        workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "abs_dequantize_host")
+
+
+def abs_profile_events(begin_event=None, end_event=None):
+    """Records the two torch CUDA events around the group-quantize kernel of later quantize calls;
+    call with no arguments to switch the hook off."""
+    lib().abs_profile_events(C.c_void_p(begin_event.cuda_event) if begin_event is not None else None,
+                             C.c_void_p(end_event.cuda_event) if end_event is not None else None)
 
 
 def abs_selftest_convert(kind: int, x_f32, out=None, stream=None):

@@ -6,6 +6,7 @@
 // consecutive row elements: 32 bytes in, 2*b + 1 bytes out.
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
+#include "abs_fast4.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -149,8 +150,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                         k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
                         k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
                     } else {
-                        k0 = fminf(fmaxf(rintf(z0), -F::M_INT), F::M_INT);
-                        k1 = fminf(fmaxf(rintf(z1), -F::M_INT), F::M_INT);
+                        // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
+                        k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);
+                        k1 = __fsub_rn(__fmaf_rn(y1, c_pre, 12582912.0f), 12582912.0f);
+                        k0 = fminf(fmaxf(k0, -F::M_INT), F::M_INT);
+                        k1 = fminf(fmaxf(k1, -F::M_INT), F::M_INT);
                     }
                     const float f0 = __fmaf_rn(k0, d_int, -x0), f1 = __fmaf_rn(k1, d_int, -x1);   // E5 (steps 8-9)
                     s_int[chain] = __fmaf_rn(f0, f0, s_int[chain]);
@@ -294,6 +298,9 @@ struct DeviceState {
 };
 DeviceState g_dev[kMaxDevices];
 
+// Optional CUDA events recorded around the group-quantize kernel (abs_profile_events).
+cudaEvent_t g_ev_quant_begin = nullptr, g_ev_quant_end = nullptr;
+
 abs_status_t device_state(DeviceState** out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ABS_ERR_CUDA;
@@ -356,6 +363,16 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const int grid = grid_for(st, ngroups, 64);
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
+    if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
+    if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
+        if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
+            const int pgrid = grid_for(st, ngroups, FMT == ABS_FMT_IF4 ? 4 : 64);   // IF4: resident blocks only
+            quantize4_fast_kernel<FMT == ABS_FMT_IF4><<<pgrid, kThreads, 0, s>>>((const uint4*)in, (uint2*)codes,
+                                                                               (uint8_t*)scales, alpha, ngroups, mul);
+            if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
     quantize_kernel<FMT, R, S><<<grid, kThreads, 0, s>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales,   \
                                                          alpha, ngroups, mul, o.had_sign_mask, k0, k1)
@@ -364,6 +381,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     else if (sr) ABS_LAUNCH_Q(false, true);
     else ABS_LAUNCH_Q(false, false);
 #undef ABS_LAUNCH_Q
+    if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
@@ -424,6 +442,11 @@ abs_status_t abs_init(int device) {
     abs_status_t rc = device_state(&st);
     cudaSetDevice(prev);
     return rc;
+}
+
+void abs_profile_events(void* quantize_begin, void* quantize_end) {
+    g_ev_quant_begin = (cudaEvent_t)quantize_begin;
+    g_ev_quant_end = (cudaEvent_t)quantize_end;
 }
 
 float abs_alpha_from_amax(abs_fmt_t fmt, float amax) {

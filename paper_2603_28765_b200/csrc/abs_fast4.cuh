@@ -1,0 +1,213 @@
+// Fast path of the group-quantize kernel for the 4-bit formats (IF4, NVFP4), round-to-nearest,
+// no Hadamard / stochastic options.  Same arithmetic as the generic kernel, bit for bit, written
+// for the sm_100a issue budget: packed f32x2 multiply / FMA for the per-element work, the integer
+// candidate rounded by one fused add of 1.5*2^23 + 8 (the low mantissa nibble of the sum is the
+// offset-binary code), three-input max for the group maximum, integer Horner packing of the codes.
+#pragma once
+#include "abs_device.cuh"
+
+namespace absq {
+
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3abs(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(fabsf(a)), "f"(fabsf(b)), "f"(fabsf(c)));
+    return d;
+}
+
+// 1.5 * 2^23 + 8: adding it to an integer-valued-after-rounding k in [-8, 7] leaves k + 8 in the
+// low mantissa nibble, so eight such sums combine into eight offset-binary nibbles without borrows.
+constexpr float kMagic8 = 12582920.0f;
+constexpr uint32_t kMagic8Bits = 0x4B400008u;
+
+// Bytes b0..b3 (each < 256) -> b0 | b1<<8 | b2<<16 | b3<<24 with multiply-adds (FMA pipe, not the ALU).
+__device__ __forceinline__ uint32_t merge_bytes(uint32_t b0, uint32_t b1, uint32_t b2, uint32_t b3) {
+    return ((b3 * 256u + b2) * 256u + b1) * 256u + b0;
+}
+
+
+// Step 4 for eight scaled values at once: four e2m1x2 converts whose bytes are packed into one word
+// inside the asm block (no byte masks), plus the half2 values of each byte for the error terms.
+__device__ __forceinline__ uint32_t e2m1x8_encode_decode(const float (&y)[8], uint32_t (&h)[4]) {
+    uint32_t w;
+    asm("{ .reg .b8 a, b, c, d;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 a, %6, %5;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b, %8, %7;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 c, %10, %9;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 d, %12, %11;\n"
+        "  cvt.rn.f16x2.e2m1x2 %1, a;\n"
+        "  cvt.rn.f16x2.e2m1x2 %2, b;\n"
+        "  cvt.rn.f16x2.e2m1x2 %3, c;\n"
+        "  cvt.rn.f16x2.e2m1x2 %4, d;\n"
+        "  mov.b32 %0, {a, b, c, d}; }"
+        : "=r"(w), "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+        : "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]), "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]));
+    return w;
+}
+__device__ __forceinline__ uint32_t e2m1x8_encode(const float (&y)[8]) {
+    uint32_t w;
+    asm("{ .reg .b8 a, b, c, d;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 a, %2, %1;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b, %4, %3;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 c, %6, %5;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 d, %8, %7;\n"
+        "  mov.b32 %0, {a, b, c, d}; }"
+        : "=r"(w)
+        : "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]), "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]));
+    return w;
+}
+
+// Per-element work of one group (steps 3-10 of Fig. 3a) once the scale is known.
+// CLAMP is the rare variant for scale bytes that are subnormal (1..7) or saturated (0x7E): there
+// |y * 7/6| can exceed 7.5, so the integer candidate must be clamped to +-7; for every other scale
+// byte |y| <= 6 * 17/16 and the rounded integer is within +-7 by construction.
+template <bool HAS_INT, bool CLAMP>
+__device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, float d, float r, uint32_t& sbyte,
+                                             uint32_t& c_lo, uint32_t& c_hi) {
+    const uint64_t R2 = pack2(r, r);
+    if constexpr (!HAS_INT) {
+#pragma unroll
+        for (int hgrp = 0; hgrp < 2; ++hgrp) {
+            float y[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                unpack2(mul2(pack2(x[8 * hgrp + 2 * i], x[8 * hgrp + 2 * i + 1]), R2), y[2 * i], y[2 * i + 1]);   // E1
+            (hgrp ? c_hi : c_lo) = e2m1x8_encode(y);                                                           // E2
+        }
+        sbyte = sb;
+    } else {
+        const float c_pre = __uint_as_float(0x3F955555u);    // fp32(7/6)
+        const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
+        const float d_int = __fmul_rn(d, c_post);
+        const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
+        const uint64_t MG2 = pack2(kMagic8, kMagic8), NMG2 = pack2(-kMagic8, -kMagic8);
+        uint64_t accF[2] = {0ull, 0ull}, accI[2] = {0ull, 0ull};             // (S0,S1) and (S2,S3) chains
+        uint32_t fw[2], kb[16];
+#pragma unroll
+        for (int hgrp = 0; hgrp < 2; ++hgrp) {
+            uint64_t X[4], Y[4];
+            float y[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                X[i] = pack2(x[8 * hgrp + 2 * i], x[8 * hgrp + 2 * i + 1]);
+                Y[i] = mul2(X[i], R2);                                       // E1 (step 3)
+                unpack2(Y[i], y[2 * i], y[2 * i + 1]);
+            }
+            uint32_t h[4];
+            fw[hgrp] = e2m1x8_encode_decode(y, h);                           // E2 (step 4) and the code values
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h[i]));
+                const uint64_t E = fma2(pack2(v.x, v.y), ND2, X[i]);         // E3: -(v*d - x); squared below
+                accF[hgrp] = fma2(E, E, accF[hgrp]);
+                uint64_t KZ = fma2(Y[i], CP2, MG2);                          // E4 (step 7): exact product, one rounding
+                if constexpr (CLAMP) {
+                    float k0, k1;
+                    unpack2(KZ, k0, k1);
+                    k0 = fminf(fmaxf(k0, kMagic8 - 7.0f), kMagic8 + 7.0f);
+                    k1 = fminf(fmaxf(k1, kMagic8 - 7.0f), kMagic8 + 7.0f);
+                    KZ = pack2(k0, k1);
+                }
+                const uint64_t KF = add2(KZ, NMG2);                          // k as a float
+                const uint64_t FI = fma2(KF, NDI2, X[i]);                    // E5 (steps 8-9)
+                accI[hgrp] = fma2(FI, FI, accI[hgrp]);
+                float kz0, kz1;
+                unpack2(KZ, kz0, kz1);
+                kb[8 * hgrp + 2 * i] = __float_as_uint(kz0);
+                kb[8 * hgrp + 2 * i + 1] = __float_as_uint(kz1);
+            }
+        }
+        // S1-S2 (step 10).
+        float f0, f1, f2, f3, i0, i1, i2, i3;
+        unpack2(accF[0], f0, f1); unpack2(accF[1], f2, f3);
+        unpack2(accI[0], i0, i1); unpack2(accI[1], i2, i3);
+        const float E_fp = __fadd_rn(__fadd_rn(f0, f1), __fadd_rn(f2, f3));
+        const float E_int = __fadd_rn(__fadd_rn(i0, i1), __fadd_rn(i2, i3));
+        const bool flag = E_int < E_fp;
+        // S3-S4: integer codes by Horner on the raw sums (each holds kMagic8Bits + k), then remove the
+        // constant part and turn offset-binary nibbles (k + 8) into two's complement (xor 8).
+        constexpr uint32_t kConst = kMagic8Bits * 0x11111111u - 0x88888888u;   // sum of (bits - (k+8)) * 16^j
+        uint32_t il = kb[7], ih = kb[15];
+#pragma unroll
+        for (int j = 6; j >= 0; --j) {
+            il = il * 16u + kb[j];
+            ih = ih * 16u + kb[8 + j];
+        }
+        il = (il - kConst) ^ 0x88888888u;
+        ih = (ih - kConst) ^ 0x88888888u;
+        c_lo = flag ? il : fw[0];
+        c_hi = flag ? ih : fw[1];
+        sbyte = sb | (flag ? 0x80u : 0u);
+    }
+}
+
+// Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
+// next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
+template <bool HAS_INT>
+__global__ void __launch_bounds__(256, HAS_INT ? 4 : 5) quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes,
+                                                             uint8_t* __restrict__ scales,
+                                                             const float* __restrict__ alpha_p, int64_t ngroups,
+                                                             float scale_mul) {
+    const float alpha = __ldg(alpha_p);
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= ngroups) return;
+    uint4 v0 = __ldg(in + 2 * g), v1 = __ldg(in + 2 * g + 1);
+    while (true) {
+        const int64_t gn = g + stride;
+        const bool more = gn < ngroups;
+        uint4 n0 = v0, n1 = v1;
+        if (more) { n0 = __ldg(in + 2 * gn); n1 = __ldg(in + 2 * gn + 1); }
+        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+        // G1: group maximum with three-input max.
+        const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
+        const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
+        const float m4 = max3abs(x[12], x[13], x[14]);
+        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
+        // G2-G3 (Eq. 2).
+        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
+        const uint32_t sb = e4m3_encode(t);
+        uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
+        if (sb != 0u) {                                                      // G4
+            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
+            const float r = __frcp_rn(d);
+            if (HAS_INT && (sb - 8u) >= 118u) encode_body4<HAS_INT, true>(x, sb, d, r, sbyte, c_lo, c_hi);
+            else encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
+        }
+        scales[g] = (uint8_t)sbyte;
+        codes[g] = make_uint2(c_lo, c_hi);
+        if (!more) break;
+        v0 = n0; v1 = n1; g = gn;
+    }
+}
+
+}  // namespace absq
