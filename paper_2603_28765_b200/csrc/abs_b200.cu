@@ -18,6 +18,30 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kMaxDevices = 64;
 
+#ifndef ABS_AMAX_UNROLL
+#define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass
+#endif
+#ifndef ABS_AMAX_BPS
+#define ABS_AMAX_BPS 8           // blocks of 256 threads per SM in the amax pass
+#endif
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while the previous
+// kernel of the stream drains; every kernel here calls pdl_wait() before its first global access.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ------------------------------------------------------------------------------------------ amax
 
 // Eq. 1, numerator: grid-wide max |x|.  Each block reduces its share and publishes it with one
@@ -29,17 +53,29 @@ template <bool RHT>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t ngroups,
                                                         uint32_t sign_mask, uint32_t* __restrict__ slot,
                                                         float* __restrict__ result, float denom) {
+    pdl_launch_dependents();
     uint32_t local = 0u;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    pdl_wait();
     if constexpr (!RHT) {
-        // |x| and max on packed bf16 pairs; 8 elements per 128-bit load.
+        // |x| and max on packed bf16 pairs; 8 elements per 128-bit load, ABS_AMAX_UNROLL loads in flight per thread.
         const int64_t nvec = ngroups * 2;
         uint32_t m0 = 0u, m1 = 0u;
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        for (; i + (ABS_AMAX_UNROLL - 1) * stride < nvec; i += ABS_AMAX_UNROLL * stride) {
+            uint4 v[ABS_AMAX_UNROLL];
+#pragma unroll
+            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) v[k] = __ldg(in + i + k * stride);
+#pragma unroll
+            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) {
+                m0 = __vmaxu2(m0, __vmaxu2(v[k].x & 0x7FFF7FFFu, v[k].y & 0x7FFF7FFFu));
+                m1 = __vmaxu2(m1, __vmaxu2(v[k].z & 0x7FFF7FFFu, v[k].w & 0x7FFF7FFFu));
+            }
+        }
+        for (; i < nvec; i += stride) {
             uint4 v = __ldg(in + i);
-            uint32_t a = v.x & 0x7FFF7FFFu, b = v.y & 0x7FFF7FFFu, c = v.z & 0x7FFF7FFFu, d = v.w & 0x7FFF7FFFu;
-            m0 = __vmaxu2(m0, __vmaxu2(a, b));
-            m1 = __vmaxu2(m1, __vmaxu2(c, d));
+            m0 = __vmaxu2(m0, __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu));
+            m1 = __vmaxu2(m1, __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
         }
         uint32_t m = __vmaxu2(m0, m1);
         local = max(m & 0xFFFFu, m >> 16) << 16;   // bf16 bits -> FP32 bits
@@ -88,6 +124,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                                                             uint32_t seed_hi) {
     using F = Fmt<FMT>;
     constexpr int B = F::BITS;
+    pdl_launch_dependents();
+    pdl_wait();
     const float alpha = __ldg(alpha_p);
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));                      // T3
     const float c_pre = F::HAS_INT ? __fdiv_rn(F::M_INT, F::M_FP) : 0.0f;
@@ -198,6 +236,8 @@ __global__ void __launch_bounds__(kThreads) dequantize_kernel(const uint8_t* __r
                                                               void* __restrict__ out) {
     using F = Fmt<FMT>;
     constexpr int B = F::BITS;
+    pdl_launch_dependents();
+    pdl_wait();
     const float alpha = __ldg(alpha_p);
     const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -348,11 +388,13 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
                          float denom, cudaStream_t s) {
     uint32_t* slot = st.ring + 4 * (st.next.fetch_add(1) % ABS_MAX_INFLIGHT);
     const bool rht = o.flags & ABS_F_HADAMARD16;
-    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, 8);
+    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, ABS_AMAX_BPS);
+    cudaError_t e;
     if (rht)
-        amax_kernel<true><<<grid, kThreads, 0, s>>>((const uint4*)in, ngroups, o.had_sign_mask, slot, result, denom);
+        e = launch_pdl(amax_kernel<true>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, result, denom);
     else
-        amax_kernel<false><<<grid, kThreads, 0, s>>>((const uint4*)in, ngroups, o.had_sign_mask, slot, result, denom);
+        e = launch_pdl(amax_kernel<false>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, result, denom);
+    if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
@@ -366,36 +408,67 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
-            const int pgrid = grid_for(st, ngroups, FMT == ABS_FMT_IF4 ? 4 : 64);   // IF4: resident blocks only
-            quantize4_fast_kernel<FMT == ABS_FMT_IF4><<<pgrid, kThreads, 0, s>>>((const uint4*)in, (uint2*)codes,
-                                                                               (uint8_t*)scales, alpha, ngroups, mul);
+            const int pgrid = grid_for(st, ngroups, FMT == ABS_FMT_IF4 ? ABS_FAST_MINB : 64);   // IF4: resident blocks only
+            constexpr bool kInt = FMT == ABS_FMT_IF4;
+            const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+            const bool i32 = ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
+            cudaError_t e;
+#define ABS_LAUNCH_F(IDX, A32)                                                                                       \
+    e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32>, pgrid, kThreads, s, (const uint4*)in, (uint2*)codes,        \
+                   (uint8_t*)scales, alpha, (IDX)ngroups, mul)
+            if (i32 && a32) ABS_LAUNCH_F(int32_t, true);
+            else if (i32) ABS_LAUNCH_F(int32_t, false);
+            else if (a32) ABS_LAUNCH_F(int64_t, true);
+            else ABS_LAUNCH_F(int64_t, false);
+#undef ABS_LAUNCH_F
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
         }
     }
+    cudaError_t eq = cudaSuccess;
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
-    quantize_kernel<FMT, R, S><<<grid, kThreads, 0, s>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales,   \
-                                                         alpha, ngroups, mul, o.had_sign_mask, k0, k1)
+    eq = launch_pdl(quantize_kernel<FMT, R, S>, grid, kThreads, s, (const uint4*)in, (uint8_t*)codes,           \
+                    (uint8_t*)scales, alpha, ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1)
     if (rht && sr) ABS_LAUNCH_Q(true, true);
     else if (rht) ABS_LAUNCH_Q(true, false);
     else if (sr) ABS_LAUNCH_Q(false, true);
     else ABS_LAUNCH_Q(false, false);
 #undef ABS_LAUNCH_Q
     if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
-    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+    return (eq == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
 
 template <int FMT>
 abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
                                    int64_t ngroups, void* out, bool fp32, cudaStream_t s) {
     const int grid = grid_for(st, ngroups, 64);
+    if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
+        if (!fp32) {
+            constexpr bool kInt = FMT == ABS_FMT_IF4;
+            const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
+            const bool i32 = ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
+            cudaError_t e;
+#define ABS_LAUNCH_D(IDX, A32)                                                                                      \
+    e = launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32>, grid, kThreads, s, (const uint2*)codes,                 \
+                   (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out)
+            if (i32 && a32) ABS_LAUNCH_D(int32_t, true);
+            else if (i32) ABS_LAUNCH_D(int32_t, false);
+            else if (a32) ABS_LAUNCH_D(int64_t, true);
+            else ABS_LAUNCH_D(int64_t, false);
+#undef ABS_LAUNCH_D
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    cudaError_t e;
     if (fp32)
-        dequantize_kernel<FMT, true><<<grid, kThreads, 0, s>>>((const uint8_t*)codes, (const uint8_t*)scales, alpha,
-                                                               ngroups, out);
+        e = launch_pdl(dequantize_kernel<FMT, true>, grid, kThreads, s, (const uint8_t*)codes, (const uint8_t*)scales, alpha,
+                       ngroups, out);
     else
-        dequantize_kernel<FMT, false><<<grid, kThreads, 0, s>>>((const uint8_t*)codes, (const uint8_t*)scales, alpha,
-                                                                ngroups, out);
-    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        e = launch_pdl(dequantize_kernel<FMT, false>, grid, kThreads, s, (const uint8_t*)codes, (const uint8_t*)scales, alpha,
+                       ngroups, out);
+    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
 
 abs_status_t check_shape(abs_fmt_t fmt, int64_t rows, int64_t cols) {

@@ -190,7 +190,41 @@ __device__ __forceinline__ void hadamard16(float (&a)[16], uint32_t sign_mask) {
     for (int i = 0; i < 16; ++i) a[i] = __fmul_rn(a[i], 0.25f);
 }
 
-// ----------------------------------------------------------------------------- loads / unpack
+// ----------------------------------------------------------------------------- loads / stores / launch order
+
+// 32 contiguous bytes per thread.  With a 32-byte aligned base one 256-bit access covers a group's
+// bf16 values, so a warp touches 1 KiB of whole sectors per instruction; otherwise two 128-bit ones.
+template <bool ALIGNED32>
+__device__ __forceinline__ void load32B(const void* p, uint32_t (&w)[8]) {
+    if constexpr (ALIGNED32) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                     : "l"(p));
+    } else {
+        const uint4 a = __ldg(reinterpret_cast<const uint4*>(p)), b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+    }
+}
+template <bool ALIGNED32>
+__device__ __forceinline__ void store32B(void* p, const uint32_t (&w)[8]) {
+    if constexpr (ALIGNED32) {
+        asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                     : "memory");
+    } else {
+        reinterpret_cast<uint4*>(p)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4*>(p)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+}
+
+// Programmatic dependent launch: every kernel lets the next kernel of the stream be scheduled
+// early and itself waits for the previous kernel's completion (and memory) before it touches
+// global memory, so only block scheduling and register set-up overlap.  Both are no-ops for a
+// kernel launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------- unpack
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4& v, float* x) {
     x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);

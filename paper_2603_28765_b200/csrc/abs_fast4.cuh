@@ -103,7 +103,7 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
         const float d_int = __fmul_rn(d, c_post);
         const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
         const uint64_t MG2 = pack2(kMagic8, kMagic8), NMG2 = pack2(-kMagic8, -kMagic8);
-        uint64_t accF[2] = {0ull, 0ull}, accI[2] = {0ull, 0ull};             // (S0,S1) and (S2,S3) chains
+        uint64_t accF[2], accI[2];                                           // (S0,S1) and (S2,S3) chains
         uint32_t fw[2], kb[16];
 #pragma unroll
         for (int hgrp = 0; hgrp < 2; ++hgrp) {
@@ -121,7 +121,7 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
             for (int i = 0; i < 4; ++i) {
                 const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h[i]));
                 const uint64_t E = fma2(pack2(v.x, v.y), ND2, X[i]);         // E3: -(v*d - x); squared below
-                accF[hgrp] = fma2(E, E, accF[hgrp]);
+                accF[hgrp] = (i == 0) ? mul2(E, E) : fma2(E, E, accF[hgrp]);   // fma(e, e, 0) == e * e
                 uint64_t KZ = fma2(Y[i], CP2, MG2);                          // E4 (step 7): exact product, one rounding
                 if constexpr (CLAMP) {
                     float k0, k1;
@@ -132,7 +132,7 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
                 }
                 const uint64_t KF = add2(KZ, NMG2);                          // k as a float
                 const uint64_t FI = fma2(KF, NDI2, X[i]);                    // E5 (steps 8-9)
-                accI[hgrp] = fma2(FI, FI, accI[hgrp]);
+                accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
                 float kz0, kz1;
                 unpack2(KZ, kz0, kz1);
                 kb[8 * hgrp + 2 * i] = __float_as_uint(kz0);
@@ -163,25 +163,30 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
     }
 }
 
+#ifndef ABS_FAST_MINB
+#define ABS_FAST_MINB 4          // resident blocks of 256 threads per SM the IF4 instance is compiled for
+#endif
+
 // Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
 // next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
-template <bool HAS_INT>
-__global__ void __launch_bounds__(256, HAS_INT ? 4 : 5) quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes,
-                                                             uint8_t* __restrict__ scales,
-                                                             const float* __restrict__ alpha_p, int64_t ngroups,
-                                                             float scale_mul) {
+// IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
+template <bool HAS_INT, typename IdxT, bool ALIGNED32>
+__global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
+quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
+                      const float* __restrict__ alpha_p, IdxT ngroups, float scale_mul) {
+    pdl_launch_dependents();
+    const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
+    IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x);
+    pdl_wait();
+    if (g >= ngroups) return;
     const float alpha = __ldg(alpha_p);
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= ngroups) return;
-    uint4 v0 = __ldg(in + 2 * g), v1 = __ldg(in + 2 * g + 1);
+    uint32_t w[8], wn[8];
+    load32B<ALIGNED32>(in + 2 * (size_t)g, w);
     while (true) {
-        const int64_t gn = g + stride;
+        const IdxT gn = g + stride;
         const bool more = gn < ngroups;
-        uint4 n0 = v0, n1 = v1;
-        if (more) { n0 = __ldg(in + 2 * gn); n1 = __ldg(in + 2 * gn + 1); }
-        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        if (more) load32B<ALIGNED32>(in + 2 * (size_t)gn, wn);
         float x[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -206,7 +211,93 @@ __global__ void __launch_bounds__(256, HAS_INT ? 4 : 5) quantize4_fast_kernel(co
         scales[g] = (uint8_t)sbyte;
         codes[g] = make_uint2(c_lo, c_hi);
         if (!more) break;
-        v0 = n0; v1 = n1; g = gn;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = wn[i];
+        g = gn;
+    }
+}
+
+
+// ----------------------------------------------------------------------------- 4-bit dequantize
+
+// FP32 -> packed bf16 pair, round to nearest even (Sec. 4.1).
+__device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// FP32 = (one f16 half of h2) + addend, one mixed-precision add (exact for the small values used here).
+__device__ __forceinline__ float half_plus_f32(uint32_t h2, bool upper, float addend) {
+    const uint16_t h = upper ? (uint16_t)(h2 >> 16) : (uint16_t)(h2 & 0xFFFFu);
+    float d;
+    asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(addend));
+    return d;
+}
+
+// Eight 4-bit codes of one word -> eight products value * d, as four packed bf16 pairs.  Branch-free:
+// both decodes are formed as f16 pairs (elements 2j, 2j+1 in register j) and selected per lane.
+//   FP decode: e2m1x2 -> f16x2 per byte; value = half + (-0).
+//   Integer decode: nibble n goes into the mantissa of the f16 constant 1024 as n ^ 8 = k + 8, so the
+//   half is 1032 + k and value = half + (-1032) = k exactly.
+template <bool HAS_INT>
+__device__ __forceinline__ void dequant_word4(uint32_t w, bool is_int, float addend, uint64_t D2, uint32_t (&out)[4]) {
+    uint32_t h[4];
+    asm("{ .reg .b8 a, b, c, d;\n"
+        "  mov.b32 {a, b, c, d}, %4;\n"
+        "  cvt.rn.f16x2.e2m1x2 %0, a;\n"
+        "  cvt.rn.f16x2.e2m1x2 %1, b;\n"
+        "  cvt.rn.f16x2.e2m1x2 %2, c;\n"
+        "  cvt.rn.f16x2.e2m1x2 %3, d; }"
+        : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(w));
+    if constexpr (HAS_INT) {
+        const uint32_t L = w & 0x0F0F0F0Fu, H = (w >> 4) & 0x0F0F0F0Fu;   // even / odd nibbles, one per byte
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            // bytes [L_j, L_j, H_j, H_j] -> keep one nibble per half, set the f16 exponent of 1024, flip bit 3
+            const uint32_t r = (__byte_perm(L, H, 0x4400u + 0x1111u * j) & 0x000F000Fu) ^ 0x64086408u;
+            h[j] = is_int ? r : h[j];
+        }
+    }
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = half_plus_f32(h[j], false, addend);
+        f[2 * j + 1] = half_plus_f32(h[j], true, addend);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float p0, p1;
+        unpack2(mul2(pack2(f[2 * j], f[2 * j + 1]), D2), p0, p1);
+        out[j] = bf16x2_rn(p0, p1);
+    }
+}
+
+template <bool HAS_INT, typename IdxT, bool ALIGNED32>
+__global__ void __launch_bounds__(256) dequantize4_fast_kernel(const uint2* __restrict__ codes,
+                                                               const uint8_t* __restrict__ scales,
+                                                               const float* __restrict__ alpha_p, IdxT ngroups,
+                                                               uint4* __restrict__ out) {
+    pdl_launch_dependents();
+    const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
+    const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
+    pdl_wait();
+    const float alpha = __ldg(alpha_p);
+    for (IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x); g < ngroups; g += stride) {
+        const uint2 c = __ldg(codes + (size_t)g);
+        const uint32_t sbyte = __ldg(scales + (size_t)g);
+        const uint32_t mag = sbyte & 0x7Fu;
+        const bool is_int = HAS_INT && (sbyte & 0x80u);
+        float Delta = e4m3_value(mag);
+        if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
+        float d = __fmul_rn(Delta, alpha);
+        if (is_int) d = __fmul_rn(d, c_post);                          // de-scale integer groups (Sec. 3)
+        const float addend = is_int ? -1032.0f : -0.0f;
+        const uint64_t D2 = pack2(d, d);
+        uint32_t lo[4], hi[4];
+        dequant_word4<HAS_INT>(c.x, is_int, addend, D2, lo);
+        dequant_word4<HAS_INT>(c.y, is_int, addend, D2, hi);
+        const uint32_t o[8] = {lo[0], lo[1], lo[2], lo[3], hi[0], hi[1], hi[2], hi[3]};
+        store32B<ALIGNED32>(out + 2 * (size_t)g, o);
     }
 }
 
