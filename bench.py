@@ -42,8 +42,9 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the group-quantize kernel per element, from the ncu capture summarised in
-# profiles/quantize_if4_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum per launch / N).
-NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = None
+# profiles/quantize4_fast_if4_cfg2.md: (dram__bytes_read.sum + dram__bytes_write.sum) per launch / N
+# = (67.12 MB + 3.82 MB) / 33 554 432 elements, captured on this same workload.
+NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = 70.94e6 / 33554432
 
 
 def step_bytes(n_elems: int) -> float:
@@ -294,7 +295,7 @@ def run_cuda(args):
     q_ms = sum(quant_ms) / len(quant_ms)
     peak, peak_src = measured_peak()
     achieved = quant_kernel_bytes(n) / (q_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "quantize_kernel<IF4> (group-quantize, Fig. 3a steps 1-10)",
+    roofline = {"bound": "hbm", "kernel": "quantize4_fast_kernel<IF4> (group-quantize, Fig. 3a steps 1-10)",
                 "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "peak_source": peak_src, "us_per_launch": round(q_ms * 1e3, 2),
                 "algorithmic_bytes_per_launch": quant_kernel_bytes(n),
