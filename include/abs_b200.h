@@ -102,6 +102,33 @@ ABS_API abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t ro
 ABS_API abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                              void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream);
 
+/* Quantize without any allocation.  (The paper has no counterpart: this entry point exists for the
+ * way the library is deployed, not for the method.)
+ *
+ * abs_quantize keeps its amax scratch in device memory that it obtains with cudaMalloc the first time
+ * it runs on a device.  Some callers cannot afford that: a serving process that has already handed
+ * every free byte of device memory to its own pool, so that a later cudaMalloc simply fails; or a
+ * latency-critical loop that must not run into the device-wide synchronisation cudaMalloc implies.
+ * For them this variant computes exactly the same outputs as abs_quantize(fmt, ...) with round to
+ * nearest and no options, but its amax pass reduces the tensor in chunks of 131072 elements whose
+ * partial maxima go to an array that is part of the library image (33 KiB on every GPU that loads
+ * the library, held until the process exits).  It calls no cudaMalloc, cudaFree or other allocating
+ * routine, and it allocates nothing through any framework.
+ *
+ *   - Limit: at most ABS_NOALLOC_MAX_ELEMS = 8192 chunks x 131072 = 1 073 741 824 elements; a larger
+ *     rows*cols returns ABS_ERR_SIZE and enqueues nothing.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current); make that first call before any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the ticket word it needs at zero
+ *     itself (a 4-byte cudaMemsetAsync on `stream`) and overwrites every partial maximum it reads, so
+ *     stale contents from earlier calls are harmless; but two calls that overlap on the GPU (different
+ *     streams, or graphs replayed concurrently) race on the array and produce wrong scales.  Serialise
+ *     them, or use abs_quantize on one of the streams.
+ * Arguments, layouts, alignment rules and the other status codes are those of abs_quantize. */
+#define ABS_NOALLOC_MAX_ELEMS ((int64_t)8192 * 8192 * 16)
+ABS_API abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
+                                          void* codes_u8, void* scales_e4m3, float* tensor_scale_f32, void* stream);
+
 /* Dequantize (Sec. 3: de-scale integer groups by M_FP/M_INT; Sec. 4.1: product in FP32, then
  * bf16 round-to-nearest-even).  out is bf16 [rows, cols], or float with ABS_F_OUT_FP32 (the only
  * flag accepted).  The Hadamard option is not inverted here. */

@@ -28,6 +28,7 @@ EXPORTS = [
     "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
+    "abs_quantize_noalloc",
 ]
 
 
@@ -72,6 +73,8 @@ def lib():
             L.abs_quantize.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
             L.abs_quantize_ex.restype = C.c_int
             L.abs_quantize_ex.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
+            L.abs_quantize_noalloc.restype = C.c_int
+            L.abs_quantize_noalloc.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
             L.abs_dequantize.restype = C.c_int
             L.abs_dequantize.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, vp]
             L.abs_dequantize_ex.restype = C.c_int
@@ -150,6 +153,19 @@ def abs_quantize(fmt: int, x, codes=None, scales=None, tensor_scale=None, opts: 
                                tensor_scale.data_ptr(), C.byref(opts) if opts is not None else None,
                                _stream_ptr(stream))
     _check(rc, "abs_quantize")
+    return codes, scales, tensor_scale
+
+
+def abs_quantize_noalloc(fmt: int, x, codes, scales, tensor_scale, stream=None):
+    """Quantize with the variant of the library that allocates nothing (see ``abs_quantize_noalloc`` in
+    the header): for processes that cannot call cudaMalloc any more.  All buffers come from the caller,
+    so nothing is allocated here either; at most 2**30 elements; do not overlap two calls on one GPU."""
+    import torch
+    rows, cols = x.shape
+    with torch.cuda.device(x.device):
+        rc = lib().abs_quantize_noalloc(fmt, x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(),
+                                        tensor_scale.data_ptr(), _stream_ptr(stream))
+    _check(rc, "abs_quantize_noalloc")
     return codes, scales, tensor_scale
 
 

@@ -471,6 +471,73 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
 
+
+// ------------------------------------------------------------------------------------------ no-allocation variant
+
+// Scratch of abs_quantize_noalloc: one partial maximum per block of the chunked amax pass plus, in
+// the last 64 words, the ticket counter.  It lives in the library image, so every GPU that loads the
+// library holds these 33 KiB until the process exits; nothing is ever allocated for it.
+#define ABS_NOALLOC_MAX_CHUNKS 8192          /* partial maxima the array can hold                 */
+#define ABS_NOALLOC_CHUNK_GROUPS 8192        /* groups of 16 elements reduced by one block        */
+static __device__ __align__(256) uint32_t g_noalloc_scratch[ABS_NOALLOC_MAX_CHUNKS + 64];
+
+// Eq. 1 without atomics on the maximum: block b reduces chunk b and stores its partial maximum in
+// scratch[b]; the block that draws the last ticket reduces the partials, writes alpha and sets the
+// ticket back to zero.  `scratch` is the device address of g_noalloc_scratch obtained on the host
+// with cudaGetSymbolAddress (the array's name is not a device address in host code).
+__global__ void __launch_bounds__(kThreads) amax_chunks_kernel(const uint4* __restrict__ in, int64_t ngroups,
+                                                               uint32_t* __restrict__ scratch,
+                                                               float* __restrict__ result, float denom) {
+    const int64_t first = (int64_t)blockIdx.x * ABS_NOALLOC_CHUNK_GROUPS * 2;       // in 128-bit vectors
+    int64_t last = first + (int64_t)ABS_NOALLOC_CHUNK_GROUPS * 2;
+    if (last > ngroups * 2) last = ngroups * 2;
+    uint32_t m0 = 0u, m1 = 0u;
+    for (int64_t i = first + threadIdx.x; i < last; i += kThreads) {
+        const uint4 v = __ldg(in + i);
+        m0 = __vmaxu2(m0, __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu));
+        m1 = __vmaxu2(m1, __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
+    }
+    const uint32_t m = __vmaxu2(m0, m1);
+    uint32_t local = __reduce_max_sync(0xFFFFFFFFu, max(m & 0xFFFFu, m >> 16) << 16);
+    __shared__ uint32_t warp_max[kThreads / 32];
+    __shared__ bool is_last;
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t bm = 0u;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) bm = max(bm, warp_max[w]);
+        scratch[blockIdx.x] = bm;
+        __threadfence();
+        is_last = atomicAdd(&scratch[ABS_NOALLOC_MAX_CHUNKS], 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    uint32_t all = 0u;
+    for (uint32_t b = threadIdx.x; b < gridDim.x; b += kThreads) all = max(all, __ldcg(scratch + b));
+    all = __reduce_max_sync(0xFFFFFFFFu, all);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = all;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t bm = 0u;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) bm = max(bm, warp_max[w]);
+        const float A = __uint_as_float(bm);
+        *result = (A == 0.0f) ? 1.0f : __fdiv_rn(A, denom);                          // Eq. 1
+        scratch[ABS_NOALLOC_MAX_CHUNKS] = 0u;
+    }
+}
+
+struct NoAllocState {
+    std::once_flag once;
+    cudaError_t err = cudaSuccess;
+    uint32_t* scratch = nullptr;     // device address of g_noalloc_scratch on this device
+    int sm_count = 148;
+};
+NoAllocState g_noalloc[kMaxDevices];
+
 abs_status_t check_shape(abs_fmt_t fmt, int64_t rows, int64_t cols) {
     if (fmt_bits((int)fmt) == 0) return ABS_ERR_FMT;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return ABS_ERR_SHAPE;
@@ -576,6 +643,48 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
 abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                           void* scales_e4m3, float* tensor_scale_f32, void* stream) {
     return abs_quantize_ex(fmt, in_bf16, rows, cols, codes_u8, scales_e4m3, tensor_scale_f32, nullptr, stream);
+}
+
+
+abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
+                                  void* scales_e4m3, float* tensor_scale_f32, void* stream) {
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if (rows * cols == 0) return ABS_OK;
+    if (!in_bf16 || !codes_u8 || !scales_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
+    if (!aligned16(in_bf16) || !aligned16(codes_u8) || !aligned16(scales_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
+        return ABS_ERR_ALIGN;
+    const int64_t ngroups = rows * cols / 16;
+    const int64_t nchunks = (ngroups + ABS_NOALLOC_CHUNK_GROUPS - 1) / ABS_NOALLOC_CHUNK_GROUPS;
+    if (nchunks > ABS_NOALLOC_MAX_CHUNKS) return ABS_ERR_SIZE;      // more partial maxima than the static array holds
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ABS_ERR_CUDA;
+    NoAllocState& na = g_noalloc[dev];
+    std::call_once(na.once, [&]() {
+        // The current device is `dev`: the address returned is the array's copy on this device.
+        na.err = cudaGetSymbolAddress((void**)&na.scratch, g_noalloc_scratch);
+        int sms = 0;
+        if (na.err == cudaSuccess) na.err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms > 0) na.sm_count = sms;
+    });
+    if (na.err != cudaSuccess || na.scratch == nullptr) return ABS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    // The array keeps whatever the last call left: the ticket must start at zero; the partial maxima
+    // need no clearing because every block overwrites its own slot before it draws a ticket.
+    if (cudaMemsetAsync(na.scratch + ABS_NOALLOC_MAX_CHUNKS, 0, sizeof(uint32_t), s) != cudaSuccess) return ABS_ERR_CUDA;
+    amax_chunks_kernel<<<(int)nchunks, kThreads, 0, s>>>((const uint4*)in_bf16, ngroups, na.scratch, tensor_scale_f32,
+                                                        fmt_mfp((int)fmt) * 448.0f);
+    if (cudaGetLastError() != cudaSuccess) return ABS_ERR_CUDA;
+    DeviceState grid_info;                 // only its SM count is read by the launchers; no ring is touched
+    grid_info.sm_count = na.sm_count;
+    const abs_opts_t o = {0, 0, 0, 0};
+    switch (fmt) {
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        default: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+    }
 }
 
 abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
