@@ -16,7 +16,6 @@ __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
 __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
-#ifndef ABS_SCALAR_F32
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
     uint64_t d;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
@@ -32,20 +31,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-#else   // timing experiment only: the same arithmetic with scalar instructions
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    float a0, a1, b0, b1, c0, c1; unpack2(a, a0, a1); unpack2(b, b0, b1); unpack2(c, c0, c1);
-    return pack2(__fmaf_rn(a0, b0, c0), __fmaf_rn(a1, b1, c1));
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    float a0, a1, b0, b1; unpack2(a, a0, a1); unpack2(b, b0, b1);
-    return pack2(__fmul_rn(a0, b0), __fmul_rn(a1, b1));
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    float a0, a1, b0, b1; unpack2(a, a0, a1); unpack2(b, b0, b1);
-    return pack2(__fadd_rn(a0, b0), __fadd_rn(a1, b1));
-}
-#endif
 __device__ __forceinline__ float max3abs(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(fabsf(a)), "f"(fabsf(b)), "f"(fabsf(c)));
@@ -131,24 +116,12 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
                 unpack2(Y[i], y[2 * i], y[2 * i + 1]);
             }
             uint32_t h[4];
-#ifndef ABL_NO_FPDEC
             fw[hgrp] = e2m1x8_encode_decode(y, h);                           // E2 (step 4) and the code values
-#else
-            fw[hgrp] = e2m1x8_encode(y); h[0] = h[1] = h[2] = h[3] = fw[hgrp];
-#endif
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-#ifndef ABL_NO_FPERR
-#ifndef ABL_NO_FPDEC
                 const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h[i]));
-#else
-                const float2 v = make_float2(__uint_as_float(h[i]), y[2 * i]);
-#endif
                 const uint64_t E = fma2(pack2(v.x, v.y), ND2, X[i]);         // E3: -(v*d - x); squared below
                 accF[hgrp] = (i == 0) ? mul2(E, E) : fma2(E, E, accF[hgrp]);   // fma(e, e, 0) == e * e
-#else
-                accF[hgrp] = X[i];
-#endif
                 uint64_t KZ = fma2(Y[i], CP2, MG2);                          // E4 (step 7): exact product, one rounding
                 if constexpr (CLAMP) {
                     float k0, k1;
@@ -157,13 +130,9 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
                     k1 = fminf(fmaxf(k1, kMagic8 - 7.0f), kMagic8 + 7.0f);
                     KZ = pack2(k0, k1);
                 }
-#ifndef ABL_NO_INTERR
                 const uint64_t KF = add2(KZ, NMG2);                          // k as a float
                 const uint64_t FI = fma2(KF, NDI2, X[i]);                    // E5 (steps 8-9)
                 accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
-#else
-                accI[hgrp] = KZ;
-#endif
                 float kz0, kz1;
                 unpack2(KZ, kz0, kz1);
                 kb[8 * hgrp + 2 * i] = __float_as_uint(kz0);
@@ -181,15 +150,11 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
         // constant part and turn offset-binary nibbles (k + 8) into two's complement (xor 8).
         constexpr uint32_t kConst = kMagic8Bits * 0x11111111u - 0x88888888u;   // sum of (bits - (k+8)) * 16^j
         uint32_t il = kb[7], ih = kb[15];
-#ifndef ABL_NO_HORNER
 #pragma unroll
         for (int j = 6; j >= 0; --j) {
             il = il * 16u + kb[j];
             ih = ih * 16u + kb[8 + j];
         }
-#else
-        il ^= kb[0] ^ kb[3]; ih ^= kb[8] ^ kb[12];
-#endif
         il = (il - kConst) ^ 0x88888888u;
         ih = (ih - kConst) ^ 0x88888888u;
         c_lo = flag ? il : fw[0];
@@ -232,11 +197,7 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
         const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
         const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
         const float m4 = max3abs(x[12], x[13], x[14]);
-#ifndef ABL_NO_MAX
         const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
-#else
-        const float gmax = fabsf(x[0]) + fabsf(x[9]);
-#endif
         // G2-G3 (Eq. 2).
         const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
         const uint32_t sb = e4m3_encode(t);
@@ -247,12 +208,8 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
             if (HAS_INT && (sb - 8u) >= 118u) encode_body4<HAS_INT, true>(x, sb, d, r, sbyte, c_lo, c_hi);
             else encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
         }
-#ifndef ABL_NO_STORE
         scales[g] = (uint8_t)sbyte;
         codes[g] = make_uint2(c_lo, c_hi);
-#else
-        if (sbyte == 0x12345u) { scales[g] = (uint8_t)sbyte; codes[g] = make_uint2(c_lo, c_hi); }
-#endif
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
