@@ -1,0 +1,92 @@
+"""Per-configuration throughput table of the library's kernels (run on a B200 machine).
+
+    python -m paper_2603_28765_b200.report [--quick]
+
+For every benchmark configuration and format it times, with CUDA events over back-to-back calls
+that rotate over enough buffer sets to defeat L2 reuse between calls:
+  T1  the group-quantize kernel alone (alpha given)          bytes = 2N + codes + scales
+  T2  abs_quantize end to end (amax pass + group-quantize)   bytes = 4N + codes + scales (DRAM basis)
+  T3  abs_dequantize                                         bytes = codes + scales + 2N
+and prints one JSON line per row.  Inputs are random bf16 tensors of the configuration's shape
+(timing does not depend on the values beyond the INT/FP mix); parity is the test suite's job.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes as C
+import json
+
+
+def main():
+    import torch
+    from . import binding as B
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true", help="fewer repetitions")
+    args = ap.parse_args()
+    L = B.lib()
+    reps = 10 if args.quick else 40
+
+    def loop_time(fn, n=reps, warm=3):
+        for i in range(warm):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    H, S, S17 = B.ABS_F_HADAMARD16, B.ABS_F_STOCHASTIC, B.ABS_F_SR_SCALE_17_16
+    rows_cfg = [
+        ("cfg2", 8192, 4096, [("if4", 0)]),
+        ("cfg3a", 4096, 14336, [("if4", 0), ("nvfp4", 0)]),
+        ("cfg3b", 14336, 4096, [("if4", 0), ("nvfp4", 0)]),
+        ("cfg4", 16384, 8192, [("if4", H | S | S17), ("if4", H | S), ("if4", S), ("if4", H), ("nvfp4", H | S | S17)]),
+        ("cfg5", 16384, 8192, [("if3", 0), ("if4", 0), ("if6_e2m3", 0), ("if6_e3m2", 0), ("nvfp4", 0)]),
+    ]
+    sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    for name, rows, cols, variants in rows_cfg:
+        n = rows * cols
+        k = max(4, int(1.0e9 // (n * 2)))
+        xs = [(torch.randn(rows, cols, device="cuda") * (1 + 3 * torch.rand(rows, 1, device="cuda"))).to(torch.bfloat16)
+              for _ in range(k)]
+        for fname, flags in variants:
+            fmt = B.FMT_NAMES[fname]
+            bits = B.FMT_BITS[fmt]
+            codes = [torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda") for _ in range(k)]
+            scales = [torch.empty(n // 16, dtype=torch.uint8, device="cuda") for _ in range(k)]
+            ts = [torch.zeros(1, dtype=torch.float32, device="cuda") for _ in range(k)]
+            outs = [torch.empty(rows, cols, dtype=torch.bfloat16, device="cuda") for _ in range(min(k, 4))]
+            o_full = B.make_opts(flags, 0x5A3C, 1234)
+            o_given = B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, 0x5A3C, 1234)
+            for i in range(k):
+                B.abs_quantize(fmt, xs[i], codes[i], scales[i], ts[i], opts=o_full)
+            torch.cuda.synchronize()
+            qa = [(fmt, xs[i].data_ptr(), rows, cols, codes[i].data_ptr(), scales[i].data_ptr(), ts[i].data_ptr(),
+                   C.byref(o_given), sp) for i in range(k)]
+            fa = [(fmt, xs[i].data_ptr(), rows, cols, codes[i].data_ptr(), scales[i].data_ptr(), ts[i].data_ptr(),
+                   C.byref(o_full), sp) for i in range(k)]
+            da = [(fmt, codes[i].data_ptr(), scales[i].data_ptr(), ts[i].data_ptr(), rows, cols,
+                   outs[i % len(outs)].data_ptr(), sp) for i in range(k)]
+            t1 = loop_time(lambda i: L.abs_quantize_ex(*qa[i % k]))
+            t2 = loop_time(lambda i: L.abs_quantize_ex(*fa[i % k]))
+            t3 = loop_time(lambda i: L.abs_dequantize(*da[i % k]))
+            outb = n * bits / 8 + n / 16
+            opt = "+".join(s for s, f in (("hadamard", H), ("sr", S), ("17/16", S17)) if flags & f) or "rtn"
+            print(json.dumps({
+                "config": name, "shape": [rows, cols], "fmt": fname, "options": opt,
+                "T1_quantize_kernel_us": round(t1 * 1e3, 1), "T1_GBs": round((2 * n + outb) / t1 / 1e6),
+                "T2_abs_quantize_us": round(t2 * 1e3, 1), "T2_dram_basis_GBs": round((4 * n + outb) / t2 / 1e6),
+                "T2_effective_GBs": round((2 * n + outb) / t2 / 1e6),
+                "T3_dequantize_us": round(t3 * 1e3, 1), "T3_GBs": round((2 * n + outb) / t3 / 1e6),
+                "elements_per_s_T2": round(n / (t2 * 1e-3)),
+            }), flush=True)
+            del codes, scales, outs
+        del xs
+
+
+if __name__ == "__main__":
+    main()
