@@ -18,9 +18,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kMaxDevices = 64;
 
-#ifndef ABS_Q4_KERNEL
-#define ABS_Q4_KERNEL quantize4_fast_kernel   // the 4-bit group-quantize kernel
-#endif
 #ifndef ABS_AMAX_UNROLL
 #define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass
 #endif
@@ -417,7 +414,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             const bool i32 = ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
             cudaError_t e;
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
-    e = launch_pdl(ABS_Q4_KERNEL<kInt, IDX, A32>, pgrid, kThreads, s, (const uint4*)in, (uint2*)codes,                \
+    e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32>, pgrid, kThreads, s, (const uint4*)in, (uint2*)codes,        \
                    (uint8_t*)scales, alpha, (IDX)ngroups, mul)
             if (i32 && a32) ABS_LAUNCH_F(int32_t, true);
             else if (i32) ABS_LAUNCH_F(int32_t, false);
