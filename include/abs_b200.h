@@ -69,7 +69,9 @@ enum {
     ABS_F_SR_SCALE_17_16 = 1u << 2, /* quantize: group scale target times 17/16 before E4M3 rounding,
                                        the 16/17 factor of Sec. 4.1, so stochastic values never clip     */
     ABS_F_ALPHA_GIVEN = 1u << 3,    /* quantize: *tensor_scale_f32 is an input; the amax pass is skipped */
-    ABS_F_OUT_FP32 = 1u << 4        /* dequantize: write the FP32 products instead of bf16               */
+    ABS_F_OUT_FP32 = 1u << 4,       /* dequantize: write the FP32 products instead of bf16               */
+    ABS_F_INDEX64 = 1u << 5         /* testing aid: run the kernel instances that index groups with 64-bit
+                                       integers (otherwise chosen only beyond 2^31 groups); same results  */
 };
 
 #define ABS_MAX_INFLIGHT 1024

@@ -21,6 +21,7 @@ ABS_F_STOCHASTIC = 1 << 1
 ABS_F_SR_SCALE_17_16 = 1 << 2
 ABS_F_ALPHA_GIVEN = 1 << 3
 ABS_F_OUT_FP32 = 1 << 4
+ABS_F_INDEX64 = 1 << 5
 
 ABS_OK = 0
 

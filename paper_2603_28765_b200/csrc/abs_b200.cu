@@ -376,7 +376,8 @@ float fmt_mfp(int fmt) {
     }
 }
 
-constexpr uint32_t kQuantFlags = ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN;
+constexpr uint32_t kQuantFlags =
+    ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN | ABS_F_INDEX64;
 
 int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
     int64_t want = (work_items + kThreads - 1) / kThreads;
@@ -411,7 +412,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             const int pgrid = grid_for(st, ngroups, FMT == ABS_FMT_IF4 ? ABS_FAST_MINB : 64);   // IF4: resident blocks only
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
-            const bool i32 = ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
+            const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
             cudaError_t e;
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
     e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32>, pgrid, kThreads, s, (const uint4*)in, (uint2*)codes,        \
@@ -441,13 +442,13 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 
 template <int FMT>
 abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
-                                   int64_t ngroups, void* out, bool fp32, cudaStream_t s) {
+                                   int64_t ngroups, void* out, bool fp32, bool index64, cudaStream_t s) {
     const int grid = grid_for(st, ngroups, 64);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
-            const bool i32 = ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
+            const bool i32 = !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
             cudaError_t e;
 #define ABS_LAUNCH_D(IDX, A32)                                                                                      \
     e = launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32>, grid, kThreads, s, (const uint2*)codes,                 \
@@ -694,7 +695,7 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
-    if ((o.flags & ~(uint32_t)ABS_F_OUT_FP32) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ~(uint32_t)(ABS_F_OUT_FP32 | ABS_F_INDEX64)) || o._pad) return ABS_ERR_FLAGS;
     if (rows * cols == 0) return ABS_OK;
     if (!codes_u8 || !scales_e4m3 || !tensor_scale_f32 || !out) return ABS_ERR_NULL;
     if (!aligned16(codes_u8) || !aligned16(scales_e4m3) || !aligned16(out) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -703,13 +704,13 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
-    const bool fp32 = o.flags & ABS_F_OUT_FP32;
+    const bool fp32 = o.flags & ABS_F_OUT_FP32, i64 = o.flags & ABS_F_INDEX64;
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
-        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
-        case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
-        case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
-        default: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, s);
+        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        default: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
     }
 }
 

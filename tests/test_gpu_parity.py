@@ -198,6 +198,93 @@ def test_alpha_given_and_worked_example(B, oracle, fmt):
         assert c[0].tobytes() == bytes([0x31, 0x76, 0, 0, 0, 0, 0, 0]) and s[0, 0] == 0xFE and a == np.float32(2 ** -6)
 
 
+def test_index64_kernel_instances(B, oracle):
+    """The 64-bit-index instances (normally chosen beyond 2^31 groups) give the same bytes."""
+    xb = I.generate("cfg2", 130, 2048)
+    for fmt in (0, 1):
+        check_case(B, oracle, fmt, xb, flags=B.ABS_F_INDEX64, dequant=False)
+        c, s, a, dev = gpu_quantize(B, fmt, xb)
+        out = B.abs_dequantize(fmt, dev[0], dev[1], dev[2], *xb.shape, opts=B.make_opts(B.ABS_F_INDEX64))
+        want = oracle.dequantize(fmt, c, s, a, *xb.shape)
+        assert_same("dequant", out.view(torch.int16).cpu().numpy().view(np.uint16), want)
+    # an input that is only 16-byte aligned takes the two-128-bit-access path
+    buf = torch.zeros(130 * 2048 + 8, dtype=torch.bfloat16, device="cuda")
+    x = buf[8:].view(130, 2048)
+    x.copy_(to_dev(xb))
+    assert x.data_ptr() % 32 == 16
+    codes, scales, ts = B.abs_quantize(1, x)
+    oc, osc, oa = oracle.quantize(1, xb)
+    assert_same("codes", codes.cpu().numpy().reshape(130, -1), oc)
+    assert_same("scales", scales.cpu().numpy().reshape(130, -1), osc)
+    obuf = torch.zeros(130 * 2048 + 8, dtype=torch.bfloat16, device="cuda")
+    out = B.abs_dequantize(1, codes, scales, ts, 130, 2048, out=obuf[8:].view(130, 2048))
+    assert_same("dequant", out.view(torch.int16).cpu().numpy().view(np.uint16), oracle.dequantize(1, oc, osc, oa, 130, 2048))
+
+
+def test_large_tensor_sampled_parity(B, oracle):
+    """2.6e9 elements (5.2 GB of bf16: byte offsets and element indices beyond 2^32 / 2^31), in the
+    launch configuration the library picks itself.  alpha is checked against torch's max; 48 sampled
+    rows plus the first and last are compared with the oracle byte for byte (quantize with the
+    stochastic option too, whose random stream is indexed by the element position)."""
+    rows, cols = 40000, 65536
+    g = torch.Generator(device="cuda").manual_seed(11)
+    block = torch.randn(500, cols, device="cuda", generator=g)
+    x = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    for r0 in range(0, rows, 500):
+        scale = 0.25 + 4 * torch.rand(500, 1, device="cuda", generator=g)
+        x[r0:r0 + 500] = (block * scale).to(torch.bfloat16)
+    x[rows - 3, cols - 5] = 77.0                                  # the maximum sits near the end
+    del block
+    amax = float(x.abs().max().float().item())
+    pick = sorted(set([0, rows - 1, rows - 3] + [int(v) for v in np.random.default_rng(3).integers(0, rows, 48)]))
+    xs = x[pick].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    for fmt, flags in ((1, 0), (1, B.ABS_F_STOCHASTIC), (0, 0)):
+        codes, scales, ts = B.abs_quantize(fmt, x, opts=B.make_opts(flags, 0, 99))
+        torch.cuda.synchronize()
+        alpha = oracle.alpha_from_amax(fmt, np.float32(amax))
+        assert np.float32(ts.item()).view(np.uint32) == np.float32(alpha).view(np.uint32)
+        cg = codes.view(rows, cols // 2)[pick].cpu().numpy()
+        sg = scales.view(rows, cols // 16)[pick].cpu().numpy()
+        for i, r in enumerate(pick):
+            if flags & B.ABS_F_STOCHASTIC:
+                # the oracle indexes the random stream by row * cols + col: give it the row offset by
+                # quantizing a tensor view that starts at row r (rows before it are never touched)
+                oc, osc = oracle_rows_with_offset(oracle, fmt, xs[i:i + 1], r, cols, alpha, flags, 99)
+            else:
+                oc, osc, _ = oracle.quantize(fmt, xs[i:i + 1], flags=B.ABS_F_ALPHA_GIVEN, alpha=alpha)
+            assert_same(f"codes row {r}", cg[i:i + 1], oc)
+            assert_same(f"scales row {r}", sg[i:i + 1], osc)
+        if flags == 0:
+            out = B.abs_dequantize(fmt, codes, scales, ts, rows, cols)
+            og = out[pick].view(torch.int16).cpu().numpy().view(np.uint16)
+            for i, r in enumerate(pick):
+                oc, osc, _ = oracle.quantize(fmt, xs[i:i + 1], flags=B.ABS_F_ALPHA_GIVEN, alpha=alpha)
+                assert_same(f"dequant row {r}", og[i:i + 1], oracle.dequantize(fmt, oc, osc, alpha, 1, cols))
+            del out
+        del codes, scales
+
+
+def oracle_rows_with_offset(oracle, fmt, row_bits, row_index, cols, alpha, flags, seed):
+    """Oracle result for one row that sits at `row_index` of a larger tensor (matters only for the
+    element index of the stochastic stream): calls the row-range entry point on a fake base pointer."""
+    import ctypes as C
+    L = oracle.lib()
+    b = oracle.fmt_bits(fmt)
+    codes = np.zeros((1, cols * b // 8), dtype=np.uint8)
+    scales = np.zeros((1, cols // 16), dtype=np.uint8)
+    row = np.ascontiguousarray(row_bits)
+    row_index = int(row_index)
+    # base pointers are shifted back by row_index rows so that row `row_index` lands on our buffers
+    in_base = row.ctypes.data - row_index * cols * 2
+    c_base = codes.ctypes.data - row_index * (cols * b // 8)
+    s_base = scales.ctypes.data - row_index * (cols // 16)
+    rc = L.abs_oracle_quantize_rows(fmt, C.c_void_p(in_base), row_index + 1, cols, row_index, row_index + 1,
+                                    C.c_float(float(alpha)), flags | oracle.F_ALPHA_GIVEN, 0, seed,
+                                    C.c_void_p(c_base), C.c_void_p(s_base), None, None)
+    assert rc == 0
+    return codes, scales
+
+
 def test_amax_entry_point(B, oracle):
     xb = I.generate("cfg2", 123, 2048)
     mask = 0x5A3C
