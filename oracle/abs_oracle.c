@@ -217,6 +217,16 @@ static void unpack_codes(const uint8_t* in, int b, uint32_t code[16]) {
     }
 }
 
+/* E4 (step 7), round-to-nearest path: integer candidate of y.  int(.) rounds the real product
+ * y * M_INT/M_FP once: the product of two floats is exact in double, then nearest integer with
+ * ties to even, clamped to +-M_INT. */
+static float int_candidate_rne(float y, float c_pre, float m_int) {
+    float kf = (float)nearbyint((double)y * (double)c_pre);
+    if (kf > m_int) kf = m_int;
+    if (kf < -m_int) kf = -m_int;
+    return kf;
+}
+
 /* ------------------------------------------------------------------ exported element-level pieces */
 
 ORACLE_API int abs_oracle_fmt_bits(int fmt) { return (fmt >= 0 && fmt < FMT_COUNT) ? FMTS[fmt].bits : -1; }
@@ -241,6 +251,12 @@ ORACLE_API uint32_t abs_oracle_fp_encode(int fmt, float y) {
     int n = build_fp_grid(F, g);
     uint32_t sign = f32_to_bits(y) >> 31;
     return (sign << (F->bits - 1)) | (uint32_t)grid_round_rne(g, n, fabsf(y));
+}
+
+/* Step 7: integer candidate k of a scaled value y (round-to-nearest path). */
+ORACLE_API int abs_oracle_int_encode(int fmt, float y) {
+    const fmt_desc* F = &FMTS[fmt];
+    return (int)int_candidate_rne(y, F->m_int / F->m_fp, F->m_int);
 }
 
 /* Step 2: E4M3 byte (0x00..0x7E) nearest to t >= 0, ties to even, saturating at 448. */
@@ -365,11 +381,7 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
                     kf = (float)grid_round_sr(intg, m_int + 1, fabsf(z), u);
                     if (f32_to_bits(z) >> 31) kf = -kf;
                 } else {
-                    /* int(.) of step 7 rounds the real product y * M_INT/M_FP once: the product of
-                     * two floats is exact in double, then nearest-integer, ties to even. */
-                    kf = (float)nearbyint((double)y * (double)c_pre);
-                    if (kf > F->m_int) kf = F->m_int;
-                    if (kf < -F->m_int) kf = -F->m_int;
+                    kf = int_candidate_rne(y, c_pre, F->m_int);
                 }
                 const int k = (int)kf;
                 q_int[i] = (uint32_t)k & ((1u << b) - 1u);   /* two's complement in b bits */

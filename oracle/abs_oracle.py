@@ -60,6 +60,8 @@ def lib():
             L.abs_oracle_fp_value.argtypes = [C.c_int, C.c_uint32]
             L.abs_oracle_fp_encode.restype = C.c_uint32
             L.abs_oracle_fp_encode.argtypes = [C.c_int, C.c_float]
+            L.abs_oracle_int_encode.restype = C.c_int
+            L.abs_oracle_int_encode.argtypes = [C.c_int, C.c_float]
             L.abs_oracle_e4m3_encode.restype = C.c_uint32
             L.abs_oracle_e4m3_encode.argtypes = [C.c_float]
             L.abs_oracle_e4m3_value.restype = C.c_float
@@ -123,6 +125,10 @@ def fp_value(fmt: int, code: int) -> np.float32:
 
 def fp_encode(fmt: int, y) -> int:
     return int(lib().abs_oracle_fp_encode(fmt, C.c_float(float(np.float32(y)))))
+
+
+def int_encode(fmt: int, y) -> int:
+    return int(lib().abs_oracle_int_encode(fmt, C.c_float(float(np.float32(y)))))
 
 
 def e4m3_encode(t) -> int:

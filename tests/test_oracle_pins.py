@@ -166,6 +166,40 @@ def test_fp_encode_nearest_ties_even_saturating(oracle, fmt):
         assert (code >> (oracle.fmt_bits(fmt) - 1)) == int(np.signbit(y))
 
 
+@pytest.mark.parametrize("fmt", IF_FMTS)
+def test_int_candidate_rounds_the_exact_product_once(oracle, fmt):
+    """Step 7: k = nearest integer (ties to even) of the real product y * fp32(M_INT/M_FP), clamped.
+    Checked in exact rational arithmetic on every bf16 y in range, on random float32 y, and on values
+    built to sit next to a half-integer product."""
+    from fractions import Fraction
+    c = Fraction(float(oracle.c_pre(fmt)))
+    top = int(oracle.m_int(fmt))
+    mfp = float(oracle.m_fp(fmt))
+
+    def exact(y):
+        p = Fraction(float(y)) * c
+        k = int(p.numerator // p.denominator)          # floor
+        frac = p - k
+        if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and k % 2 == 1):
+            k += 1
+        return max(-top, min(top, k))
+
+    ys = [v for v in I.bf16_bits_to_f32(np.arange(0x3C00, 0x4100, dtype=np.uint16)) if abs(v) <= 1.3 * mfp]
+    rng = np.random.default_rng(77)
+    ys += list(rng.uniform(-1.3 * mfp, 1.3 * mfp, 3000).astype(np.float32))
+    for k in range(-top - 2, top + 2):                   # neighbours of every half-integer product
+        y0 = np.float32((k + 0.5) / float(c))
+        for _ in range(4):
+            ys += [y0, -y0]
+            y0 = np.nextafter(y0, np.float32(np.inf))
+        y0 = np.float32((k + 0.5) / float(c))
+        for _ in range(4):
+            y0 = np.nextafter(y0, np.float32(-np.inf))
+            ys.append(y0)
+    for y in ys:
+        assert oracle.int_encode(fmt, y) == exact(y), (fmt, float(y))
+
+
 def test_e4m3_matches_torch_cast(oracle):
     """In range, the scale rounding is torch's float8_e4m3fn cast (nearest, ties to even)."""
     torch = pytest.importorskip("torch")
