@@ -44,15 +44,16 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream
 
 // ------------------------------------------------------------------------------------------ amax
 
-// Eq. 1, numerator: grid-wide max |x|.  Each block reduces its share and publishes it with one
-// atomicMax on the bit pattern (non-negative floats order like unsigned integers); the last block
-// to finish (ticket counter) turns the maximum into alpha (or returns the raw maximum), writes it
-// to the caller's slot and re-arms the scratch slot for the next call.
-//   slot[0] = running max bits, slot[1] = ticket counter; both are 0 between calls.
-template <bool RHT>
+// Eq. 1, numerator: grid-wide max |x|.  Each block reduces its share and publishes it with one 64-bit
+// atomicMax of (generation << 32) | bit pattern (non-negative floats order like unsigned integers; a
+// larger generation beats whatever an earlier call left in the slot, so nothing is ever cleared).
+//   TICKET = false: that is all; the quantize kernel of the same call turns the maximum into alpha.
+//   TICKET = true (abs_amax): the last block to finish (ticket counter in slot word 2, re-armed by
+//   that block) writes the maximum (or alpha when denom != 0) to `result`.
+template <bool RHT, bool TICKET>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t ngroups,
-                                                        uint32_t sign_mask, uint32_t* __restrict__ slot,
-                                                        float* __restrict__ result, float denom) {
+                                                        uint32_t sign_mask, unsigned long long* __restrict__ slot,
+                                                        uint32_t gen, float* __restrict__ result, float denom) {
     pdl_launch_dependents();
     uint32_t local = 0u;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -91,42 +92,44 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
     }
     local = __reduce_max_sync(0xFFFFFFFFu, local);
     __shared__ uint32_t warp_max[kThreads / 32];
-    __shared__ bool is_last;
     if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local;
     __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t m = 0u;
 #pragma unroll
         for (int w = 0; w < kThreads / 32; ++w) m = max(m, warp_max[w]);
-        atomicMax(&slot[0], m);
-        __threadfence();
-        uint32_t ticket = atomicAdd(&slot[1], 1u);
-        is_last = (ticket == gridDim.x - 1);
-        if (is_last) {
+        const unsigned long long tagged = ((unsigned long long)gen << 32) | m;
+        atomicMax(slot, tagged);
+        if constexpr (TICKET) {
+            uint32_t* ticket_word = reinterpret_cast<uint32_t*>(slot) + 2;
             __threadfence();
-            float A = __uint_as_float(atomicMax(&slot[0], 0u));
-            float out = A;
-            if (denom != 0.0f) out = (A == 0.0f) ? 1.0f : __fdiv_rn(A, denom);   // Eq. 1
-            *result = out;
-            slot[0] = 0u;
-            slot[1] = 0u;
+            const uint32_t ticket = atomicAdd(ticket_word, 1u);
+            if (ticket == gridDim.x - 1) {
+                __threadfence();
+                const unsigned long long v = atomicMax(slot, tagged);     // read the final value
+                const float A = __uint_as_float((uint32_t)v);
+                float out = A;
+                if (denom != 0.0f) out = (A == 0.0f) ? 1.0f : __fdiv_rn(A, denom);   // Eq. 1
+                *result = out;
+                *ticket_word = 0u;
+            }
         }
     }
 }
 
 // ------------------------------------------------------------------------------------------ quantize
 
-template <int FMT, bool RHT, bool SR>
+template <int FMT, bool RHT, bool SR, bool FROM_SLOT>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
                                                             uint8_t* __restrict__ scales,
-                                                            const float* __restrict__ alpha_p, int64_t ngroups,
+                                                            const AlphaSrc alpha_src, int64_t ngroups,
                                                             float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
                                                             uint32_t seed_hi) {
     using F = Fmt<FMT>;
     constexpr int B = F::BITS;
     pdl_launch_dependents();
     pdl_wait();
-    const float alpha = __ldg(alpha_p);
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                        // T2
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));                      // T3
     const float c_pre = F::HAS_INT ? __fdiv_rn(F::M_INT, F::M_FP) : 0.0f;
     const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
@@ -331,8 +334,7 @@ __global__ void selftest_kernel(int kind, const float* __restrict__ in, int64_t 
 struct DeviceState {
     std::once_flag once;
     cudaError_t init_err = cudaSuccess;
-    uint32_t* ring = nullptr;          // ABS_MAX_INFLIGHT slots of 4 words (amax bits, ticket, pad, pad)
-    float* amax_alpha = nullptr;       // unused spare floats, one per slot (alpha hand-off for abs_amax)
+    uint32_t* ring = nullptr;          // ABS_MAX_INFLIGHT slots of 16 bytes: tagged maximum (u64), ticket (u32), pad
     std::atomic<uint32_t> next{0};
     int sm_count = 148;
 };
@@ -385,23 +387,42 @@ int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
     return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
 }
 
-abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const abs_opts_t& o, float* result,
-                         float denom, cudaStream_t s) {
-    uint32_t* slot = st.ring + 4 * (st.next.fetch_add(1) % ABS_MAX_INFLIGHT);
+// Takes the next scratch slot and generation of this device.  Generations grow by one per call; when
+// the 32-bit counter wraps (after 2^32 calls) the ring is cleared once, after the device went idle.
+abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen) {
+    uint32_t g = st.next.fetch_add(1) + 1;
+    if (g == 0) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return ABS_ERR_CUDA;
+        if (cudaMemset(st.ring, 0, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t)) != cudaSuccess) return ABS_ERR_CUDA;
+        g = st.next.fetch_add(1) + 1;
+    }
+    *gen = g;
+    *slot = reinterpret_cast<unsigned long long*>(st.ring + 4 * (g % ABS_MAX_INFLIGHT));
+    return ABS_OK;
+}
+
+// ticket = true: the kernel itself writes max |x| (denom == 0) or alpha to `result` (abs_amax).
+// ticket = false: the maximum stays in the slot for the quantize kernel of the same call.
+abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const abs_opts_t& o, bool ticket,
+                         unsigned long long* slot, uint32_t gen, float* result, float denom, cudaStream_t s) {
     const bool rht = o.flags & ABS_F_HADAMARD16;
     const int grid = grid_for(st, rht ? ngroups : ngroups * 2, ABS_AMAX_BPS);
     cudaError_t e;
-    if (rht)
-        e = launch_pdl(amax_kernel<true>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, result, denom);
-    else
-        e = launch_pdl(amax_kernel<false>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, result, denom);
+#define ABS_LAUNCH_A(R, T)                                                                                          \
+    e = launch_pdl(amax_kernel<R, T>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, \
+                   gen, result, denom)
+    if (rht && ticket) ABS_LAUNCH_A(true, true);
+    else if (rht) ABS_LAUNCH_A(true, false);
+    else if (ticket) ABS_LAUNCH_A(false, true);
+    else ABS_LAUNCH_A(false, false);
+#undef ABS_LAUNCH_A
     if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
 template <int FMT>
 abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
-                                 const float* alpha, const abs_opts_t& o, cudaStream_t s) {
+                                 const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s) {
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const int grid = grid_for(st, ngroups, 64);
@@ -415,8 +436,10 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
             cudaError_t e;
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
-    e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32>, pgrid, kThreads, s, (const uint4*)in, (uint2*)codes,        \
-                   (uint8_t*)scales, alpha, (IDX)ngroups, mul)
+    e = alpha.slot ? launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, true>, pgrid, kThreads, s, (const uint4*)in,    \
+                                (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, mul)                            \
+                   : launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, false>, pgrid, kThreads, s, (const uint4*)in,   \
+                                (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, mul)
             if (i32 && a32) ABS_LAUNCH_F(int32_t, true);
             else if (i32) ABS_LAUNCH_F(int32_t, false);
             else if (a32) ABS_LAUNCH_F(int64_t, true);
@@ -429,8 +452,12 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     }
     cudaError_t eq = cudaSuccess;
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
-    eq = launch_pdl(quantize_kernel<FMT, R, S>, grid, kThreads, s, (const uint4*)in, (uint8_t*)codes,           \
-                    (uint8_t*)scales, alpha, ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1)
+    eq = alpha.slot ? launch_pdl(quantize_kernel<FMT, R, S, true>, grid, kThreads, s, (const uint4*)in,         \
+                                 (uint8_t*)codes, (uint8_t*)scales, alpha, ngroups, mul,                        \
+                                 (uint32_t)o.had_sign_mask, k0, k1)                                             \
+                    : launch_pdl(quantize_kernel<FMT, R, S, false>, grid, kThreads, s, (const uint4*)in,        \
+                                 (uint8_t*)codes, (uint8_t*)scales, alpha, ngroups, mul,                        \
+                                 (uint32_t)o.had_sign_mask, k0, k1)
     if (rht && sr) ABS_LAUNCH_Q(true, true);
     else if (rht) ABS_LAUNCH_Q(true, false);
     else if (sr) ABS_LAUNCH_Q(false, true);
@@ -610,7 +637,10 @@ abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs
     if (!aligned16(in_bf16)) return ABS_ERR_ALIGN;
     DeviceState* st = nullptr;
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
-    return launch_amax(*st, in_bf16, rows * cols / 16, o, amax_f32, 0.0f, s);
+    unsigned long long* slot = nullptr;
+    uint32_t gen = 0;
+    if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+    return launch_amax(*st, in_bf16, rows * cols / 16, o, true, slot, gen, amax_f32, 0.0f, s);
 }
 
 abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
@@ -628,16 +658,24 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
-        rc = launch_amax(*st, in_bf16, ngroups, o, tensor_scale_f32, fmt_mfp((int)fmt) * 448.0f, s);
+        unsigned long long* slot = nullptr;
+        uint32_t gen = 0;
+        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        const float denom = fmt_mfp((int)fmt) * 448.0f;
+        rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
         if (rc != ABS_OK) return rc;
+        src.slot = slot;
+        src.gen = gen;
+        src.denom = denom;
     }
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        default: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        default: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
     }
 }
 
@@ -679,12 +717,13 @@ abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t ro
     DeviceState grid_info;                 // only its SM count is read by the launchers; no ring is touched
     grid_info.sm_count = na.sm_count;
     const abs_opts_t o = {0, 0, 0, 0};
+    const AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};   // alpha was written by the chunked pass
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF4: return launch_quantize_fmt<1>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF3: return launch_quantize_fmt<2>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
-        default: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, tensor_scale_f32, o, s);
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        default: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
     }
 }
 

@@ -224,6 +224,27 @@ __device__ __forceinline__ void store32B(void* p, const uint32_t (&w)[8]) {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// How a quantize kernel learns alpha (Eq. 1): either a float the caller supplied, or the running
+// maximum that the amax pass of the same call left in a scratch slot.  The slot holds
+// (generation << 32) | bits(max |x|): every call uses a larger generation, so a 64-bit atomicMax never
+// needs the slot cleared and the amax pass needs no "last block" epilogue.
+struct AlphaSrc {
+    const float* alpha_p;                 // used when slot == nullptr
+    const unsigned long long* slot;       // tagged maximum written by amax_kernel
+    uint32_t gen;                         // generation of this call
+    float denom;                          // M_FP * 448
+    float* alpha_out;                     // where alpha is published for the caller
+};
+template <bool FROM_SLOT>
+__device__ __forceinline__ float resolve_alpha(const AlphaSrc& a) {
+    if constexpr (!FROM_SLOT) return __ldg(a.alpha_p);
+    const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(a.slot);
+    const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
+    const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                   // Eq. 1
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.alpha_out = alpha;
+    return alpha;
+}
+
 // ----------------------------------------------------------------------------- unpack
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4& v, float* x) {

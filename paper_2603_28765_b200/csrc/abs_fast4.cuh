@@ -170,16 +170,16 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
 // Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
 // next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
 // IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
-template <bool HAS_INT, typename IdxT, bool ALIGNED32>
+template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT>
 __global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
 quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                      const float* __restrict__ alpha_p, IdxT ngroups, float scale_mul) {
+                      const AlphaSrc alpha_src, IdxT ngroups, float scale_mul) {
     pdl_launch_dependents();
     const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
     IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x);
     pdl_wait();
     if (g >= ngroups) return;
-    const float alpha = __ldg(alpha_p);
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     uint32_t w[8], wn[8];
     load32B<ALIGNED32>(in + 2 * (size_t)g, w);
