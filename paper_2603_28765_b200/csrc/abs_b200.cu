@@ -435,16 +435,22 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
             cudaError_t e;
+#define ABS_LAUNCH_F3(IDX, A32, SLOT, MUL)                                                                           \
+    e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL>, pgrid, kThreads, s, (const uint4*)in,            \
+                   (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups)
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
-    e = alpha.slot ? launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, true>, pgrid, kThreads, s, (const uint4*)in,    \
-                                (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, mul)                            \
-                   : launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, false>, pgrid, kThreads, s, (const uint4*)in,   \
-                                (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, mul)
+    do {                                                                                                             \
+        if (alpha.slot && mul != 1.0f) ABS_LAUNCH_F3(IDX, A32, true, true);                                          \
+        else if (alpha.slot) ABS_LAUNCH_F3(IDX, A32, true, false);                                                   \
+        else if (mul != 1.0f) ABS_LAUNCH_F3(IDX, A32, false, true);                                                  \
+        else ABS_LAUNCH_F3(IDX, A32, false, false);                                                                  \
+    } while (0)
             if (i32 && a32) ABS_LAUNCH_F(int32_t, true);
             else if (i32) ABS_LAUNCH_F(int32_t, false);
             else if (a32) ABS_LAUNCH_F(int64_t, true);
             else ABS_LAUNCH_F(int64_t, false);
 #undef ABS_LAUNCH_F
+#undef ABS_LAUNCH_F3
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;

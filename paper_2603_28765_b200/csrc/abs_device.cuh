@@ -235,14 +235,22 @@ struct AlphaSrc {
     float denom;                          // M_FP * 448
     float* alpha_out;                     // where alpha is published for the caller
 };
+// Must be called by every thread of the block (it synchronises): thread 0 reads the slot, divides once
+// (Eq. 1) and shares alpha through shared memory, so one-group-per-thread launches do not pay a division
+// per thread.  Block 0 also publishes alpha for the caller.
 template <bool FROM_SLOT>
 __device__ __forceinline__ float resolve_alpha(const AlphaSrc& a) {
     if constexpr (!FROM_SLOT) return __ldg(a.alpha_p);
-    const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(a.slot);
-    const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
-    const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                   // Eq. 1
-    if (blockIdx.x == 0 && threadIdx.x == 0) *a.alpha_out = alpha;
-    return alpha;
+    __shared__ float alpha_shared;
+    if (threadIdx.x == 0) {
+        const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(a.slot);
+        const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
+        const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                   // Eq. 1
+        alpha_shared = alpha;
+        if (blockIdx.x == 0) *a.alpha_out = alpha;
+    }
+    __syncthreads();
+    return alpha_shared;
 }
 
 // ----------------------------------------------------------------------------- unpack

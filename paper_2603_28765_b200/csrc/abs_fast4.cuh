@@ -170,16 +170,16 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
 // Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
 // next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
 // IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
-template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT>
+template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT, bool SCALE_MUL>
 __global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
 quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                      const AlphaSrc alpha_src, IdxT ngroups, float scale_mul) {
+                      const AlphaSrc alpha_src, IdxT ngroups) {
     pdl_launch_dependents();
     const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
     IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x);
     pdl_wait();
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
     if (g >= ngroups) return;
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     uint32_t w[8], wn[8];
     load32B<ALIGNED32>(in + 2 * (size_t)g, w);
@@ -199,14 +199,17 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
         const float m4 = max3abs(x[12], x[13], x[14]);
         const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
         // G2-G3 (Eq. 2).
-        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
+        float t = __fmul_rn(gmax, inv_a6);
+        if constexpr (SCALE_MUL) t = __fmul_rn(t, 1.0625f);                 // the 17/16 option
         const uint32_t sb = e4m3_encode(t);
+        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
+        const float r = __frcp_rn(d);
         uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
-        if (sb != 0u) {                                                      // G4
-            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
-            const float r = __frcp_rn(d);
-            if (HAS_INT && (sb - 8u) >= 118u) encode_body4<HAS_INT, true>(x, sb, d, r, sbyte, c_lo, c_hi);
-            else encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
+        if ((sb - 8u) >= 118u) {
+            // rare path: zero scale (G4: all codes 0), subnormal scale bytes 1..7 and the saturated 0x7E
+            if (sb != 0u) encode_body4<HAS_INT, HAS_INT>(x, sb, d, r, sbyte, c_lo, c_hi);
+        } else {
+            encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
         }
         scales[g] = (uint8_t)sbyte;
         codes[g] = make_uint2(c_lo, c_hi);
