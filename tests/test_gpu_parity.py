@@ -402,3 +402,20 @@ def test_full_size_parity(B, oracle, name, fmts, opt):
             assert 0.05 < frac < 0.999, (name, fmt, frac)
     if opt == "HS17":       # the extra row of the gradient configuration: 17/16 option off
         check_case(B, oracle, 1, xb, flags=flags & ~B.ABS_F_SR_SCALE_17_16, mask=mask, seed=seed, dequant=False)
+
+
+def test_sr_bias_signature_on_gpu(B):
+    """App. B on the CUDA path: averaged over seeds, NVFP4 with stochastic rounding leaves every
+    magnitude bin unchanged, IF4 moves the near-maximal values of a group outward, by well under
+    5 % of the group maximum, and only a small share of the elements sits in the affected bins."""
+    from paper_2603_28765_b200 import sr_bias
+    res = sr_bias.run(trials=200, rows=256, cols=4096, scale_option=True)
+    nv = {round(b["rel_lo"], 1): b for b in res["nvfp4"]}
+    i4 = {round(b["rel_lo"], 1): b for b in res["if4"]}
+    for lo, b in nv.items():
+        assert abs(b["mean_change_over_gmax"]) < 3e-3, ("nvfp4", lo, b)
+    top = i4[0.9]
+    assert 3e-3 < top["mean_change_over_gmax"] < 5e-2, top
+    assert top["share"] < 0.12
+    for lo in (0.1, 0.2, 0.3, 0.4):
+        assert abs(i4[lo]["mean_change_over_gmax"]) < 6e-3, (lo, i4[lo])
