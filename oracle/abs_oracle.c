@@ -38,7 +38,8 @@
 
 #define ORACLE_API __attribute__((visibility("default")))
 
-enum { FMT_NVFP4 = 0, FMT_IF4 = 1, FMT_IF3 = 2, FMT_IF6_E2M3 = 3, FMT_IF6_E3M2 = 4, FMT_COUNT = 5 };
+enum { FMT_NVFP4 = 0, FMT_IF4 = 1, FMT_IF3 = 2, FMT_IF6_E2M3 = 3, FMT_IF6_E3M2 = 4,
+       FMT_NVFP4_BS8 = 5, FMT_IF4_BS8 = 6, FMT_IF3_BS8 = 7, FMT_COUNT = 8 };   /* BS8: one scale per 8 values (Sec. 5.1, Table 5) */
 
 enum {
     F_HADAMARD16 = 1u << 0,
@@ -55,14 +56,18 @@ typedef struct {
     int has_int;            /* 0 for plain NVFP4 (procedure stops after step 4)          */
     float m_fp;             /* largest FP magnitude: 6, 4, 7.5, 28                       */
     float m_int;            /* largest integer magnitude: 7, 3, 31, 31                   */
+    int group;              /* values per scale: 16, or 8 for the block-size-8 variants  */
 } fmt_desc;
 
 static const fmt_desc FMTS[FMT_COUNT] = {
-    /* NVFP4    */ {2, 1, 1, 4, 0, 6.0f, 0.0f},
-    /* IF4      */ {2, 1, 1, 4, 1, 6.0f, 7.0f},
-    /* IF3      */ {2, 0, 1, 3, 1, 4.0f, 3.0f},
-    /* IF6-E2M3 */ {2, 3, 1, 6, 1, 7.5f, 31.0f},
-    /* IF6-E3M2 */ {3, 2, 3, 6, 1, 28.0f, 31.0f},
+    /* NVFP4     */ {2, 1, 1, 4, 0, 6.0f, 0.0f, 16},
+    /* IF4       */ {2, 1, 1, 4, 1, 6.0f, 7.0f, 16},
+    /* IF3       */ {2, 0, 1, 3, 1, 4.0f, 3.0f, 16},
+    /* IF6-E2M3  */ {2, 3, 1, 6, 1, 7.5f, 31.0f, 16},
+    /* IF6-E3M2  */ {3, 2, 3, 6, 1, 28.0f, 31.0f, 16},
+    /* NVFP4-BS8 */ {2, 1, 1, 4, 0, 6.0f, 0.0f, 8},
+    /* IF4-BS8   */ {2, 1, 1, 4, 1, 6.0f, 7.0f, 8},
+    /* IF3-BS8   */ {2, 0, 1, 3, 1, 4.0f, 3.0f, 8},
 };
 
 /* ------------------------------------------------------------------ small helpers */
@@ -184,17 +189,19 @@ static void load_group(const uint16_t* in_bf16, uint32_t flags, uint16_t sign_ma
 /* ------------------------------------------------------------------ error sum */
 
 /* Sum of squares of 16 errors in the fixed order: four fused chains over the element sets
- * {0,2,4,6}, {1,3,5,7}, {8,10,12,14}, {9,11,13,15}, then (S0+S1)+(S2+S3).  (Fig. 3a steps
+ * {0,2,4,6}, {1,3,5,7}, {8,10,12,14}, {9,11,13,15}, then (S0+S1)+(S2+S3); a group of 8 values
+ * has the first two chains and the sum S0+S1.  (Fig. 3a steps
  * 6 and 9 print a mean, but the printed value 46.0 is the sum; n = 16 is constant, so the
  * comparison of step 10 is the same either way.) */
-static float sum16_sq(const float e[16]) {
-    float s[4];
-    for (int c = 0; c < 4; ++c) {
+static float sum16_sq(const float* e, int n) {
+    float s[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int c = 0; c < n / 4; ++c) {
         int first = (c & 1) + 8 * (c >> 1);
         float acc = 0.0f;
         for (int k = 0; k < 4; ++k) { float v = e[first + 2 * k]; acc = fmaf(v, v, acc); }
         s[c] = acc;
     }
+    if (n == 8) return s[0] + s[1];          /* a group of 8 has the first two chains only */
     return (s[0] + s[1]) + (s[2] + s[3]);
 }
 
@@ -230,6 +237,7 @@ static float int_candidate_rne(float y, float c_pre, float m_int) {
 /* ------------------------------------------------------------------ exported element-level pieces */
 
 ORACLE_API int abs_oracle_fmt_bits(int fmt) { return (fmt >= 0 && fmt < FMT_COUNT) ? FMTS[fmt].bits : -1; }
+ORACLE_API int abs_oracle_fmt_group(int fmt) { return (fmt >= 0 && fmt < FMT_COUNT) ? FMTS[fmt].group : -1; }
 ORACLE_API float abs_oracle_fmt_mfp(int fmt) { return FMTS[fmt].m_fp; }
 ORACLE_API float abs_oracle_fmt_mint(int fmt) { return FMTS[fmt].m_int; }
 /* c_pre = fp32(M_INT / M_FP), c_post = fp32(M_FP / M_INT) (the "6/7 method" constants). */
@@ -305,8 +313,8 @@ ORACLE_API float abs_oracle_alpha(int fmt, float amax) {
 /* ------------------------------------------------------------------ quantize */
 
 /* Quantize rows [row0,row1) of a row-major bf16 matrix with tensor scale alpha.
- * Outputs: codes (rows x cols*b/8 bytes), scales (rows x cols/16 bytes); optional per-group
- * E_FP / E_INT (rows x cols/16 floats each, may be NULL) for the selection invariants. */
+ * Outputs: codes (rows x cols*b/8 bytes), scales (rows x cols/G bytes, G = values per scale); optional
+ * per-group E_FP / E_INT (rows x cols/G floats each, may be NULL) for the selection invariants. */
 ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_t rows, int64_t cols,
                                         int64_t row0, int64_t row1, float alpha, uint32_t flags,
                                         uint16_t sign_mask, uint64_t sr_seed, uint8_t* codes,
@@ -327,80 +335,89 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
     const float c_post = F->has_int ? F->m_fp / F->m_int : 0.0f;
     const int64_t gpr = cols / 16;
 
+    const int G = F->group;                 /* values per scale */
+    const int nsub = 16 / G;                /* groups per aligned block of 16 (the Hadamard block) */
+
     for (int64_t r = row0; r < row1; ++r)
         for (int64_t gi = 0; gi < gpr; ++gi) {
             float x[16];
             load_group(in_bf16 + r * cols + gi * 16, flags, sign_mask, x);
             uint8_t* code_out = codes + (r * gpr + gi) * (2 * b);
-            uint8_t* scale_out = scales + (r * gpr + gi);
-            uint32_t q_fp[16], q_int[16];
-            float e_fp[16], e_int[16];
+            uint32_t chosen[16];
+            for (int sub = 0; sub < nsub; ++sub) {
+                const float* xs = x + sub * G;
+                const int64_t sidx = (r * gpr + gi) * nsub + sub;
+                uint32_t q_fp[16], q_int[16];
+                float e_fp[16], e_int[16];
 
-            /* G1: group maximum (exact). */
-            float gmax = 0.0f;
-            for (int i = 0; i < 16; ++i) { float a = fabsf(x[i]); if (a > gmax) gmax = a; }
-            /* G2 (Eq. 2; steps 1-2): t = gmax / (alpha * M_FP), as a multiply by the reciprocal. */
-            float t = gmax * inv_a6;
-            if (flags & F_SR_SCALE_17_16) t = t * 1.0625f;
-            /* G3: E4M3 round-to-nearest-even, saturating. */
-            uint32_t sb = (uint32_t)grid_round_rne(e4g, ne4, t);
-            /* G4: a scale that rounds to zero encodes an all-zero group. */
-            if (sb == 0) {
-                memset(code_out, 0, (size_t)(2 * b));
-                *scale_out = 0x00;
-                if (dbg_e_fp) dbg_e_fp[r * gpr + gi] = 0.0f;
-                if (dbg_e_int) dbg_e_int[r * gpr + gi] = 0.0f;
-                continue;
-            }
-            /* G5: decoded block scale, combined scale and its reciprocal. */
-            const float Delta = (float)e4g[sb];
-            const float d = Delta * alpha;
-            const float rcp = 1.0f / d;
-            const float d_int = d * c_post;
-
-            for (int i = 0; i < 16; ++i) {
-                const float xi = x[i];
-                float u = 0.0f;
-                if (flags & F_STOCHASTIC) u = sr_uniform(sr_seed, (uint64_t)(r * cols + gi * 16 + i));
-                /* E1 (step 3). */
-                const float y = xi * rcp;
-                const uint32_t ysign = f32_to_bits(y) >> 31;
-                /* E2 (step 4): FP candidate code. */
-                int mi = (flags & F_STOCHASTIC) ? grid_round_sr(fpg, nfp, fabsf(y), u)
-                                                : grid_round_rne(fpg, nfp, fabsf(y));
-                q_fp[i] = (ysign << (b - 1)) | (uint32_t)mi;
-                /* E3 (steps 5-6): error of the dequantized FP candidate, one fused rounding. */
-                float vfp = (float)fpg[mi];
-                if (ysign) vfp = -vfp;
-                e_fp[i] = fmaf(vfp, d, -xi);
-                if (!F->has_int) continue;
-                /* E4 (step 7): integer candidate of y * M_INT / M_FP, clamped to +-M_INT. */
-                float kf;
-                if (flags & F_STOCHASTIC) {
-                    const float z = y * c_pre;   /* the stochastic draw needs the FP32 value itself */
-                    kf = (float)grid_round_sr(intg, m_int + 1, fabsf(z), u);
-                    if (f32_to_bits(z) >> 31) kf = -kf;
-                } else {
-                    kf = int_candidate_rne(y, c_pre, F->m_int);
+                /* G1: group maximum (exact). */
+                float gmax = 0.0f;
+                for (int i = 0; i < G; ++i) { float a = fabsf(xs[i]); if (a > gmax) gmax = a; }
+                /* G2 (Eq. 2; steps 1-2): t = gmax / (alpha * M_FP), as a multiply by the reciprocal. */
+                float t = gmax * inv_a6;
+                if (flags & F_SR_SCALE_17_16) t = t * 1.0625f;
+                /* G3: E4M3 round-to-nearest-even, saturating. */
+                uint32_t sb = (uint32_t)grid_round_rne(e4g, ne4, t);
+                /* G4: a scale that rounds to zero encodes an all-zero group. */
+                if (sb == 0) {
+                    for (int i = 0; i < G; ++i) chosen[sub * G + i] = 0u;
+                    scales[sidx] = 0x00;
+                    if (dbg_e_fp) dbg_e_fp[sidx] = 0.0f;
+                    if (dbg_e_int) dbg_e_int[sidx] = 0.0f;
+                    continue;
                 }
-                const int k = (int)kf;
-                q_int[i] = (uint32_t)k & ((1u << b) - 1u);   /* two's complement in b bits */
-                /* E5 (steps 8-9): error of the dequantized integer candidate. */
-                e_int[i] = fmaf((float)k, d_int, -xi);
-            }
+                /* G5: decoded block scale, combined scale and its reciprocal. */
+                const float Delta = (float)e4g[sb];
+                const float d = Delta * alpha;
+                const float rcp = 1.0f / d;
+                const float d_int = d * c_post;
 
-            /* S1-S3 (step 10): keep the integer candidate iff its error is strictly smaller. */
-            int flag = 0;
-            float E_fp = sum16_sq(e_fp), E_int = 0.0f;
-            if (F->has_int) {
-                E_int = sum16_sq(e_int);
-                flag = (E_int < E_fp) ? 1 : 0;
+                for (int i = 0; i < G; ++i) {
+                    const float xi = xs[i];
+                    float u = 0.0f;
+                    if (flags & F_STOCHASTIC)
+                        u = sr_uniform(sr_seed, (uint64_t)(r * cols + gi * 16 + sub * G + i));
+                    /* E1 (step 3). */
+                    const float y = xi * rcp;
+                    const uint32_t ysign = f32_to_bits(y) >> 31;
+                    /* E2 (step 4): FP candidate code. */
+                    int mi = (flags & F_STOCHASTIC) ? grid_round_sr(fpg, nfp, fabsf(y), u)
+                                                    : grid_round_rne(fpg, nfp, fabsf(y));
+                    q_fp[i] = (ysign << (b - 1)) | (uint32_t)mi;
+                    /* E3 (steps 5-6): error of the dequantized FP candidate, one fused rounding. */
+                    float vfp = (float)fpg[mi];
+                    if (ysign) vfp = -vfp;
+                    e_fp[i] = fmaf(vfp, d, -xi);
+                    if (!F->has_int) continue;
+                    /* E4 (step 7): integer candidate of y * M_INT / M_FP, clamped to +-M_INT. */
+                    float kf;
+                    if (flags & F_STOCHASTIC) {
+                        const float z = y * c_pre;   /* the stochastic draw needs the FP32 value itself */
+                        kf = (float)grid_round_sr(intg, m_int + 1, fabsf(z), u);
+                        if (f32_to_bits(z) >> 31) kf = -kf;
+                    } else {
+                        kf = int_candidate_rne(y, c_pre, F->m_int);
+                    }
+                    const int k = (int)kf;
+                    q_int[i] = (uint32_t)k & ((1u << b) - 1u);   /* two's complement in b bits */
+                    /* E5 (steps 8-9): error of the dequantized integer candidate. */
+                    e_int[i] = fmaf((float)k, d_int, -xi);
+                }
+
+                /* S1-S3 (step 10): keep the integer candidate iff its error is strictly smaller. */
+                int flag = 0;
+                float E_fp = sum16_sq(e_fp, G), E_int = 0.0f;
+                if (F->has_int) {
+                    E_int = sum16_sq(e_int, G);
+                    flag = (E_int < E_fp) ? 1 : 0;
+                }
+                if (dbg_e_fp) dbg_e_fp[sidx] = E_fp;
+                if (dbg_e_int) dbg_e_int[sidx] = E_int;
+                scales[sidx] = (uint8_t)(sb | ((uint32_t)flag << 7));
+                for (int i = 0; i < G; ++i) chosen[sub * G + i] = flag ? q_int[i] : q_fp[i];
             }
-            if (dbg_e_fp) dbg_e_fp[r * gpr + gi] = E_fp;
-            if (dbg_e_int) dbg_e_int[r * gpr + gi] = E_int;
-            *scale_out = (uint8_t)(sb | ((uint32_t)flag << 7));
-            /* S4. */
-            pack_codes(flag ? q_int : q_fp, b, code_out);
+            /* S4: the 16 codes of the block form one little-endian bitstream, whatever the group size. */
+            pack_codes(chosen, b, code_out);
         }
     return 0;
 }
@@ -417,16 +434,17 @@ ORACLE_API int abs_oracle_dequantize_rows(int fmt, const uint8_t* codes, const u
     const int b = F->bits;
     const float c_post = F->has_int ? F->m_fp / F->m_int : 0.0f;
     const int64_t gpr = cols / 16;
+    const int G = F->group, nsub = 16 / G;
     for (int64_t r = row0; r < row1; ++r)
         for (int64_t gi = 0; gi < gpr; ++gi) {
-            const uint8_t sbyte = scales[r * gpr + gi];
-            const int flag = sbyte >> 7;
-            const float Delta = abs_oracle_e4m3_value(sbyte);
-            float d = Delta * alpha;
-            if (flag) d = d * c_post;
             uint32_t code[16];
             unpack_codes(codes + (r * gpr + gi) * (2 * b), b, code);
             for (int i = 0; i < 16; ++i) {
+                const uint8_t sbyte = scales[(r * gpr + gi) * nsub + i / G];
+                const int flag = sbyte >> 7;
+                const float Delta = abs_oracle_e4m3_value(sbyte);
+                float d = Delta * alpha;
+                if (flag) d = d * c_post;
                 float v;
                 if (flag) {
                     int k = (int)code[i];

@@ -21,8 +21,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "abs_oracle.c")
 _LIB = os.path.join(_HERE, "libabs_oracle.so")
 
-FMT_NVFP4, FMT_IF4, FMT_IF3, FMT_IF6_E2M3, FMT_IF6_E3M2 = range(5)
-FMT_NAMES = {"nvfp4": 0, "if4": 1, "if3": 2, "if6_e2m3": 3, "if6_e3m2": 4}
+FMT_NVFP4, FMT_IF4, FMT_IF3, FMT_IF6_E2M3, FMT_IF6_E3M2, FMT_NVFP4_BS8, FMT_IF4_BS8, FMT_IF3_BS8 = range(8)
+FMT_NAMES = {"nvfp4": 0, "if4": 1, "if3": 2, "if6_e2m3": 3, "if6_e3m2": 4, "nvfp4_bs8": 5, "if4_bs8": 6, "if3_bs8": 7}
 
 F_HADAMARD16 = 1 << 0
 F_STOCHASTIC = 1 << 1
@@ -53,6 +53,8 @@ def lib():
             u8p, u16p, f32p, u32p = (C.POINTER(t) for t in (C.c_uint8, C.c_uint16, C.c_float, C.c_uint32))
             L.abs_oracle_fmt_bits.restype = C.c_int
             L.abs_oracle_fmt_bits.argtypes = [C.c_int]
+            L.abs_oracle_fmt_group.restype = C.c_int
+            L.abs_oracle_fmt_group.argtypes = [C.c_int]
             for name in ("abs_oracle_fmt_mfp", "abs_oracle_fmt_mint", "abs_oracle_c_pre", "abs_oracle_c_post"):
                 getattr(L, name).restype = C.c_float
                 getattr(L, name).argtypes = [C.c_int]
@@ -95,12 +97,17 @@ def fmt_bits(fmt: int) -> int:
     return lib().abs_oracle_fmt_bits(fmt)
 
 
+def fmt_group(fmt: int) -> int:
+    """Values that share one scale: 16, or 8 for the block-size-8 variants."""
+    return lib().abs_oracle_fmt_group(fmt)
+
+
 def codes_bytes(fmt: int, rows: int, cols: int) -> int:
     return rows * cols * fmt_bits(fmt) // 8
 
 
-def scales_bytes(rows: int, cols: int) -> int:
-    return rows * cols // 16
+def scales_bytes(rows: int, cols: int, fmt: int = 0) -> int:
+    return rows * cols // fmt_group(fmt)
 
 
 def c_pre(fmt):
@@ -222,10 +229,11 @@ def quantize(fmt: int, x_bf16_bits, flags: int = 0, sign_mask: int = 0, sr_seed:
         alpha = np.float32(alpha)
     else:
         alpha = alpha_from_amax(fmt, amax(a, flags, sign_mask, threads))
+    G = fmt_group(fmt)
     codes = np.zeros((rows, cols * b // 8), dtype=np.uint8)
-    scales = np.zeros((rows, cols // 16), dtype=np.uint8)
-    efp = np.zeros((rows, cols // 16), dtype=np.float32) if debug else None
-    eint = np.zeros((rows, cols // 16), dtype=np.float32) if debug else None
+    scales = np.zeros((rows, cols // G), dtype=np.uint8)
+    efp = np.zeros((rows, cols // G), dtype=np.float32) if debug else None
+    eint = np.zeros((rows, cols // G), dtype=np.float32) if debug else None
 
     def work(rr):
         rc = L.abs_oracle_quantize_rows(fmt, a.ctypes.data, rows, cols, rr[0], rr[1], C.c_float(float(alpha)),
@@ -249,7 +257,7 @@ def dequantize(fmt: int, codes, scales, alpha, rows: int, cols: int, out_fp32: b
     """Inverse path. Returns bf16 bit patterns (uint16) or float32 when ``out_fp32``."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     scales = np.ascontiguousarray(scales, dtype=np.uint8)
-    assert codes.size == codes_bytes(fmt, rows, cols) and scales.size == scales_bytes(rows, cols)
+    assert codes.size == codes_bytes(fmt, rows, cols) and scales.size == scales_bytes(rows, cols, fmt)
     out = np.zeros((rows, cols), dtype=np.float32 if out_fp32 else np.uint16)
     L = lib()
 

@@ -590,3 +590,97 @@ def test_sr_scale_option_prevents_clipping(oracle):
         assert (ymax.max() > 6.0 * (1 + 1e-6)) == expect_clip
         if not expect_clip:
             assert ymax[s >= 8].max() <= 6.0 * (1 + 1e-6)
+
+
+# --------------------------------------------------------------------------- block size 8 (Sec. 5.1, Table 5)
+
+BS8 = {5: 0, 6: 1, 7: 2}          # block-size-8 format -> its 16-value sibling
+
+
+def test_bs8_bits_per_parameter(oracle):
+    g = read_golden("format_facts.txt")
+    for key, fmt in (("if3_bs8", 7), ("if4_bs8", 6), ("nvfp4_bs8", 5)):
+        bpp = (oracle.codes_bytes(fmt, 1, 16) + oracle.scales_bytes(1, 16, fmt)) * 8 / 16
+        assert bpp == float(g["bits_per_param_" + key][0])
+        assert oracle.fmt_group(fmt) == 8 and oracle.fmt_bits(fmt) == oracle.fmt_bits(BS8[fmt])
+
+
+@pytest.mark.parametrize("fmt", sorted(BS8))
+def test_bs8_equals_16_on_duplicated_halves(oracle, fmt):
+    """A block whose two halves are identical: the 16-value format's single scale, flag and codes must
+    equal the two (identical) groups of the block-size-8 format -- the sum of 16 squared errors is then
+    exactly twice the sum of 8, so even the selection agrees.  Links BS8 to the pinned 16-value path."""
+    half = CASES["cfg5"][:24, :256].reshape(24, 32, 8)
+    xb = np.concatenate([half, half], axis=2).reshape(24, 512)
+    c8, s8, a8 = oracle.quantize(fmt, xb)
+    c16, s16, a16 = oracle.quantize(BS8[fmt], xb)
+    assert a8 == a16
+    assert np.array_equal(c8, c16)
+    assert np.array_equal(s8[:, 0::2], s16) and np.array_equal(s8[:, 1::2], s16)
+    d8 = oracle.dequantize(fmt, c8, s8, a8, 24, 512)
+    assert np.array_equal(d8, oracle.dequantize(BS8[fmt], c16, s16, a16, 24, 512))
+
+
+@pytest.mark.parametrize("fmt", [6, 7])
+@pytest.mark.parametrize("case", ["cfg1", "cfg2", "cfg4", "wide_dynamic_range", "tiny_row", "zeros_3x48"])
+def test_bs8_selection_invariants(oracle, fmt, case):
+    xb = CASES[case]
+    rows, cols = xb.shape
+    c, s, a, efp, eint = oracle.quantize(fmt, xb, debug=True)
+    assert s.shape == (rows, cols // 8)
+    flag = (s >> 7).astype(bool)
+    assert np.all(eint[flag] < efp[flag]) and np.all(~(eint[~flag] < efp[~flag]))
+    assert not np.any(s == 0x80)
+    # FP groups are the FP-only format's groups, byte for byte
+    cn, sn, an = oracle.quantize(5 if fmt == 6 else fmt, xb)
+    if fmt == 6:
+        assert an == a and np.array_equal(s & 0x7F, sn)
+        b = 4
+        g4 = c.reshape(rows, cols // 8, b)
+        gn = cn.reshape(rows, cols // 8, b)
+        assert np.array_equal(g4[~flag], gn[~flag])
+
+
+@pytest.mark.parametrize("fmt", sorted(BS8))
+def test_bs8_bruteforce_elements(oracle, fmt):
+    """Every stored code is (up to float32 near-ties) the closest grid point for the group's scale."""
+    xb = CASES["cfg5"][:8, :128]
+    rows, cols = xb.shape
+    b = oracle.fmt_bits(fmt)
+    g = np.array(fp_grid(BS8[fmt]))
+    fpvals = np.concatenate([g, -g])
+    mint = int(oracle.m_int(fmt))
+    xf = I.bf16_bits_to_f32(xb).astype(np.float64)
+    c, s, a = oracle.quantize(fmt, xb)
+    for r in range(rows):
+        codes = unpack_bitstream(c[r], b).reshape(-1, 8)
+        for gi in range(cols // 8):
+            sb = int(s[r, gi])
+            x = xf[r, gi * 8:(gi + 1) * 8]
+            if sb == 0:
+                assert not codes[gi].any()
+                continue
+            d = float(np.float32(oracle.e4m3_value(sb)) * np.float32(a))
+            slack = 1e-6 * np.abs(x) + 1e-30
+            if sb >> 7:
+                d_i = float(np.float32(d) * oracle.c_post(fmt))
+                k = codes[gi].astype(np.int64)
+                k = np.where(k >= (1 << (b - 1)), k - (1 << b), k)
+                best = np.abs(np.arange(-mint, mint + 1)[None, :] * d_i - x[:, None]).min(axis=1)
+                assert np.all(np.abs(k * d_i - x) <= best + slack)
+            else:
+                v = fpvals[(codes[gi] & (len(g) - 1)) + len(g) * (codes[gi] >> (b - 1))]
+                best = np.abs(fpvals[None, :] * d - x[:, None]).min(axis=1)
+                assert np.all(np.abs(v * d - x) <= best + slack)
+
+
+def test_bs8_has_lower_error_than_16(oracle):
+    """Finer scales cannot be worse on N(0,1): the ordering behind Table 5's BS8 rows."""
+    xb = I.generate("cfg1", 256, 1024)
+    xf = I.bf16_bits_to_f32(xb).astype(np.float64)
+    for f8, f16 in BS8.items():
+        mse = {}
+        for f in (f8, f16):
+            c, s, a = oracle.quantize(f, xb, threads=4)
+            mse[f] = np.mean((oracle.dequantize(f, c, s, a, 256, 1024, out_fp32=True, threads=4) - xf) ** 2)
+        assert mse[f8] < 0.85 * mse[f16], (f8, mse)
