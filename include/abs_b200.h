@@ -47,7 +47,12 @@ typedef enum {
     ABS_FMT_IF4 = 1,
     ABS_FMT_IF3 = 2,
     ABS_FMT_IF6_E2M3 = 3,
-    ABS_FMT_IF6_E3M2 = 4
+    ABS_FMT_IF6_E3M2 = 4,
+    /* Block-size-8 variants (Sec. 5.1, Table 5): one E4M3 scale per 8 values instead of 16; codes are
+     * laid out exactly as for the 16-value sibling, the scale array is [rows, cols/8]. */
+    ABS_FMT_NVFP4_BS8 = 5,
+    ABS_FMT_IF4_BS8 = 6,
+    ABS_FMT_IF3_BS8 = 7
 } abs_fmt_t;
 
 typedef enum {
@@ -83,7 +88,8 @@ typedef struct {
     uint64_t sr_seed;       /* stochastic rounding: Philox key                                    */
 } abs_opts_t;
 
-/* Sizes of the outputs of abs_quantize: rows*cols*b/8 and rows*cols/16 bytes (0 on bad arguments). */
+/* Sizes of the outputs of abs_quantize: rows*cols*b/8 and rows*cols/16 bytes (rows*cols/8 for the
+ * block-size-8 formats); 0 on bad arguments. */
 ABS_API size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
 ABS_API size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
 ABS_API const char* abs_status_string(abs_status_t status);

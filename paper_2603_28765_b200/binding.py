@@ -12,9 +12,11 @@ import threading
 
 from . import build as _build
 
-ABS_FMT_NVFP4, ABS_FMT_IF4, ABS_FMT_IF3, ABS_FMT_IF6_E2M3, ABS_FMT_IF6_E3M2 = range(5)
-FMT_NAMES = {"nvfp4": 0, "if4": 1, "if3": 2, "if6_e2m3": 3, "if6_e3m2": 4}
-FMT_BITS = {0: 4, 1: 4, 2: 3, 3: 6, 4: 6}
+(ABS_FMT_NVFP4, ABS_FMT_IF4, ABS_FMT_IF3, ABS_FMT_IF6_E2M3, ABS_FMT_IF6_E3M2, ABS_FMT_NVFP4_BS8, ABS_FMT_IF4_BS8,
+ ABS_FMT_IF3_BS8) = range(8)
+FMT_NAMES = {"nvfp4": 0, "if4": 1, "if3": 2, "if6_e2m3": 3, "if6_e3m2": 4, "nvfp4_bs8": 5, "if4_bs8": 6, "if3_bs8": 7}
+FMT_BITS = {0: 4, 1: 4, 2: 3, 3: 6, 4: 6, 5: 4, 6: 4, 7: 3}
+FMT_GROUP = {0: 16, 1: 16, 2: 16, 3: 16, 4: 16, 5: 8, 6: 8, 7: 8}
 
 ABS_F_HADAMARD16 = 1 << 0
 ABS_F_STOCHASTIC = 1 << 1
@@ -146,7 +148,7 @@ def abs_quantize(fmt: int, x, codes=None, scales=None, tensor_scale=None, opts: 
         codes = torch.empty(max(L.abs_codes_bytes(fmt, rows, cols), 1) if cols % 16 == 0 else 1, dtype=torch.uint8,
                             device=x.device)
     if scales is None:
-        scales = torch.empty(max(rows * cols // 16, 1), dtype=torch.uint8, device=x.device)
+        scales = torch.empty(max(rows * cols // FMT_GROUP[fmt], 1), dtype=torch.uint8, device=x.device)
     if tensor_scale is None:
         tensor_scale = torch.zeros(1, dtype=torch.float32, device=x.device)
     with torch.cuda.device(x.device):

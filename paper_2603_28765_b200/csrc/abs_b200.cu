@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                                                             float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
                                                             uint32_t seed_hi) {
     using F = Fmt<FMT>;
-    constexpr int B = F::BITS;
+    constexpr int B = F::BITS, G = F::GROUP, NSUB = 16 / G;
     pdl_launch_dependents();
     pdl_wait();
     const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                        // T2
@@ -141,83 +141,89 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
         unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
         if constexpr (RHT) hadamard16(x, sign_mask);
 
-        // G1-G3 (Eq. 2, steps 1-2).
-        float gmax = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) gmax = fmaxf(gmax, fabsf(x[i]));
-        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
-        const uint32_t sb = e4m3_encode(t);
-
-        uint32_t w[3] = {0u, 0u, 0u};
-        uint32_t sbyte = 0u;
-        if (sb != 0u) {                                                               // G4
-            const float d = __fmul_rn(e4m3_value(sb), alpha);                         // G5
-            const float r = __frcp_rn(d);
-            const float d_int = __fmul_rn(d, c_post);
-
-            uint32_t rnd[8];
-            if constexpr (SR) {
-                const uint64_t i8 = (uint64_t)g * 2u;
-                uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
-                uint4 p1 = philox4x32_10((uint32_t)(i8 + 1), (uint32_t)((i8 + 1) >> 32), seed_lo, seed_hi);
-                rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;
-                rnd[4] = p1.x; rnd[5] = p1.y; rnd[6] = p1.z; rnd[7] = p1.w;
-            }
-
-            uint32_t q_fp[16], q_int[16];
-            float s_fp[4] = {0.f, 0.f, 0.f, 0.f}, s_int[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int i = 0; i < 16; i += 2) {
-                const float x0 = x[i], x1 = x[i + 1];
-                float y0 = __fmul_rn(x0, r), y1 = __fmul_rn(x1, r);                    // E1 (step 3)
-                float u0 = 0.f, u1 = 0.f;
-                float yq0 = y0, yq1 = y1;
-                if constexpr (SR) {
-                    u0 = __fmul_rn(__fadd_rn((float)(rnd[i >> 1] & 0xFFFFu), 0.5f), 1.0f / 65536.0f);
-                    u1 = __fmul_rn(__fadd_rn((float)(rnd[i >> 1] >> 16), 0.5f), 1.0f / 65536.0f);
-                    yq0 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y0), F::M_FP, u0), y0);
-                    yq1 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y1), F::M_FP, u1), y1);
-                }
-                float v0, v1;
-                fp_encode_pair<F::EK>(yq0, yq1, q_fp[i], q_fp[i + 1], v0, v1);         // E2 (step 4)
-                const int chain = ((i >> 3) << 1);                                     // elements 0-7 -> S0,S1; 8-15 -> S2,S3
-                if constexpr (F::HAS_INT) {
-                    const float e0 = __fmaf_rn(v0, d, -x0), e1 = __fmaf_rn(v1, d, -x1);   // E3 (steps 5-6)
-                    s_fp[chain] = __fmaf_rn(e0, e0, s_fp[chain]);
-                    s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
-                    const float z0 = __fmul_rn(y0, c_pre), z1 = __fmul_rn(y1, c_pre);     // E4 (step 7)
-                    float k0, k1;
-                    if constexpr (SR) {
-                        k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
-                        k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
-                    } else {
-                        // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
-                        k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);
-                        k1 = __fsub_rn(__fmaf_rn(y1, c_pre, 12582912.0f), 12582912.0f);
-                        k0 = fminf(fmaxf(k0, -F::M_INT), F::M_INT);
-                        k1 = fminf(fmaxf(k1, -F::M_INT), F::M_INT);
-                    }
-                    const float f0 = __fmaf_rn(k0, d_int, -x0), f1 = __fmaf_rn(k1, d_int, -x1);   // E5 (steps 8-9)
-                    s_int[chain] = __fmaf_rn(f0, f0, s_int[chain]);
-                    s_int[chain + 1] = __fmaf_rn(f1, f1, s_int[chain + 1]);
-                    q_int[i] = (uint32_t)__float2int_rn(k0) & ((1u << B) - 1u);
-                    q_int[i + 1] = (uint32_t)__float2int_rn(k1) & ((1u << B) - 1u);
-                }
-            }
-            uint32_t flag = 0u;
-            if constexpr (F::HAS_INT) {                                                // S1-S2 (step 10)
-                const float E_fp = __fadd_rn(__fadd_rn(s_fp[0], s_fp[1]), __fadd_rn(s_fp[2], s_fp[3]));
-                const float E_int = __fadd_rn(__fadd_rn(s_int[0], s_int[1]), __fadd_rn(s_int[2], s_int[3]));
-                flag = (E_int < E_fp) ? 1u : 0u;
-                if (flag) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) q_fp[i] = q_int[i];
-                }
-            }
-            sbyte = sb | (flag << 7);                                                 // S3
-            pack_codes<B>(q_fp, w);                                                   // S4
+        uint32_t rnd[8];
+        if constexpr (SR) {
+            const uint64_t i8 = (uint64_t)g * 2u;
+            uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
+            uint4 p1 = philox4x32_10((uint32_t)(i8 + 1), (uint32_t)((i8 + 1) >> 32), seed_lo, seed_hi);
+            rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;
+            rnd[4] = p1.x; rnd[5] = p1.y; rnd[6] = p1.z; rnd[7] = p1.w;
         }
-        scales[g] = (uint8_t)sbyte;
+
+        // One or two groups (GROUP = 16 or 8 values per scale) inside the aligned block of 16.
+        uint32_t chosen[16];
+#pragma unroll
+        for (int sub = 0; sub < NSUB; ++sub) {
+            const int e0i = sub * G;
+            // G1-G3 (Eq. 2, steps 1-2).
+            float gmax = 0.0f;
+#pragma unroll
+            for (int i = 0; i < G; ++i) gmax = fmaxf(gmax, fabsf(x[e0i + i]));
+            const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
+            const uint32_t sb = e4m3_encode(t);
+            uint32_t sbyte = 0u;
+#pragma unroll
+            for (int i = 0; i < G; ++i) chosen[e0i + i] = 0u;
+            if (sb != 0u) {                                                           // G4
+                const float d = __fmul_rn(e4m3_value(sb), alpha);                     // G5
+                const float r = __frcp_rn(d);
+                const float d_int = __fmul_rn(d, c_post);
+                uint32_t q_fp[G], q_int[G];
+                float s_fp[4] = {0.f, 0.f, 0.f, 0.f}, s_int[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int i = 0; i < G; i += 2) {
+                    const float x0 = x[e0i + i], x1 = x[e0i + i + 1];
+                    float y0 = __fmul_rn(x0, r), y1 = __fmul_rn(x1, r);                // E1 (step 3)
+                    float u0 = 0.f, u1 = 0.f;
+                    float yq0 = y0, yq1 = y1;
+                    if constexpr (SR) {
+                        const uint32_t rw = rnd[(e0i + i) >> 1];
+                        u0 = __fmul_rn(__fadd_rn((float)(rw & 0xFFFFu), 0.5f), 1.0f / 65536.0f);
+                        u1 = __fmul_rn(__fadd_rn((float)(rw >> 16), 0.5f), 1.0f / 65536.0f);
+                        yq0 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y0), F::M_FP, u0), y0);
+                        yq1 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y1), F::M_FP, u1), y1);
+                    }
+                    float v0, v1;
+                    fp_encode_pair<F::EK>(yq0, yq1, q_fp[i], q_fp[i + 1], v0, v1);     // E2 (step 4)
+                    const int chain = ((i >> 3) << 1);                                 // elements 0-7 -> S0,S1; 8-15 -> S2,S3
+                    if constexpr (F::HAS_INT) {
+                        const float e0 = __fmaf_rn(v0, d, -x0), e1 = __fmaf_rn(v1, d, -x1);   // E3 (steps 5-6)
+                        s_fp[chain] = __fmaf_rn(e0, e0, s_fp[chain]);
+                        s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
+                        const float z0 = __fmul_rn(y0, c_pre), z1 = __fmul_rn(y1, c_pre);     // E4 (step 7)
+                        float k0, k1;
+                        if constexpr (SR) {
+                            k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
+                            k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
+                        } else {
+                            // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
+                            k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);
+                            k1 = __fsub_rn(__fmaf_rn(y1, c_pre, 12582912.0f), 12582912.0f);
+                            k0 = fminf(fmaxf(k0, -F::M_INT), F::M_INT);
+                            k1 = fminf(fmaxf(k1, -F::M_INT), F::M_INT);
+                        }
+                        const float f0 = __fmaf_rn(k0, d_int, -x0), f1 = __fmaf_rn(k1, d_int, -x1);   // E5 (steps 8-9)
+                        s_int[chain] = __fmaf_rn(f0, f0, s_int[chain]);
+                        s_int[chain + 1] = __fmaf_rn(f1, f1, s_int[chain + 1]);
+                        q_int[i] = (uint32_t)__float2int_rn(k0) & ((1u << B) - 1u);
+                        q_int[i + 1] = (uint32_t)__float2int_rn(k1) & ((1u << B) - 1u);
+                    }
+                }
+                uint32_t flag = 0u;
+                if constexpr (F::HAS_INT) {                                            // S1-S2 (step 10)
+                    // a group of 8 leaves the last two chains at +0, so this is S0 + S1 for it
+                    const float E_fp = __fadd_rn(__fadd_rn(s_fp[0], s_fp[1]), __fadd_rn(s_fp[2], s_fp[3]));
+                    const float E_int = __fadd_rn(__fadd_rn(s_int[0], s_int[1]), __fadd_rn(s_int[2], s_int[3]));
+                    flag = (E_int < E_fp) ? 1u : 0u;
+                }
+#pragma unroll
+                for (int i = 0; i < G; ++i) chosen[e0i + i] = (F::HAS_INT && flag) ? q_int[i] : q_fp[i];
+                sbyte = sb | (flag << 7);                                             // S3
+            }
+            scales[g * NSUB + sub] = (uint8_t)sbyte;
+        }
+        uint32_t w[3];
+        pack_codes<B>(chosen, w);                                                     // S4
         if constexpr (B == 4) {
             *reinterpret_cast<uint2*>(codes + g * 8) = make_uint2(w[0], w[1]);
         } else if constexpr (B == 6) {
@@ -238,7 +244,7 @@ __global__ void __launch_bounds__(kThreads) dequantize_kernel(const uint8_t* __r
                                                               const float* __restrict__ alpha_p, int64_t ngroups,
                                                               void* __restrict__ out) {
     using F = Fmt<FMT>;
-    constexpr int B = F::BITS;
+    constexpr int B = F::BITS, G = F::GROUP, NSUB = 16 / G;
     pdl_launch_dependents();
     pdl_wait();
     const float alpha = __ldg(alpha_p);
@@ -256,15 +262,24 @@ __global__ void __launch_bounds__(kThreads) dequantize_kernel(const uint8_t* __r
             const uint16_t* p = reinterpret_cast<const uint16_t*>(codes + g * 6);
             w[0] = (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 16); w[1] = (uint32_t)__ldg(p + 2);
         }
-        const uint32_t sbyte = __ldg(scales + g);
-        const uint32_t flag = sbyte >> 7, mag = sbyte & 0x7Fu;
-        float Delta = e4m3_value(mag);
-        if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
-        float d = __fmul_rn(Delta, alpha);
-        if (F::HAS_INT && flag) d = __fmul_rn(d, c_post);              // de-scale integer groups (Sec. 3)
+        uint32_t flags[NSUB];
+        float ds[NSUB];
+#pragma unroll
+        for (int sub = 0; sub < NSUB; ++sub) {
+            const uint32_t sbyte = __ldg(scales + g * NSUB + sub);
+            const uint32_t mag = sbyte & 0x7Fu;
+            flags[sub] = sbyte >> 7;
+            float Delta = e4m3_value(mag);
+            if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
+            float d = __fmul_rn(Delta, alpha);
+            if (F::HAS_INT && flags[sub]) d = __fmul_rn(d, c_post);        // de-scale integer groups (Sec. 3)
+            ds[sub] = d;
+        }
         float o[16];
 #pragma unroll
         for (int i = 0; i < 16; i += 2) {
+            const uint32_t flag = flags[i / G];
+            const float d = ds[i / G];
             const uint32_t c0 = extract_code<B>(w, i), c1 = extract_code<B>(w, i + 1);
             float v0, v1;
             if (F::HAS_INT && flag) {
@@ -361,18 +376,20 @@ abs_status_t device_state(DeviceState** out) {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+int fmt_group(int fmt) { return (fmt >= ABS_FMT_NVFP4_BS8 && fmt <= ABS_FMT_IF3_BS8) ? 8 : 16; }
+
 int fmt_bits(int fmt) {
     switch (fmt) {
-        case ABS_FMT_NVFP4: case ABS_FMT_IF4: return 4;
-        case ABS_FMT_IF3: return 3;
+        case ABS_FMT_NVFP4: case ABS_FMT_IF4: case ABS_FMT_NVFP4_BS8: case ABS_FMT_IF4_BS8: return 4;
+        case ABS_FMT_IF3: case ABS_FMT_IF3_BS8: return 3;
         case ABS_FMT_IF6_E2M3: case ABS_FMT_IF6_E3M2: return 6;
         default: return 0;
     }
 }
 float fmt_mfp(int fmt) {
     switch (fmt) {
-        case ABS_FMT_NVFP4: case ABS_FMT_IF4: return 6.0f;
-        case ABS_FMT_IF3: return 4.0f;
+        case ABS_FMT_NVFP4: case ABS_FMT_IF4: case ABS_FMT_NVFP4_BS8: case ABS_FMT_IF4_BS8: return 6.0f;
+        case ABS_FMT_IF3: case ABS_FMT_IF3_BS8: return 4.0f;
         case ABS_FMT_IF6_E2M3: return 7.5f;
         default: return 28.0f;
     }
@@ -591,7 +608,7 @@ size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
 
 size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
     if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
-    return (size_t)rows * (size_t)cols / 16;
+    return (size_t)rows * (size_t)cols / (size_t)fmt_group((int)fmt);
 }
 
 const char* abs_status_string(abs_status_t status) {
@@ -681,7 +698,10 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
         case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
         case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
         case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        default: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        default: return launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
     }
 }
 
@@ -729,7 +749,10 @@ abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t ro
         case ABS_FMT_IF4: return launch_quantize_fmt<1>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
         case ABS_FMT_IF3: return launch_quantize_fmt<2>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
         case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        default: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        default: return launch_quantize_fmt<7>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
     }
 }
 
@@ -755,7 +778,10 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
         case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        default: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF6_E3M2: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_NVFP4_BS8: return launch_dequantize_fmt<5>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF4_BS8: return launch_dequantize_fmt<6>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        default: return launch_dequantize_fmt<7>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
     }
 }
 
@@ -771,7 +797,7 @@ static size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
 size_t abs_host_workspace_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
     if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
     const size_t n = (size_t)rows * (size_t)cols;
-    return round256(n * 4) + round256(abs_codes_bytes(fmt, rows, cols)) + round256(n / 16) + 256;
+    return round256(n * 4) + round256(abs_codes_bytes(fmt, rows, cols)) + round256(abs_scales_bytes(fmt, rows, cols)) + 256;
 }
 
 abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t rows, int64_t cols,
@@ -784,7 +810,7 @@ abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t 
     if (!aligned16(d_workspace)) return ABS_ERR_ALIGN;
     if (workspace_bytes < abs_host_workspace_bytes(fmt, rows, cols)) return ABS_ERR_SIZE;
     const size_t n = (size_t)rows * (size_t)cols;
-    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = n / 16;
+    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = abs_scales_bytes(fmt, rows, cols);
     uint8_t* base = (uint8_t*)d_workspace;
     uint8_t* d_in = base;
     uint8_t* d_codes = d_in + round256(n * 4);
@@ -812,7 +838,7 @@ abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const
     if (!aligned16(d_workspace)) return ABS_ERR_ALIGN;
     if (workspace_bytes < abs_host_workspace_bytes(fmt, rows, cols)) return ABS_ERR_SIZE;
     const size_t n = (size_t)rows * (size_t)cols;
-    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = n / 16;
+    const size_t cb = abs_codes_bytes(fmt, rows, cols), sb = abs_scales_bytes(fmt, rows, cols);
     const bool fp32 = opts && (opts->flags & ABS_F_OUT_FP32);
     uint8_t* base = (uint8_t*)d_workspace;
     uint8_t* d_out = base;

@@ -16,25 +16,30 @@ enum ElemKind { EK_E2M1 = 0, EK_E2M0 = 1, EK_E2M3 = 2, EK_E3M2 = 3 };
 // Format traits: (M_FP, M_INT, bits) per Sec. 3 (IF4) and the Sec. 5.1 footnote (IF3, IF6).
 template <int FMT> struct Fmt;
 template <> struct Fmt<0> {  // NVFP4: Fig. 3a stops after step 4
-    static constexpr int BITS = 4; static constexpr bool HAS_INT = false; static constexpr ElemKind EK = EK_E2M1;
+    static constexpr int BITS = 4; static constexpr int GROUP = 16; static constexpr bool HAS_INT = false; static constexpr ElemKind EK = EK_E2M1;
     static constexpr float M_FP = 6.0f, M_INT = 0.0f; static constexpr int EMIN = 0, MBITS = 1;
 };
 template <> struct Fmt<1> {  // IF4
-    static constexpr int BITS = 4; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M1;
+    static constexpr int BITS = 4; static constexpr int GROUP = 16; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M1;
     static constexpr float M_FP = 6.0f, M_INT = 7.0f; static constexpr int EMIN = 0, MBITS = 1;
 };
 template <> struct Fmt<2> {  // IF3: E2M0 or INT3
-    static constexpr int BITS = 3; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M0;
+    static constexpr int BITS = 3; static constexpr int GROUP = 16; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M0;
     static constexpr float M_FP = 4.0f, M_INT = 3.0f; static constexpr int EMIN = 0, MBITS = 0;
 };
 template <> struct Fmt<3> {  // IF6-E2M3
-    static constexpr int BITS = 6; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M3;
+    static constexpr int BITS = 6; static constexpr int GROUP = 16; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E2M3;
     static constexpr float M_FP = 7.5f, M_INT = 31.0f; static constexpr int EMIN = 0, MBITS = 3;
 };
 template <> struct Fmt<4> {  // IF6-E3M2
-    static constexpr int BITS = 6; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E3M2;
+    static constexpr int BITS = 6; static constexpr int GROUP = 16; static constexpr bool HAS_INT = true; static constexpr ElemKind EK = EK_E3M2;
     static constexpr float M_FP = 28.0f, M_INT = 31.0f; static constexpr int EMIN = -2, MBITS = 2;
 };
+
+// Block-size-8 variants (Sec. 5.1, Table 5): the same element formats with one scale per 8 values.
+template <> struct Fmt<5> : Fmt<0> { static constexpr int GROUP = 8; };   // NVFP4-BS8
+template <> struct Fmt<6> : Fmt<1> { static constexpr int GROUP = 8; };   // IF4-BS8
+template <> struct Fmt<7> : Fmt<2> { static constexpr int GROUP = 8; };   // IF3-BS8
 
 // ----------------------------------------------------------------------------- conversions
 

@@ -45,7 +45,8 @@ def main():
         ("cfg3a", 4096, 14336, [("if4", 0), ("nvfp4", 0)]),
         ("cfg3b", 14336, 4096, [("if4", 0), ("nvfp4", 0)]),
         ("cfg4", 16384, 8192, [("if4", H | S | S17), ("if4", H | S), ("if4", S), ("if4", H), ("nvfp4", H | S | S17)]),
-        ("cfg5", 16384, 8192, [("if3", 0), ("if4", 0), ("if6_e2m3", 0), ("if6_e3m2", 0), ("nvfp4", 0)]),
+        ("cfg5", 16384, 8192, [("if3", 0), ("if4", 0), ("if6_e2m3", 0), ("if6_e3m2", 0), ("nvfp4", 0),
+                               ("if4_bs8", 0), ("if3_bs8", 0), ("nvfp4_bs8", 0)]),
     ]
     sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     for name, rows, cols, variants in rows_cfg:
@@ -57,7 +58,7 @@ def main():
             fmt = B.FMT_NAMES[fname]
             bits = B.FMT_BITS[fmt]
             codes = [torch.empty(n * bits // 8, dtype=torch.uint8, device="cuda") for _ in range(k)]
-            scales = [torch.empty(n // 16, dtype=torch.uint8, device="cuda") for _ in range(k)]
+            scales = [torch.empty(n // B.FMT_GROUP[fmt], dtype=torch.uint8, device="cuda") for _ in range(k)]
             ts = [torch.zeros(1, dtype=torch.float32, device="cuda") for _ in range(k)]
             outs = [torch.empty(rows, cols, dtype=torch.bfloat16, device="cuda") for _ in range(min(k, 4))]
             o_full = B.make_opts(flags, 0x5A3C, 1234)
@@ -74,7 +75,7 @@ def main():
             t1 = loop_time(lambda i: L.abs_quantize_ex(*qa[i % k]))
             t2 = loop_time(lambda i: L.abs_quantize_ex(*fa[i % k]))
             t3 = loop_time(lambda i: L.abs_dequantize(*da[i % k]))
-            outb = n * bits / 8 + n / 16
+            outb = n * bits / 8 + n / B.FMT_GROUP[fmt]
             opt = "+".join(s for s, f in (("hadamard", H), ("sr", S), ("17/16", S17)) if flags & f) or "rtn"
             print(json.dumps({
                 "config": name, "shape": [rows, cols], "fmt": fname, "options": opt,

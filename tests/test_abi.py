@@ -38,7 +38,9 @@ def test_sizes(B):
     assert B.abs_codes_bytes(B.ABS_FMT_IF6_E2M3, 2, 32) == 48
     assert B.abs_codes_bytes(B.ABS_FMT_IF6_E3M2, 2, 32) == 48
     assert B.abs_scales_bytes(B.ABS_FMT_IF4, 8192, 4096) == 8192 * 4096 // 16
-    assert B.abs_codes_bytes(B.ABS_FMT_IF4, 2, 30) == 0 and B.abs_codes_bytes(7, 2, 32) == 0
+    assert B.abs_scales_bytes(B.ABS_FMT_IF4_BS8, 8192, 4096) == 8192 * 4096 // 8
+    assert B.abs_codes_bytes(B.ABS_FMT_IF4_BS8, 2, 32) == 32 and B.abs_codes_bytes(B.ABS_FMT_IF3_BS8, 2, 32) == 24
+    assert B.abs_codes_bytes(B.ABS_FMT_IF4, 2, 30) == 0 and B.abs_codes_bytes(17, 2, 32) == 0
     assert B.abs_codes_bytes(B.ABS_FMT_IF4, -2, 32) == 0
     assert B.abs_host_workspace_bytes(B.ABS_FMT_IF4, 16, 64) >= 16 * 64 * 2 + 16 * 64 // 2 + 64 + 4
 
@@ -60,7 +62,7 @@ def test_alpha_from_amax_is_eq1(B):
 def test_host_side_validation_needs_no_gpu(B):
     L = B.lib()
     dummy = ctypes.c_void_p(0x1000)      # never dereferenced: validation fails first
-    assert L.abs_quantize(9, dummy, 4, 64, dummy, dummy, dummy, None) == 4      # format
+    assert L.abs_quantize(19, dummy, 4, 64, dummy, dummy, dummy, None) == 4     # format
     assert L.abs_quantize(1, dummy, 4, 60, dummy, dummy, dummy, None) == 2      # cols % 16
     assert L.abs_quantize(1, dummy, -4, 64, dummy, dummy, dummy, None) == 2
     assert L.abs_quantize(1, None, 4, 64, dummy, dummy, dummy, None) == 1       # null
