@@ -110,6 +110,18 @@ ABS_API abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t ro
 ABS_API abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                              void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream);
 
+/* Quantize the transpose (Sec. 4.1: for the weight-gradient product both operands are quantized along
+ * the token dimension, i.e. down the columns of a [tokens, features] matrix).  `in_bf16` is the same
+ * row-major [rows, cols] matrix as for abs_quantize; the outputs are exactly what abs_quantize would
+ * give for its transpose [cols, rows]: groups are 16 consecutive rows of one column,
+ *   codes_t_u8    [cols, rows*b/8]   scales_t_e4m3 [cols, rows/16]   alpha as for abs_quantize.
+ * The transpose is never materialised.  rows and cols must be multiples of 16; formats ABS_FMT_IF4 and
+ * ABS_FMT_NVFP4; the only flag accepted is ABS_F_ALPHA_GIVEN.  abs_dequantize(fmt, ..., cols, rows, ...)
+ * turns the result back into the transposed matrix. */
+ABS_API abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
+                                             void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
+                                             const abs_opts_t* opts, void* stream);
+
 /* Quantize without any allocation.  (The paper has no counterpart: this entry point exists for the
  * way the library is deployed, not for the method.)
  *

@@ -31,7 +31,7 @@ EXPORTS = [
     "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
-    "abs_quantize_noalloc",
+    "abs_quantize_noalloc", "abs_quantize_transposed",
 ]
 
 
@@ -76,6 +76,8 @@ def lib():
             L.abs_quantize.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
             L.abs_quantize_ex.restype = C.c_int
             L.abs_quantize_ex.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
+            L.abs_quantize_transposed.restype = C.c_int
+            L.abs_quantize_transposed.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
             L.abs_quantize_noalloc.restype = C.c_int
             L.abs_quantize_noalloc.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
             L.abs_dequantize.restype = C.c_int
@@ -157,6 +159,27 @@ def abs_quantize(fmt: int, x, codes=None, scales=None, tensor_scale=None, opts: 
                                _stream_ptr(stream))
     _check(rc, "abs_quantize")
     return codes, scales, tensor_scale
+
+
+def abs_quantize_transposed(fmt: int, x, codes_t=None, scales_t=None, tensor_scale=None, opts: AbsOpts | None = None,
+                            stream=None):
+    """Quantize the transpose of the CUDA bf16 matrix ``x`` [rows, cols] (groups of 16 down the columns)
+    without materialising it.  Returns (codes_t u8 [cols*rows*b/8], scales_t u8 [cols*rows/16], alpha)."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    rows, cols = x.shape
+    if codes_t is None:
+        codes_t = torch.empty(max(rows * cols * FMT_BITS[fmt] // 8, 1), dtype=torch.uint8, device=x.device)
+    if scales_t is None:
+        scales_t = torch.empty(max(rows * cols // 16, 1), dtype=torch.uint8, device=x.device)
+    if tensor_scale is None:
+        tensor_scale = torch.zeros(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        rc = lib().abs_quantize_transposed(fmt, x.data_ptr(), rows, cols, codes_t.data_ptr(), scales_t.data_ptr(),
+                                           tensor_scale.data_ptr(), C.byref(opts) if opts is not None else None,
+                                           _stream_ptr(stream))
+    _check(rc, "abs_quantize_transposed")
+    return codes_t, scales_t, tensor_scale
 
 
 def abs_quantize_noalloc(fmt: int, x, codes, scales, tensor_scale, stream=None):

@@ -711,6 +711,58 @@ abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int6
 }
 
 
+abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
+                                     void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
+                                     const abs_opts_t* opts, void* stream) {
+    abs_opts_t o = {0, 0, 0, 0};
+    if (opts) o = *opts;
+    if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
+    if (rows < 0 || cols < 0 || (cols % 16) != 0 || (rows % 16) != 0) return ABS_ERR_SHAPE;
+    if ((o.flags & ~(uint32_t)ABS_F_ALPHA_GIVEN) || o._pad) return ABS_ERR_FLAGS;
+    if (rows * cols == 0) return ABS_OK;
+    if (!in_bf16 || !codes_t_u8 || !scales_t_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
+    if (!aligned16(in_bf16) || !aligned16(codes_t_u8) || !aligned16(scales_t_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
+        return ABS_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t ngroups = rows * cols / 16;
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
+        unsigned long long* slot = nullptr;
+        uint32_t gen = 0;
+        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        const float denom = 6.0f * 448.0f;
+        abs_status_t rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+        if (rc != ABS_OK) return rc;
+        src.slot = slot;
+        src.gen = gen;
+        src.denom = denom;
+    }
+    const int64_t rblocks = rows / 16;
+    cudaLaunchConfig_t cfg = {};
+    const int64_t tiles_y = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
+    cfg.gridDim = dim3((unsigned)((cols + kTransTileCols - 1) / kTransTileCols), (unsigned)(tiles_y < 65535 ? tiles_y : 65535));
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    const uint16_t* in = (const uint16_t*)in_bf16;
+    uint2* ct = (uint2*)codes_t_u8;
+    uint8_t* stp = (uint8_t*)scales_t_e4m3;
+    if (fmt == ABS_FMT_IF4)
+        e = src.slot ? cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<true, true>, in, ct, stp, src, rows, cols)
+                     : cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<true, false>, in, ct, stp, src, rows, cols);
+    else
+        e = src.slot ? cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<false, true>, in, ct, stp, src, rows, cols)
+                     : cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<false, false>, in, ct, stp, src, rows, cols);
+    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
+}
+
 abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                                   void* scales_e4m3, float* tensor_scale_f32, void* stream) {
     abs_status_t rc = check_shape(fmt, rows, cols);

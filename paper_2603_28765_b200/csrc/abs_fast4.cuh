@@ -221,6 +221,92 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
 }
 
 
+// ----------------------------------------------------------------------------- transposed quantize
+
+// Quantizes the TRANSPOSE of a row-major [rows, cols] matrix without materialising it: groups are 16
+// consecutive ROWS of one column (Sec. 4.1: both operands of the weight-gradient product are quantized
+// along the token dimension).  Output = what the plain kernel would give for the [cols, rows] matrix:
+// codes_t [cols, rows/2 bytes], scales_t [cols, rows/16].
+// A block stages a tile of 64 rows x 256 columns in shared memory with coalesced 128-bit loads; thread
+// c then encodes the four groups of its column (rows 0-15, 16-31, 32-47, 48-63 of the tile), reading its
+// values down the column.  Those four groups are neighbours in the transposed output, so their codes
+// leave as one 256-bit store and their scale bytes as one 32-bit store whenever the tile is complete
+// and the output addresses allow it.
+constexpr int kTransTileCols = 256;
+constexpr int kTransTileRowBlocks = 4;
+
+template <bool HAS_INT, bool FROM_SLOT>
+__global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_t* __restrict__ in,
+                                                                   uint2* __restrict__ codes_t,
+                                                                   uint8_t* __restrict__ scales_t,
+                                                                   const AlphaSrc alpha_src, int64_t rows, int64_t cols) {
+    __shared__ __align__(16) uint16_t tile[16 * kTransTileRowBlocks][kTransTileCols];
+    pdl_launch_dependents();
+    pdl_wait();
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
+    const int64_t rblocks = rows / 16;
+    const int64_t c0 = (int64_t)blockIdx.x * kTransTileCols;
+    const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);          // multiple of 16
+    const int64_t ntiles_y = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
+    // vector stores need 32-byte aligned code addresses and 4-byte aligned scale addresses for every column
+    const bool vec_ok = (rblocks % kTransTileRowBlocks) == 0 &&
+                        ((reinterpret_cast<uintptr_t>(codes_t) & 31u) == 0) && ((reinterpret_cast<uintptr_t>(scales_t) & 3u) == 0);
+    for (int64_t ty = blockIdx.y; ty < ntiles_y; ty += gridDim.y) {
+        const int64_t rb0 = ty * kTransTileRowBlocks;
+        const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
+        const int chunks_per_row = ncols / 8;
+        for (int ch = threadIdx.x; ch < 16 * nrb * chunks_per_row; ch += blockDim.x) {
+            const int r = ch / chunks_per_row, q = ch - r * chunks_per_row;
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(in + (rb0 * 16 + r) * cols + c0) + q);
+            *reinterpret_cast<uint4*>(&tile[r][q * 8]) = v;
+        }
+        __syncthreads();
+        const int c = threadIdx.x;
+        if (c < ncols) {
+            uint32_t cw[2 * kTransTileRowBlocks];
+            uint32_t sbytes = 0u;
+#pragma unroll 1
+            for (int k = 0; k < nrb; ++k) {
+                float x[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) x[i] = __uint_as_float((uint32_t)tile[16 * k + i][c] << 16);
+                const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
+                const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
+                const float m4 = max3abs(x[12], x[13], x[14]);
+                const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));   // G1
+                const float t = __fmul_rn(gmax, inv_a6);                                 // G2
+                const uint32_t sb = e4m3_encode(t);                                      // G3
+                const float d = __fmul_rn(e4m3_value(sb), alpha);                        // G5
+                const float r = __frcp_rn(d);
+                uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
+                if ((sb - 8u) >= 118u) {
+                    if (sb != 0u) encode_body4<HAS_INT, HAS_INT>(x, sb, d, r, sbyte, c_lo, c_hi);
+                } else {
+                    encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
+                }
+                const int64_t g = (c0 + c) * rblocks + rb0 + k;      // group index in the transposed matrix
+                if (vec_ok) {
+                    // k is a runtime index: select the slot without dynamic register indexing
+#pragma unroll
+                    for (int j = 0; j < kTransTileRowBlocks; ++j)
+                        if (j == k) { cw[2 * j] = c_lo; cw[2 * j + 1] = c_hi; }
+                    sbytes |= sbyte << (8 * k);
+                } else {
+                    scales_t[g] = (uint8_t)sbyte;
+                    codes_t[g] = make_uint2(c_lo, c_hi);
+                }
+            }
+            if (vec_ok) {
+                const int64_t g0 = (c0 + c) * rblocks + rb0;
+                store32B<true>(codes_t + g0, reinterpret_cast<const uint32_t(&)[8]>(cw));
+                *reinterpret_cast<uint32_t*>(scales_t + g0) = sbytes;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // ----------------------------------------------------------------------------- 4-bit dequantize
 
 // FP32 -> packed bf16 pair, round to nearest even (Sec. 4.1).

@@ -419,3 +419,36 @@ def test_sr_bias_signature_on_gpu(B):
     assert top["share"] < 0.12
     for lo in (0.1, 0.2, 0.3, 0.4):
         assert abs(i4[lo]["mean_change_over_gmax"]) < 6e-3, (lo, i4[lo])
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_transposed_quantize_equals_quantize_of_transpose(B, oracle, fmt):
+    """abs_quantize_transposed(X) must give the bytes the oracle gives for X^T (the plain definition),
+    on shapes with several column tiles, a ragged last tile and many row blocks; dequantizing with
+    swapped dimensions returns the transposed matrix's dequantization."""
+    for name, rows, cols in (("cfg2", 304, 4096), ("cfg3a", 64, 14336), ("cfg5", 2048, 1040), ("cfg1", 16, 16)):
+        xb = I.generate(name, rows, cols)
+        xt = np.ascontiguousarray(xb.T)
+        ct, st, ts = B.abs_quantize_transposed(fmt, to_dev(xb))
+        torch.cuda.synchronize()
+        oc, osc, oa = oracle.quantize(fmt, xt, threads=THREADS)
+        assert np.float32(ts.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+        assert_same("scales_t", st.cpu().numpy().reshape(cols, -1), osc)
+        assert_same("codes_t", ct.cpu().numpy().reshape(cols, -1), oc)
+        out = B.abs_dequantize(fmt, ct, st, ts, cols, rows)
+        assert_same("dequant_t", out.view(torch.int16).cpu().numpy().view(np.uint16),
+                    oracle.dequantize(fmt, oc, osc, oa, cols, rows, threads=THREADS))
+    # alpha given, and the argument checks
+    xb = I.generate("cfg5", 64, 256)
+    ts = torch.tensor([0.02], dtype=torch.float32, device="cuda")
+    ct, st, _ = B.abs_quantize_transposed(fmt, to_dev(xb), tensor_scale=ts, opts=B.make_opts(B.ABS_F_ALPHA_GIVEN))
+    oc, osc, _ = oracle.quantize(fmt, np.ascontiguousarray(xb.T), flags=oracle.F_ALPHA_GIVEN, alpha=0.02)
+    assert_same("codes_t", ct.cpu().numpy().reshape(256, -1), oc)
+    L = B.lib()
+    x = to_dev(xb)
+    assert L.abs_quantize_transposed(2, x.data_ptr(), 64, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(), None, None) == 4
+    assert L.abs_quantize_transposed(1, x.data_ptr(), 40, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(), None, None) == 2
+    import ctypes
+    sr = B.make_opts(B.ABS_F_STOCHASTIC)
+    assert L.abs_quantize_transposed(1, x.data_ptr(), 64, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(),
+                                     ctypes.byref(sr), None) == 5
