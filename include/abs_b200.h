@@ -75,6 +75,9 @@ enum {
                                        the 16/17 factor of Sec. 4.1, so stochastic values never clip     */
     ABS_F_ALPHA_GIVEN = 1u << 3,    /* quantize: *tensor_scale_f32 is an input; the amax pass is skipped */
     ABS_F_OUT_FP32 = 1u << 4,       /* dequantize: write the FP32 products instead of bf16               */
+    ABS_F_SCALES_SWIZZLED = 1u << 6, /* quantize / dequantize, ABS_FMT_NVFP4 and ABS_FMT_IF4 only: the scale array uses
+                                       the 128x4-tile layout that Blackwell block-scaled tensor-core MMAs read
+                                       (see abs_scales_bytes_swizzled) instead of row-major [rows, cols/16]      */
     ABS_F_INDEX64 = 1u << 5         /* testing aid: run the kernel instances that index groups with 64-bit
                                        integers (otherwise chosen only beyond 2^31 groups); same results  */
 };
@@ -93,6 +96,14 @@ typedef struct {
 ABS_API size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
 ABS_API size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
 ABS_API const char* abs_status_string(abs_status_t status);
+
+/* Size of the scale array with ABS_F_SCALES_SWIZZLED.  (Sec. 3 notes that a group stored as FP4 is an
+ * NVFP4 group; this option stores the scales where NVFP4 tensor-core kernels expect them.)  The scale of
+ * row r, group k (k = column / 16) lives at byte
+ *     ((r / 128) * ceil(K / 4) + k / 4) * 512 + (r % 32) * 16 + ((r % 128) / 32) * 4 + k % 4,   K = cols / 16,
+ * i.e. tiles of 128 rows x 4 scales, 512 bytes each, tiles ordered row-major.  The array is padded to whole
+ * tiles: ceil(rows / 128) * ceil(K / 4) * 512 bytes; the library never writes the padding bytes. */
+ABS_API size_t abs_scales_bytes_swizzled(abs_fmt_t fmt, int64_t rows, int64_t cols);
 
 /* Allocates the per-device scratch ring of `device` now (synchronous).  Optional: the first
  * quantize call on a device does the same. */

@@ -279,3 +279,18 @@ def dequantize(fmt: int, codes, scales, alpha, rows: int, cols: int, out_fp32: b
 def bf16_bits_to_f32(bits) -> np.ndarray:
     """Exact widening of bf16 bit patterns to float32 (a dtype view, no rounding)."""
     return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def swizzle_scales(scales: np.ndarray, fill: int = 0) -> np.ndarray:
+    """Row-major scale bytes [rows, K] -> the 128x4-tile layout that Blackwell block-scaled tensor-core
+    MMAs read (the layout NVFP4 kernels use for their E4M3 scales; Sec. 3: an FP group IS an NVFP4
+    group).  Written as the layout's definition: pad to whole 128 x 4 tiles; tiles in row-major order;
+    inside a tile the 128 rows are split as (row // 32, row % 32) and stored with row % 32 slowest,
+    then row // 32, then the 4 scales of the row.  Padding bytes get ``fill``."""
+    s = np.asarray(scales, dtype=np.uint8)
+    rows, k = s.shape
+    mt, kt = -(-rows // 128), -(-k // 4)
+    padded = np.full((mt * 128, kt * 4), fill, dtype=np.uint8)
+    padded[:rows, :k] = s
+    tiles = padded.reshape(mt, 4, 32, kt, 4)           # [tile row, row // 32, row % 32, tile col, scale]
+    return np.ascontiguousarray(tiles.transpose(0, 3, 2, 1, 4)).reshape(-1)   # [mt, kt, row % 32, row // 32, scale]

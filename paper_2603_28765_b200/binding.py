@@ -24,6 +24,7 @@ ABS_F_SR_SCALE_17_16 = 1 << 2
 ABS_F_ALPHA_GIVEN = 1 << 3
 ABS_F_OUT_FP32 = 1 << 4
 ABS_F_INDEX64 = 1 << 5
+ABS_F_SCALES_SWIZZLED = 1 << 6
 
 ABS_OK = 0
 
@@ -31,7 +32,7 @@ EXPORTS = [
     "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
-    "abs_quantize_noalloc", "abs_quantize_transposed",
+    "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled",
 ]
 
 
@@ -68,6 +69,8 @@ def lib():
             L.abs_codes_bytes.argtypes = [C.c_int, i64, i64]
             L.abs_scales_bytes.restype = sz
             L.abs_scales_bytes.argtypes = [C.c_int, i64, i64]
+            L.abs_scales_bytes_swizzled.restype = sz
+            L.abs_scales_bytes_swizzled.argtypes = [C.c_int, i64, i64]
             L.abs_status_string.restype = C.c_char_p
             L.abs_status_string.argtypes = [C.c_int]
             L.abs_init.restype = C.c_int
@@ -129,6 +132,10 @@ def abs_scales_bytes(fmt: int, rows: int, cols: int) -> int:
     return lib().abs_scales_bytes(fmt, rows, cols)
 
 
+def abs_scales_bytes_swizzled(fmt: int, rows: int, cols: int) -> int:
+    return lib().abs_scales_bytes_swizzled(fmt, rows, cols)
+
+
 def abs_alpha_from_amax(fmt: int, amax: float) -> float:
     return lib().abs_alpha_from_amax(fmt, amax)
 
@@ -150,7 +157,10 @@ def abs_quantize(fmt: int, x, codes=None, scales=None, tensor_scale=None, opts: 
         codes = torch.empty(max(L.abs_codes_bytes(fmt, rows, cols), 1) if cols % 16 == 0 else 1, dtype=torch.uint8,
                             device=x.device)
     if scales is None:
-        scales = torch.empty(max(rows * cols // FMT_GROUP[fmt], 1), dtype=torch.uint8, device=x.device)
+        if opts is not None and (opts.flags & ABS_F_SCALES_SWIZZLED):
+            scales = torch.zeros(max(L.abs_scales_bytes_swizzled(fmt, rows, cols), 1), dtype=torch.uint8, device=x.device)
+        else:
+            scales = torch.empty(max(rows * cols // FMT_GROUP[fmt], 1), dtype=torch.uint8, device=x.device)
     if tensor_scale is None:
         tensor_scale = torch.zeros(1, dtype=torch.float32, device=x.device)
     with torch.cuda.device(x.device):

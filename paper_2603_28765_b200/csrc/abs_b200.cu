@@ -395,8 +395,8 @@ float fmt_mfp(int fmt) {
     }
 }
 
-constexpr uint32_t kQuantFlags =
-    ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN | ABS_F_INDEX64;
+constexpr uint32_t kQuantFlags = ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN |
+                                 ABS_F_INDEX64 | ABS_F_SCALES_SWIZZLED;
 
 int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
     int64_t want = (work_items + kThreads - 1) / kThreads;
@@ -439,7 +439,7 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
 
 template <int FMT>
 abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
-                                 const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s) {
+                                 const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s, int64_t cols = 0) {
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const int grid = grid_for(st, ngroups, 64);
@@ -452,9 +452,13 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
             cudaError_t e;
+            const bool swz = o.flags & ABS_F_SCALES_SWIZZLED;
+            const uint32_t gpr = swz ? (uint32_t)(cols / 16) : 0u, ktiles = (gpr + 3u) / 4u;
 #define ABS_LAUNCH_F3(IDX, A32, SLOT, MUL)                                                                           \
-    e = launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL>, pgrid, kThreads, s, (const uint4*)in,            \
-                   (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups)
+    e = swz ? launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL, true>, pgrid, kThreads, s,                  \
+                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles)         \
+            : launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL, false>, pgrid, kThreads, s,                 \
+                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles)
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
     do {                                                                                                             \
         if (alpha.slot && mul != 1.0f) ABS_LAUNCH_F3(IDX, A32, true, true);                                          \
@@ -492,7 +496,8 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 
 template <int FMT>
 abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
-                                   int64_t ngroups, void* out, bool fp32, bool index64, cudaStream_t s) {
+                                   int64_t ngroups, void* out, bool fp32, bool index64, cudaStream_t s,
+                                   int64_t swz_cols = 0) {
     const int grid = grid_for(st, ngroups, 64);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
@@ -500,9 +505,13 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
             const bool i32 = !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
             cudaError_t e;
+            const bool swz = swz_cols > 0;
+            const uint32_t gpr = (uint32_t)(swz_cols / 16), ktiles = (gpr + 3u) / 4u;
 #define ABS_LAUNCH_D(IDX, A32)                                                                                      \
-    e = launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32>, grid, kThreads, s, (const uint2*)codes,                 \
-                   (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out)
+    e = swz ? launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32, true>, grid, kThreads, s, (const uint2*)codes,     \
+                         (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out, gpr, ktiles)                     \
+            : launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32, false>, grid, kThreads, s, (const uint2*)codes,    \
+                         (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out, gpr, ktiles)
             if (i32 && a32) ABS_LAUNCH_D(int32_t, true);
             else if (i32) ABS_LAUNCH_D(int32_t, false);
             else if (a32) ABS_LAUNCH_D(int64_t, true);
@@ -606,6 +615,12 @@ size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
     return (size_t)rows * (size_t)cols / 16 * (size_t)(2 * fmt_bits((int)fmt));
 }
 
+size_t abs_scales_bytes_swizzled(abs_fmt_t fmt, int64_t rows, int64_t cols) {
+    if (check_shape(fmt, rows, cols) != ABS_OK || (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4)) return 0;
+    const size_t k = (size_t)cols / 16;
+    return (((size_t)rows + 127) / 128) * ((k + 3) / 4) * 512;
+}
+
 size_t abs_scales_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
     if (check_shape(fmt, rows, cols) != ABS_OK) return 0;
     return (size_t)rows * (size_t)cols / (size_t)fmt_group((int)fmt);
@@ -673,6 +688,10 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if ((o.flags & ~kQuantFlags) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_SCALES_SWIZZLED) &&
+        ((fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) || (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC)) ||
+         cols / 16 > 0x7FFFFFFF || rows > 0x7FFFFFFF))
+        return ABS_ERR_FLAGS;      // the tiled scale layout exists for the 4-bit round-to-nearest kernels only
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !codes_u8 || !scales_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(codes_u8) || !aligned16(scales_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -694,14 +713,14 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
         src.denom = denom;
     }
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        default: return launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        default: return launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
     }
 }
 
@@ -815,7 +834,10 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
-    if ((o.flags & ~(uint32_t)(ABS_F_OUT_FP32 | ABS_F_INDEX64)) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ~(uint32_t)(ABS_F_OUT_FP32 | ABS_F_INDEX64 | ABS_F_SCALES_SWIZZLED)) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_SCALES_SWIZZLED) &&
+        ((fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) || (o.flags & ABS_F_OUT_FP32) || cols / 16 > 0x7FFFFFFF || rows > 0x7FFFFFFF))
+        return ABS_ERR_FLAGS;
     if (rows * cols == 0) return ABS_OK;
     if (!codes_u8 || !scales_e4m3 || !tensor_scale_f32 || !out) return ABS_ERR_NULL;
     if (!aligned16(codes_u8) || !aligned16(scales_e4m3) || !aligned16(out) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -825,9 +847,10 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
     const bool fp32 = o.flags & ABS_F_OUT_FP32, i64 = o.flags & ABS_F_INDEX64;
+    const int64_t swz_cols = (o.flags & ABS_F_SCALES_SWIZZLED) ? cols : 0;
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
+        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
         case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF6_E3M2: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);

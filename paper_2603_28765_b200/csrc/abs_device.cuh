@@ -258,6 +258,19 @@ __device__ __forceinline__ float resolve_alpha(const AlphaSrc& a) {
     return alpha_shared;
 }
 
+// Byte offset of the scale of (row, k-th group of the row) in the 128x4-tile layout read by Blackwell
+// block-scaled MMAs; ktiles = ceil(groups_per_row / 4).
+__device__ __forceinline__ size_t swizzled_scale_offset(uint32_t row, uint32_t k, uint32_t ktiles) {
+    return ((size_t)(row >> 7) * ktiles + (k >> 2)) * 512u + (row & 31u) * 16u + ((row >> 5) & 3u) * 4u + (k & 3u);
+}
+// Where group g's scale byte goes: row-major, or the tiled layout when `gpr` (groups per row) is non-zero.
+template <bool SWZ>
+__device__ __forceinline__ size_t scale_offset(size_t g, uint32_t gpr, uint32_t ktiles) {
+    if constexpr (!SWZ) return g;
+    const uint32_t row = (uint32_t)(g / gpr);
+    return swizzled_scale_offset(row, (uint32_t)(g - (size_t)row * gpr), ktiles);
+}
+
 // ----------------------------------------------------------------------------- unpack
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4& v, float* x) {

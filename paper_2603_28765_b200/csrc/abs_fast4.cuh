@@ -170,10 +170,10 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
 // Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
 // next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
 // IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
-template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT, bool SCALE_MUL>
+template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT, bool SCALE_MUL, bool SWZ>
 __global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
 quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                      const AlphaSrc alpha_src, IdxT ngroups) {
+                      const AlphaSrc alpha_src, IdxT ngroups, uint32_t gpr, uint32_t ktiles) {
     pdl_launch_dependents();
     const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
     IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x);
@@ -211,7 +211,7 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
         } else {
             encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
         }
-        scales[g] = (uint8_t)sbyte;
+        scales[scale_offset<SWZ>((size_t)g, gpr, ktiles)] = (uint8_t)sbyte;
         codes[g] = make_uint2(c_lo, c_hi);
         if (!more) break;
 #pragma unroll
@@ -361,11 +361,11 @@ __device__ __forceinline__ void dequant_word4(uint32_t w, bool is_int, float add
     }
 }
 
-template <bool HAS_INT, typename IdxT, bool ALIGNED32>
+template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool SWZ>
 __global__ void __launch_bounds__(256) dequantize4_fast_kernel(const uint2* __restrict__ codes,
                                                                const uint8_t* __restrict__ scales,
                                                                const float* __restrict__ alpha_p, IdxT ngroups,
-                                                               uint4* __restrict__ out) {
+                                                               uint4* __restrict__ out, uint32_t gpr, uint32_t ktiles) {
     pdl_launch_dependents();
     const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
     const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
@@ -373,7 +373,7 @@ __global__ void __launch_bounds__(256) dequantize4_fast_kernel(const uint2* __re
     const float alpha = __ldg(alpha_p);
     for (IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x); g < ngroups; g += stride) {
         const uint2 c = __ldg(codes + (size_t)g);
-        const uint32_t sbyte = __ldg(scales + (size_t)g);
+        const uint32_t sbyte = __ldg(scales + scale_offset<SWZ>((size_t)g, gpr, ktiles));
         const uint32_t mag = sbyte & 0x7Fu;
         const bool is_int = HAS_INT && (sbyte & 0x80u);
         float Delta = e4m3_value(mag);

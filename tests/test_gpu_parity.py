@@ -452,3 +452,32 @@ def test_transposed_quantize_equals_quantize_of_transpose(B, oracle, fmt):
     sr = B.make_opts(B.ABS_F_STOCHASTIC)
     assert L.abs_quantize_transposed(1, x.data_ptr(), 64, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(),
                                      ctypes.byref(sr), None) == 5
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_swizzled_scale_layout(B, oracle, fmt):
+    """ABS_F_SCALES_SWIZZLED: same codes and alpha, scale bytes permuted into the 128x4-tile layout (the
+    oracle builds that layout by reshapes from the row-major scales); padding bytes stay untouched; the
+    dequantize option reads the same layout back."""
+    for name, rows, cols in (("cfg2", 300, 4096), ("cfg5", 129, 208), ("cfg1", 256, 1024)):
+        xb = I.generate(name, rows, cols)
+        oc, osc, oa = oracle.quantize(fmt, xb, threads=THREADS)
+        x = to_dev(xb)
+        nsw = B.abs_scales_bytes_swizzled(fmt, rows, cols)
+        assert nsw == -(-rows // 128) * -(-(cols // 16) // 4) * 512
+        scales = torch.full((nsw,), 0xEE, dtype=torch.uint8, device="cuda")
+        opts = B.make_opts(B.ABS_F_SCALES_SWIZZLED)
+        codes, scales, ts = B.abs_quantize(fmt, x, scales=scales, opts=opts)
+        torch.cuda.synchronize()
+        assert np.float32(ts.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+        assert_same("codes", codes.cpu().numpy().reshape(rows, -1), oc)
+        assert_same("swizzled scales", scales.cpu().numpy(), oracle.swizzle_scales(osc, fill=0xEE))
+        out = B.abs_dequantize(fmt, codes, scales, ts, rows, cols, opts=opts)
+        assert_same("dequant", out.view(torch.int16).cpu().numpy().view(np.uint16),
+                    oracle.dequantize(fmt, oc, osc, oa, rows, cols, threads=THREADS))
+    L = B.lib()
+    import ctypes
+    bad = B.make_opts(B.ABS_F_SCALES_SWIZZLED)
+    assert L.abs_quantize_ex(2, x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(), ts.data_ptr(),
+                             ctypes.byref(bad), None) == 5          # IF3 has no tensor-core layout
+    assert B.abs_scales_bytes_swizzled(2, 128, 64) == 0

@@ -684,3 +684,25 @@ def test_bs8_has_lower_error_than_16(oracle):
             c, s, a = oracle.quantize(f, xb, threads=4)
             mse[f] = np.mean((oracle.dequantize(f, c, s, a, 256, 1024, out_fp32=True, threads=4) - xf) ** 2)
         assert mse[f8] < 0.85 * mse[f16], (f8, mse)
+
+
+# --------------------------------------------------------------------------- tensor-core scale layout
+
+def test_swizzled_scale_layout_definition(oracle):
+    """The 128x4-tile layout against its closed-form byte offset, on shapes with ragged tiles."""
+    for rows, k in ((128, 4), (300, 13), (1, 1), (257, 64)):
+        s = (np.arange(rows * k, dtype=np.int64) * 7 % 251 + 1).astype(np.uint8).reshape(rows, k)
+        out = oracle.swizzle_scales(s, fill=0)
+        kt = -(-k // 4)
+        assert out.size == -(-rows // 128) * kt * 512
+        seen = np.zeros(out.size, bool)
+        for r in range(rows):
+            for c in range(k):
+                off = ((r // 128) * kt + c // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + c % 4
+                assert out[off] == s[r, c]
+                seen[off] = True
+        assert not out[~seen].any()                      # padding untouched
+        # one 512-byte tile holds exactly rows 128t..128t+127 x scales 4u..4u+3
+        tile0 = out[:512]
+        want = set(s[:128, :4].reshape(-1).tolist()) | {0}
+        assert set(tile0.tolist()) <= want
