@@ -759,10 +759,13 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
         src.denom = denom;
     }
     const int64_t rblocks = rows / 16;
+    const int64_t ntiles = ((cols + kTransTileCols - 1) / kTransTileCols) *
+                           ((rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks);
+    const int64_t resident = (int64_t)st->sm_count * 3;        // 64 KiB of shared memory per block: 3 blocks per SM
     cudaLaunchConfig_t cfg = {};
-    const int64_t tiles_y = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
-    cfg.gridDim = dim3((unsigned)((cols + kTransTileCols - 1) / kTransTileCols), (unsigned)(tiles_y < 65535 ? tiles_y : 65535));
+    cfg.gridDim = dim3((unsigned)(ntiles < resident ? ntiles : resident));
     cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kTransSmemBytes;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -773,12 +776,15 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     const uint16_t* in = (const uint16_t*)in_bf16;
     uint2* ct = (uint2*)codes_t_u8;
     uint8_t* stp = (uint8_t*)scales_t_e4m3;
-    if (fmt == ABS_FMT_IF4)
-        e = src.slot ? cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<true, true>, in, ct, stp, src, rows, cols)
-                     : cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<true, false>, in, ct, stp, src, rows, cols);
-    else
-        e = src.slot ? cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<false, true>, in, ct, stp, src, rows, cols)
-                     : cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<false, false>, in, ct, stp, src, rows, cols);
+#define ABS_LAUNCH_T(I, S)                                                                                          \
+    do {                                                                                                            \
+        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
+                                 kTransSmemBytes);                                                                  \
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S>, in, ct, stp, src, rows, cols); \
+    } while (0)
+    if (fmt == ABS_FMT_IF4) { if (src.slot) ABS_LAUNCH_T(true, true); else ABS_LAUNCH_T(true, false); }
+    else { if (src.slot) ABS_LAUNCH_T(false, true); else ABS_LAUNCH_T(false, false); }
+#undef ABS_LAUNCH_T
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
 

@@ -227,56 +227,100 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
 // consecutive ROWS of one column (Sec. 4.1: both operands of the weight-gradient product are quantized
 // along the token dimension).  Output = what the plain kernel would give for the [cols, rows] matrix:
 // codes_t [cols, rows/2 bytes], scales_t [cols, rows/16].
-// A block stages a tile of 64 rows x 256 columns in shared memory with coalesced 128-bit loads; thread
-// c then encodes the four groups of its column (rows 0-15, 16-31, 32-47, 48-63 of the tile), reading its
-// values down the column.  Those four groups are neighbours in the transposed output, so their codes
-// leave as one 256-bit store and their scale bytes as one 32-bit store whenever the tile is complete
-// and the output addresses allow it.
+// Persistent blocks walk over tiles of 64 rows x 256 columns.  A tile is brought into shared memory with
+// 16-byte asynchronous copies (cp.async), double buffered: the copies of the block's next tile are in
+// flight while it encodes the current one.  Thread c reads its column's values down the tile and encodes
+// the four groups of 16 rows; those are neighbours in the transposed output, so their codes leave as one
+// 256-bit store and their scale bytes as one 32-bit store whenever the tile is complete and the output
+// addresses allow it.
+#ifndef ABS_TRANS_UNROLL
+#define ABS_TRANS_UNROLL 4
+#endif
+constexpr int kTransUnroll = ABS_TRANS_UNROLL;
 constexpr int kTransTileCols = 256;
 constexpr int kTransTileRowBlocks = 4;
+constexpr int kTransStageElems = 16 * kTransTileRowBlocks * kTransTileCols;        // bf16 elements per stage
+constexpr int kTransSmemBytes = 2 * kTransStageElems * 2;                           // two stages
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 template <bool HAS_INT, bool FROM_SLOT>
 __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_t* __restrict__ in,
                                                                    uint2* __restrict__ codes_t,
                                                                    uint8_t* __restrict__ scales_t,
                                                                    const AlphaSrc alpha_src, int64_t rows, int64_t cols) {
-    __shared__ __align__(16) uint16_t tile[16 * kTransTileRowBlocks][kTransTileCols];
+    extern __shared__ __align__(16) uint16_t trans_smem[];
     pdl_launch_dependents();
     pdl_wait();
     const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     const int64_t rblocks = rows / 16;
-    const int64_t c0 = (int64_t)blockIdx.x * kTransTileCols;
-    const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);          // multiple of 16
-    const int64_t ntiles_y = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
+    const int64_t ntx = (cols + kTransTileCols - 1) / kTransTileCols;
+    const int64_t nty = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
+    const int64_t ntiles = ntx * nty;
     // vector stores need 32-byte aligned code addresses and 4-byte aligned scale addresses for every column
     const bool vec_ok = (rblocks % kTransTileRowBlocks) == 0 &&
                         ((reinterpret_cast<uintptr_t>(codes_t) & 31u) == 0) && ((reinterpret_cast<uintptr_t>(scales_t) & 3u) == 0);
-    for (int64_t ty = blockIdx.y; ty < ntiles_y; ty += gridDim.y) {
-        const int64_t rb0 = ty * kTransTileRowBlocks;
-        const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
-        const int chunks_per_row = ncols / 8;
-        for (int ch = threadIdx.x; ch < 16 * nrb * chunks_per_row; ch += blockDim.x) {
-            const int r = ch / chunks_per_row, q = ch - r * chunks_per_row;
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(in + (rb0 * 16 + r) * cols + c0) + q);
-            *reinterpret_cast<uint4*>(&tile[r][q * 8]) = v;
+
+    // issue the asynchronous copies of tile t into stage s (one commit group per call, possibly empty)
+    auto issue = [&](int64_t t, int s) {
+        if (t < ntiles) {
+            const int64_t ty = t / ntx, tx = t - ty * ntx;
+            const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
+            const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
+            const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
+            uint16_t* stage = trans_smem + s * kTransStageElems;
+            const uint16_t* src = in + rb0 * 16 * cols + c0;
+            if (ncols == kTransTileCols) {               // full-width tile: 32 chunks of 16 bytes per row
+                for (int ch = threadIdx.x; ch < 16 * nrb * (kTransTileCols / 8); ch += blockDim.x) {
+                    const int r = ch >> 5, q = ch & 31;
+                    cp_async16(stage + r * kTransTileCols + q * 8, src + (int64_t)r * cols + q * 8);
+                }
+            } else {                                     // ragged last column tile
+                const int chunks_per_row = ncols / 8;
+                for (int ch = threadIdx.x; ch < 16 * nrb * chunks_per_row; ch += blockDim.x) {
+                    const int r = ch / chunks_per_row, q = ch - r * chunks_per_row;
+                    cp_async16(stage + r * kTransTileCols + q * 8, src + (int64_t)r * cols + q * 8);
+                }
+            }
         }
-        __syncthreads();
+        cp_async_commit();
+    };
+
+    int s = 0;
+    int64_t t = blockIdx.x;
+    issue(t, 0);
+    for (; t < ntiles; t += gridDim.x, s ^= 1) {
+        issue(t + gridDim.x, s ^ 1);                 // prefetch the block's next tile into the other stage
+        cp_async_wait_all_but_one();                 // this thread's copies of tile t have landed
+        __syncthreads();                             // ... and everybody else's
+        const int64_t ty = t / ntx, tx = t - ty * ntx;
+        const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
+        const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
+        const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
+        const uint16_t* stage = trans_smem + s * kTransStageElems;
         const int c = threadIdx.x;
         if (c < ncols) {
             uint32_t cw[2 * kTransTileRowBlocks];
             uint32_t sbytes = 0u;
-#pragma unroll 1
-            for (int k = 0; k < nrb; ++k) {
+#pragma unroll kTransUnroll
+            for (int k = 0; k < kTransTileRowBlocks; ++k) {
+                if (k >= nrb) break;
                 float x[16];
+                const uint16_t* colp = stage + 16 * k * kTransTileCols + c;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) x[i] = __uint_as_float((uint32_t)tile[16 * k + i][c] << 16);
+                for (int i = 0; i < 16; ++i) x[i] = __uint_as_float((uint32_t)colp[i * kTransTileCols] << 16);
                 const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
                 const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
                 const float m4 = max3abs(x[12], x[13], x[14]);
                 const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));   // G1
-                const float t = __fmul_rn(gmax, inv_a6);                                 // G2
-                const uint32_t sb = e4m3_encode(t);                                      // G3
+                const float tt = __fmul_rn(gmax, inv_a6);                                // G2
+                const uint32_t sb = e4m3_encode(tt);                                     // G3
                 const float d = __fmul_rn(e4m3_value(sb), alpha);                        // G5
                 const float r = __frcp_rn(d);
                 uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
@@ -303,7 +347,7 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
                 *reinterpret_cast<uint32_t*>(scales_t + g0) = sbytes;
             }
         }
-        __syncthreads();
+        __syncthreads();                             // the stage may be overwritten by the next prefetch
     }
 }
 
