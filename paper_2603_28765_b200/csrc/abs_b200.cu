@@ -737,7 +737,7 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     if (opts) o = *opts;
     if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
     if (rows < 0 || cols < 0 || (cols % 16) != 0 || (rows % 16) != 0) return ABS_ERR_SHAPE;
-    if ((o.flags & ~(uint32_t)ABS_F_ALPHA_GIVEN) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ~(uint32_t)(ABS_F_ALPHA_GIVEN | ABS_F_HADAMARD16)) || o._pad) return ABS_ERR_FLAGS;
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !codes_t_u8 || !scales_t_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(codes_t_u8) || !aligned16(scales_t_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -746,18 +746,7 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
-    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
-    if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
-        unsigned long long* slot = nullptr;
-        uint32_t gen = 0;
-        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
-        const float denom = 6.0f * 448.0f;
-        abs_status_t rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
-        if (rc != ABS_OK) return rc;
-        src.slot = slot;
-        src.gen = gen;
-        src.denom = denom;
-    }
+    const bool rht = o.flags & ABS_F_HADAMARD16;
     const int64_t rblocks = rows / 16;
     const int64_t ntiles = ((cols + kTransTileCols - 1) / kTransTileCols) *
                            ((rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks);
@@ -772,18 +761,46 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e;
+    cudaError_t e = cudaSuccess;
     const uint16_t* in = (const uint16_t*)in_bf16;
     uint2* ct = (uint2*)codes_t_u8;
     uint8_t* stp = (uint8_t*)scales_t_e4m3;
-#define ABS_LAUNCH_T(I, S)                                                                                          \
+    const uint32_t mask = o.had_sign_mask;
+#define ABS_LAUNCH_T(I, S, R, M, SLOT, GEN)                                                                         \
     do {                                                                                                            \
-        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
+        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  kTransSmemBytes);                                                                  \
-        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S>, in, ct, stp, src, rows, cols); \
+        if (e == cudaSuccess)                                                                                       \
+            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, M>, in, ct, stp, src, rows, cols, mask, \
+                                   SLOT, GEN);                                                                      \
     } while (0)
-    if (fmt == ABS_FMT_IF4) { if (src.slot) ABS_LAUNCH_T(true, true); else ABS_LAUNCH_T(true, false); }
-    else { if (src.slot) ABS_LAUNCH_T(false, true); else ABS_LAUNCH_T(false, false); }
+
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
+        unsigned long long* slot = nullptr;
+        uint32_t gen = 0;
+        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        const float denom = 6.0f * 448.0f;
+        if (rht) {
+            // the maximum is taken over the transformed column groups: same tile walk, MODE 1
+            ABS_LAUNCH_T(false, false, true, 1, slot, gen);
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+        } else {
+            abs_status_t rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+            if (rc != ABS_OK) return rc;
+        }
+        src.slot = slot;
+        src.gen = gen;
+        src.denom = denom;
+    }
+    unsigned long long* no_slot = nullptr;
+    if (fmt == ABS_FMT_IF4) {
+        if (rht) { if (src.slot) ABS_LAUNCH_T(true, true, true, 0, no_slot, 0u); else ABS_LAUNCH_T(true, false, true, 0, no_slot, 0u); }
+        else { if (src.slot) ABS_LAUNCH_T(true, true, false, 0, no_slot, 0u); else ABS_LAUNCH_T(true, false, false, 0, no_slot, 0u); }
+    } else {
+        if (rht) { if (src.slot) ABS_LAUNCH_T(false, true, true, 0, no_slot, 0u); else ABS_LAUNCH_T(false, false, true, 0, no_slot, 0u); }
+        else { if (src.slot) ABS_LAUNCH_T(false, true, false, 0, no_slot, 0u); else ABS_LAUNCH_T(false, false, false, 0, no_slot, 0u); }
+    }
 #undef ABS_LAUNCH_T
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }

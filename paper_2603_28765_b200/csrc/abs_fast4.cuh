@@ -249,16 +249,24 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
-template <bool HAS_INT, bool FROM_SLOT>
+// MODE 0: quantize.  MODE 1: only the maximum of the Hadamard-transformed column groups (the amax pass of
+// the transposed path with the Hadamard option; publishes a tagged maximum like amax_kernel).
+template <bool HAS_INT, bool FROM_SLOT, bool RHT, int MODE>
 __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_t* __restrict__ in,
                                                                    uint2* __restrict__ codes_t,
                                                                    uint8_t* __restrict__ scales_t,
-                                                                   const AlphaSrc alpha_src, int64_t rows, int64_t cols) {
+                                                                   const AlphaSrc alpha_src, int64_t rows, int64_t cols,
+                                                                   uint32_t sign_mask, unsigned long long* amax_slot,
+                                                                   uint32_t amax_gen) {
     extern __shared__ __align__(16) uint16_t trans_smem[];
     pdl_launch_dependents();
     pdl_wait();
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2
-    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
+    float alpha = 1.0f, inv_a6 = 1.0f;
+    if constexpr (MODE == 0) {
+        alpha = resolve_alpha<FROM_SLOT>(alpha_src);                         // T2
+        inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                          // T3
+    }
+    uint32_t local_max = 0u;
     const int64_t rblocks = rows / 16;
     const int64_t ntx = (cols + kTransTileCols - 1) / kTransTileCols;
     const int64_t nty = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
@@ -315,6 +323,12 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
                 const uint16_t* colp = stage + 16 * k * kTransTileCols + c;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) x[i] = __uint_as_float((uint32_t)colp[i * kTransTileCols] << 16);
+                if constexpr (RHT) hadamard16(x, sign_mask);         // along the group, i.e. down the column
+                if constexpr (MODE == 1) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) local_max = max(local_max, __float_as_uint(x[i]) & 0x7FFFFFFFu);
+                    continue;
+                }
                 const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
                 const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
                 const float m4 = max3abs(x[12], x[13], x[14]);
@@ -341,13 +355,25 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
                     codes_t[g] = make_uint2(c_lo, c_hi);
                 }
             }
-            if (vec_ok) {
+            if (MODE == 0 && vec_ok) {
                 const int64_t g0 = (c0 + c) * rblocks + rb0;
                 store32B<true>(codes_t + g0, reinterpret_cast<const uint32_t(&)[8]>(cw));
                 *reinterpret_cast<uint32_t*>(scales_t + g0) = sbytes;
             }
         }
         __syncthreads();                             // the stage may be overwritten by the next prefetch
+    }
+    if constexpr (MODE == 1) {
+        __shared__ uint32_t warp_max[8];
+        local_max = __reduce_max_sync(0xFFFFFFFFu, local_max);
+        if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local_max;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t m = 0u;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) m = max(m, warp_max[w]);
+            atomicMax(amax_slot, ((unsigned long long)amax_gen << 32) | m);
+        }
     }
 }
 

@@ -438,6 +438,17 @@ def test_transposed_quantize_equals_quantize_of_transpose(B, oracle, fmt):
         out = B.abs_dequantize(fmt, ct, st, ts, cols, rows)
         assert_same("dequant_t", out.view(torch.int16).cpu().numpy().view(np.uint16),
                     oracle.dequantize(fmt, oc, osc, oa, cols, rows, threads=THREADS))
+    # with the Hadamard option (Sec. 4.1: transform, then quantize, both along the token dimension)
+    mask = oracle.hadamard_sign_mask(31)
+    for name, rows, cols in (("cfg4", 320, 2048), ("cfg2", 64, 528)):
+        xb = I.generate(name, rows, cols)
+        ct, st, ts = B.abs_quantize_transposed(fmt, to_dev(xb), opts=B.make_opts(B.ABS_F_HADAMARD16, mask))
+        torch.cuda.synchronize()
+        oc, osc, oa = oracle.quantize(fmt, np.ascontiguousarray(xb.T), flags=oracle.F_HADAMARD16, sign_mask=mask,
+                                      threads=THREADS)
+        assert np.float32(ts.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+        assert_same("scales_t rht", st.cpu().numpy().reshape(cols, -1), osc)
+        assert_same("codes_t rht", ct.cpu().numpy().reshape(cols, -1), oc)
     # alpha given, and the argument checks
     xb = I.generate("cfg5", 64, 256)
     ts = torch.tensor([0.02], dtype=torch.float32, device="cuda")
