@@ -46,7 +46,10 @@ enum {
     F_STOCHASTIC = 1u << 1,
     F_SR_SCALE_17_16 = 1u << 2,
     F_ALPHA_GIVEN = 1u << 3,
-    F_OUT_FP32 = 1u << 4
+    F_OUT_FP32 = 1u << 4,
+    F_FP_GROUPS_ONLY = 1u << 7,   /* dequantize: groups stored as integers come out as +0          */
+    F_INT_GROUPS_RAW = 1u << 8    /* dequantize: FP groups come out as +0; integer groups as k * Delta * alpha,
+                                     without the M_FP/M_INT de-scale (the MAC applies it on the scale path) */
 };
 
 /* Element format of the floating-point candidate plus the integer alternative. */
@@ -425,10 +428,11 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
 /* ------------------------------------------------------------------ dequantize */
 
 /* Dequantize rows [row0,row1): value(code) * (Delta * alpha [* M_FP/M_INT for integer groups]),
- * product in FP32, then BF16 round-to-nearest-even (or FP32 when out_fp32 != 0). */
+ * product in FP32, then BF16 round-to-nearest-even (or FP32 when out_fp32 != 0).  `select` splits the
+ * tensor for the MAC arithmetic of Sec. 5.2: FP groups only, or integer groups only and without de-scale. */
 ORACLE_API int abs_oracle_dequantize_rows(int fmt, const uint8_t* codes, const uint8_t* scales, float alpha,
                                           int64_t rows, int64_t cols, int64_t row0, int64_t row1,
-                                          int out_fp32, void* out) {
+                                          int out_fp32, void* out, uint32_t select) {
     if (fmt < 0 || fmt >= FMT_COUNT || cols % 16 != 0 || row0 < 0 || row1 > rows) return 1;
     const fmt_desc* F = &FMTS[fmt];
     const int b = F->bits;
@@ -444,7 +448,8 @@ ORACLE_API int abs_oracle_dequantize_rows(int fmt, const uint8_t* codes, const u
                 const int flag = sbyte >> 7;
                 const float Delta = abs_oracle_e4m3_value(sbyte);
                 float d = Delta * alpha;
-                if (flag) d = d * c_post;
+                if (flag && !(select & F_INT_GROUPS_RAW)) d = d * c_post;
+                const int masked = (flag && (select & F_FP_GROUPS_ONLY)) || (!flag && (select & F_INT_GROUPS_RAW));
                 float v;
                 if (flag) {
                     int k = (int)code[i];
@@ -453,7 +458,7 @@ ORACLE_API int abs_oracle_dequantize_rows(int fmt, const uint8_t* codes, const u
                 } else {
                     v = abs_oracle_fp_value(fmt, code[i]);
                 }
-                const float o = v * d;
+                const float o = masked ? 0.0f : v * d;
                 const int64_t at = r * cols + gi * 16 + i;
                 if (out_fp32) ((float*)out)[at] = o;
                 else ((uint16_t*)out)[at] = f32_to_bf16_rne(o);

@@ -29,6 +29,8 @@ F_STOCHASTIC = 1 << 1
 F_SR_SCALE_17_16 = 1 << 2
 F_ALPHA_GIVEN = 1 << 3
 F_OUT_FP32 = 1 << 4
+F_FP_GROUPS_ONLY = 1 << 7
+F_INT_GROUPS_RAW = 1 << 8
 
 _lock = threading.Lock()
 _lib = None
@@ -86,7 +88,7 @@ def lib():
                                                    C.c_void_p, C.c_void_p, C.c_void_p]
             L.abs_oracle_dequantize_rows.restype = C.c_int
             L.abs_oracle_dequantize_rows.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_float, C.c_int64,
-                                                     C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_void_p]
+                                                     C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_uint32]
             _lib = L
     return _lib
 
@@ -253,8 +255,10 @@ def quantize(fmt: int, x_bf16_bits, flags: int = 0, sign_mask: int = 0, sr_seed:
     return codes, scales, alpha
 
 
-def dequantize(fmt: int, codes, scales, alpha, rows: int, cols: int, out_fp32: bool = False, threads: int = 1):
-    """Inverse path. Returns bf16 bit patterns (uint16) or float32 when ``out_fp32``."""
+def dequantize(fmt: int, codes, scales, alpha, rows: int, cols: int, out_fp32: bool = False, threads: int = 1,
+               select: int = 0):
+    """Inverse path. Returns bf16 bit patterns (uint16) or float32 when ``out_fp32``.  ``select`` =
+    F_FP_GROUPS_ONLY or F_INT_GROUPS_RAW gives one half of the split used for the MAC arithmetic."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     scales = np.ascontiguousarray(scales, dtype=np.uint8)
     assert codes.size == codes_bytes(fmt, rows, cols) and scales.size == scales_bytes(rows, cols, fmt)
@@ -263,7 +267,7 @@ def dequantize(fmt: int, codes, scales, alpha, rows: int, cols: int, out_fp32: b
 
     def work(rr):
         rc = L.abs_oracle_dequantize_rows(fmt, codes.ctypes.data, scales.ctypes.data, C.c_float(float(alpha)),
-                                          rows, cols, rr[0], rr[1], int(out_fp32), out.ctypes.data)
+                                          rows, cols, rr[0], rr[1], int(out_fp32), out.ctypes.data, select)
         if rc != 0:
             raise ValueError("abs_oracle_dequantize_rows rejected its arguments")
 
@@ -294,3 +298,19 @@ def swizzle_scales(scales: np.ndarray, fill: int = 0) -> np.ndarray:
     padded[:rows, :k] = s
     tiles = padded.reshape(mt, 4, 32, kt, 4)           # [tile row, row // 32, row % 32, tile col, scale]
     return np.ascontiguousarray(tiles.transpose(0, 3, 2, 1, 4)).reshape(-1)   # [mt, kt, row % 32, row // 32, scale]
+
+
+def mac_matmul_reference(fmt: int, qa, qb, m: int, n: int, k: int) -> np.ndarray:
+    """C = A B^T for two quantized operands (A: [m, k], B: [n, k], groups along k) with the arithmetic of
+    the paper's MAC unit (Sec. 5.2), in float64: inside a group pair the decoded codes are multiplied and
+    summed exactly; the sum is scaled by Delta_a * Delta_b and by 1, 6/7 or 36/49 when none, one or both
+    groups are integer groups; the tensor scales multiply the total.  qa, qb = (codes, scales, alpha)."""
+    parts = []
+    for codes, scales, alpha, rows in ((qa[0], qa[1], qa[2], m), (qb[0], qb[1], qb[2], n)):
+        fp = dequantize(fmt, codes, scales, 1.0, rows, k, out_fp32=True, select=F_FP_GROUPS_ONLY).astype(np.float64)
+        it = dequantize(fmt, codes, scales, 1.0, rows, k, out_fp32=True, select=F_INT_GROUPS_RAW).astype(np.float64)
+        parts.append((fp, it, float(alpha)))
+    (af, ai, aa), (bf, bi, ab) = parts
+    c67 = float(m_fp(fmt)) / float(m_int(fmt))
+    c = af @ bf.T + c67 * (af @ bi.T + ai @ bf.T) + (c67 * c67) * (ai @ bi.T)
+    return c * (aa * ab)

@@ -706,3 +706,38 @@ def test_swizzled_scale_layout_definition(oracle):
         tile0 = out[:512]
         want = set(s[:128, :4].reshape(-1).tolist()) | {0}
         assert set(tile0.tolist()) <= want
+
+
+# --------------------------------------------------------------------------- MAC semantics (Sec. 5.2)
+
+def test_split_dequantize_recombines(oracle):
+    """FP-group part + (M_FP/M_INT) * raw integer-group part == the ordinary dequantization, and both
+    parts are exactly representable in bf16 (a 4-bit code times a 4-bit-mantissa scale)."""
+    xb = CASES["cfg5"]
+    rows, cols = xb.shape
+    c, s, a = oracle.quantize(1, xb)
+    full = oracle.dequantize(1, c, s, 1.0, rows, cols, out_fp32=True).astype(np.float64)
+    fp = oracle.dequantize(1, c, s, 1.0, rows, cols, out_fp32=True, select=oracle.F_FP_GROUPS_ONLY)
+    it = oracle.dequantize(1, c, s, 1.0, rows, cols, out_fp32=True, select=oracle.F_INT_GROUPS_RAW)
+    flag = np.repeat((s >> 7).astype(bool), 16, axis=1)
+    assert not fp[flag].any() and not it[~flag].any()
+    assert np.array_equal(fp[~flag].astype(np.float64), full[~flag])
+    assert np.allclose(it[flag].astype(np.float64) * (6.0 / 7.0), full[flag], rtol=1e-6)
+    for part in (fp, it):
+        assert np.array_equal(I.bf16_bits_to_f32(I.f32_to_bf16_bits(part)), part)
+
+
+def test_mac_constants_and_reference(oracle):
+    """Sec. 5.2: 6/7 for one integer operand, 36/49 for two.  On a tiny case the reference equals the
+    dot product of the ordinary dequantized operands (same real number, different rounding)."""
+    g = read_golden("format_facts.txt")
+    one = float(g["mac_rescale_one_int"][0]) / float(g["mac_rescale_one_int"][1])
+    two = float(g["mac_rescale_two_int"][0]) / float(g["mac_rescale_two_int"][1])
+    assert abs(one * one - two) < 1e-15
+    a = I.generate("cfg1", 32, 256)
+    b = I.generate("cfg5", 48, 256)
+    qa, qb = oracle.quantize(1, a), oracle.quantize(1, b)
+    ref = oracle.mac_matmul_reference(1, qa, qb, 32, 48, 256)
+    da = oracle.dequantize(1, *qa, 32, 256, out_fp32=True).astype(np.float64)
+    db = oracle.dequantize(1, *qb, 48, 256, out_fp32=True).astype(np.float64)
+    assert np.abs(ref - da @ db.T).max() <= 1e-5 * np.abs(ref).max()    # cancellation: compare on the result's scale
