@@ -78,6 +78,11 @@ enum {
     ABS_F_SCALES_SWIZZLED = 1u << 6, /* quantize / dequantize, ABS_FMT_NVFP4 and ABS_FMT_IF4 only: the scale array uses
                                        the 128x4-tile layout that Blackwell block-scaled tensor-core MMAs read
                                        (see abs_scales_bytes_swizzled) instead of row-major [rows, cols/16]      */
+    ABS_F_FP_GROUPS_ONLY = 1u << 7,  /* dequantize (ABS_FMT_IF4, bf16 output): groups stored as integers come out as +0    */
+    ABS_F_INT_GROUPS_RAW = 1u << 8,  /* dequantize (ABS_FMT_IF4, bf16 output): FP groups come out as +0 and integer groups as
+                                       k * Delta * alpha WITHOUT the 6/7 de-scale.  Both halves are exact in bf16, so
+                                       the MAC arithmetic of Sec. 5.2 (factors 1, 6/7, 36/49 applied in FP32 on the
+                                       scale path) can be reproduced with four plain bf16 GEMMs                      */
     ABS_F_INDEX64 = 1u << 5         /* testing aid: run the kernel instances that index groups with 64-bit
                                        integers (otherwise chosen only beyond 2^31 groups); same results  */
 };

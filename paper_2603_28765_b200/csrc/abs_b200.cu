@@ -497,7 +497,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 template <int FMT>
 abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
                                    int64_t ngroups, void* out, bool fp32, bool index64, cudaStream_t s,
-                                   int64_t swz_cols = 0) {
+                                   int64_t swz_cols = 0, int sel = 0) {
     const int grid = grid_for(st, ngroups, 64);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
@@ -507,16 +507,22 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
             cudaError_t e;
             const bool swz = swz_cols > 0;
             const uint32_t gpr = (uint32_t)(swz_cols / 16), ktiles = (gpr + 3u) / 4u;
+#define ABS_LAUNCH_D3(IDX, A32, SW, SE)                                                                              \
+    e = launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32, SW, SE>, grid, kThreads, s, (const uint2*)codes,         \
+                   (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out, gpr, ktiles)
 #define ABS_LAUNCH_D(IDX, A32)                                                                                      \
-    e = swz ? launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32, true>, grid, kThreads, s, (const uint2*)codes,     \
-                         (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out, gpr, ktiles)                     \
-            : launch_pdl(dequantize4_fast_kernel<kInt, IDX, A32, false>, grid, kThreads, s, (const uint2*)codes,    \
-                         (const uint8_t*)scales, alpha, (IDX)ngroups, (uint4*)out, gpr, ktiles)
+    do {                                                                                                            \
+        if (sel == 1) ABS_LAUNCH_D3(IDX, A32, false, 1);                                                            \
+        else if (sel == 2) ABS_LAUNCH_D3(IDX, A32, false, 2);                                                       \
+        else if (swz) ABS_LAUNCH_D3(IDX, A32, true, 0);                                                             \
+        else ABS_LAUNCH_D3(IDX, A32, false, 0);                                                                     \
+    } while (0)
             if (i32 && a32) ABS_LAUNCH_D(int32_t, true);
             else if (i32) ABS_LAUNCH_D(int32_t, false);
             else if (a32) ABS_LAUNCH_D(int64_t, true);
             else ABS_LAUNCH_D(int64_t, false);
 #undef ABS_LAUNCH_D
+#undef ABS_LAUNCH_D3
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
         }
@@ -857,7 +863,12 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
-    if ((o.flags & ~(uint32_t)(ABS_F_OUT_FP32 | ABS_F_INDEX64 | ABS_F_SCALES_SWIZZLED)) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ~(uint32_t)(ABS_F_OUT_FP32 | ABS_F_INDEX64 | ABS_F_SCALES_SWIZZLED | ABS_F_FP_GROUPS_ONLY | ABS_F_INT_GROUPS_RAW)) || o._pad)
+        return ABS_ERR_FLAGS;
+    const uint32_t split = o.flags & (ABS_F_FP_GROUPS_ONLY | ABS_F_INT_GROUPS_RAW);
+    if (split && (fmt != ABS_FMT_IF4 || split == (ABS_F_FP_GROUPS_ONLY | ABS_F_INT_GROUPS_RAW) ||
+                  (o.flags & (ABS_F_OUT_FP32 | ABS_F_SCALES_SWIZZLED))))
+        return ABS_ERR_FLAGS;      // the split exists for IF4 with bf16 output and row-major scales
     if ((o.flags & ABS_F_SCALES_SWIZZLED) &&
         ((fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) || (o.flags & ABS_F_OUT_FP32) || cols / 16 > 0x7FFFFFFF || rows > 0x7FFFFFFF))
         return ABS_ERR_FLAGS;
@@ -871,9 +882,10 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     const int64_t ngroups = rows * cols / 16;
     const bool fp32 = o.flags & ABS_F_OUT_FP32, i64 = o.flags & ABS_F_INDEX64;
     const int64_t swz_cols = (o.flags & ABS_F_SCALES_SWIZZLED) ? cols : 0;
+    const int sel = (o.flags & ABS_F_FP_GROUPS_ONLY) ? 1 : ((o.flags & ABS_F_INT_GROUPS_RAW) ? 2 : 0);
     switch (fmt) {
         case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
-        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
+        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols, sel);
         case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
         case ABS_FMT_IF6_E3M2: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);

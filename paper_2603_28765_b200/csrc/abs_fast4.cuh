@@ -431,7 +431,9 @@ __device__ __forceinline__ void dequant_word4(uint32_t w, bool is_int, float add
     }
 }
 
-template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool SWZ>
+// SEL 0: ordinary dequantize.  SEL 1: FP groups only (integer groups -> +0).  SEL 2: integer groups only and
+// without the 6/7 de-scale (FP groups -> +0): the two exact halves used for the MAC arithmetic of Sec. 5.2.
+template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool SWZ, int SEL>
 __global__ void __launch_bounds__(256) dequantize4_fast_kernel(const uint2* __restrict__ codes,
                                                                const uint8_t* __restrict__ scales,
                                                                const float* __restrict__ alpha_p, IdxT ngroups,
@@ -449,13 +451,17 @@ __global__ void __launch_bounds__(256) dequantize4_fast_kernel(const uint2* __re
         float Delta = e4m3_value(mag);
         if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
         float d = __fmul_rn(Delta, alpha);
-        if (is_int) d = __fmul_rn(d, c_post);                          // de-scale integer groups (Sec. 3)
+        if (is_int && SEL != 2) d = __fmul_rn(d, c_post);              // de-scale integer groups (Sec. 3)
         const float addend = is_int ? -1032.0f : -0.0f;
         const uint64_t D2 = pack2(d, d);
         uint32_t lo[4], hi[4];
         dequant_word4<HAS_INT>(c.x, is_int, addend, D2, lo);
         dequant_word4<HAS_INT>(c.y, is_int, addend, D2, hi);
-        const uint32_t o[8] = {lo[0], lo[1], lo[2], lo[3], hi[0], hi[1], hi[2], hi[3]};
+        uint32_t o[8] = {lo[0], lo[1], lo[2], lo[3], hi[0], hi[1], hi[2], hi[3]};
+        if ((SEL == 1 && is_int) || (SEL == 2 && !is_int)) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o[j] = 0u;                      // the other half of the split: +0
+        }
         store32B<ALIGNED32>(out + 2 * (size_t)g, o);
     }
 }

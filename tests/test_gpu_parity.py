@@ -492,3 +492,41 @@ def test_swizzled_scale_layout(B, oracle, fmt):
     assert L.abs_quantize_ex(2, x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(), ts.data_ptr(),
                              ctypes.byref(bad), None) == 5          # IF3 has no tensor-core layout
     assert B.abs_scales_bytes_swizzled(2, 128, 64) == 0
+
+
+def test_split_dequantize_and_mac_matmul(B, oracle):
+    """Sec. 5.2 on the GPU.  (1) The two halves of the split dequantize are byte-identical to the oracle's.
+    (2) matmul_mac (four exact-product BF16 GEMMs + FP32 factors 1, 6/7, 36/49) agrees with the float64 MAC
+    reference to FP32-accumulation accuracy.  (3) The paper's own emulation (dequantize to BF16, one GEMM)
+    is the same product up to the BF16 rounding of the operands -- visibly less accurate, as expected.
+    Tolerances: a K-term FP32 sum carries about sqrt(K) * 2^-24 relative error on the scale of the result;
+    BF16 operands carry 2^-9 per element, i.e. about 2^-9 / sqrt(K) .. 2^-9 on the result."""
+    from paper_2603_28765_b200 import gemm
+    m, n, k = 192, 160, 1024
+    a = I.generate("cfg2", m, k)
+    b = I.generate("cfg3a", n, k, seed=9)
+    qa_o, qb_o = oracle.quantize(1, a, threads=THREADS), oracle.quantize(1, b, threads=THREADS)
+    qa = B.abs_quantize(1, to_dev(a))
+    qb = B.abs_quantize(1, to_dev(b))
+    for flag, sel in ((B.ABS_F_FP_GROUPS_ONLY, oracle.F_FP_GROUPS_ONLY), (B.ABS_F_INT_GROUPS_RAW, oracle.F_INT_GROUPS_RAW)):
+        got = B.abs_dequantize(1, qa[0], qa[1], qa[2], m, k, opts=B.make_opts(flag))
+        want = oracle.dequantize(1, qa_o[0], qa_o[1], qa_o[2], m, k, select=sel, threads=THREADS)
+        assert_same("split half", got.view(torch.int16).cpu().numpy().view(np.uint16), want)
+    ref = oracle.mac_matmul_reference(1, qa_o, qb_o, m, n, k)
+    scale = np.abs(ref).max()
+    c_mac = gemm.matmul_mac(qa, qb, m, n, k).double().cpu().numpy()
+    c_emu = gemm.matmul_emulated(qa, qb, m, n, k).double().cpu().numpy()
+    err_mac = np.abs(c_mac - ref).max() / scale
+    err_emu = np.abs(c_emu - ref).max() / scale
+    assert err_mac < 2e-5, err_mac
+    assert err_emu < 4e-3, err_emu
+    assert err_mac < 0.1 * err_emu, (err_mac, err_emu)
+    import ctypes
+    both = B.make_opts(B.ABS_F_FP_GROUPS_ONLY | B.ABS_F_INT_GROUPS_RAW)
+    out = torch.empty((m, k), dtype=torch.bfloat16, device="cuda")
+    L = B.lib()
+    assert L.abs_dequantize_ex(1, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), m, k, out.data_ptr(),
+                               ctypes.byref(both), None) == 5
+    one = B.make_opts(B.ABS_F_FP_GROUPS_ONLY)
+    assert L.abs_dequantize_ex(0, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), m, k, out.data_ptr(),
+                               ctypes.byref(one), None) == 5
