@@ -1,12 +1,14 @@
-// Kernels and C ABI of the B200 IF4 / IF3 / IF6 / NVFP4 quantize-dequantize library.
+// Host side and C ABI of the B200 IF4 / IF3 / IF6 / NVFP4 quantize-dequantize library: argument
+// validation, per-device scratch, kernel selection and launches.
 //
-// Path (paper Sec. 3): amax_kernel (Eq. 1, grid-wide max -> alpha) -> quantize_kernel (Eq. 2 and
-// Fig. 3a steps 1-10 per 16-value group, flag in the scale's sign bit, packed codes);
-// dequantize_kernel is the inverse (Sec. 3, Sec. 4.1).  One thread owns one group of 16
-// consecutive row elements: 32 bytes in, 2*b + 1 bytes out.
+// Path (paper Sec. 3): amax_kernel (Eq. 1, grid-wide max) -> group-quantize kernel (Eq. 2 and Fig. 3a
+// steps 1-10 per 16-value group, flag in the scale's sign bit, packed codes); the dequantize kernels are
+// the inverse (Sec. 3, Sec. 4.1).  Kernels: abs_generic.cuh (amax, every format and option),
+// abs_fast4.cuh (the 4-bit round-to-nearest fast paths, transposed quantize), abs_device.cuh (building blocks).
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
 #include "abs_fast4.cuh"
+#include "abs_generic.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -15,15 +17,7 @@ using namespace absq;
 
 namespace {
 
-constexpr int kThreads = 256;
 constexpr int kMaxDevices = 64;
-
-#ifndef ABS_AMAX_UNROLL
-#define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass
-#endif
-#ifndef ABS_AMAX_BPS
-#define ABS_AMAX_BPS 8           // blocks of 256 threads per SM in the amax pass
-#endif
 
 // Launch with programmatic stream serialization: the kernel may be scheduled while the previous
 // kernel of the stream drains; every kernel here calls pdl_wait() before its first global access.
@@ -40,308 +34,6 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
-// ------------------------------------------------------------------------------------------ amax
-
-// Eq. 1, numerator: grid-wide max |x|.  Each block reduces its share and publishes it with one 64-bit
-// atomicMax of (generation << 32) | bit pattern (non-negative floats order like unsigned integers; a
-// larger generation beats whatever an earlier call left in the slot, so nothing is ever cleared).
-//   TICKET = false: that is all; the quantize kernel of the same call turns the maximum into alpha.
-//   TICKET = true (abs_amax): the last block to finish (ticket counter in slot word 2, re-armed by
-//   that block) writes the maximum (or alpha when denom != 0) to `result`.
-template <bool RHT, bool TICKET>
-__global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict__ in, int64_t ngroups,
-                                                        uint32_t sign_mask, unsigned long long* __restrict__ slot,
-                                                        uint32_t gen, float* __restrict__ result, float denom) {
-    pdl_launch_dependents();
-    uint32_t local = 0u;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    pdl_wait();
-    if constexpr (!RHT) {
-        // |x| and max on packed bf16 pairs; 8 elements per 128-bit load, ABS_AMAX_UNROLL loads in flight per thread.
-        const int64_t nvec = ngroups * 2;
-        uint32_t m0 = 0u, m1 = 0u;
-        int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-        for (; i + (ABS_AMAX_UNROLL - 1) * stride < nvec; i += ABS_AMAX_UNROLL * stride) {
-            uint4 v[ABS_AMAX_UNROLL];
-#pragma unroll
-            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) v[k] = __ldg(in + i + k * stride);
-#pragma unroll
-            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) {
-                m0 = __vmaxu2(m0, __vmaxu2(v[k].x & 0x7FFF7FFFu, v[k].y & 0x7FFF7FFFu));
-                m1 = __vmaxu2(m1, __vmaxu2(v[k].z & 0x7FFF7FFFu, v[k].w & 0x7FFF7FFFu));
-            }
-        }
-        for (; i < nvec; i += stride) {
-            uint4 v = __ldg(in + i);
-            m0 = __vmaxu2(m0, __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu));
-            m1 = __vmaxu2(m1, __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
-        }
-        uint32_t m = __vmaxu2(m0, m1);
-        local = max(m & 0xFFFFu, m >> 16) << 16;   // bf16 bits -> FP32 bits
-    } else {
-        for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
-            float x[16];
-            unpack_bf16x8(__ldg(in + 2 * g), x);
-            unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
-            hadamard16(x, sign_mask);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) local = max(local, __float_as_uint(x[i]) & 0x7FFFFFFFu);
-        }
-    }
-    local = __reduce_max_sync(0xFFFFFFFFu, local);
-    __shared__ uint32_t warp_max[kThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t m = 0u;
-#pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) m = max(m, warp_max[w]);
-        const unsigned long long tagged = ((unsigned long long)gen << 32) | m;
-        atomicMax(slot, tagged);
-        if constexpr (TICKET) {
-            uint32_t* ticket_word = reinterpret_cast<uint32_t*>(slot) + 2;
-            __threadfence();
-            const uint32_t ticket = atomicAdd(ticket_word, 1u);
-            if (ticket == gridDim.x - 1) {
-                __threadfence();
-                const unsigned long long v = atomicMax(slot, tagged);     // read the final value
-                const float A = __uint_as_float((uint32_t)v);
-                float out = A;
-                if (denom != 0.0f) out = (A == 0.0f) ? 1.0f : __fdiv_rn(A, denom);   // Eq. 1
-                *result = out;
-                *ticket_word = 0u;
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------ quantize
-
-template <int FMT, bool RHT, bool SR, bool FROM_SLOT>
-__global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
-                                                            uint8_t* __restrict__ scales,
-                                                            const AlphaSrc alpha_src, int64_t ngroups,
-                                                            float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
-                                                            uint32_t seed_hi) {
-    using F = Fmt<FMT>;
-    constexpr int B = F::BITS, G = F::GROUP, NSUB = 16 / G;
-    pdl_launch_dependents();
-    pdl_wait();
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                        // T2
-    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));                      // T3
-    const float c_pre = F::HAS_INT ? __fdiv_rn(F::M_INT, F::M_FP) : 0.0f;
-    const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-
-    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
-        float x[16];
-        unpack_bf16x8(__ldg(in + 2 * g), x);
-        unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
-        if constexpr (RHT) hadamard16(x, sign_mask);
-
-        uint32_t rnd[8];
-        if constexpr (SR) {
-            const uint64_t i8 = (uint64_t)g * 2u;
-            uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
-            uint4 p1 = philox4x32_10((uint32_t)(i8 + 1), (uint32_t)((i8 + 1) >> 32), seed_lo, seed_hi);
-            rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;
-            rnd[4] = p1.x; rnd[5] = p1.y; rnd[6] = p1.z; rnd[7] = p1.w;
-        }
-
-        // One or two groups (GROUP = 16 or 8 values per scale) inside the aligned block of 16.
-        uint32_t chosen[16];
-#pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-            const int e0i = sub * G;
-            // G1-G3 (Eq. 2, steps 1-2).
-            float gmax = 0.0f;
-#pragma unroll
-            for (int i = 0; i < G; ++i) gmax = fmaxf(gmax, fabsf(x[e0i + i]));
-            const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
-            const uint32_t sb = e4m3_encode(t);
-            uint32_t sbyte = 0u;
-#pragma unroll
-            for (int i = 0; i < G; ++i) chosen[e0i + i] = 0u;
-            if (sb != 0u) {                                                           // G4
-                const float d = __fmul_rn(e4m3_value(sb), alpha);                     // G5
-                const float r = __frcp_rn(d);
-                const float d_int = __fmul_rn(d, c_post);
-                uint32_t q_fp[G], q_int[G];
-                float s_fp[4] = {0.f, 0.f, 0.f, 0.f}, s_int[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int i = 0; i < G; i += 2) {
-                    const float x0 = x[e0i + i], x1 = x[e0i + i + 1];
-                    float y0 = __fmul_rn(x0, r), y1 = __fmul_rn(x1, r);                // E1 (step 3)
-                    float u0 = 0.f, u1 = 0.f;
-                    float yq0 = y0, yq1 = y1;
-                    if constexpr (SR) {
-                        const uint32_t rw = rnd[(e0i + i) >> 1];
-                        u0 = __fmul_rn(__fadd_rn((float)(rw & 0xFFFFu), 0.5f), 1.0f / 65536.0f);
-                        u1 = __fmul_rn(__fadd_rn((float)(rw >> 16), 0.5f), 1.0f / 65536.0f);
-                        yq0 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y0), F::M_FP, u0), y0);
-                        yq1 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y1), F::M_FP, u1), y1);
-                    }
-                    float v0, v1;
-                    fp_encode_pair<F::EK>(yq0, yq1, q_fp[i], q_fp[i + 1], v0, v1);     // E2 (step 4)
-                    const int chain = ((i >> 3) << 1);                                 // elements 0-7 -> S0,S1; 8-15 -> S2,S3
-                    if constexpr (F::HAS_INT) {
-                        const float e0 = __fmaf_rn(v0, d, -x0), e1 = __fmaf_rn(v1, d, -x1);   // E3 (steps 5-6)
-                        s_fp[chain] = __fmaf_rn(e0, e0, s_fp[chain]);
-                        s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
-                        const float z0 = __fmul_rn(y0, c_pre), z1 = __fmul_rn(y1, c_pre);     // E4 (step 7)
-                        float k0, k1;
-                        if constexpr (SR) {
-                            k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
-                            k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
-                        } else {
-                            // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
-                            k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);
-                            k1 = __fsub_rn(__fmaf_rn(y1, c_pre, 12582912.0f), 12582912.0f);
-                            k0 = fminf(fmaxf(k0, -F::M_INT), F::M_INT);
-                            k1 = fminf(fmaxf(k1, -F::M_INT), F::M_INT);
-                        }
-                        const float f0 = __fmaf_rn(k0, d_int, -x0), f1 = __fmaf_rn(k1, d_int, -x1);   // E5 (steps 8-9)
-                        s_int[chain] = __fmaf_rn(f0, f0, s_int[chain]);
-                        s_int[chain + 1] = __fmaf_rn(f1, f1, s_int[chain + 1]);
-                        q_int[i] = (uint32_t)__float2int_rn(k0) & ((1u << B) - 1u);
-                        q_int[i + 1] = (uint32_t)__float2int_rn(k1) & ((1u << B) - 1u);
-                    }
-                }
-                uint32_t flag = 0u;
-                if constexpr (F::HAS_INT) {                                            // S1-S2 (step 10)
-                    // a group of 8 leaves the last two chains at +0, so this is S0 + S1 for it
-                    const float E_fp = __fadd_rn(__fadd_rn(s_fp[0], s_fp[1]), __fadd_rn(s_fp[2], s_fp[3]));
-                    const float E_int = __fadd_rn(__fadd_rn(s_int[0], s_int[1]), __fadd_rn(s_int[2], s_int[3]));
-                    flag = (E_int < E_fp) ? 1u : 0u;
-                }
-#pragma unroll
-                for (int i = 0; i < G; ++i) chosen[e0i + i] = (F::HAS_INT && flag) ? q_int[i] : q_fp[i];
-                sbyte = sb | (flag << 7);                                             // S3
-            }
-            scales[g * NSUB + sub] = (uint8_t)sbyte;
-        }
-        uint32_t w[3];
-        pack_codes<B>(chosen, w);                                                     // S4
-        if constexpr (B == 4) {
-            *reinterpret_cast<uint2*>(codes + g * 8) = make_uint2(w[0], w[1]);
-        } else if constexpr (B == 6) {
-            uint32_t* p = reinterpret_cast<uint32_t*>(codes + g * 12);
-            p[0] = w[0]; p[1] = w[1]; p[2] = w[2];
-        } else {
-            uint16_t* p = reinterpret_cast<uint16_t*>(codes + g * 6);
-            p[0] = (uint16_t)w[0]; p[1] = (uint16_t)(w[0] >> 16); p[2] = (uint16_t)w[1];
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------ dequantize
-
-template <int FMT, bool OUT_FP32>
-__global__ void __launch_bounds__(kThreads) dequantize_kernel(const uint8_t* __restrict__ codes,
-                                                              const uint8_t* __restrict__ scales,
-                                                              const float* __restrict__ alpha_p, int64_t ngroups,
-                                                              void* __restrict__ out) {
-    using F = Fmt<FMT>;
-    constexpr int B = F::BITS, G = F::GROUP, NSUB = 16 / G;
-    pdl_launch_dependents();
-    pdl_wait();
-    const float alpha = __ldg(alpha_p);
-    const float c_post = F::HAS_INT ? __fdiv_rn(F::M_FP, F::M_INT) : 0.0f;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
-        uint32_t w[3] = {0u, 0u, 0u};
-        if constexpr (B == 4) {
-            uint2 v = __ldg(reinterpret_cast<const uint2*>(codes + g * 8));
-            w[0] = v.x; w[1] = v.y;
-        } else if constexpr (B == 6) {
-            const uint32_t* p = reinterpret_cast<const uint32_t*>(codes + g * 12);
-            w[0] = __ldg(p); w[1] = __ldg(p + 1); w[2] = __ldg(p + 2);
-        } else {
-            const uint16_t* p = reinterpret_cast<const uint16_t*>(codes + g * 6);
-            w[0] = (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 16); w[1] = (uint32_t)__ldg(p + 2);
-        }
-        uint32_t flags[NSUB];
-        float ds[NSUB];
-#pragma unroll
-        for (int sub = 0; sub < NSUB; ++sub) {
-            const uint32_t sbyte = __ldg(scales + g * NSUB + sub);
-            const uint32_t mag = sbyte & 0x7Fu;
-            flags[sub] = sbyte >> 7;
-            float Delta = e4m3_value(mag);
-            if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
-            float d = __fmul_rn(Delta, alpha);
-            if (F::HAS_INT && flags[sub]) d = __fmul_rn(d, c_post);        // de-scale integer groups (Sec. 3)
-            ds[sub] = d;
-        }
-        float o[16];
-#pragma unroll
-        for (int i = 0; i < 16; i += 2) {
-            const uint32_t flag = flags[i / G];
-            const float d = ds[i / G];
-            const uint32_t c0 = extract_code<B>(w, i), c1 = extract_code<B>(w, i + 1);
-            float v0, v1;
-            if (F::HAS_INT && flag) {
-                v0 = (float)((int32_t)(c0 << (32 - B)) >> (32 - B));   // sign-extend b bits
-                v1 = (float)((int32_t)(c1 << (32 - B)) >> (32 - B));
-            } else {
-                float2 v = fp_decode_pair<F::EK>(c0, c1);
-                v0 = v.x; v1 = v.y;
-            }
-            o[i] = __fmul_rn(v0, d);
-            o[i + 1] = __fmul_rn(v1, d);
-        }
-        if constexpr (OUT_FP32) {
-            float4* p = reinterpret_cast<float4*>(out) + g * 4;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) p[k] = make_float4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
-        } else {
-            uint32_t pk[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);   // FP32 -> bf16, nearest even
-                pk[k] = *reinterpret_cast<uint32_t*>(&h);
-            }
-            uint4* p = reinterpret_cast<uint4*>(out) + g * 2;
-            p[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            p[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------ self-test hook
-
-__global__ void selftest_kernel(int kind, const float* __restrict__ in, int64_t n, void* __restrict__ out) {
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-        const float v = in[i];
-        uint32_t c0 = 0, c1 = 0;
-        float v0, v1;
-        if (kind < 16) {
-            uint32_t r = 0;
-            switch (kind) {
-                case 0: r = e4m3_encode(v); break;
-                case 1: fp_encode_pair<EK_E2M1>(v, 0.f, c0, c1, v0, v1); r = c0; break;
-                case 2: fp_encode_pair<EK_E2M0>(v, 0.f, c0, c1, v0, v1); r = c0; break;
-                case 3: fp_encode_pair<EK_E2M3>(v, 0.f, c0, c1, v0, v1); r = c0; break;
-                case 4: fp_encode_pair<EK_E3M2>(v, 0.f, c0, c1, v0, v1); r = c0; break;
-                default: r = (uint32_t)__float2int_rn(rintf(v)) & 0xFFu; break;
-            }
-            reinterpret_cast<uint8_t*>(out)[i] = (uint8_t)r;
-        } else {
-            const uint32_t code = (uint32_t)v;
-            float r;
-            switch (kind - 16) {
-                case 0: r = e4m3_value(code & 0x7Fu); break;
-                case 1: r = fp_decode_pair<EK_E2M1>(code, 0u).x; break;
-                case 2: r = fp_decode_pair<EK_E2M0>(code, 0u).x; break;
-                case 3: r = fp_decode_pair<EK_E2M3>(code, 0u).x; break;
-                default: r = fp_decode_pair<EK_E3M2>(code, 0u).x; break;
-            }
-            reinterpret_cast<float*>(out)[i] = r;
-        }
-    }
 }
 
 // ------------------------------------------------------------------------------------------ host state

@@ -178,11 +178,13 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
     const IdxT stride = (IdxT)(gridDim.x * blockDim.x);
     IdxT g = (IdxT)(blockIdx.x * blockDim.x + threadIdx.x);
     pdl_wait();
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
-    if (g >= ngroups) return;
-    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
+    // The first group's load goes out before alpha is resolved: its latency hides the alpha read.
     uint32_t w[8], wn[8];
-    load32B<ALIGNED32>(in + 2 * (size_t)g, w);
+    const bool active = g < ngroups;
+    if (active) load32B<ALIGNED32>(in + 2 * (size_t)g, w);
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    if (!active) return;
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     while (true) {
         const IdxT gn = g + stride;
         const bool more = gn < ngroups;
