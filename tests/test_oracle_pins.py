@@ -548,6 +548,57 @@ def test_sr_keeps_representable_and_brackets(oracle):
         assert np.all((d == lo) | (d == hi))
 
 
+@pytest.mark.parametrize("fmt", [0, 2, 3, 4])
+def test_sr_index_probability_is_the_fractional_position(oracle, fmt):
+    """App. B: a value between grid points lo < a < hi rounds up with probability (a-lo)/(hi-lo), and a
+    grid point stays put.  Counted over all 65536 values the centred noise can take; built from the
+    grid alone (searchsorted), not from the oracle's piecewise index map."""
+    g = np.array(fp_grid(fmt), dtype=np.float64)
+    noise = ((np.arange(65536) + 0.5) / 65536.0 - 0.5).astype(np.float32)
+    rng = np.random.default_rng(100 + fmt)
+    samples = list(g) + [float(np.float32(v)) for v in rng.uniform(0, g[-1], 40)]
+    samples += [float(g[-1]) * 1.5, float(g[1]) * 0.25, float(g[-2] + g[-1]) / 2]
+    for a in samples:
+        idx = np.array([oracle.fp_index_sr(fmt, a, float(n)) for n in noise[::16]])   # 4096 evenly spaced draws
+        ac = min(a, g[-1])
+        lo = int(np.searchsorted(g, ac, side="right") - 1)
+        if g[lo] == ac:
+            assert np.all(idx == lo), (fmt, a)
+            continue
+        assert set(np.unique(idx)) <= {lo, lo + 1}
+        p = (ac - g[lo]) / (g[lo + 1] - g[lo])
+        assert abs((idx == lo + 1).mean() - p) <= 1.0 / 4096 + 1e-9, (fmt, a, p)
+
+
+def test_sr_int_candidate_probability(oracle):
+    """The integer candidate under SR: floor or ceil of y*7/6, up with probability frac, clamped to +-7.
+    Read back from the codes of groups the selection gives to the integer grid."""
+    rows, cols = 1, 16
+    for y_target in (0.3, 2.25, -4.6, 5.9, -6.0):
+        z = y_target * 7.0 / 6.0
+        ups = 0
+        n = 0
+        for seed in range(400):
+            x = np.zeros((rows, cols), np.float32)
+            x[0, :] = [6, 6 * 5 / 7, 6 * 3 / 7, 6 * 1 / 7, -6 * 5 / 7, -6 * 3 / 7, 0, 0, 0, 0, 0, 0, 0, 0, 0, y_target]
+            xb = I.f32_to_bf16_bits(x)
+            yb = float(I.bf16_bits_to_f32(xb)[0, 15])
+            zb = yb * 7.0 / 6.0
+            c, s, a = oracle.quantize(1, xb, flags=oracle.F_STOCHASTIC | oracle.F_ALPHA_GIVEN, alpha=1.0 / 64,
+                                      sr_seed=seed)
+            if not (s[0, 0] & 0x80):
+                continue
+            code = (int(c[0, 7]) >> 4) & 0xF
+            k = code - 16 if code >= 8 else code
+            assert k in (int(np.floor(zb)), int(np.ceil(zb))), (y_target, k)
+            ups += k == int(np.ceil(zb))
+            n += 1
+        assert n > 100
+        frac = zb - np.floor(zb)
+        if frac > 0:
+            assert abs(ups / n - frac) < 4.5 * np.sqrt(frac * (1 - frac) / n) + 1e-3, (y_target, ups / n, frac)
+
+
 def test_sr_bias_signature(oracle):
     """App. B: NVFP4 with stochastic rounding is unbiased; IF4's selection on the stochastic
     candidates pushes near-maximal values slightly up.  Checked with the 17/16 scale option on
