@@ -410,11 +410,14 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
                     /* E4 (step 7): integer candidate of y * M_INT / M_FP, clamped to +-M_INT. */
                     float kf;
                     if (flags & F_STOCHASTIC) {
-                        /* the same noise, added to the exact product with one rounding, then nearest-even:
-                         * rounds up with probability frac(y * c_pre); clamp as in the deterministic path */
-                        kf = nearbyintf(fmaf(y, c_pre, noise));
+                        /* like the FP candidate, on the magnitude clamped to M_FP and with the same noise:
+                         * |k| = nearest-even of fma(a, c_pre, n), so it rounds up with probability
+                         * frac(a * c_pre); the sign of y goes back on afterwards (rounding is symmetric) */
+                        float ay = fabsf(y);
+                        if (ay > F->m_fp) ay = F->m_fp;
+                        kf = nearbyintf(fmaf(ay, c_pre, noise));
                         if (kf > F->m_int) kf = F->m_int;
-                        if (kf < -F->m_int) kf = -F->m_int;
+                        if (ysign) kf = -kf;
                     } else {
                         kf = int_candidate_rne(y, c_pre, F->m_int);
                     }

@@ -8,6 +8,7 @@
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
 #include "abs_fast4.cuh"
+#include "abs_opt4.cuh"
 #include "abs_generic.cuh"
 
 #include <atomic>
@@ -96,6 +97,21 @@ int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
     return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
 }
 
+// Grid of a grid-stride kernel that keeps `resident_per_sm` blocks on every SM: a whole number of waves of
+// resident blocks, chosen so that a thread handles about `target_iters` work items.  A few items per thread
+// amortise the prologue and keep the prefetch running; several waves let blocks that start later overlap
+// their first loads with the arithmetic of the others (measured: about seven items per thread is best for
+// the IF4 kernel, 10 % faster than one wave of long-running blocks).
+int grid_waves(const DeviceState& st, int64_t work_items, int resident_per_sm, int target_iters) {
+    const int64_t want = (work_items + kThreads - 1) / kThreads;
+    const int64_t resident = (int64_t)st.sm_count * resident_per_sm;
+    if (want <= resident) return (int)(want < 1 ? 1 : want);
+    int64_t waves = (want + (int64_t)target_iters * resident / 2) / ((int64_t)target_iters * resident);
+    if (waves < 1) waves = 1;
+    const int64_t grid = waves * resident;
+    return (int)(grid < want ? grid : want);
+}
+
 // Takes the next scratch slot and generation of this device.  Generations grow by one per call; when
 // the 32-bit counter wraps (after 2^32 calls) the ring is cleared once, after the device went idle.
 abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen) {
@@ -129,6 +145,13 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
+#ifndef ABS_FAST_ITERS
+#define ABS_FAST_ITERS 7          // groups per thread the IF4 round-to-nearest kernel is launched for
+#endif
+#ifndef ABS_OPT_ITERS
+#define ABS_OPT_ITERS 12          // same for the Hadamard / stochastic-rounding kernel
+#endif
+
 template <int FMT>
 abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
                                  const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s, int64_t cols = 0) {
@@ -139,7 +162,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
-            const int pgrid = grid_for(st, ngroups, FMT == ABS_FMT_IF4 ? ABS_FAST_MINB : 64);   // IF4: resident blocks only
+            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(st, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_for(st, ngroups, 64);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
@@ -164,6 +187,29 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             else ABS_LAUNCH_F(int64_t, false);
 #undef ABS_LAUNCH_F
 #undef ABS_LAUNCH_F3
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+            if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
+        // Hadamard / stochastic-rounding options of the 4-bit formats: the packed persistent kernel
+        const int ogrid = grid_waves(st, ngroups, opt_blocks_per_sm(sr), ABS_OPT_ITERS);
+        if (!(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)ogrid * kThreads) {
+            constexpr bool kInt = FMT == ABS_FMT_IF4;
+            const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+            cudaError_t e;
+#define ABS_LAUNCH_O(R, S)                                                                                        \
+    e = alpha.slot ? launch_pdl(quantize4_opt_kernel<kInt, R, S, true>, ogrid, kThreads, s, (const uint4*)in,     \
+                                (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
+                                (uint32_t)o.had_sign_mask, k0, k1, a32)                                           \
+                   : launch_pdl(quantize4_opt_kernel<kInt, R, S, false>, ogrid, kThreads, s, (const uint4*)in,    \
+                                (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
+                                (uint32_t)o.had_sign_mask, k0, k1, a32)
+            if (rht && sr) ABS_LAUNCH_O(true, true);
+            else if (rht) ABS_LAUNCH_O(true, false);
+            else ABS_LAUNCH_O(false, true);
+#undef ABS_LAUNCH_O
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;

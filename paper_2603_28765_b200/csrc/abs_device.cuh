@@ -171,10 +171,12 @@ __device__ __forceinline__ uint32_t sr_index_fp(float a, float noise) {
     int idx = __float2int_rn(__fadd_rn(phi, noise));
     return (uint32_t)min(max(idx, 0), TOP);
 }
-// Integer candidate under stochastic rounding: nearest-even of fma(y, c_pre, n), clamped to +-M_INT.
-__device__ __forceinline__ float sr_round_int(float y, float c_pre, float noise, float m_int) {
-    const float k = rintf(__fmaf_rn(y, c_pre, noise));
-    return fminf(fmaxf(k, -m_int), m_int);
+// Integer candidate under stochastic rounding, on the magnitude like the FP one: |k| = nearest-even of
+// fma(min(|y|, M_FP), c_pre, n), at most M_INT; the sign of y goes back on afterwards.
+__device__ __forceinline__ float sr_round_int(float y, float c_pre, float noise, float m_fp, float m_int) {
+    const float a = (fabsf(y) > m_fp) ? m_fp : fabsf(y);
+    const float k = fminf(rintf(__fmaf_rn(a, c_pre, noise)), m_int);
+    return copysignf(k, y);
 }
 // Centred noise of a 16-bit random field h: n = (h + 1/2) * 2^-16 - 1/2, exact in FP32.
 __device__ __forceinline__ float sr_noise(uint32_t h) {

@@ -167,8 +167,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                         s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
                         float k0, k1;                                                         // E4 (step 7)
                         if constexpr (SR) {
-                            k0 = sr_round_int(y0, c_pre, n0, F::M_INT);
-                            k1 = sr_round_int(y1, c_pre, n1, F::M_INT);
+                            k0 = sr_round_int(y0, c_pre, n0, F::M_FP, F::M_INT);
+                            k1 = sr_round_int(y1, c_pre, n1, F::M_FP, F::M_INT);
                         } else {
                             // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
                             k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);
