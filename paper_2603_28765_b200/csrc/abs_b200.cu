@@ -145,6 +145,12 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
+#ifndef ABS_NV_ITERS
+#define ABS_NV_ITERS 5            // groups per thread of the NVFP4 round-to-nearest kernel (5 resident blocks per SM)
+#endif
+#ifndef ABS_DEQ_ITERS
+#define ABS_DEQ_ITERS 2           // groups per thread of the 4-bit dequantize kernel
+#endif
 #ifndef ABS_FAST_ITERS
 #define ABS_FAST_ITERS 7          // groups per thread the IF4 round-to-nearest kernel is launched for
 #endif
@@ -162,7 +168,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
-            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(st, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_for(st, ngroups, 64);
+            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(st, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(st, ngroups, 5, ABS_NV_ITERS);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
@@ -240,6 +246,7 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
+            const int grid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);    // 31 registers: 8 resident blocks per SM
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
             const bool i32 = !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
             cudaError_t e;

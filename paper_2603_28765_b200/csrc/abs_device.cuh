@@ -183,6 +183,31 @@ __device__ __forceinline__ float sr_noise(uint32_t h) {
     return __fsub_rn(__fmul_rn(__fadd_rn((float)h, 0.5f), 1.0f / 65536.0f), 0.5f);
 }
 
+// ----------------------------------------------------------------------------- packed f32x2 arithmetic
+
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 // ----------------------------------------------------------------------------- Hadamard option
 
 // 16-point transform of one group held in registers: sign flips from the mask, natural-order
@@ -205,6 +230,36 @@ __device__ __forceinline__ void hadamard16(float (&a)[16], uint32_t sign_mask) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) a[i] = __fmul_rn(a[i], 0.25f);
 }
+
+// 16-point transform of one group given as eight bf16x2 words: sign flips on the packed words (smask has
+// bit 15 / 31 of word i set where elements 2i / 2i+1 are negated), the h = 1 stage inside each pair with
+// scalar adds, the h = 2, 4, 8 stages on whole pairs with packed add and fused (p - q = fma(q, -1, p), one
+// rounding), then times 1/4.  Natural-order Sylvester butterflies, every result rounded to FP32.
+__device__ __forceinline__ void hadamard16_packed(const uint32_t (&w)[8], const uint32_t (&smask)[8], float (&x)[16]) {
+    uint64_t P[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t v = w[i] ^ smask[i];
+        const float p = __uint_as_float(v << 16), q = __uint_as_float(v & 0xFFFF0000u);
+        P[i] = pack2(__fadd_rn(p, q), __fsub_rn(p, q));
+    }
+    const uint64_t NEG1 = pack2(-1.0f, -1.0f), QUARTER = pack2(0.25f, 0.25f);
+#pragma unroll
+    for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+        for (int base = 0; base < 8; base += 2 * h) {
+#pragma unroll
+            for (int j = base; j < base + h; ++j) {
+                const uint64_t p = P[j], q = P[j + h];
+                P[j] = add2(p, q);
+                P[j + h] = fma2(q, NEG1, p);
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) unpack2(mul2(P[i], QUARTER), x[2 * i], x[2 * i + 1]);
+}
+
 
 // ----------------------------------------------------------------------------- loads / stores / launch order
 

@@ -9,10 +9,13 @@ namespace absq {
 constexpr int kThreads = 256;
 
 #ifndef ABS_AMAX_UNROLL
-#define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass
+#define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass (input not 32-byte aligned)
+#endif
+#ifndef ABS_AMAX_V8
+#define ABS_AMAX_V8 2            // 256-bit loads in flight per thread when the input is 32-byte aligned
 #endif
 #ifndef ABS_AMAX_BPS
-#define ABS_AMAX_BPS 8           // blocks of 256 threads per SM in the amax pass
+#define ABS_AMAX_BPS 4           // blocks of 256 threads per SM in the amax pass
 #endif
 
 // ------------------------------------------------------------------------------------------ amax
@@ -32,10 +35,34 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     pdl_wait();
     if constexpr (!RHT) {
-        // |x| and max on packed bf16 pairs; 8 elements per 128-bit load, ABS_AMAX_UNROLL loads in flight per thread.
+        // |x| and max on packed bf16 pairs
         const int64_t nvec = ngroups * 2;
         uint32_t m0 = 0u, m1 = 0u;
         int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        if ((reinterpret_cast<uintptr_t>(in) & 31u) == 0) {
+            // 256-bit loads: one group of 16 values per load, ABS_AMAX_V8 loads in flight per thread
+            for (; i + (ABS_AMAX_V8 - 1) * stride < ngroups; i += ABS_AMAX_V8 * stride) {
+                uint32_t w[ABS_AMAX_V8][8];
+#pragma unroll
+                for (int k = 0; k < ABS_AMAX_V8; ++k) load32B<true>(in + 2 * (i + k * stride), w[k]);
+#pragma unroll
+                for (int k = 0; k < ABS_AMAX_V8; ++k) {
+                    m0 = __vmaxu2(m0, __vmaxu2(__vmaxu2(w[k][0] & 0x7FFF7FFFu, w[k][1] & 0x7FFF7FFFu),
+                                               __vmaxu2(w[k][2] & 0x7FFF7FFFu, w[k][3] & 0x7FFF7FFFu)));
+                    m1 = __vmaxu2(m1, __vmaxu2(__vmaxu2(w[k][4] & 0x7FFF7FFFu, w[k][5] & 0x7FFF7FFFu),
+                                               __vmaxu2(w[k][6] & 0x7FFF7FFFu, w[k][7] & 0x7FFF7FFFu)));
+                }
+            }
+            for (; i < ngroups; i += stride) {
+                uint32_t w[8];
+                load32B<true>(in + 2 * i, w);
+                m0 = __vmaxu2(m0, __vmaxu2(__vmaxu2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu),
+                                           __vmaxu2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu)));
+                m1 = __vmaxu2(m1, __vmaxu2(__vmaxu2(w[4] & 0x7FFF7FFFu, w[5] & 0x7FFF7FFFu),
+                                           __vmaxu2(w[6] & 0x7FFF7FFFu, w[7] & 0x7FFF7FFFu)));
+            }
+            i = nvec;
+        }
         for (; i + (ABS_AMAX_UNROLL - 1) * stride < nvec; i += ABS_AMAX_UNROLL * stride) {
             uint4 v[ABS_AMAX_UNROLL];
 #pragma unroll
@@ -54,14 +81,37 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
         uint32_t m = __vmaxu2(m0, m1);
         local = max(m & 0xFFFFu, m >> 16) << 16;   // bf16 bits -> FP32 bits
     } else {
-        for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
-            float x[16];
-            unpack_bf16x8(__ldg(in + 2 * g), x);
-            unpack_bf16x8(__ldg(in + 2 * g + 1), x + 8);
-            hadamard16(x, sign_mask);
+        // maximum of the Hadamard-transformed groups: packed butterflies, next group's load in flight
+        uint32_t smask[8];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) local = max(local, __float_as_uint(x[i]) & 0x7FFFFFFFu);
+        for (int i = 0; i < 8; ++i)
+            smask[i] = (((sign_mask >> (2 * i)) & 1u) << 15) | (((sign_mask >> (2 * i + 1)) & 1u) << 31);
+        const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+        int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        uint32_t w[8], wn[8];
+        if (g < ngroups) {
+            if (a32) load32B<true>(in + 2 * g, w);
+            else load32B<false>(in + 2 * g, w);
         }
+        float m0 = 0.0f, m1 = 0.0f;
+        while (g < ngroups) {
+            const int64_t gn = g + stride;
+            if (gn < ngroups) {
+                if (a32) load32B<true>(in + 2 * gn, wn);
+                else load32B<false>(in + 2 * gn, wn);
+            }
+            float x[16];
+            hadamard16_packed(w, smask, x);
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+                m0 = fmaxf(m0, fmaxf(fabsf(x[i]), fabsf(x[i + 1])));
+                m1 = fmaxf(m1, fmaxf(fabsf(x[i + 2]), fabsf(x[i + 3])));
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = wn[i];
+            g = gn;
+        }
+        local = __float_as_uint(fmaxf(m0, m1));
     }
     local = __reduce_max_sync(0xFFFFFFFFu, local);
     __shared__ uint32_t warp_max[kThreads / 32];

@@ -22,35 +22,6 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 }
 __device__ __forceinline__ uint32_t sign_of(float y) { return __float_as_uint(y) & 0x80000000u; }
 
-// 16-point transform of one group given as eight bf16x2 words: sign flips on the packed words (smask has
-// bit 15 / 31 of word i set where elements 2i / 2i+1 are negated), the h = 1 stage inside each pair with
-// scalar adds, the h = 2, 4, 8 stages on whole pairs with packed add and fused (p - q = fma(q, -1, p), one
-// rounding), then times 1/4.  Natural-order Sylvester butterflies, every result rounded to FP32.
-__device__ __forceinline__ void hadamard16_packed(const uint32_t (&w)[8], const uint32_t (&smask)[8], float (&x)[16]) {
-    uint64_t P[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t v = w[i] ^ smask[i];
-        const float p = __uint_as_float(v << 16), q = __uint_as_float(v & 0xFFFF0000u);
-        P[i] = pack2(__fadd_rn(p, q), __fsub_rn(p, q));
-    }
-    const uint64_t NEG1 = pack2(-1.0f, -1.0f), QUARTER = pack2(0.25f, 0.25f);
-#pragma unroll
-    for (int h = 1; h < 8; h <<= 1) {
-#pragma unroll
-        for (int base = 0; base < 8; base += 2 * h) {
-#pragma unroll
-            for (int j = base; j < base + h; ++j) {
-                const uint64_t p = P[j], q = P[j + h];
-                P[j] = add2(p, q);
-                P[j + h] = fma2(q, NEG1, p);
-            }
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) unpack2(mul2(P[i], QUARTER), x[2 * i], x[2 * i + 1]);
-}
-
 // Per-element work of one group under stochastic rounding (steps 3-10 of Fig. 3a with both candidates
 // rounded stochastically, App. B).  rnd[i] holds the two 16-bit random fields of elements 2i (low half)
 // and 2i+1.  For E2M1 the index map is phi(a) = min(2a, a + 2, a/2 + 4) and its inverse, the value of an
