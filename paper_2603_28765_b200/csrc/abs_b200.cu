@@ -9,6 +9,7 @@
 #include "abs_device.cuh"
 #include "abs_fast4.cuh"
 #include "abs_opt4.cuh"
+#include "abs_fastx.cuh"
 #include "abs_generic.cuh"
 
 #include <atomic>
@@ -145,6 +146,9 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
+#ifndef ABS_IF6_ITERS
+#define ABS_IF6_ITERS 7           // groups per thread of the 6-bit round-to-nearest kernel
+#endif
 #ifndef ABS_NV_ITERS
 #define ABS_NV_ITERS 5            // groups per thread of the NVFP4 round-to-nearest kernel (5 resident blocks per SM)
 #endif
@@ -216,6 +220,37 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             else if (rht) ABS_LAUNCH_O(true, false);
             else ABS_LAUNCH_O(false, true);
 #undef ABS_LAUNCH_O
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+            if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
+        // block-size-8 variants of the 4-bit formats, round-to-nearest: two groups of 8 per thread
+        constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
+        const int bgrid = grid_waves(st, ngroups, kInt ? 4 : 5, kInt ? 7 : 5);
+        if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
+            const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+            const cudaError_t e =
+                alpha.slot ? launch_pdl(quantize4_bs8_kernel<kInt, true>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32)
+                           : launch_pdl(quantize4_bs8_kernel<kInt, false>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32);
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+            if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
+        // 6-bit formats, round-to-nearest
+        const int sgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
+        if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
+            const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+            const cudaError_t e =
+                alpha.slot ? launch_pdl(quantize6_fast_kernel<FMT, true>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32)
+                           : launch_pdl(quantize6_fast_kernel<FMT, false>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32);
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;

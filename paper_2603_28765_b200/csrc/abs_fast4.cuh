@@ -39,7 +39,7 @@ __device__ __forceinline__ uint32_t e2m1x8_encode_decode(const float (&y)[8], ui
         "  cvt.rn.f16x2.e2m1x2 %3, c;\n"
         "  cvt.rn.f16x2.e2m1x2 %4, d;\n"
         "  mov.b32 %0, {a, b, c, d}; }"
-        : "=r"(w), "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+        : "=&r"(w), "=&r"(h[0]), "=&r"(h[1]), "=&r"(h[2]), "=&r"(h[3])
         : "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]), "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]));
     return w;
 }

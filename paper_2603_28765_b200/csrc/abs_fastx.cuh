@@ -1,0 +1,283 @@
+// Packed round-to-nearest group-quantize kernels for the formats beside IF4 / NVFP4: the block-size-8
+// variants of the 4-bit formats (Sec. 5.1, Table 5) and the 6-bit formats IF6-E2M3 / IF6-E3M2 (Sec. 5.1).  Same
+// arithmetic as the generic kernel, bit for bit, in the style of abs_fast4.cuh: persistent grid-stride
+// threads that prefetch the next 32 bytes, f32x2 arithmetic, magic-number integer rounding, Horner packing.
+#pragma once
+#include "abs_fast4.cuh"
+
+namespace absq {
+
+// ----------------------------------------------------------------------------- 4-bit, one scale per 8 values
+
+// Steps 3-10 of Fig. 3a for one group of EIGHT values (one 32-bit word of codes).  The error sums of a
+// group of 8 are S0 + S1 (the other two chains of the 16-value order are +0).
+template <bool HAS_INT, bool CLAMP>
+__device__ __forceinline__ void encode_half4(const float* x, uint32_t sb, float d, float r, uint32_t& sbyte,
+                                             uint32_t& cword) {
+    const uint64_t R2 = pack2(r, r);
+    float y[8];
+    uint64_t X[4], Y[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        X[i] = pack2(x[2 * i], x[2 * i + 1]);
+        Y[i] = mul2(X[i], R2);                                               // E1 (step 3)
+        unpack2(Y[i], y[2 * i], y[2 * i + 1]);
+    }
+    if constexpr (!HAS_INT) {
+        cword = e2m1x8_encode(y);                                            // E2
+        sbyte = sb;
+    } else {
+        const float c_pre = __uint_as_float(0x3F955555u);    // fp32(7/6)
+        const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
+        const float d_int = __fmul_rn(d, c_post);
+        const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
+        const uint64_t MG2 = pack2(kMagic8, kMagic8), NMG2 = pack2(-kMagic8, -kMagic8);
+        uint64_t accF = 0, accI = 0;
+        uint32_t h[4], kb[8];
+        const uint32_t fw = e2m1x8_encode_decode(y, h);                      // E2 (step 4) and the code values
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h[i]));
+            const uint64_t E = fma2(pack2(v.x, v.y), ND2, X[i]);             // E3, negated; squared below
+            accF = (i == 0) ? mul2(E, E) : fma2(E, E, accF);
+            uint64_t KZ = fma2(Y[i], CP2, MG2);                              // E4 (step 7)
+            if constexpr (CLAMP) {
+                float k0, k1;
+                unpack2(KZ, k0, k1);
+                k0 = fminf(fmaxf(k0, kMagic8 - 7.0f), kMagic8 + 7.0f);
+                k1 = fminf(fmaxf(k1, kMagic8 - 7.0f), kMagic8 + 7.0f);
+                KZ = pack2(k0, k1);
+            }
+            const uint64_t FI = fma2(add2(KZ, NMG2), NDI2, X[i]);            // E5 (steps 8-9)
+            accI = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI);
+            float kz0, kz1;
+            unpack2(KZ, kz0, kz1);
+            kb[2 * i] = __float_as_uint(kz0);
+            kb[2 * i + 1] = __float_as_uint(kz1);
+        }
+        float f0, f1, i0, i1;
+        unpack2(accF, f0, f1);
+        unpack2(accI, i0, i1);
+        const bool flag = __fadd_rn(i0, i1) < __fadd_rn(f0, f1);             // S1-S2 (step 10)
+        constexpr uint32_t kConst = kMagic8Bits * 0x11111111u - 0x88888888u;
+        uint32_t il = kb[7];
+#pragma unroll
+        for (int j = 6; j >= 0; --j) il = il * 16u + kb[j];
+        il = (il - kConst) ^ 0x88888888u;
+        cword = flag ? il : fw;
+        sbyte = sb | (flag ? 0x80u : 0u);
+    }
+}
+
+// One thread per aligned block of 16 values = two groups of 8: two scales, one 64-bit store of codes and
+// one 16-bit store of scale bytes.  scale_mul is 17/16 with that option and 1 otherwise.
+template <bool HAS_INT, bool FROM_SLOT>
+__global__ void __launch_bounds__(256, HAS_INT ? 4 : 5)
+quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint16_t* __restrict__ scales,
+                     const AlphaSrc alpha_src, int32_t nblocks16, float scale_mul, bool aligned32) {
+    pdl_launch_dependents();
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    pdl_wait();
+    uint32_t w[8], wn[8];
+    const bool active = g < nblocks16;
+    if (active) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
+        else load32B<false>(in + 2 * (size_t)g, w);
+    }
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    if (!active) return;
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < nblocks16;
+        if (more) {
+            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
+            else load32B<false>(in + 2 * (size_t)gn, wn);
+        }
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+        uint32_t cw[2], sbytes = 0u;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float* xs = x + 8 * h;
+            const float gmax = max3abs(max3abs(xs[0], xs[1], xs[2]), max3abs(xs[3], xs[4], xs[5]), fmaxf(fabsf(xs[6]), fabsf(xs[7])));   // G1
+            const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);   // G2
+            const uint32_t sb = e4m3_encode(t);                              // G3
+            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
+            const float r = __frcp_rn(d);
+            uint32_t sbyte = 0u, c = 0u;
+            if ((sb - 8u) >= 118u) {
+                if (sb != 0u) encode_half4<HAS_INT, HAS_INT>(xs, sb, d, r, sbyte, c);      // G4: zero scale -> zeros
+            } else {
+                encode_half4<HAS_INT, false>(xs, sb, d, r, sbyte, c);
+            }
+            cw[h] = c;
+            sbytes |= sbyte << (8 * h);
+        }
+        scales[g] = (uint16_t)sbytes;
+        codes[g] = make_uint2(cw[0], cw[1]);
+        if (!more) break;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = wn[i];
+        g = gn;
+    }
+}
+
+// ----------------------------------------------------------------------------- 6-bit formats (IF6)
+
+constexpr float kMagic32 = 12582944.0f;               // 1.5 * 2^23 + 32: the low six mantissa bits of k + kMagic32 are k + 32
+constexpr uint32_t kMagic32Bits = 0x4B400020u;
+
+// Step 4 for eight scaled values: four 6-bit x2 converts (one code per byte) give the eight code bytes
+// as two words; the half2 values of the codes are then decoded from the 16-bit halves of those words.
+template <ElemKind EK>
+__device__ __forceinline__ void fp6x8_encode_decode(const float (&y)[8], uint32_t (&h)[4], uint32_t& w0, uint32_t& w1) {
+    if constexpr (EK == EK_E2M3) {
+        w0 = e2m3x2_encode(y[0], y[1]) | (e2m3x2_encode(y[2], y[3]) << 16);
+        w1 = e2m3x2_encode(y[4], y[5]) | (e2m3x2_encode(y[6], y[7]) << 16);
+        asm("{ .reg .b16 lo, hi;\n"
+            "  mov.b32 {lo, hi}, %2;\n"
+            "  cvt.rn.f16x2.e2m3x2 %0, lo;\n"
+            "  cvt.rn.f16x2.e2m3x2 %1, hi; }" : "=&r"(h[0]), "=&r"(h[1]) : "r"(w0));
+        asm("{ .reg .b16 lo, hi;\n"
+            "  mov.b32 {lo, hi}, %2;\n"
+            "  cvt.rn.f16x2.e2m3x2 %0, lo;\n"
+            "  cvt.rn.f16x2.e2m3x2 %1, hi; }" : "=&r"(h[2]), "=&r"(h[3]) : "r"(w1));
+    } else {
+        w0 = e3m2x2_encode(y[0], y[1]) | (e3m2x2_encode(y[2], y[3]) << 16);
+        w1 = e3m2x2_encode(y[4], y[5]) | (e3m2x2_encode(y[6], y[7]) << 16);
+        asm("{ .reg .b16 lo, hi;\n"
+            "  mov.b32 {lo, hi}, %2;\n"
+            "  cvt.rn.f16x2.e3m2x2 %0, lo;\n"
+            "  cvt.rn.f16x2.e3m2x2 %1, hi; }" : "=&r"(h[0]), "=&r"(h[1]) : "r"(w0));
+        asm("{ .reg .b16 lo, hi;\n"
+            "  mov.b32 {lo, hi}, %2;\n"
+            "  cvt.rn.f16x2.e3m2x2 %0, lo;\n"
+            "  cvt.rn.f16x2.e3m2x2 %1, hi; }" : "=&r"(h[2]), "=&r"(h[3]) : "r"(w1));
+    }
+}
+
+// Four 6-bit codes, one per byte of w, squeezed into 24 bits (code j at bit 6j) with multiply-adds:
+// b0 + b1*2^8 + b2*2^16 + b3*2^24  ->  pairs (b0 + b1*2^6) at bits 0 and 16  ->  b0 + b1*2^6 + b2*2^12 + b3*2^18.
+__device__ __forceinline__ uint32_t squeeze6x4(uint32_t w) {
+    const uint32_t t = w - 192u * ((w >> 8) & 0x00FF00FFu);
+    return t - 0xF000u * (t >> 16);
+}
+
+// Steps 3-10 of Fig. 3a for one group of 16 values of a 6-bit format; the 96 bits of codes leave as
+// three words.  The integer candidate is always clamped: |y| reaches M_FP * 17/16, and 31 * 17/16 > 31.5.
+template <ElemKind EK>
+__device__ __forceinline__ void encode_body6(const float (&x)[16], uint32_t sb, float d, float r, float c_pre,
+                                             float c_post, uint32_t& sbyte, uint32_t (&cw)[3]) {
+    const uint64_t R2 = pack2(r, r);
+    const float d_int = __fmul_rn(d, c_post);
+    const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
+    const uint64_t MG2 = pack2(kMagic32, kMagic32), NMG2 = pack2(-kMagic32, -kMagic32);
+    uint64_t accF[2], accI[2];
+    uint32_t fchunk[4], ichunk[4];
+#pragma unroll
+    for (int hgrp = 0; hgrp < 2; ++hgrp) {
+        uint64_t X[4], Y[4];
+        float y[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            X[i] = pack2(x[8 * hgrp + 2 * i], x[8 * hgrp + 2 * i + 1]);
+            Y[i] = mul2(X[i], R2);                                           // E1 (step 3)
+            unpack2(Y[i], y[2 * i], y[2 * i + 1]);
+        }
+        uint32_t h[4], w0, w1, kb[8];
+        fp6x8_encode_decode<EK>(y, h, w0, w1);                               // E2 (step 4) and the code values
+        fchunk[2 * hgrp] = squeeze6x4(w0);
+        fchunk[2 * hgrp + 1] = squeeze6x4(w1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&h[i]));
+            const uint64_t E = fma2(pack2(v.x, v.y), ND2, X[i]);             // E3, negated; squared below
+            accF[hgrp] = (i == 0) ? mul2(E, E) : fma2(E, E, accF[hgrp]);
+            float k0, k1;
+            unpack2(fma2(Y[i], CP2, MG2), k0, k1);                           // E4 (step 7): exact product, one rounding
+            k0 = fminf(fmaxf(k0, kMagic32 - 31.0f), kMagic32 + 31.0f);
+            k1 = fminf(fmaxf(k1, kMagic32 - 31.0f), kMagic32 + 31.0f);
+            const uint64_t FI = fma2(add2(pack2(k0, k1), NMG2), NDI2, X[i]); // E5 (steps 8-9)
+            accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
+            kb[2 * i] = __float_as_uint(k0);
+            kb[2 * i + 1] = __float_as_uint(k1);
+        }
+        // integer codes: Horner over four raw sums (each kMagic32Bits + k + 32), constant part removed,
+        // offset-binary fields (k + 32) turned into two's complement (flip bit 5 of every field)
+        constexpr uint32_t kConst = (kMagic32Bits - 32u) * (1u + 64u + 4096u + 262144u);   // leaves the fields k + 32
+        ichunk[2 * hgrp] = ((((kb[3] * 64u + kb[2]) * 64u + kb[1]) * 64u + kb[0]) - kConst) ^ 0x820820u;
+        ichunk[2 * hgrp + 1] = ((((kb[7] * 64u + kb[6]) * 64u + kb[5]) * 64u + kb[4]) - kConst) ^ 0x820820u;
+    }
+    float f0, f1, f2, f3, i0, i1, i2, i3;
+    unpack2(accF[0], f0, f1); unpack2(accF[1], f2, f3);
+    unpack2(accI[0], i0, i1); unpack2(accI[1], i2, i3);
+    const float E_fp = __fadd_rn(__fadd_rn(f0, f1), __fadd_rn(f2, f3));         // S1-S2 (step 10)
+    const float E_int = __fadd_rn(__fadd_rn(i0, i1), __fadd_rn(i2, i3));
+    const bool flag = E_int < E_fp;
+    const uint32_t c0 = flag ? ichunk[0] : fchunk[0], c1 = flag ? ichunk[1] : fchunk[1];
+    const uint32_t c2 = flag ? ichunk[2] : fchunk[2], c3 = flag ? ichunk[3] : fchunk[3];
+    cw[0] = c0 | (c1 << 24);                                                    // S4: 4 x 24 bits -> 3 words
+    cw[1] = (c1 >> 8) | (c2 << 16);
+    cw[2] = (c2 >> 16) | (c3 << 8);
+    sbyte = sb | (flag ? 0x80u : 0u);                                           // S3
+}
+
+template <int FMT, bool FROM_SLOT>
+__global__ void __launch_bounds__(256, 3)
+quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32) {
+    using F = Fmt<FMT>;
+    pdl_launch_dependents();
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    pdl_wait();
+    uint32_t w[8], wn[8];
+    const bool active = g < ngroups;
+    if (active) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
+        else load32B<false>(in + 2 * (size_t)g, w);
+    }
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    if (!active) return;
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));               // T3
+    const float c_pre = __fdiv_rn(F::M_INT, F::M_FP), c_post = __fdiv_rn(F::M_FP, F::M_INT);
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < ngroups;
+        if (more) {
+            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
+            else load32B<false>(in + 2 * (size_t)gn, wn);
+        }
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+        const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);                        // G1
+        const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
+        const float m4 = max3abs(x[12], x[13], x[14]);
+        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
+        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);       // G2
+        const uint32_t sb = e4m3_encode(t);                                  // G3
+        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
+        const float r = __frcp_rn(d);
+        uint32_t sbyte = 0u, cw[3] = {0u, 0u, 0u};
+        if (sb != 0u) encode_body6<F::EK>(x, sb, d, r, c_pre, c_post, sbyte, cw);   // G4: zero scale -> zeros
+        scales[g] = (uint8_t)sbyte;
+        uint32_t* cp = codes + 3 * (size_t)g;
+        cp[0] = cw[0]; cp[1] = cw[1]; cp[2] = cw[2];
+        if (!more) break;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = wn[i];
+        g = gn;
+    }
+}
+
+}  // namespace absq

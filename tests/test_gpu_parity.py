@@ -356,6 +356,27 @@ def test_argument_validation_on_device(B):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+def test_input_aligned_to_16_but_not_32_bytes(B, oracle, fmt):
+    """The kernels use 256-bit loads when the input allows it; a tensor that starts 16 bytes into an
+    allocation takes their 128-bit fallbacks (plain, Hadamard + stochastic rounding, amax)."""
+    xb = I.generate("cfg2", 70, 1024)
+    rows, cols = xb.shape
+    buf = torch.zeros(rows * cols + 8, dtype=torch.bfloat16, device="cuda")
+    assert buf.data_ptr() % 32 == 0
+    x = buf[8:].view(rows, cols)
+    x.copy_(to_dev(xb))
+    assert x.data_ptr() % 32 == 16
+    mask = oracle.hadamard_sign_mask(5)
+    for flags in (0, B.ABS_F_HADAMARD16 | B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16):
+        codes, scales, ts = B.abs_quantize(fmt, x, opts=B.make_opts(flags, mask, 1234))
+        torch.cuda.synchronize()
+        oc, os_, oa = oracle.quantize(fmt, xb, flags=flags, sign_mask=mask, sr_seed=1234)
+        assert np.float32(ts.item()) == oa
+        assert_same("codes", codes.cpu().numpy()[:oc.size].reshape(oc.shape), oc)
+        assert_same("scales", scales.cpu().numpy()[:os_.size].reshape(os_.shape), os_)
+
+
 def test_guard_bands_stay_untouched(B, oracle):
     """Outputs are written inside their buffers only: sentinel bytes around them survive."""
     for fmt in ALL_FMTS:
