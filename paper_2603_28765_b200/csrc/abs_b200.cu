@@ -256,6 +256,21 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
         }
     }
+    if constexpr (FMT == ABS_FMT_IF3) {
+        // IF3, round-to-nearest
+        const int tgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
+        if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
+            const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
+            const cudaError_t e =
+                alpha.slot ? launch_pdl(quantize3_fast_kernel<true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32)
+                           : launch_pdl(quantize3_fast_kernel<false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32);
+            if (e != cudaSuccess) return ABS_ERR_CUDA;
+            if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
+            return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
     cudaError_t eq = cudaSuccess;
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
     eq = alpha.slot ? launch_pdl(quantize_kernel<FMT, R, S, true>, grid, kThreads, s, (const uint4*)in,         \

@@ -1,5 +1,5 @@
 // Packed round-to-nearest group-quantize kernels for the formats beside IF4 / NVFP4: the block-size-8
-// variants of the 4-bit formats (Sec. 5.1, Table 5) and the 6-bit formats IF6-E2M3 / IF6-E3M2 (Sec. 5.1).  Same
+// variants of the 4-bit formats (Sec. 5.1, Table 5), the 6-bit formats IF6-E2M3 / IF6-E3M2 and IF3 (Sec. 5.1).  Same
 // arithmetic as the generic kernel, bit for bit, in the style of abs_fast4.cuh: persistent grid-stride
 // threads that prefetch the next 32 bytes, f32x2 arithmetic, magic-number integer rounding, Horner packing.
 #pragma once
@@ -273,6 +273,163 @@ quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
         scales[g] = (uint8_t)sbyte;
         uint32_t* cp = codes + 3 * (size_t)g;
         cp[0] = cw[0]; cp[1] = cw[1]; cp[2] = cw[2];
+        if (!more) break;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i] = wn[i];
+        g = gn;
+    }
+}
+
+// ----------------------------------------------------------------------------- 3-bit format (IF3)
+
+constexpr float kMagic4 = 12582916.0f;                // 1.5 * 2^23 + 4: the low three mantissa bits of k + kMagic4 are k + 4
+constexpr uint32_t kMagic4Bits = 0x4B400004u;
+constexpr float kMagic0 = 12582912.0f;                // 1.5 * 2^23
+constexpr uint32_t kMagic0Bits = 0x4B400000u;
+
+// Sign bits of eight bf16 values (four bf16x2 words) moved to bits 3j+2, the sign position of 3-bit code j.
+// PRMT collects the four high bytes of two words (signs at bits 7, 15, 23, 31); the high half of a product
+// with 2^27 + 2^22 + 2^17 + 2^12 drops them at bits 2, 5, 8, 11 (all sixteen partial products fall on
+// different bits, so nothing carries; the mask removes the strays).
+__device__ __forceinline__ uint32_t sign_bits3x8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+    const uint32_t a = __umulhi(__byte_perm(w0, w1, 0x7531) & 0x80808080u, 0x08421000u) & 0x924u;
+    const uint32_t b = __umulhi(__byte_perm(w2, w3, 0x7531) & 0x80808080u, 0x08421000u) & 0x924u;
+    return a | (b << 12);
+}
+
+// Steps 3-10 of Fig. 3a for one group of 16 values of IF3 (E2M0 magnitudes {0, 1, 2, 4} or INT3).
+// E2M0 has no hardware convert.  Round-to-nearest-even onto {0, 1, 2, 4} of a = min(|y|, 4) is the sum of
+// two exact integer roundings, RNE(min(a, 2)) + 2 * RNE(max(a - 2, 0) / 2): the first covers 0..2 (ties
+// 0.5 -> 0, 1.5 -> 2), the second the step from 2 to 4 (tie 3 -> 2); the code index is the sum of the two
+// rounded integers.  Errors are taken on magnitudes (|x| and |v| carry the same sign, so the squares agree).
+// CLAMP as in the 4-bit kernel: only subnormal or saturated scale bytes let |y * 3/4| pass 3.5.
+template <bool CLAMP>
+__device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_t (&w)[8], uint32_t sb, float d, float r,
+                                             uint32_t& sbyte, uint32_t& c_lo, uint32_t& c_hi) {
+    const float c_pre = 0.75f, c_post = __fdiv_rn(4.0f, 3.0f);
+    const float d_int = __fmul_rn(d, c_post);
+    const uint64_t R2 = pack2(r, r), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
+    const uint64_t MG = pack2(kMagic0, kMagic0), NMG = pack2(-kMagic0, -kMagic0);
+    const uint64_t MG4 = pack2(kMagic4, kMagic4), NMG4 = pack2(-kMagic4, -kMagic4);
+    const uint64_t NTWO = pack2(-2.0f, -2.0f), HALF = pack2(0.5f, 0.5f), TWO = pack2(2.0f, 2.0f);
+    float sF[4];
+    uint64_t accI[2];
+    uint32_t fchunk[2], ichunk[2];
+#pragma unroll
+    for (int hgrp = 0; hgrp < 2; ++hgrp) {
+        uint32_t ib[8], kb[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = 8 * hgrp + 2 * i;
+            const uint64_t X = pack2(x[e], x[e + 1]);
+            const uint64_t Y = mul2(X, R2);                                  // E1 (step 3)
+            float y0, y1;
+            unpack2(Y, y0, y1);
+            // E2 (step 4): E2M0 index and value of the magnitude
+            const float a0 = fminf(fabsf(y0), 4.0f), a1 = fminf(fabsf(y1), 4.0f);
+            float u0, u1;
+            unpack2(add2(pack2(a0, a1), NTWO), u0, u1);                      // a - 2: exact for a in [2, 4], unused below 2
+            const uint64_t M1 = add2(pack2(fminf(a0, 2.0f), fminf(a1, 2.0f)), MG);            // RNE(min(a, 2)) + magic
+            const uint64_t M2 = fma2(pack2(fmaxf(u0, 0.0f), fmaxf(u1, 0.0f)), HALF, MG);      // RNE(max(a - 2, 0) / 2) + magic
+            float m10, m11, m20, m21;
+            unpack2(M1, m10, m11);
+            unpack2(M2, m20, m21);
+            ib[2 * i] = __float_as_uint(m10) + __float_as_uint(m20);         // 2 * kMagic0Bits + index
+            ib[2 * i + 1] = __float_as_uint(m11) + __float_as_uint(m21);
+            float v0, v1;
+            unpack2(fma2(add2(M2, NMG), TWO, add2(M1, NMG)), v0, v1);        // the E2M0 magnitude: r1 + 2 * r2
+            // E3 (steps 5-6) on magnitudes
+            const float e0 = __fmaf_rn(v0, -d, fabsf(x[e])), e1 = __fmaf_rn(v1, -d, fabsf(x[e + 1]));
+            const int ch = 2 * hgrp;
+            sF[ch] = (i == 0) ? __fmul_rn(e0, e0) : __fmaf_rn(e0, e0, sF[ch]);
+            sF[ch + 1] = (i == 0) ? __fmul_rn(e1, e1) : __fmaf_rn(e1, e1, sF[ch + 1]);
+            // E4-E5 (steps 7-9): integer candidate, signed
+            uint64_t KZ = fma2(Y, CP2, MG4);
+            if constexpr (CLAMP) {
+                float k0, k1;
+                unpack2(KZ, k0, k1);
+                k0 = fminf(fmaxf(k0, kMagic4 - 3.0f), kMagic4 + 3.0f);
+                k1 = fminf(fmaxf(k1, kMagic4 - 3.0f), kMagic4 + 3.0f);
+                KZ = pack2(k0, k1);
+            }
+            const uint64_t FI = fma2(add2(KZ, NMG4), NDI2, X);
+            accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
+            float kz0, kz1;
+            unpack2(KZ, kz0, kz1);
+            kb[2 * i] = __float_as_uint(kz0);
+            kb[2 * i + 1] = __float_as_uint(kz1);
+        }
+        // eight 3-bit fields by Horner on the raw sums; the constant parts are removed afterwards
+        constexpr uint32_t kS8 = 0x249249u;                                  // 1 + 8 + ... + 8^7
+        constexpr uint32_t kConstF = 2u * kMagic0Bits * kS8;                 // leaves the indices 0..3
+        constexpr uint32_t kConstI = (kMagic4Bits - 4u) * kS8;               // leaves the fields k + 4
+        uint32_t fc = ib[7], ic = kb[7];
+#pragma unroll
+        for (int j = 6; j >= 0; --j) {
+            fc = fc * 8u + ib[j];
+            ic = ic * 8u + kb[j];
+        }
+        fchunk[hgrp] = (fc - kConstF) | sign_bits3x8(w[4 * hgrp], w[4 * hgrp + 1], w[4 * hgrp + 2], w[4 * hgrp + 3]);
+        ichunk[hgrp] = (ic - kConstI) ^ 0x924924u;                           // offset-binary -> two's complement
+    }
+    float i0, i1, i2, i3;
+    unpack2(accI[0], i0, i1); unpack2(accI[1], i2, i3);
+    const float E_fp = __fadd_rn(__fadd_rn(sF[0], sF[1]), __fadd_rn(sF[2], sF[3]));   // S1-S2 (step 10)
+    const float E_int = __fadd_rn(__fadd_rn(i0, i1), __fadd_rn(i2, i3));
+    const bool flag = E_int < E_fp;
+    const uint32_t c0 = flag ? ichunk[0] : fchunk[0], c1 = flag ? ichunk[1] : fchunk[1];
+    c_lo = c0 | (c1 << 24);                                                  // S4: 2 x 24 bits -> 48 bits
+    c_hi = c1 >> 8;
+    sbyte = sb | (flag ? 0x80u : 0u);                                        // S3
+}
+
+template <bool FROM_SLOT>
+__global__ void __launch_bounds__(256, 3)
+quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32) {
+    pdl_launch_dependents();
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    pdl_wait();
+    uint32_t w[8], wn[8];
+    const bool active = g < ngroups;
+    if (active) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
+        else load32B<false>(in + 2 * (size_t)g, w);
+    }
+    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    if (!active) return;
+    const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 4.0f));                  // T3
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < ngroups;
+        if (more) {
+            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
+            else load32B<false>(in + 2 * (size_t)gn, wn);
+        }
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+        const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);                        // G1
+        const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
+        const float m4 = max3abs(x[12], x[13], x[14]);
+        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
+        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);       // G2
+        const uint32_t sb = e4m3_encode(t);                                  // G3
+        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
+        const float r = __frcp_rn(d);
+        uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
+        if ((sb - 8u) >= 118u) {
+            if (sb != 0u) encode_body3<true>(x, w, sb, d, r, sbyte, c_lo, c_hi);             // G4: zero scale -> zeros
+        } else {
+            encode_body3<false>(x, w, sb, d, r, sbyte, c_lo, c_hi);
+        }
+        scales[g] = (uint8_t)sbyte;
+        uint16_t* cp = codes + 3 * (size_t)g;                                // 6 bytes per group
+        cp[0] = (uint16_t)c_lo; cp[1] = (uint16_t)(c_lo >> 16); cp[2] = (uint16_t)c_hi;
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
