@@ -1,6 +1,9 @@
 """Per-configuration throughput table of the library's kernels (run on a B200 machine).
 
-    python -m paper_2603_28765_b200.report [--quick]
+    python -m paper_2603_28765_b200.report [--quick] [--only CFG[:FMT]] [--rows R]
+
+``--only cfg4:if4 --rows 4096 --quick`` restricts the run to one configuration (and format) at a reduced
+row count: the small case to put under a profiler.
 
 For every benchmark configuration and format it times, with CUDA events over back-to-back calls
 that rotate over enough buffer sets to defeat L2 reuse between calls:
@@ -23,6 +26,8 @@ def main():
 
     ap = argparse.ArgumentParser()
     ap.add_argument("--quick", action="store_true", help="fewer repetitions")
+    ap.add_argument("--only", default="", help="one configuration, optionally one format: cfg4 or cfg4:if4")
+    ap.add_argument("--rows", type=int, default=0, help="override the row count (smaller case for profiling)")
     args = ap.parse_args()
     L = B.lib()
     reps = 10 if args.quick else 40
@@ -49,7 +54,14 @@ def main():
                                ("if4_bs8", 0), ("if3_bs8", 0), ("nvfp4_bs8", 0)]),
     ]
     sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    only_cfg, _, only_fmt = args.only.partition(":")
     for name, rows, cols, variants in rows_cfg:
+        if only_cfg and name != only_cfg:
+            continue
+        if only_fmt:
+            variants = [v for v in variants if v[0] == only_fmt]
+        if args.rows:
+            rows = args.rows
         n = rows * cols
         k = max(4, int(1.0e9 // (n * 2)))
         xs = [(torch.randn(rows, cols, device="cuda") * (1 + 3 * torch.rand(rows, 1, device="cuda"))).to(torch.bfloat16)
