@@ -132,8 +132,10 @@ ABS_API abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t
  * give for its transpose [cols, rows]: groups are 16 consecutive rows of one column,
  *   codes_t_u8    [cols, rows*b/8]   scales_t_e4m3 [cols, rows/16]   alpha as for abs_quantize.
  * The transpose is never materialised.  rows and cols must be multiples of 16; formats ABS_FMT_IF4 and
- * ABS_FMT_NVFP4; flags accepted: ABS_F_ALPHA_GIVEN and ABS_F_HADAMARD16 (the transform then runs along the
- * groups, i.e. down the columns: the paper's recipe for both operands of the weight-gradient product).  abs_dequantize(fmt, ..., cols, rows, ...)
+ * ABS_FMT_NVFP4; flags accepted: ABS_F_ALPHA_GIVEN, ABS_F_HADAMARD16 (the transform then runs along the
+ * groups, i.e. down the columns: the paper's recipe for both operands of the weight-gradient product),
+ * ABS_F_STOCHASTIC and ABS_F_SR_SCALE_17_16 (App. B; element indices, hence the random stream, are those of
+ * the transposed matrix); any other flag is ABS_ERR_FLAGS.  abs_dequantize(fmt, ..., cols, rows, ...)
  * turns the result back into the transposed matrix. */
 ABS_API abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
                                              void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,

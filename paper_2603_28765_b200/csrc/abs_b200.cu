@@ -10,6 +10,7 @@
 #include "abs_fast4.cuh"
 #include "abs_opt4.cuh"
 #include "abs_fastx.cuh"
+#include "abs_trans4.cuh"
 #include "abs_generic.cuh"
 
 #include <atomic>
@@ -538,7 +539,8 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     if (opts) o = *opts;
     if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
     if (rows < 0 || cols < 0 || (cols % 16) != 0 || (rows % 16) != 0) return ABS_ERR_SHAPE;
-    if ((o.flags & ~(uint32_t)(ABS_F_ALPHA_GIVEN | ABS_F_HADAMARD16)) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ~(uint32_t)(ABS_F_ALPHA_GIVEN | ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16)) || o._pad)
+        return ABS_ERR_FLAGS;
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !codes_t_u8 || !scales_t_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(codes_t_u8) || !aligned16(scales_t_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -567,15 +569,18 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     uint2* ct = (uint2*)codes_t_u8;
     uint8_t* stp = (uint8_t*)scales_t_e4m3;
     const uint32_t mask = o.had_sign_mask;
-#define ABS_LAUNCH_T(I, S, R, M, SLOT, GEN)                                                                         \
+#define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
     do {                                                                                                            \
-        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, Q, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  kTransSmemBytes);                                                                  \
         if (e == cudaSuccess)                                                                                       \
-            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, M>, in, ct, stp, src, rows, cols, mask, \
-                                   SLOT, GEN);                                                                      \
+            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, Q, M>, in, ct, stp, src, rows, cols, mask, \
+                                   SLOT, GEN, mul, k0, k1);                                                         \
     } while (0)
 
+    const bool sr = o.flags & ABS_F_STOCHASTIC;
+    const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
+    const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;
@@ -584,7 +589,7 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
         const float denom = 6.0f * 448.0f;
         if (rht) {
             // the maximum is taken over the transformed column groups: same tile walk, MODE 1
-            ABS_LAUNCH_T(false, false, true, 1, slot, gen);
+            ABS_LAUNCH_T(false, false, true, false, 1, slot, gen);
             if (e != cudaSuccess) return ABS_ERR_CUDA;
         } else {
             abs_status_t rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
@@ -595,13 +600,22 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
         src.denom = denom;
     }
     unsigned long long* no_slot = nullptr;
-    if (fmt == ABS_FMT_IF4) {
-        if (rht) { if (src.slot) ABS_LAUNCH_T(true, true, true, 0, no_slot, 0u); else ABS_LAUNCH_T(true, false, true, 0, no_slot, 0u); }
-        else { if (src.slot) ABS_LAUNCH_T(true, true, false, 0, no_slot, 0u); else ABS_LAUNCH_T(true, false, false, 0, no_slot, 0u); }
-    } else {
-        if (rht) { if (src.slot) ABS_LAUNCH_T(false, true, true, 0, no_slot, 0u); else ABS_LAUNCH_T(false, false, true, 0, no_slot, 0u); }
-        else { if (src.slot) ABS_LAUNCH_T(false, true, false, 0, no_slot, 0u); else ABS_LAUNCH_T(false, false, false, 0, no_slot, 0u); }
-    }
+#define ABS_LAUNCH_T2(I, R, Q)                                                                                      \
+    do {                                                                                                            \
+        if (src.slot) ABS_LAUNCH_T(I, true, R, Q, 0, no_slot, 0u);                                                  \
+        else ABS_LAUNCH_T(I, false, R, Q, 0, no_slot, 0u);                                                          \
+    } while (0)
+#define ABS_LAUNCH_T3(I)                                                                                            \
+    do {                                                                                                            \
+        if (rht && sr) ABS_LAUNCH_T2(I, true, true);                                                                \
+        else if (rht) ABS_LAUNCH_T2(I, true, false);                                                                \
+        else if (sr) ABS_LAUNCH_T2(I, false, true);                                                                 \
+        else ABS_LAUNCH_T2(I, false, false);                                                                        \
+    } while (0)
+    if (fmt == ABS_FMT_IF4) ABS_LAUNCH_T3(true);
+    else ABS_LAUNCH_T3(false);
+#undef ABS_LAUNCH_T3
+#undef ABS_LAUNCH_T2
 #undef ABS_LAUNCH_T
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }

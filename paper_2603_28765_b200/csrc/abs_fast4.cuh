@@ -200,162 +200,6 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
 }
 
 
-// ----------------------------------------------------------------------------- transposed quantize
-
-// Quantizes the TRANSPOSE of a row-major [rows, cols] matrix without materialising it: groups are 16
-// consecutive ROWS of one column (Sec. 4.1: both operands of the weight-gradient product are quantized
-// along the token dimension).  Output = what the plain kernel would give for the [cols, rows] matrix:
-// codes_t [cols, rows/2 bytes], scales_t [cols, rows/16].
-// Persistent blocks walk over tiles of 64 rows x 256 columns.  A tile is brought into shared memory with
-// 16-byte asynchronous copies (cp.async), double buffered: the copies of the block's next tile are in
-// flight while it encodes the current one.  Thread c reads its column's values down the tile and encodes
-// the four groups of 16 rows; those are neighbours in the transposed output, so their codes leave as one
-// 256-bit store and their scale bytes as one 32-bit store whenever the tile is complete and the output
-// addresses allow it.
-#ifndef ABS_TRANS_UNROLL
-#define ABS_TRANS_UNROLL 4
-#endif
-constexpr int kTransUnroll = ABS_TRANS_UNROLL;
-constexpr int kTransTileCols = 256;
-constexpr int kTransTileRowBlocks = 4;
-constexpr int kTransStageElems = 16 * kTransTileRowBlocks * kTransTileCols;        // bf16 elements per stage
-constexpr int kTransSmemBytes = 2 * kTransStageElems * 2;                           // two stages
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
-
-// MODE 0: quantize.  MODE 1: only the maximum of the Hadamard-transformed column groups (the amax pass of
-// the transposed path with the Hadamard option; publishes a tagged maximum like amax_kernel).
-template <bool HAS_INT, bool FROM_SLOT, bool RHT, int MODE>
-__global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_t* __restrict__ in,
-                                                                   uint2* __restrict__ codes_t,
-                                                                   uint8_t* __restrict__ scales_t,
-                                                                   const AlphaSrc alpha_src, int64_t rows, int64_t cols,
-                                                                   uint32_t sign_mask, unsigned long long* amax_slot,
-                                                                   uint32_t amax_gen) {
-    extern __shared__ __align__(16) uint16_t trans_smem[];
-    pdl_launch_dependents();
-    pdl_wait();
-    float alpha = 1.0f, inv_a6 = 1.0f;
-    if constexpr (MODE == 0) {
-        alpha = resolve_alpha<FROM_SLOT>(alpha_src);                         // T2
-        inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                          // T3
-    }
-    uint32_t local_max = 0u;
-    const int64_t rblocks = rows / 16;
-    const int64_t ntx = (cols + kTransTileCols - 1) / kTransTileCols;
-    const int64_t nty = (rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks;
-    const int64_t ntiles = ntx * nty;
-    // vector stores need 32-byte aligned code addresses and 4-byte aligned scale addresses for every column
-    const bool vec_ok = (rblocks % kTransTileRowBlocks) == 0 &&
-                        ((reinterpret_cast<uintptr_t>(codes_t) & 31u) == 0) && ((reinterpret_cast<uintptr_t>(scales_t) & 3u) == 0);
-
-    // issue the asynchronous copies of tile t into stage s (one commit group per call, possibly empty)
-    auto issue = [&](int64_t t, int s) {
-        if (t < ntiles) {
-            const int64_t ty = t / ntx, tx = t - ty * ntx;
-            const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
-            const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
-            const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
-            uint16_t* stage = trans_smem + s * kTransStageElems;
-            const uint16_t* src = in + rb0 * 16 * cols + c0;
-            if (ncols == kTransTileCols) {               // full-width tile: 32 chunks of 16 bytes per row
-                for (int ch = threadIdx.x; ch < 16 * nrb * (kTransTileCols / 8); ch += blockDim.x) {
-                    const int r = ch >> 5, q = ch & 31;
-                    cp_async16(stage + r * kTransTileCols + q * 8, src + (int64_t)r * cols + q * 8);
-                }
-            } else {                                     // ragged last column tile
-                const int chunks_per_row = ncols / 8;
-                for (int ch = threadIdx.x; ch < 16 * nrb * chunks_per_row; ch += blockDim.x) {
-                    const int r = ch / chunks_per_row, q = ch - r * chunks_per_row;
-                    cp_async16(stage + r * kTransTileCols + q * 8, src + (int64_t)r * cols + q * 8);
-                }
-            }
-        }
-        cp_async_commit();
-    };
-
-    int s = 0;
-    int64_t t = blockIdx.x;
-    issue(t, 0);
-    for (; t < ntiles; t += gridDim.x, s ^= 1) {
-        issue(t + gridDim.x, s ^ 1);                 // prefetch the block's next tile into the other stage
-        cp_async_wait_all_but_one();                 // this thread's copies of tile t have landed
-        __syncthreads();                             // ... and everybody else's
-        const int64_t ty = t / ntx, tx = t - ty * ntx;
-        const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
-        const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
-        const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
-        const uint16_t* stage = trans_smem + s * kTransStageElems;
-        const int c = threadIdx.x;
-        if (c < ncols) {
-            uint32_t cw[2 * kTransTileRowBlocks];
-            uint32_t sbytes = 0u;
-#pragma unroll kTransUnroll
-            for (int k = 0; k < kTransTileRowBlocks; ++k) {
-                if (k >= nrb) break;
-                float x[16];
-                const uint16_t* colp = stage + 16 * k * kTransTileCols + c;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) x[i] = __uint_as_float((uint32_t)colp[i * kTransTileCols] << 16);
-                if constexpr (RHT) hadamard16(x, sign_mask);         // along the group, i.e. down the column
-                if constexpr (MODE == 1) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) local_max = max(local_max, __float_as_uint(x[i]) & 0x7FFFFFFFu);
-                    continue;
-                }
-                const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
-                const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
-                const float m4 = max3abs(x[12], x[13], x[14]);
-                const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));   // G1
-                const float tt = __fmul_rn(gmax, inv_a6);                                // G2
-                const uint32_t sb = e4m3_encode(tt);                                     // G3
-                const float d = __fmul_rn(e4m3_value(sb), alpha);                        // G5
-                const float r = __frcp_rn(d);
-                uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
-                if ((sb - 8u) >= 118u) {
-                    if (sb != 0u) encode_body4<HAS_INT, HAS_INT>(x, sb, d, r, sbyte, c_lo, c_hi);
-                } else {
-                    encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
-                }
-                const int64_t g = (c0 + c) * rblocks + rb0 + k;      // group index in the transposed matrix
-                if (vec_ok) {
-                    // k is a runtime index: select the slot without dynamic register indexing
-#pragma unroll
-                    for (int j = 0; j < kTransTileRowBlocks; ++j)
-                        if (j == k) { cw[2 * j] = c_lo; cw[2 * j + 1] = c_hi; }
-                    sbytes |= sbyte << (8 * k);
-                } else {
-                    scales_t[g] = (uint8_t)sbyte;
-                    codes_t[g] = make_uint2(c_lo, c_hi);
-                }
-            }
-            if (MODE == 0 && vec_ok) {
-                const int64_t g0 = (c0 + c) * rblocks + rb0;
-                store32B<true>(codes_t + g0, reinterpret_cast<const uint32_t(&)[8]>(cw));
-                *reinterpret_cast<uint32_t*>(scales_t + g0) = sbytes;
-            }
-        }
-        __syncthreads();                             // the stage may be overwritten by the next prefetch
-    }
-    if constexpr (MODE == 1) {
-        __shared__ uint32_t warp_max[8];
-        local_max = __reduce_max_sync(0xFFFFFFFFu, local_max);
-        if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = local_max;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t m = 0u;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) m = max(m, warp_max[w]);
-            atomicMax(amax_slot, ((unsigned long long)amax_gen << 32) | m);
-        }
-    }
-}
-
 // ----------------------------------------------------------------------------- 4-bit dequantize
 
 // FP32 -> packed bf16 pair, round to nearest even (Sec. 4.1).

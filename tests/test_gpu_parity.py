@@ -470,6 +470,17 @@ def test_transposed_quantize_equals_quantize_of_transpose(B, oracle, fmt):
         assert np.float32(ts.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
         assert_same("scales_t rht", st.cpu().numpy().reshape(cols, -1), osc)
         assert_same("codes_t rht", ct.cpu().numpy().reshape(cols, -1), oc)
+    # the gradient recipe of Sec. 4.1 / App. B along the token dimension: Hadamard, stochastic rounding, 17/16
+    for flags in (B.ABS_F_STOCHASTIC, B.ABS_F_HADAMARD16 | B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16):
+        for name, rows, cols in (("cfg4", 320, 2048), ("cfg2", 80, 528)):
+            xb = I.generate(name, rows, cols)
+            ct, st, ts = B.abs_quantize_transposed(fmt, to_dev(xb), opts=B.make_opts(flags, mask, 0xABCDEF0123))
+            torch.cuda.synchronize()
+            oc, osc, oa = oracle.quantize(fmt, np.ascontiguousarray(xb.T), flags=flags, sign_mask=mask,
+                                          sr_seed=0xABCDEF0123, threads=THREADS)
+            assert np.float32(ts.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+            assert_same("scales_t sr", st.cpu().numpy().reshape(cols, -1), osc)
+            assert_same("codes_t sr", ct.cpu().numpy().reshape(cols, -1), oc)
     # alpha given, and the argument checks
     xb = I.generate("cfg5", 64, 256)
     ts = torch.tensor([0.02], dtype=torch.float32, device="cuda")
@@ -481,9 +492,9 @@ def test_transposed_quantize_equals_quantize_of_transpose(B, oracle, fmt):
     assert L.abs_quantize_transposed(2, x.data_ptr(), 64, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(), None, None) == 4
     assert L.abs_quantize_transposed(1, x.data_ptr(), 40, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(), None, None) == 2
     import ctypes
-    sr = B.make_opts(B.ABS_F_STOCHASTIC)
+    bad = B.make_opts(B.ABS_F_SCALES_SWIZZLED)
     assert L.abs_quantize_transposed(1, x.data_ptr(), 64, 256, ct.data_ptr(), st.data_ptr(), ts.data_ptr(),
-                                     ctypes.byref(sr), None) == 5
+                                     ctypes.byref(bad), None) == 5
 
 
 @pytest.mark.parametrize("fmt", [0, 1])
