@@ -257,15 +257,16 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
         }
     }
-    if constexpr (FMT == ABS_FMT_IF3) {
-        // IF3, round-to-nearest
+    if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
+        // IF3 and its block-size-8 variant, round-to-nearest
+        constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
         const int tgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const cudaError_t e =
-                alpha.slot ? launch_pdl(quantize3_fast_kernel<true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                alpha.slot ? launch_pdl(quantize3_fast_kernel<kG, true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
                                         (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32)
-                           : launch_pdl(quantize3_fast_kernel<false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                           : launch_pdl(quantize3_fast_kernel<kG, false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
                                         (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32);
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
@@ -321,6 +322,33 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
 #undef ABS_LAUNCH_D3
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
+        const int bgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
+            constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
+            const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
+            const cudaError_t e8 =
+                a32 ? launch_pdl(dequantize4_bs8_kernel<kInt, true>, bgrid, kThreads, s, (const uint2*)codes,
+                                 (const uint16_t*)scales, alpha, (int32_t)ngroups, (uint4*)out)
+                    : launch_pdl(dequantize4_bs8_kernel<kInt, false>, bgrid, kThreads, s, (const uint2*)codes,
+                                 (const uint16_t*)scales, alpha, (int32_t)ngroups, (uint4*)out);
+            return (e8 == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
+    if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
+        // 3-bit codes widened to nibbles and decoded like the 4-bit formats
+        const int tgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
+            constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
+            const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
+            const cudaError_t e3 =
+                a32 ? launch_pdl(dequantize3_fast_kernel<kG, true>, tgrid, kThreads, s, (const uint16_t*)codes,
+                                 (const uint8_t*)scales, alpha, (int32_t)ngroups, (uint4*)out)
+                    : launch_pdl(dequantize3_fast_kernel<kG, false>, tgrid, kThreads, s, (const uint16_t*)codes,
+                                 (const uint8_t*)scales, alpha, (int32_t)ngroups, (uint4*)out);
+            return (e3 == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
         }
     }
     cudaError_t e;

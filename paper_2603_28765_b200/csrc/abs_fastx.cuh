@@ -297,85 +297,89 @@ __device__ __forceinline__ uint32_t sign_bits3x8(uint32_t w0, uint32_t w1, uint3
     return a | (b << 12);
 }
 
-// Steps 3-10 of Fig. 3a for one group of 16 values of IF3 (E2M0 magnitudes {0, 1, 2, 4} or INT3).
+// Candidates of EIGHT values of IF3 (E2M0 magnitudes {0, 1, 2, 4} or INT3), steps 3-9 of Fig. 3a: the
+// 24-bit chunks of FP and integer codes and the two error chains (even / odd elements) of each candidate.
 // E2M0 has no hardware convert.  Round-to-nearest-even onto {0, 1, 2, 4} of a = min(|y|, 4) is the sum of
 // two exact integer roundings, RNE(min(a, 2)) + 2 * RNE(max(a - 2, 0) / 2): the first covers 0..2 (ties
 // 0.5 -> 0, 1.5 -> 2), the second the step from 2 to 4 (tie 3 -> 2); the code index is the sum of the two
-// rounded integers.  Errors are taken on magnitudes (|x| and |v| carry the same sign, so the squares agree).
-// CLAMP as in the 4-bit kernel: only subnormal or saturated scale bytes let |y * 3/4| pass 3.5.
+// rounded integers.  FP errors are taken on magnitudes (|x| and |v| carry the same sign, so the squares
+// agree).  CLAMP as in the 4-bit kernel: only subnormal or saturated scale bytes let |y * 3/4| pass 3.5.
+// w holds the four bf16x2 words of the eight values (for their sign bits).
 template <bool CLAMP>
-__device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_t (&w)[8], uint32_t sb, float d, float r,
-                                             uint32_t& sbyte, uint32_t& c_lo, uint32_t& c_hi) {
+__device__ __forceinline__ void candidates3x8(const float* x, const uint32_t* w, float d, float r, uint32_t& fchunk,
+                                              uint32_t& ichunk, float& f0, float& f1, float& i0, float& i1) {
     const float c_pre = 0.75f, c_post = __fdiv_rn(4.0f, 3.0f);
     const float d_int = __fmul_rn(d, c_post);
     const uint64_t R2 = pack2(r, r), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
     const uint64_t MG = pack2(kMagic0, kMagic0), NMG = pack2(-kMagic0, -kMagic0);
     const uint64_t MG4 = pack2(kMagic4, kMagic4), NMG4 = pack2(-kMagic4, -kMagic4);
     const uint64_t NTWO = pack2(-2.0f, -2.0f), HALF = pack2(0.5f, 0.5f), TWO = pack2(2.0f, 2.0f);
-    float sF[4];
-    uint64_t accI[2];
-    uint32_t fchunk[2], ichunk[2];
+    uint64_t accI = 0;
+    uint32_t ib[8], kb[8];
 #pragma unroll
-    for (int hgrp = 0; hgrp < 2; ++hgrp) {
-        uint32_t ib[8], kb[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int e = 8 * hgrp + 2 * i;
-            const uint64_t X = pack2(x[e], x[e + 1]);
-            const uint64_t Y = mul2(X, R2);                                  // E1 (step 3)
-            float y0, y1;
-            unpack2(Y, y0, y1);
-            // E2 (step 4): E2M0 index and value of the magnitude
-            const float a0 = fminf(fabsf(y0), 4.0f), a1 = fminf(fabsf(y1), 4.0f);
-            float u0, u1;
-            unpack2(add2(pack2(a0, a1), NTWO), u0, u1);                      // a - 2: exact for a in [2, 4], unused below 2
-            const uint64_t M1 = add2(pack2(fminf(a0, 2.0f), fminf(a1, 2.0f)), MG);            // RNE(min(a, 2)) + magic
-            const uint64_t M2 = fma2(pack2(fmaxf(u0, 0.0f), fmaxf(u1, 0.0f)), HALF, MG);      // RNE(max(a - 2, 0) / 2) + magic
-            float m10, m11, m20, m21;
-            unpack2(M1, m10, m11);
-            unpack2(M2, m20, m21);
-            ib[2 * i] = __float_as_uint(m10) + __float_as_uint(m20);         // 2 * kMagic0Bits + index
-            ib[2 * i + 1] = __float_as_uint(m11) + __float_as_uint(m21);
-            float v0, v1;
-            unpack2(fma2(add2(M2, NMG), TWO, add2(M1, NMG)), v0, v1);        // the E2M0 magnitude: r1 + 2 * r2
-            // E3 (steps 5-6) on magnitudes
-            const float e0 = __fmaf_rn(v0, -d, fabsf(x[e])), e1 = __fmaf_rn(v1, -d, fabsf(x[e + 1]));
-            const int ch = 2 * hgrp;
-            sF[ch] = (i == 0) ? __fmul_rn(e0, e0) : __fmaf_rn(e0, e0, sF[ch]);
-            sF[ch + 1] = (i == 0) ? __fmul_rn(e1, e1) : __fmaf_rn(e1, e1, sF[ch + 1]);
-            // E4-E5 (steps 7-9): integer candidate, signed
-            uint64_t KZ = fma2(Y, CP2, MG4);
-            if constexpr (CLAMP) {
-                float k0, k1;
-                unpack2(KZ, k0, k1);
-                k0 = fminf(fmaxf(k0, kMagic4 - 3.0f), kMagic4 + 3.0f);
-                k1 = fminf(fmaxf(k1, kMagic4 - 3.0f), kMagic4 + 3.0f);
-                KZ = pack2(k0, k1);
-            }
-            const uint64_t FI = fma2(add2(KZ, NMG4), NDI2, X);
-            accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
-            float kz0, kz1;
-            unpack2(KZ, kz0, kz1);
-            kb[2 * i] = __float_as_uint(kz0);
-            kb[2 * i + 1] = __float_as_uint(kz1);
+    for (int i = 0; i < 4; ++i) {
+        const uint64_t X = pack2(x[2 * i], x[2 * i + 1]);
+        const uint64_t Y = mul2(X, R2);                                      // E1 (step 3)
+        float y0, y1;
+        unpack2(Y, y0, y1);
+        // E2 (step 4): E2M0 index and value of the magnitude
+        const float a0 = fminf(fabsf(y0), 4.0f), a1 = fminf(fabsf(y1), 4.0f);
+        float u0, u1;
+        unpack2(add2(pack2(a0, a1), NTWO), u0, u1);                          // a - 2: exact for a in [2, 4], unused below 2
+        const uint64_t M1 = add2(pack2(fminf(a0, 2.0f), fminf(a1, 2.0f)), MG);                // RNE(min(a, 2)) + magic
+        const uint64_t M2 = fma2(pack2(fmaxf(u0, 0.0f), fmaxf(u1, 0.0f)), HALF, MG);          // RNE(max(a - 2, 0) / 2) + magic
+        float m10, m11, m20, m21;
+        unpack2(M1, m10, m11);
+        unpack2(M2, m20, m21);
+        ib[2 * i] = __float_as_uint(m10) + __float_as_uint(m20);             // 2 * kMagic0Bits + index
+        ib[2 * i + 1] = __float_as_uint(m11) + __float_as_uint(m21);
+        float v0, v1;
+        unpack2(fma2(add2(M2, NMG), TWO, add2(M1, NMG)), v0, v1);            // the E2M0 magnitude: r1 + 2 * r2
+        // E3 (steps 5-6) on magnitudes
+        const float e0 = __fmaf_rn(v0, -d, fabsf(x[2 * i])), e1 = __fmaf_rn(v1, -d, fabsf(x[2 * i + 1]));
+        f0 = (i == 0) ? __fmul_rn(e0, e0) : __fmaf_rn(e0, e0, f0);
+        f1 = (i == 0) ? __fmul_rn(e1, e1) : __fmaf_rn(e1, e1, f1);
+        // E4-E5 (steps 7-9): integer candidate, signed
+        uint64_t KZ = fma2(Y, CP2, MG4);
+        if constexpr (CLAMP) {
+            float k0, k1;
+            unpack2(KZ, k0, k1);
+            k0 = fminf(fmaxf(k0, kMagic4 - 3.0f), kMagic4 + 3.0f);
+            k1 = fminf(fmaxf(k1, kMagic4 - 3.0f), kMagic4 + 3.0f);
+            KZ = pack2(k0, k1);
         }
-        // eight 3-bit fields by Horner on the raw sums; the constant parts are removed afterwards
-        constexpr uint32_t kS8 = 0x249249u;                                  // 1 + 8 + ... + 8^7
-        constexpr uint32_t kConstF = 2u * kMagic0Bits * kS8;                 // leaves the indices 0..3
-        constexpr uint32_t kConstI = (kMagic4Bits - 4u) * kS8;               // leaves the fields k + 4
-        uint32_t fc = ib[7], ic = kb[7];
-#pragma unroll
-        for (int j = 6; j >= 0; --j) {
-            fc = fc * 8u + ib[j];
-            ic = ic * 8u + kb[j];
-        }
-        fchunk[hgrp] = (fc - kConstF) | sign_bits3x8(w[4 * hgrp], w[4 * hgrp + 1], w[4 * hgrp + 2], w[4 * hgrp + 3]);
-        ichunk[hgrp] = (ic - kConstI) ^ 0x924924u;                           // offset-binary -> two's complement
+        const uint64_t FI = fma2(add2(KZ, NMG4), NDI2, X);
+        accI = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI);
+        float kz0, kz1;
+        unpack2(KZ, kz0, kz1);
+        kb[2 * i] = __float_as_uint(kz0);
+        kb[2 * i + 1] = __float_as_uint(kz1);
     }
-    float i0, i1, i2, i3;
-    unpack2(accI[0], i0, i1); unpack2(accI[1], i2, i3);
-    const float E_fp = __fadd_rn(__fadd_rn(sF[0], sF[1]), __fadd_rn(sF[2], sF[3]));   // S1-S2 (step 10)
-    const float E_int = __fadd_rn(__fadd_rn(i0, i1), __fadd_rn(i2, i3));
+    unpack2(accI, i0, i1);
+    // eight 3-bit fields by Horner on the raw sums; the constant parts are removed afterwards
+    constexpr uint32_t kS8 = 0x249249u;                                      // 1 + 8 + ... + 8^7
+    constexpr uint32_t kConstF = 2u * kMagic0Bits * kS8;                     // leaves the indices 0..3
+    constexpr uint32_t kConstI = (kMagic4Bits - 4u) * kS8;                   // leaves the fields k + 4
+    uint32_t fc = ib[7], ic = kb[7];
+#pragma unroll
+    for (int j = 6; j >= 0; --j) {
+        fc = fc * 8u + ib[j];
+        ic = ic * 8u + kb[j];
+    }
+    fchunk = (fc - kConstF) | sign_bits3x8(w[0], w[1], w[2], w[3]);
+    ichunk = (ic - kConstI) ^ 0x924924u;                                     // offset-binary -> two's complement
+}
+
+// Steps 3-10 for one group of 16 values: both halves under one scale, selection on (S0 + S1) + (S2 + S3).
+template <bool CLAMP>
+__device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_t (&w)[8], uint32_t sb, float d, float r,
+                                             uint32_t& sbyte, uint32_t& c_lo, uint32_t& c_hi) {
+    uint32_t fchunk[2], ichunk[2];
+    float f[4], in[4];
+    candidates3x8<CLAMP>(x, w, d, r, fchunk[0], ichunk[0], f[0], f[1], in[0], in[1]);
+    candidates3x8<CLAMP>(x + 8, w + 4, d, r, fchunk[1], ichunk[1], f[2], f[3], in[2], in[3]);
+    const float E_fp = __fadd_rn(__fadd_rn(f[0], f[1]), __fadd_rn(f[2], f[3]));       // S1-S2 (step 10)
+    const float E_int = __fadd_rn(__fadd_rn(in[0], in[1]), __fadd_rn(in[2], in[3]));
     const bool flag = E_int < E_fp;
     const uint32_t c0 = flag ? ichunk[0] : fchunk[0], c1 = flag ? ichunk[1] : fchunk[1];
     c_lo = c0 | (c1 << 24);                                                  // S4: 2 x 24 bits -> 48 bits
@@ -383,7 +387,8 @@ __device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_
     sbyte = sb | (flag ? 0x80u : 0u);                                        // S3
 }
 
-template <bool FROM_SLOT>
+// G = 16: one scale per thread's 16 values.  G = 8 (IF3-BS8): each half has its own scale and selection.
+template <int G, bool FROM_SLOT>
 __global__ void __launch_bounds__(256, 3)
 quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes, uint8_t* __restrict__ scales,
                       const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32) {
@@ -413,27 +418,144 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
             x[2 * i] = __uint_as_float(w[i] << 16);
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
-        const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);                        // G1
-        const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
-        const float m4 = max3abs(x[12], x[13], x[14]);
-        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
-        const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);       // G2
-        const uint32_t sb = e4m3_encode(t);                                  // G3
-        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
-        const float r = __frcp_rn(d);
-        uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
-        if ((sb - 8u) >= 118u) {
-            if (sb != 0u) encode_body3<true>(x, w, sb, d, r, sbyte, c_lo, c_hi);             // G4: zero scale -> zeros
+        uint32_t c_lo = 0u, c_hi = 0u;
+        if constexpr (G == 16) {
+            const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);                    // G1
+            const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
+            const float m4 = max3abs(x[12], x[13], x[14]);
+            const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
+            const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);   // G2
+            const uint32_t sb = e4m3_encode(t);                              // G3
+            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
+            const float r = __frcp_rn(d);
+            uint32_t sbyte = 0u;
+            if ((sb - 8u) >= 118u) {
+                if (sb != 0u) encode_body3<true>(x, w, sb, d, r, sbyte, c_lo, c_hi);         // G4: zero scale -> zeros
+            } else {
+                encode_body3<false>(x, w, sb, d, r, sbyte, c_lo, c_hi);
+            }
+            scales[g] = (uint8_t)sbyte;
         } else {
-            encode_body3<false>(x, w, sb, d, r, sbyte, c_lo, c_hi);
+            uint32_t chunk[2] = {0u, 0u}, sbytes = 0u;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float* xs = x + 8 * h;
+                const float gmax = max3abs(max3abs(xs[0], xs[1], xs[2]), max3abs(xs[3], xs[4], xs[5]),
+                                           fmaxf(fabsf(xs[6]), fabsf(xs[7])));              // G1
+                const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
+                const uint32_t sb = e4m3_encode(t);
+                const float d = __fmul_rn(e4m3_value(sb), alpha);
+                const float r = __frcp_rn(d);
+                if (sb != 0u) {
+                    uint32_t fc, ic;
+                    float f0, f1, i0, i1;
+                    if ((sb - 8u) >= 118u) candidates3x8<true>(xs, w + 4 * h, d, r, fc, ic, f0, f1, i0, i1);
+                    else candidates3x8<false>(xs, w + 4 * h, d, r, fc, ic, f0, f1, i0, i1);
+                    const bool flag = __fadd_rn(i0, i1) < __fadd_rn(f0, f1);  // a group of 8: S0 + S1
+                    chunk[h] = flag ? ic : fc;
+                    sbytes |= (sb | (flag ? 0x80u : 0u)) << (8 * h);
+                }
+            }
+            c_lo = chunk[0] | (chunk[1] << 24);
+            c_hi = chunk[1] >> 8;
+            reinterpret_cast<uint16_t*>(scales)[g] = (uint16_t)sbytes;
         }
-        scales[g] = (uint8_t)sbyte;
-        uint16_t* cp = codes + 3 * (size_t)g;                                // 6 bytes per group
+        uint16_t* cp = codes + 3 * (size_t)g;                                // 6 bytes per block of 16
         cp[0] = (uint16_t)c_lo; cp[1] = (uint16_t)(c_lo >> 16); cp[2] = (uint16_t)c_hi;
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
         g = gn;
+    }
+}
+
+// ----------------------------------------------------------------------------- 3-bit dequantize
+
+// Eight 3-bit fields of a 24-bit chunk (field j at bit 3j) spread to the low three bits of eight nibbles:
+// 12-bit halves to 16-bit halves, 6-bit pairs to bytes, 3-bit fields to nibbles, each step one mask and
+// one multiply-add (moving a part left by s bits adds (2^s - 1) times that part).
+__device__ __forceinline__ uint32_t spread3to4(uint32_t x) {
+    const uint32_t y = x + (x >> 12) * 0xF000u;
+    const uint32_t z = y + (y & 0x0FC00FC0u) * 3u;
+    return z + (z & 0x38383838u);
+}
+
+// IF3 / IF3-BS8 dequantize through the 4-bit decoder: an E2M0 code s|ee is the E2M1 code s|ee|0 (values
+// 0, 1, 2, 4 are the E2M1 codes with a zero mantissa bit), and a 3-bit two's-complement integer sign-extends
+// to a nibble.  One thread per aligned block of 16 values; G = 8 gives each word of eight codes its own scale.
+template <int G, bool ALIGNED32>
+__global__ void __launch_bounds__(256) dequantize3_fast_kernel(const uint16_t* __restrict__ codes,
+                                                               const uint8_t* __restrict__ scales,
+                                                               const float* __restrict__ alpha_p, int32_t nblocks16,
+                                                               uint4* __restrict__ out) {
+    constexpr int NSUB = 16 / G;
+    pdl_launch_dependents();
+    const float c_post = __fdiv_rn(4.0f, 3.0f);
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    pdl_wait();
+    const float alpha = __ldg(alpha_p);
+    for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < nblocks16; g += stride) {
+        const uint16_t* cp = codes + 3 * (size_t)g;
+        const uint32_t c0 = __ldg(cp), c1 = __ldg(cp + 1), c2 = __ldg(cp + 2);
+        const uint32_t chunk[2] = {c0 | ((c1 & 0xFFu) << 16), (c1 >> 8) | (c2 << 8)};
+        uint32_t sb[2];
+        if constexpr (NSUB == 2) {
+            const uint32_t two = __ldg(reinterpret_cast<const uint16_t*>(scales) + g);
+            sb[0] = two & 0xFFu; sb[1] = two >> 8;
+        } else {
+            sb[0] = sb[1] = __ldg(scales + g);
+        }
+        uint32_t o[8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t mag = sb[h] & 0x7Fu;
+            const bool is_int = sb[h] & 0x80u;
+            float Delta = e4m3_value(mag);
+            if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
+            float d = __fmul_rn(Delta, alpha);
+            if (is_int) d = __fmul_rn(d, c_post);                          // de-scale integer groups (Sec. 3)
+            const uint32_t u = spread3to4(chunk[h]);
+            const uint32_t w = is_int ? (u + (u & 0x44444444u) * 2u) : (u << 1);
+            uint32_t r[4];
+            dequant_word4<true>(w, is_int, is_int ? -1032.0f : -0.0f, pack2(d, d), r);
+            o[4 * h] = r[0]; o[4 * h + 1] = r[1]; o[4 * h + 2] = r[2]; o[4 * h + 3] = r[3];
+        }
+        store32B<ALIGNED32>(out + 2 * (size_t)g, o);
+    }
+}
+
+// ----------------------------------------------------------------------------- 4-bit dequantize, one scale per 8 values
+
+// One thread per aligned block of 16 values: each word of eight codes has its own scale byte.
+template <bool HAS_INT, bool ALIGNED32>
+__global__ void __launch_bounds__(256) dequantize4_bs8_kernel(const uint2* __restrict__ codes,
+                                                              const uint16_t* __restrict__ scales,
+                                                              const float* __restrict__ alpha_p, int32_t nblocks16,
+                                                              uint4* __restrict__ out) {
+    pdl_launch_dependents();
+    const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    pdl_wait();
+    const float alpha = __ldg(alpha_p);
+    for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < nblocks16; g += stride) {
+        const uint2 c = __ldg(codes + (size_t)g);
+        const uint32_t two = __ldg(scales + g);
+        const uint32_t cw[2] = {c.x, c.y};
+        uint32_t o[8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t sbyte = (two >> (8 * h)) & 0xFFu;
+            const uint32_t mag = sbyte & 0x7Fu;
+            const bool is_int = HAS_INT && (sbyte & 0x80u);
+            float Delta = e4m3_value(mag);
+            if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
+            float d = __fmul_rn(Delta, alpha);
+            if (is_int) d = __fmul_rn(d, c_post);                          // de-scale integer groups (Sec. 3)
+            uint32_t r[4];
+            dequant_word4<HAS_INT>(cw[h], is_int, is_int ? -1032.0f : -0.0f, pack2(d, d), r);
+            o[4 * h] = r[0]; o[4 * h + 1] = r[1]; o[4 * h + 2] = r[2]; o[4 * h + 3] = r[3];
+        }
+        store32B<ALIGNED32>(out + 2 * (size_t)g, o);
     }
 }
 
