@@ -120,29 +120,17 @@ static int grid_round_rne(const double* g, int n, float a) {
     return (lo & 1) ? lo + 1 : lo;
 }
 
-/* Stochastic rounding (Sec. 4.1, App. B) is done in the INDEX domain of a grid.  For a minifloat
- * the map phi from a magnitude a to its fractional index (grid point g_i -> i, linear in between) is
- * concave and piecewise linear, one affine piece per binade:
- *     piece 0 (zero, subnormals and the first normal binade, common step s0):  a / s0
- *     piece e (binade 2^(e-bias) .. 2^(e-bias+1), step s_e = 2^(e-bias-mbits)): a / s_e + (e-1) * 2^mbits
- * so phi(a) = min over the pieces.  With centred noise n = u - 1/2 in (-1/2, 1/2) the stochastically
- * rounded index is round-to-nearest-even of phi(a) + n: it is the upper neighbour with probability
- * frac(phi) = (a - lo) / (hi - lo) and never leaves [lo, hi].  Every operation is an FP32 operation
- * in the order written (a / s is exact, adding the offset rounds once, adding n rounds once). */
-static int fp_index_sr(const fmt_desc* F, float a, float noise) {
-    const int mb = F->mbits, emax = (1 << F->ebits) - 1;
-    if (a > F->m_fp) a = F->m_fp;
-    float phi = a * ldexpf(1.0f, F->bias + mb - 1);                       /* piece 0: a / s0 */
-    for (int e = 2; e <= emax; ++e) {
-        const float piece = a * ldexpf(1.0f, F->bias + mb - e) + (float)((e - 1) << mb);
-        if (piece < phi) phi = piece;
-    }
-    const float t = phi + noise;
-    int idx = (int)nearbyintf(t);                                         /* ties to even */
-    const int top = (1 << (F->bits - 1)) - 1;
-    if (idx < 0) idx = 0;
-    if (idx > top) idx = top;
-    return idx;
+/* Stochastic rounding on a sorted magnitude grid (Sec. 4.1, App. B): a is clamped to the
+ * top; an exact grid value stays; otherwise round up with probability (a-lo)/(hi-lo),
+ * realised as "u < p" with u in (0,1). */
+static int grid_round_sr(const double* g, int n, float a, float u) {
+    if (!(a < g[n - 1])) return n - 1;
+    int lo = 0;
+    while (lo + 1 < n && g[lo + 1] <= (double)a) ++lo;
+    float flo = (float)g[lo], fhi = (float)g[lo + 1];
+    if (a == flo) return lo;
+    float p = (a - flo) / (fhi - flo);
+    return (u < p) ? lo + 1 : lo;
 }
 
 /* ------------------------------------------------------------------ Philox4x32-10 */
@@ -174,9 +162,6 @@ static float sr_uniform(uint64_t seed, uint64_t idx) {
     uint32_t h = (w[(idx & 7) >> 1] >> (16 * (idx & 1))) & 0xFFFFu;
     return ((float)h + 0.5f) * (1.0f / 65536.0f);
 }
-
-/* Centred noise of element idx: n = u - 1/2 = (h - 32767.5) * 2^-16, exact in FP32. */
-static float sr_noise(uint64_t seed, uint64_t idx) { return sr_uniform(seed, idx) - 0.5f; }
 
 /* ------------------------------------------------------------------ Hadamard option */
 
@@ -302,8 +287,12 @@ ORACLE_API void abs_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t k
     philox4x32_10(ctr, key, out);
 }
 ORACLE_API float abs_oracle_sr_uniform(uint64_t seed, uint64_t idx) { return sr_uniform(seed, idx); }
-/* Stochastic FP index of a magnitude for a given centred noise (element-level piece for the pins). */
-ORACLE_API int abs_oracle_fp_index_sr(int fmt, float a, float noise) { return fp_index_sr(&FMTS[fmt], a, noise); }
+/* Stochastically rounded index of a magnitude on a format's FP grid for a given u (element-level piece for the pins). */
+ORACLE_API int abs_oracle_fp_sr(int fmt, float a, float u) {
+    double g[64];
+    const int n = build_fp_grid(&FMTS[fmt], g);
+    return grid_round_sr(g, n, a, u);
+}
 ORACLE_API void abs_oracle_hadamard16(const float in[16], uint16_t sign_mask, float out[16]) {
     hadamard16(in, sign_mask, out);
 }
@@ -342,9 +331,11 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
     if (fmt < 0 || fmt >= FMT_COUNT || cols % 16 != 0 || row0 < 0 || row1 > rows) return 1;
     const fmt_desc* F = &FMTS[fmt];
     const int b = F->bits;
-    double fpg[64], e4g[127];
+    const int m_int = (int)F->m_int;
+    double fpg[64], e4g[127], intg[64];
     const int nfp = build_fp_grid(F, fpg);
     const int ne4 = build_e4m3_grid(e4g);
+    for (int i = 0; i <= m_int; ++i) intg[i] = (double)i;
 
     /* T3: per-tensor constants. */
     const float a6 = alpha * F->m_fp;
@@ -392,14 +383,14 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
 
                 for (int i = 0; i < G; ++i) {
                     const float xi = xs[i];
-                    float noise = 0.0f;
+                    float u = 0.0f;
                     if (flags & F_STOCHASTIC)
-                        noise = sr_noise(sr_seed, (uint64_t)(r * cols + gi * 16 + sub * G + i));
+                        u = sr_uniform(sr_seed, (uint64_t)(r * cols + gi * 16 + sub * G + i));
                     /* E1 (step 3). */
                     const float y = xi * rcp;
                     const uint32_t ysign = f32_to_bits(y) >> 31;
                     /* E2 (step 4): FP candidate code. */
-                    int mi = (flags & F_STOCHASTIC) ? fp_index_sr(F, fabsf(y), noise)
+                    int mi = (flags & F_STOCHASTIC) ? grid_round_sr(fpg, nfp, fabsf(y), u)
                                                     : grid_round_rne(fpg, nfp, fabsf(y));
                     q_fp[i] = (ysign << (b - 1)) | (uint32_t)mi;
                     /* E3 (steps 5-6): error of the dequantized FP candidate, one fused rounding. */
@@ -410,14 +401,9 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
                     /* E4 (step 7): integer candidate of y * M_INT / M_FP, clamped to +-M_INT. */
                     float kf;
                     if (flags & F_STOCHASTIC) {
-                        /* like the FP candidate, on the magnitude clamped to M_FP and with the same noise:
-                         * |k| = nearest-even of fma(a, c_pre, n), so it rounds up with probability
-                         * frac(a * c_pre); the sign of y goes back on afterwards (rounding is symmetric) */
-                        float ay = fabsf(y);
-                        if (ay > F->m_fp) ay = F->m_fp;
-                        kf = nearbyintf(fmaf(ay, c_pre, noise));
-                        if (kf > F->m_int) kf = F->m_int;
-                        if (ysign) kf = -kf;
+                        const float z = y * c_pre;   /* the stochastic draw needs the FP32 value itself */
+                        kf = (float)grid_round_sr(intg, m_int + 1, fabsf(z), u);
+                        if (f32_to_bits(z) >> 31) kf = -kf;
                     } else {
                         kf = int_candidate_rne(y, c_pre, F->m_int);
                     }

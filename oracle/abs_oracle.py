@@ -72,10 +72,10 @@ def lib():
             L.abs_oracle_e4m3_value.argtypes = [C.c_uint32]
             L.abs_oracle_philox4x32_10.restype = None
             L.abs_oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
-            L.abs_oracle_fp_index_sr.restype = C.c_int
-            L.abs_oracle_fp_index_sr.argtypes = [C.c_int, C.c_float, C.c_float]
             L.abs_oracle_sr_uniform.restype = C.c_float
             L.abs_oracle_sr_uniform.argtypes = [C.c_uint64, C.c_uint64]
+            L.abs_oracle_fp_sr.restype = C.c_int
+            L.abs_oracle_fp_sr.argtypes = [C.c_int, C.c_float, C.c_float]
             L.abs_oracle_hadamard16.restype = None
             L.abs_oracle_hadamard16.argtypes = [f32p, C.c_uint16, f32p]
             L.abs_oracle_f32_to_bf16.restype = C.c_uint16
@@ -162,9 +162,9 @@ def sr_uniform(seed: int, idx: int) -> np.float32:
     return np.float32(lib().abs_oracle_sr_uniform(seed, idx))
 
 
-def fp_index_sr(fmt: int, a, noise) -> int:
-    """Stochastically rounded FP grid index of magnitude ``a`` for centred noise in (-1/2, 1/2)."""
-    return int(lib().abs_oracle_fp_index_sr(fmt, C.c_float(float(np.float32(a))), C.c_float(float(np.float32(noise)))))
+def fp_sr(fmt: int, a: float, u: float) -> int:
+    """Index on the FP grid of ``fmt`` that the magnitude ``a`` rounds to stochastically for the uniform ``u``."""
+    return int(lib().abs_oracle_fp_sr(fmt, float(a), float(u)))
 
 
 def hadamard16(x16, sign_mask: int) -> np.ndarray:

@@ -151,36 +151,25 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
-// Stochastic rounding works in the index domain of the grid (Sec. 4.1, App. B).  The map phi from a
-// magnitude to its fractional grid index is concave and piecewise linear, one affine piece per binade:
-//     piece 0 (subnormals and the first normal binade, step s0 = 2^(EMIN - MBITS)):  a / s0
-//     piece e (step s_e = 2^(e - 1 + EMIN - MBITS)):                                  a / s_e + (e-1) * 2^MBITS
-// so phi is the minimum over the pieces.  With centred noise n = u - 1/2 the rounded index is
-// nearest-even of phi + n: the upper neighbour with probability frac(phi).  FP32 throughout, in this order.
-template <class F>
-__device__ __forceinline__ uint32_t sr_index_fp(float a, float noise) {
-    constexpr int TOP = (1 << (F::BITS - 1)) - 1, EMAX = TOP >> F::MBITS;
-    a = (a > F::M_FP) ? F::M_FP : a;
-    float phi = __fmul_rn(a, __uint_as_float((uint32_t)(127 + F::MBITS - F::EMIN) << 23));
-#pragma unroll
-    for (int e = 2; e <= EMAX; ++e) {
-        const float piece = __fadd_rn(__fmul_rn(a, __uint_as_float((uint32_t)(127 + F::MBITS - F::EMIN + 1 - e) << 23)),
-                                      (float)((e - 1) << F::MBITS));
-        phi = (piece < phi) ? piece : phi;
-    }
-    int idx = __float2int_rn(__fadd_rn(phi, noise));
-    return (uint32_t)min(max(idx, 0), TOP);
+// Stochastic rounding of a magnitude onto a minifloat grid with MBITS mantissa bits and smallest
+// normal exponent EMIN: clamp to the top; step s = 2^(max(exponent, EMIN) - MBITS); lo = floor to
+// the step; round up iff u < (a - lo) / s.  All operations are exact in FP32.
+template <int EMIN, int MBITS>
+__device__ __forceinline__ float sr_round_fp(float a, float top, float u) {
+    a = fminf(a, top);
+    int e = (int)(__float_as_uint(a) >> 23) - 127;
+    e = max(e, EMIN);
+    float s = __uint_as_float((uint32_t)(e - MBITS + 127) << 23);
+    float inv_s = __uint_as_float((uint32_t)(MBITS - e + 127) << 23);
+    float lo = __fmul_rn(floorf(__fmul_rn(a, inv_s)), s);
+    float p = __fmul_rn(__fsub_rn(a, lo), inv_s);
+    return (u < p) ? __fadd_rn(lo, s) : lo;
 }
-// Integer candidate under stochastic rounding, on the magnitude like the FP one: |k| = nearest-even of
-// fma(min(|y|, M_FP), c_pre, n), at most M_INT; the sign of y goes back on afterwards.
-__device__ __forceinline__ float sr_round_int(float y, float c_pre, float noise, float m_fp, float m_int) {
-    const float a = (fabsf(y) > m_fp) ? m_fp : fabsf(y);
-    const float k = fminf(rintf(__fmaf_rn(a, c_pre, noise)), m_int);
-    return copysignf(k, y);
-}
-// Centred noise of a 16-bit random field h: n = (h + 1/2) * 2^-16 - 1/2, exact in FP32.
-__device__ __forceinline__ float sr_noise(uint32_t h) {
-    return __fsub_rn(__fmul_rn(__fadd_rn((float)h, 0.5f), 1.0f / 65536.0f), 0.5f);
+__device__ __forceinline__ float sr_round_int(float a, float top, float u) {
+    a = fminf(a, top);
+    float lo = floorf(a);
+    float p = __fsub_rn(a, lo);
+    return (u < p) ? __fadd_rn(lo, 1.0f) : lo;
 }
 
 // ----------------------------------------------------------------------------- packed f32x2 arithmetic

@@ -197,28 +197,27 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                 for (int i = 0; i < G; i += 2) {
                     const float x0 = x[e0i + i], x1 = x[e0i + i + 1];
                     float y0 = __fmul_rn(x0, r), y1 = __fmul_rn(x1, r);                // E1 (step 3)
-                    float n0 = 0.f, n1 = 0.f;
-                    float v0, v1;
-                    if constexpr (SR) {                                                // E2 under stochastic rounding
+                    float u0 = 0.f, u1 = 0.f;
+                    float yq0 = y0, yq1 = y1;
+                    if constexpr (SR) {
                         const uint32_t rw = rnd[(e0i + i) >> 1];
-                        n0 = sr_noise(rw & 0xFFFFu);
-                        n1 = sr_noise(rw >> 16);
-                        q_fp[i] = sr_index_fp<F>(fabsf(y0), n0) | ((__float_as_uint(y0) >> 31) << (B - 1));
-                        q_fp[i + 1] = sr_index_fp<F>(fabsf(y1), n1) | ((__float_as_uint(y1) >> 31) << (B - 1));
-                        const float2 v = fp_decode_pair<F::EK>(q_fp[i], q_fp[i + 1]);
-                        v0 = v.x; v1 = v.y;
-                    } else {
-                        fp_encode_pair<F::EK>(y0, y1, q_fp[i], q_fp[i + 1], v0, v1);   // E2 (step 4)
+                        u0 = __fmul_rn(__fadd_rn((float)(rw & 0xFFFFu), 0.5f), 1.0f / 65536.0f);
+                        u1 = __fmul_rn(__fadd_rn((float)(rw >> 16), 0.5f), 1.0f / 65536.0f);
+                        yq0 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y0), F::M_FP, u0), y0);
+                        yq1 = copysignf(sr_round_fp<F::EMIN, F::MBITS>(fabsf(y1), F::M_FP, u1), y1);
                     }
+                    float v0, v1;
+                    fp_encode_pair<F::EK>(yq0, yq1, q_fp[i], q_fp[i + 1], v0, v1);     // E2 (step 4)
                     const int chain = ((i >> 3) << 1);                                 // elements 0-7 -> S0,S1; 8-15 -> S2,S3
                     if constexpr (F::HAS_INT) {
                         const float e0 = __fmaf_rn(v0, d, -x0), e1 = __fmaf_rn(v1, d, -x1);   // E3 (steps 5-6)
                         s_fp[chain] = __fmaf_rn(e0, e0, s_fp[chain]);
                         s_fp[chain + 1] = __fmaf_rn(e1, e1, s_fp[chain + 1]);
-                        float k0, k1;                                                         // E4 (step 7)
+                        const float z0 = __fmul_rn(y0, c_pre), z1 = __fmul_rn(y1, c_pre);     // E4 (step 7)
+                        float k0, k1;
                         if constexpr (SR) {
-                            k0 = sr_round_int(y0, c_pre, n0, F::M_FP, F::M_INT);
-                            k1 = sr_round_int(y1, c_pre, n1, F::M_FP, F::M_INT);
+                            k0 = copysignf(sr_round_int(fabsf(z0), F::M_INT, u0), z0);
+                            k1 = copysignf(sr_round_int(fabsf(z1), F::M_INT, u1), z1);
                         } else {
                             // round-half-even of the exact product y * c_pre (one rounding): fused add of 1.5 * 2^23
                             k0 = __fsub_rn(__fmaf_rn(y0, c_pre, 12582912.0f), 12582912.0f);

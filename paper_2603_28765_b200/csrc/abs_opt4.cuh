@@ -22,26 +22,43 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 }
 __device__ __forceinline__ uint32_t sign_of(float y) { return __float_as_uint(y) & 0x80000000u; }
 
+__device__ __forceinline__ uint64_t add2_rp(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rp.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2_rp(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // Per-element work of one group under stochastic rounding (steps 3-10 of Fig. 3a with both candidates
-// rounded stochastically, App. B).  rnd[i] holds the two 16-bit random fields of elements 2i (low half)
-// and 2i+1.  For E2M1 the index map is phi(a) = min(2a, a + 2, a/2 + 4) and its inverse, the value of an
-// index, is max(i/2, i - 2, 2i - 8).  No clamp of the integer candidate is needed: a <= 6 gives
-// fma(a, 7/6, n) < 7.5.
+// rounded stochastically, App. B).  rnd[i] holds the two 16-bit random fields h of elements 2i (low half)
+// and 2i+1; u = (h + 1/2) * 2^-16.
+//
+// The rule "lo if a == lo, else hi iff u < (a - lo) / (hi - lo)" is evaluated as a ceiling.  With phi the
+// grid's fractional-index map (grid point g_i -> i, linear in between), the rounded index is ceil(phi(a) - u):
+// for phi = n + f it is n when u >= f and n + 1 when u < f.  For E2M1 phi(a) = min(2a, a + 2, a/2 + 4); the
+// pieces, the subtraction of u and the final add of 1.5 * 2^23 (which leaves the ceiling in the low mantissa
+// bits) all round toward +infinity, and that changes nothing: u is an odd multiple of 2^-17, every rounding
+// here is to a grid at least as fine as 2^-21, so a sum rounded up crosses neither u nor an integer that the
+// exact sum does not reach.  The value of an index is max(i/2, i - 2, 2i - 8).  The integer candidate is the
+// same ceiling on |z|, z = y * 7/6 rounded to FP32 as in the round-to-nearest path, clamped to 7.
 template <bool HAS_INT>
 __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint32_t (&rnd)[8], uint32_t sb, float d,
                                                 float r, uint32_t& sbyte, uint32_t& c_lo, uint32_t& c_hi) {
     const uint64_t R2 = pack2(r, r);
     const uint64_t TWO = pack2(2.0f, 2.0f), HALF = pack2(0.5f, 0.5f), FOUR = pack2(4.0f, 4.0f);
     const uint64_t MG = pack2(kMagic, kMagic), NMG = pack2(-kMagic, -kMagic);
-    const uint64_t SC16 = pack2(1.0f / 65536.0f, 1.0f / 65536.0f), N128 = pack2(-128.0f, -128.0f);
-    const float cn = 1.0f / 131072.0f - 0.5f;                                  // 2^-17 - 1/2, exact
-    const uint64_t CN = pack2(cn, cn);
+    const uint64_t NSC16 = pack2(-1.0f / 65536.0f, -1.0f / 65536.0f), P128 = pack2(128.0f, 128.0f);
+    const uint64_t NH17 = pack2(-1.0f / 131072.0f, -1.0f / 131072.0f);
 
     const float c_pre = __uint_as_float(0x3F955555u);    // fp32(7/6)
     const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
     const float d_int = __fmul_rn(d, c_post);
     const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
-    const uint64_t MG8 = pack2(kMagic8, kMagic8), NMG8 = pack2(-kMagic8, -kMagic8);
+    const uint64_t MG8 = pack2(kMagic8, kMagic8);
     const uint64_t NTWO = pack2(-2.0f, -2.0f), NEIGHT = pack2(-8.0f, -8.0f);
 
     uint64_t accF[2], accI[2];
@@ -53,23 +70,24 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
         for (int i = 0; i < 4; ++i) {
             const int e = 8 * hgrp + 2 * i;
             const uint64_t X = pack2(x[e], x[e + 1]);
+            const uint64_t Y = mul2(X, R2);                                    // E1 (step 3)
             float y0, y1;
-            unpack2(mul2(X, R2), y0, y1);                                      // E1 (step 3)
+            unpack2(Y, y0, y1);
             ys[2 * i] = y0; ys[2 * i + 1] = y1;
-            // centred noise n = (h + 1/2) * 2^-16 - 1/2 from the 16-bit fields, exact: 2^23 + h as a float first
+            // -u = -(h + 1/2) * 2^-16 from the 16-bit fields, exact: 2^23 + h as a float first
             const uint32_t rw = rnd[e >> 1];
             const float m0 = __uint_as_float((rw & 0xFFFFu) | 0x4B000000u);
             const float m1 = __uint_as_float(__byte_perm(rw, 0x4B00u, 0x5432));
-            const uint64_t N = add2(fma2(pack2(m0, m1), SC16, N128), CN);
-            // E2 under stochastic rounding: fractional index, plus noise, nearest-even
+            const uint64_t NU = add2(fma2(pack2(m0, m1), NSC16, P128), NH17);
+            // E2 under stochastic rounding: index = ceil(phi(a) - u)
             const float a0 = fminf(fabsf(y0), 6.0f), a1 = fminf(fabsf(y1), 6.0f);
             const uint64_t A = pack2(a0, a1);
             float p00, p01, p10, p11, p20, p21;
-            unpack2(add2(A, A), p00, p01);
-            unpack2(add2(A, TWO), p10, p11);
-            unpack2(fma2(A, HALF, FOUR), p20, p21);
+            unpack2(add2(A, A), p00, p01);                                     // exact
+            unpack2(add2_rp(A, TWO), p10, p11);
+            unpack2(fma2_rp(A, HALF, FOUR), p20, p21);
             const uint64_t PHI = pack2(min3f(p00, p10, p20), min3f(p01, p11, p21));
-            const uint64_t IM = add2(add2(PHI, N), MG);                        // low mantissa bits = index 0..7
+            const uint64_t IM = add2_rp(add2_rp(PHI, NU), MG);                 // low mantissa bits = index 0..7
             float im0, im1;
             unpack2(IM, im0, im1);
             ib[e] = __float_as_uint(im0);
@@ -86,20 +104,19 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
                 vs[2 * i] = vs0; vs[2 * i + 1] = vs1;
                 const uint64_t E = fma2(pack2(vs0, vs1), ND2, X);              // E3 (steps 5-6), negated; squared below
                 accF[hgrp] = (i == 0) ? mul2(E, E) : fma2(E, E, accF[hgrp]);
-                // E4 (step 7) under stochastic rounding: |k| = RNE(fma(a, 7/6, n)); magnitude and noise carry
-                // the sign of y so that the sum below is the signed k directly (rounding is symmetric)
-                const float as0 = __uint_as_float(__float_as_uint(a0) | sign_of(y0));
-                const float as1 = __uint_as_float(__float_as_uint(a1) | sign_of(y1));
-                float n0, n1;
-                unpack2(N, n0, n1);
-                const float ns0 = __uint_as_float(__float_as_uint(n0) ^ sign_of(y0));
-                const float ns1 = __uint_as_float(__float_as_uint(n1) ^ sign_of(y1));
-                const uint64_t KM = add2(fma2(pack2(as0, as1), CP2, pack2(ns0, ns1)), MG8);
-                const uint64_t KF = add2(KM, NMG8);
-                const uint64_t FI = fma2(KF, NDI2, X);                         // E5 (steps 8-9)
+                // E4 (step 7) under stochastic rounding: |k| = ceil(min(|z|, 7) - u), sign of z put back
+                float z0, z1;
+                unpack2(mul2(Y, CP2), z0, z1);
+                const uint64_t AZ = pack2(fminf(fabsf(z0), 7.0f), fminf(fabsf(z1), 7.0f));
+                float k0, k1;
+                unpack2(add2(add2_rp(add2_rp(AZ, NU), MG), NMG), k0, k1);
+                const float ks0 = __uint_as_float((__float_as_uint(k0) & 0x7FFFFFFFu) | sign_of(z0));
+                const float ks1 = __uint_as_float((__float_as_uint(k1) & 0x7FFFFFFFu) | sign_of(z1));
+                const uint64_t KS = pack2(ks0, ks1);
+                const uint64_t FI = fma2(KS, NDI2, X);                         // E5 (steps 8-9)
                 accI[hgrp] = (i == 0) ? mul2(FI, FI) : fma2(FI, FI, accI[hgrp]);
                 float km0, km1;
-                unpack2(KM, km0, km1);
+                unpack2(add2(KS, MG8), km0, km1);                              // low nibble = k + 8
                 kb[e] = __float_as_uint(km0);
                 kb[e + 1] = __float_as_uint(km1);
             }

@@ -551,15 +551,15 @@ def test_sr_keeps_representable_and_brackets(oracle):
 @pytest.mark.parametrize("fmt", [0, 2, 3, 4])
 def test_sr_index_probability_is_the_fractional_position(oracle, fmt):
     """App. B: a value between grid points lo < a < hi rounds up with probability (a-lo)/(hi-lo), and a
-    grid point stays put.  Counted over all 65536 values the centred noise can take; built from the
-    grid alone (searchsorted), not from the oracle's piecewise index map."""
+    grid point stays put.  Counted over evenly spaced values of the 16-bit uniform; built from the grid
+    alone (searchsorted), not from the oracle's own bracket search."""
     g = np.array(fp_grid(fmt), dtype=np.float64)
-    noise = ((np.arange(65536) + 0.5) / 65536.0 - 0.5).astype(np.float32)
+    us = ((np.arange(65536) + 0.5) / 65536.0).astype(np.float32)[::16]      # 4096 evenly spaced draws
     rng = np.random.default_rng(100 + fmt)
     samples = list(g) + [float(np.float32(v)) for v in rng.uniform(0, g[-1], 40)]
     samples += [float(g[-1]) * 1.5, float(g[1]) * 0.25, float(g[-2] + g[-1]) / 2]
     for a in samples:
-        idx = np.array([oracle.fp_index_sr(fmt, a, float(n)) for n in noise[::16]])   # 4096 evenly spaced draws
+        idx = np.array([oracle.fp_sr(fmt, a, float(u)) for u in us])
         ac = min(a, g[-1])
         lo = int(np.searchsorted(g, ac, side="right") - 1)
         if g[lo] == ac:
@@ -568,6 +568,7 @@ def test_sr_index_probability_is_the_fractional_position(oracle, fmt):
         assert set(np.unique(idx)) <= {lo, lo + 1}
         p = (ac - g[lo]) / (g[lo + 1] - g[lo])
         assert abs((idx == lo + 1).mean() - p) <= 1.0 / 4096 + 1e-9, (fmt, a, p)
+        assert np.array_equal(idx == lo + 1, us.astype(np.float64) < p)     # "u < p" itself
 
 
 def test_sr_int_candidate_probability(oracle):
