@@ -337,6 +337,20 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
             return (e8 == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
         }
     }
+    if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
+        const int sgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
+            constexpr ElemKind kEK = Fmt<FMT>::EK;
+            const float c_post = Fmt<FMT>::M_FP / Fmt<FMT>::M_INT;         // IEEE single division, as in the generic kernel
+            const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
+            const cudaError_t e6 =
+                a32 ? launch_pdl(dequantize6_fast_kernel<kEK, true>, sgrid, kThreads, s, (const uint32_t*)codes,
+                                 (const uint8_t*)scales, alpha, (int32_t)ngroups, (uint4*)out, c_post)
+                    : launch_pdl(dequantize6_fast_kernel<kEK, false>, sgrid, kThreads, s, (const uint32_t*)codes,
+                                 (const uint8_t*)scales, alpha, (int32_t)ngroups, (uint4*)out, c_post);
+            return (e6 == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
+        }
+    }
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // 3-bit codes widened to nibbles and decoded like the 4-bit formats
         const int tgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);

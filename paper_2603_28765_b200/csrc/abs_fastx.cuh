@@ -559,4 +559,68 @@ __global__ void __launch_bounds__(256) dequantize4_bs8_kernel(const uint2* __res
     }
 }
 
+// ----------------------------------------------------------------------------- 6-bit dequantize
+
+// Four 6-bit fields of a 24-bit chunk (field j at bit 6j) spread to one field per byte: the inverse of
+// squeeze6x4, again one mask and one multiply-add per step.
+__device__ __forceinline__ uint32_t spread6to8(uint32_t c) {
+    const uint32_t t = c + (c >> 12) * 0xF000u;
+    return t + (t & 0x0FC00FC0u) * 3u;
+}
+
+// IF6 dequantize: one thread per group of 16 (three words of codes in, 32 bytes of bf16 out).  Branch-free
+// like the 4-bit kernel: the FP decode is the hardware convert to f16 pairs, the integer decode places the
+// field k + 32 (field xor 32) in the mantissa of the f16 constant 1024, so the half is 1056 + k; one shared
+// tail adds -0 or -1056 in FP32, multiplies by the group scale and rounds to bf16 pairs.
+template <ElemKind EK, bool ALIGNED32>
+__global__ void __launch_bounds__(256) dequantize6_fast_kernel(const uint32_t* __restrict__ codes,
+                                                               const uint8_t* __restrict__ scales,
+                                                               const float* __restrict__ alpha_p, int32_t ngroups,
+                                                               uint4* __restrict__ out, float c_post) {
+    pdl_launch_dependents();
+    const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    pdl_wait();
+    const float alpha = __ldg(alpha_p);
+    for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < ngroups; g += stride) {
+        const uint32_t* cp = codes + 3 * (size_t)g;
+        const uint32_t w0 = __ldg(cp), w1 = __ldg(cp + 1), w2 = __ldg(cp + 2);
+        const uint32_t sbyte = __ldg(scales + g);
+        const uint32_t mag = sbyte & 0x7Fu;
+        const bool is_int = sbyte & 0x80u;
+        float Delta = e4m3_value(mag);
+        if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);            // E4M3 NaN propagates
+        float d = __fmul_rn(Delta, alpha);
+        if (is_int) d = __fmul_rn(d, c_post);                              // de-scale integer groups (Sec. 3)
+        const float addend = is_int ? -1056.0f : -0.0f;
+        const uint64_t D2 = pack2(d, d);
+        const uint32_t chunk[4] = {w0 & 0xFFFFFFu, (w0 >> 24) | ((w1 & 0xFFFFu) << 8), (w1 >> 16) | ((w2 & 0xFFu) << 16), w2 >> 8};
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t bytes = spread6to8(chunk[q]);                   // codes 4q .. 4q+3, one per byte
+            uint32_t h0, h1;
+            if constexpr (EK == EK_E2M3) {
+                asm("{ .reg .b16 lo, hi;\n"
+                    "  mov.b32 {lo, hi}, %2;\n"
+                    "  cvt.rn.f16x2.e2m3x2 %0, lo;\n"
+                    "  cvt.rn.f16x2.e2m3x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
+            } else {
+                asm("{ .reg .b16 lo, hi;\n"
+                    "  mov.b32 {lo, hi}, %2;\n"
+                    "  cvt.rn.f16x2.e3m2x2 %0, lo;\n"
+                    "  cvt.rn.f16x2.e3m2x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
+            }
+            const uint32_t r0 = __byte_perm(bytes, 0u, 0x4140) ^ 0x64206420u;   // halves 1056 + k of codes 4q, 4q+1
+            const uint32_t r1 = __byte_perm(bytes, 0u, 0x4342) ^ 0x64206420u;   // ... of codes 4q+2, 4q+3
+            const uint32_t s0 = is_int ? r0 : h0, s1 = is_int ? r1 : h1;
+            float p0, p1, p2, p3;
+            unpack2(mul2(pack2(half_plus_f32(s0, false, addend), half_plus_f32(s0, true, addend)), D2), p0, p1);
+            unpack2(mul2(pack2(half_plus_f32(s1, false, addend), half_plus_f32(s1, true, addend)), D2), p2, p3);
+            o[2 * q] = bf16x2_rn(p0, p1);
+            o[2 * q + 1] = bf16x2_rn(p2, p3);
+        }
+        store32B<ALIGNED32>(out + 2 * (size_t)g, o);
+    }
+}
+
 }  // namespace absq
