@@ -133,7 +133,10 @@ abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen
 abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const abs_opts_t& o, bool ticket,
                          unsigned long long* slot, uint32_t gen, float* result, float denom, cudaStream_t s) {
     const bool rht = o.flags & ABS_F_HADAMARD16;
-    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, ABS_AMAX_BPS);
+#ifndef ABS_AMAX_RHT_BPS
+#define ABS_AMAX_RHT_BPS ABS_AMAX_BPS
+#endif
+    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, rht ? ABS_AMAX_RHT_BPS : ABS_AMAX_BPS);
     cudaError_t e;
 #define ABS_LAUNCH_A(R, T)                                                                                          \
     e = launch_pdl(amax_kernel<R, T>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, \

@@ -197,6 +197,12 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ float max3abs(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(fabsf(a)), "f"(fabsf(b)), "f"(fabsf(c)));
+    return d;
+}
+
 // ----------------------------------------------------------------------------- Hadamard option
 
 // 16-point transform of one group held in registers: sign flips from the mask, natural-order
@@ -224,6 +230,9 @@ __device__ __forceinline__ void hadamard16(float (&a)[16], uint32_t sign_mask) {
 // bit 15 / 31 of word i set where elements 2i / 2i+1 are negated), the h = 1 stage inside each pair with
 // scalar adds, the h = 2, 4, 8 stages on whole pairs with packed add and fused (p - q = fma(q, -1, p), one
 // rounding), then times 1/4.  Natural-order Sylvester butterflies, every result rounded to FP32.
+// SCALE = false leaves out the final factor 1/4 (for a maximum it can be applied once at the end:
+// rounding is monotone, so max_i fl(x_i / 4) = fl(max_i x_i / 4)).
+template <bool SCALE = true>
 __device__ __forceinline__ void hadamard16_packed(const uint32_t (&w)[8], const uint32_t (&smask)[8], float (&x)[16]) {
     uint64_t P[8];
 #pragma unroll
@@ -246,7 +255,7 @@ __device__ __forceinline__ void hadamard16_packed(const uint32_t (&w)[8], const 
         }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) unpack2(mul2(P[i], QUARTER), x[2 * i], x[2 * i + 1]);
+    for (int i = 0; i < 8; ++i) unpack2(SCALE ? mul2(P[i], QUARTER) : P[i], x[2 * i], x[2 * i + 1]);
 }
 
 

@@ -8,11 +8,6 @@
 
 namespace absq {
 
-__device__ __forceinline__ float max3abs(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(fabsf(a)), "f"(fabsf(b)), "f"(fabsf(c)));
-    return d;
-}
 
 // 1.5 * 2^23 + 8: adding it to an integer-valued-after-rounding k in [-8, 7] leaves k + 8 in the
 // low mantissa nibble, so eight such sums combine into eight offset-binary nibbles without borrows.

@@ -101,17 +101,17 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
                 else load32B<false>(in + 2 * gn, wn);
             }
             float x[16];
-            hadamard16_packed(w, smask, x);
+            hadamard16_packed<false>(w, smask, x);                      // times 1/4 once, after the maximum
 #pragma unroll
             for (int i = 0; i < 16; i += 4) {
-                m0 = fmaxf(m0, fmaxf(fabsf(x[i]), fabsf(x[i + 1])));
-                m1 = fmaxf(m1, fmaxf(fabsf(x[i + 2]), fabsf(x[i + 3])));
+                m0 = max3abs(m0, x[i], x[i + 1]);
+                m1 = max3abs(m1, x[i + 2], x[i + 3]);
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) w[i] = wn[i];
             g = gn;
         }
-        local = __float_as_uint(fmaxf(m0, m1));
+        local = __float_as_uint(__fmul_rn(fmaxf(m0, m1), 0.25f));
     }
     local = __reduce_max_sync(0xFFFFFFFFu, local);
     __shared__ uint32_t warp_max[kThreads / 32];
