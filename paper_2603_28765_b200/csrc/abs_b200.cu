@@ -598,9 +598,18 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     const int64_t rblocks = rows / 16;
     const int64_t ntiles = ((cols + kTransTileCols - 1) / kTransTileCols) *
                            ((rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks);
-    const int64_t resident = (int64_t)st->sm_count * 3;        // 64 KiB of shared memory per block: 3 blocks per SM
+    // 64 KiB of shared memory per block: 3 blocks per SM.  The arithmetic-bound variants (IF4, options) run
+    // best as several waves with about four tiles per block; plain NVFP4 as one wave of persistent blocks.
+    const int64_t resident = (int64_t)st->sm_count * 3;
+    const bool heavy = fmt == ABS_FMT_IF4 || (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC));
+    int64_t tgrid = ntiles < resident ? ntiles : resident;
+    if (heavy && ntiles > resident) {
+        int64_t waves = (ntiles + 2 * resident) / (4 * resident);
+        if (waves < 1) waves = 1;
+        tgrid = waves * resident < ntiles ? waves * resident : ntiles;
+    }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(ntiles < resident ? ntiles : resident));
+    cfg.gridDim = dim3((unsigned)tgrid);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kTransSmemBytes;
     cfg.stream = s;
