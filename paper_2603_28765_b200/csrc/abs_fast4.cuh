@@ -139,8 +139,9 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
 #define ABS_FAST_MINB 4          // resident blocks of 256 threads per SM the IF4 instance is compiled for
 #endif
 
-// Persistent grid-stride kernel: every thread encodes groups g, g + stride, ... and fetches the
-// next group's 32 bytes before it works on the current one, so loads stay in flight under the math.
+// Grid-stride kernel: every thread encodes groups g, g + stride, ... (a handful of them: the host sizes the
+// grid as a few waves of resident blocks) and fetches the next group's 32 bytes before it works on the
+// current one, so loads stay in flight under the math.
 // IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
 template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT, bool SCALE_MUL, bool SWZ>
 __global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
