@@ -1,6 +1,6 @@
 """Per-configuration throughput table of the library's kernels (run on a B200 machine).
 
-    python -m paper_2603_28765_b200.report [--quick] [--only CFG[:FMT]] [--rows R]
+    python -m paper_2603_28765_b200.report [--quick] [--only CFG[:FMT]] [--rows R] [--transposed]
 
 ``--only cfg4:if4 --rows 4096 --quick`` restricts the run to one configuration (and format) at a reduced
 row count: the small case to put under a profiler.
@@ -10,7 +10,8 @@ that rotate over enough buffer sets to defeat L2 reuse between calls:
   T1  the group-quantize kernel alone (alpha given)          bytes = 2N + codes + scales
   T2  abs_quantize end to end (amax pass + group-quantize)   bytes = 4N + codes + scales (DRAM basis)
   T3  abs_dequantize                                         bytes = codes + scales + 2N
-and prints one JSON line per row.  Inputs are random bf16 tensors of the configuration's shape
+and prints one JSON line per row.  With ``--transposed`` it times abs_quantize_transposed instead (the kernel
+alone, alpha given; the same bytes move), for IF4 and NVFP4 with and without the gradient options.  Inputs are random bf16 tensors of the configuration's shape
 (timing does not depend on the values beyond the INT/FP mix); parity is the test suite's job.
 """
 from __future__ import annotations
@@ -28,6 +29,7 @@ def main():
     ap.add_argument("--quick", action="store_true", help="fewer repetitions")
     ap.add_argument("--only", default="", help="one configuration, optionally one format: cfg4 or cfg4:if4")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (smaller case for profiling)")
+    ap.add_argument("--transposed", action="store_true", help="time abs_quantize_transposed (groups down the columns)")
     args = ap.parse_args()
     L = B.lib()
     reps = 10 if args.quick else 40
@@ -55,6 +57,32 @@ def main():
     ]
     sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     only_cfg, _, only_fmt = args.only.partition(":")
+    if args.transposed:
+        for name, rows, cols in (("cfg2", 8192, 4096), ("cfg4", 16384, 8192)):
+            if only_cfg and name != only_cfg:
+                continue
+            if args.rows:
+                rows = args.rows
+            n = rows * cols
+            k = max(4, int(1.0e9 // (n * 2)))
+            xs = [torch.randn(rows, cols, device="cuda").to(torch.bfloat16) for _ in range(k)]
+            codes = [torch.empty(n // 2, dtype=torch.uint8, device="cuda") for _ in range(k)]
+            scales = [torch.empty(n // 16, dtype=torch.uint8, device="cuda") for _ in range(k)]
+            ts = [torch.full((1,), 0.01, dtype=torch.float32, device="cuda") for _ in range(k)]
+            for fname, flags in (("if4", 0), ("nvfp4", 0), ("if4", H), ("if4", H | S | S17), ("nvfp4", H | S | S17)):
+                if only_fmt and fname != only_fmt:
+                    continue
+                fmt = B.FMT_NAMES[fname]
+                og = B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, 0x5A3C, 1234)
+                a = [(fmt, xs[i].data_ptr(), rows, cols, codes[i].data_ptr(), scales[i].data_ptr(), ts[i].data_ptr(),
+                      C.byref(og), sp) for i in range(k)]
+                t = loop_time(lambda i: L.abs_quantize_transposed(*a[i % k]))
+                opt = "+".join(s for s, f in (("hadamard", H), ("sr", S), ("17/16", S17)) if flags & f) or "rtn"
+                print(json.dumps({"config": name, "shape": [rows, cols], "fmt": fname, "options": opt, "transposed": True,
+                                  "T1_quantize_kernel_us": round(t * 1e3, 1),
+                                  "T1_GBs": round(2.5625 * n / t / 1e6)}), flush=True)
+            del xs, codes, scales
+        return
     for name, rows, cols, variants in rows_cfg:
         if only_cfg and name != only_cfg:
             continue
