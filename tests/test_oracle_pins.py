@@ -96,6 +96,12 @@ def test_table1_mse_normal(oracle):
         d = oracle.dequantize(fmt, c, s, a, 1024, 1024, out_fp32=True, threads=4).astype(np.float64)
         mse = np.mean((d - xf) ** 2) * 1e3
         assert abs(mse - float(g[name][0])) < 0.12, (name, mse)
+    # the per-group error sums of the two candidates (steps 5-6 and 8-9 of Fig. 3a), before selection: the FP
+    # candidate alone is NVFP4, the integer candidate alone is NVINT4 up to where the E4M3 rounding falls
+    c, s, a, e_fp, e_int = oracle.quantize(1, xb, threads=4, debug=True)
+    assert abs(e_fp.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVFP4"][0])) < 0.12
+    assert abs(e_int.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVINT4"][0])) < 0.12
+    assert abs(np.minimum(e_fp, e_int).astype(np.float64).sum() / xb.size * 1e3 - float(g["IF4"][0])) < 0.12
 
 
 def test_format_facts(oracle):
