@@ -190,7 +190,10 @@ ABS_API float abs_alpha_from_amax(abs_fmt_t fmt, float amax);
 /* Host-buffer variants: `*_host` pointers are HOST memory (pinned memory makes the copies
  * asynchronous), `d_workspace` is a device buffer of at least abs_host_workspace_bytes() bytes.
  * Each call copies its inputs to the device, runs the same kernels as above, copies the results
- * back and returns after synchronising `stream`. */
+ * back and returns after synchronising `stream`.  abs_dequantize_host works in four row chunks and
+ * copies each finished chunk back on a second, library-owned stream (created on first use, one per
+ * device, ordered against `stream` by events) while the next chunk is uploaded and decoded; calls
+ * on the same device are serialised by the library. */
 ABS_API size_t abs_host_workspace_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols);
 ABS_API abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t rows, int64_t cols,
                                void* codes_u8_host, void* scales_e4m3_host, float* tensor_scale_f32_host,

@@ -41,12 +41,19 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, cudaStream
 
 // ------------------------------------------------------------------------------------------ host state
 
+constexpr int kHostChunks = 4;        // row chunks of abs_dequantize_host
+
 struct DeviceState {
     std::once_flag once;
     cudaError_t init_err = cudaSuccess;
     uint32_t* ring = nullptr;          // ABS_MAX_INFLIGHT slots of 16 bytes: tagged maximum (u64), ticket (u32), pad
     std::atomic<uint32_t> next{0};
     int sm_count = 148;
+    // abs_dequantize_host: a second stream for the device-to-host copies and the events that order it
+    std::mutex host_mu;
+    cudaStream_t d2h_stream = nullptr;
+    cudaEvent_t chunk_done[kHostChunks] = {};
+    cudaEvent_t d2h_done = nullptr;
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -821,6 +828,42 @@ abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const
     uint8_t* d_scales = d_codes + round256(cb);
     float* d_alpha = (float*)(d_scales + round256(sb));
     cudaStream_t s = (cudaStream_t)stream;
+    // Row chunks: the device-to-host copy of one chunk (second stream) overlaps the host-to-device copy and
+    // the kernel of the next.  Chunk boundaries are multiples of 16 rows, which keeps every section pointer
+    // 16-byte aligned; the tiled scale layout does not split by rows and takes the single-shot path below.
+    const int64_t chunk_rows = ((rows + kHostChunks - 1) / kHostChunks + 15) / 16 * 16;
+    DeviceState* st = nullptr;
+    if (rows >= 16 * kHostChunks && !(opts && (opts->flags & ABS_F_SCALES_SWIZZLED)) && device_state(&st) == ABS_OK) {
+        std::lock_guard<std::mutex> lock(st->host_mu);
+        if (!st->d2h_stream) {
+            bool ok = cudaStreamCreateWithFlags(&st->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+            for (int i = 0; ok && i < kHostChunks; ++i)
+                ok = cudaEventCreateWithFlags(&st->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
+            ok = ok && cudaEventCreateWithFlags(&st->d2h_done, cudaEventDisableTiming) == cudaSuccess;
+            if (!ok) return ABS_ERR_CUDA;
+        }
+        if (cudaMemcpyAsync(d_alpha, tensor_scale_f32_host, 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
+        const size_t out_row = (size_t)cols * (fp32 ? 4 : 2);
+        int i = 0;
+        for (int64_t r0 = 0; r0 < rows; r0 += chunk_rows, ++i) {
+            const int64_t nr = rows - r0 < chunk_rows ? rows - r0 : chunk_rows;
+            const size_t c0 = abs_codes_bytes(fmt, r0, cols), cn = abs_codes_bytes(fmt, nr, cols);
+            const size_t s0 = abs_scales_bytes(fmt, r0, cols), sn = abs_scales_bytes(fmt, nr, cols);
+            if (cudaMemcpyAsync(d_codes + c0, (const uint8_t*)codes_u8_host + c0, cn, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+                cudaMemcpyAsync(d_scales + s0, (const uint8_t*)scales_e4m3_host + s0, sn, cudaMemcpyHostToDevice, s) != cudaSuccess)
+                return ABS_ERR_CUDA;
+            rc = abs_dequantize_ex(fmt, d_codes + c0, d_scales + s0, d_alpha, nr, cols, d_out + (size_t)r0 * out_row, opts, stream);
+            if (rc != ABS_OK) return rc;
+            if (cudaEventRecord(st->chunk_done[i], s) != cudaSuccess ||
+                cudaStreamWaitEvent(st->d2h_stream, st->chunk_done[i], 0) != cudaSuccess ||
+                cudaMemcpyAsync((uint8_t*)out_host + (size_t)r0 * out_row, d_out + (size_t)r0 * out_row, (size_t)nr * out_row,
+                                cudaMemcpyDeviceToHost, st->d2h_stream) != cudaSuccess)
+                return ABS_ERR_CUDA;
+        }
+        if (cudaEventRecord(st->d2h_done, st->d2h_stream) != cudaSuccess || cudaStreamWaitEvent(s, st->d2h_done, 0) != cudaSuccess)
+            return ABS_ERR_CUDA;
+        return cudaStreamSynchronize(s) == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+    }
     if (cudaMemcpyAsync(d_codes, codes_u8_host, cb, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
     if (cudaMemcpyAsync(d_scales, scales_e4m3_host, sb, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
     if (cudaMemcpyAsync(d_alpha, tensor_scale_f32_host, 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;

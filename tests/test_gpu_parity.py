@@ -315,10 +315,13 @@ def test_back_to_back_calls_reuse_scratch(B, oracle):
         assert np.array_equal(s.cpu().numpy().reshape(64, -1), want[k][1])
 
 
-def test_host_buffer_entry_points(B, oracle):
-    xb = I.generate("cfg5", 96, 1024)
+@pytest.mark.parametrize("rows", [48, 96, 1000])
+def test_host_buffer_entry_points(B, oracle, rows):
+    """Host-buffer calls; from 64 rows on abs_dequantize_host works in row chunks on two streams (the last
+    chunk of 1000 rows is shorter than the others)."""
+    xb = I.generate("cfg5", rows, 1024)
     rows, cols = xb.shape
-    for fmt in (1, 3):
+    for fmt in ALL_FMTS:
         ws = torch.empty(B.abs_host_workspace_bytes(fmt, rows, cols), dtype=torch.uint8, device="cuda")
         xh = torch.from_numpy(xb.view(np.int16)).pin_memory()
         ch = torch.empty(B.abs_codes_bytes(fmt, rows, cols), dtype=torch.uint8).pin_memory()
