@@ -34,7 +34,7 @@ EXPORTS = [
     "abs_codes_bytes", "abs_scales_bytes", "abs_status_string", "abs_init", "abs_quantize", "abs_quantize_ex",
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
-    "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled",
+    "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled", "abs_quantize_dequantize",
 ]
 
 
@@ -83,6 +83,8 @@ def lib():
             L.abs_quantize_ex.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
             L.abs_quantize_transposed.restype = C.c_int
             L.abs_quantize_transposed.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp]
+            L.abs_quantize_dequantize.restype = C.c_int
+            L.abs_quantize_dequantize.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp, op, vp]
             L.abs_quantize_noalloc.restype = C.c_int
             L.abs_quantize_noalloc.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, vp]
             L.abs_dequantize.restype = C.c_int
@@ -192,6 +194,26 @@ def abs_quantize_transposed(fmt: int, x, codes_t=None, scales_t=None, tensor_sca
                                            _stream_ptr(stream))
     _check(rc, "abs_quantize_transposed")
     return codes_t, scales_t, tensor_scale
+
+
+def abs_quantize_dequantize(fmt: int, x, out=None, codes=None, scales=None, tensor_scale=None,
+                            opts: AbsOpts | None = None, stream=None):
+    """Quantize the CUDA bf16 matrix ``x`` and dequantize it in the same pass (the emulation of Sec. 4.1).
+    ``codes`` and ``scales`` are optional outputs (both or neither).  Returns (out bf16 [rows, cols], alpha)."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    rows, cols = x.shape
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.bfloat16, device=x.device)
+    if tensor_scale is None:
+        tensor_scale = torch.zeros(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        rc = lib().abs_quantize_dequantize(fmt, x.data_ptr(), rows, cols, out.data_ptr(),
+                                           codes.data_ptr() if codes is not None else None,
+                                           scales.data_ptr() if scales is not None else None, tensor_scale.data_ptr(),
+                                           C.byref(opts) if opts is not None else None, _stream_ptr(stream))
+    _check(rc, "abs_quantize_dequantize")
+    return out, tensor_scale
 
 
 def abs_quantize_noalloc(fmt: int, x, codes, scales, tensor_scale, stream=None):

@@ -217,18 +217,18 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     }
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         // Hadamard / stochastic-rounding options of the 4-bit formats: the packed persistent kernel
-        const int ogrid = grid_waves(st, ngroups, opt_blocks_per_sm(sr), ABS_OPT_ITERS);
+        const int ogrid = grid_waves(st, ngroups, opt_blocks_per_sm(sr, rht), ABS_OPT_ITERS);
         if (!(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)ogrid * kThreads) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             cudaError_t e;
 #define ABS_LAUNCH_O(R, S)                                                                                        \
-    e = alpha.slot ? launch_pdl(quantize4_opt_kernel<kInt, R, S, true>, ogrid, kThreads, s, (const uint4*)in,     \
+    e = alpha.slot ? launch_pdl(quantize4_opt_kernel<kInt, R, S, true, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, a32)                                           \
-                   : launch_pdl(quantize4_opt_kernel<kInt, R, S, false>, ogrid, kThreads, s, (const uint4*)in,    \
+                                (uint32_t)o.had_sign_mask, k0, k1, a32, (uint4*)nullptr, false, true)             \
+                   : launch_pdl(quantize4_opt_kernel<kInt, R, S, false, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, a32)
+                                (uint32_t)o.had_sign_mask, k0, k1, a32, (uint4*)nullptr, false, true)
             if (rht && sr) ABS_LAUNCH_O(true, true);
             else if (rht) ABS_LAUNCH_O(true, false);
             else ABS_LAUNCH_O(false, true);
@@ -578,6 +578,69 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
         case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
         default: return launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
     }
+}
+
+abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* out_bf16,
+                                     void* codes_u8, void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts,
+                                     void* stream) {
+    abs_opts_t o = {0, 0, 0, 0};
+    if (opts) o = *opts;
+    abs_status_t rc = check_shape(fmt, rows, cols);
+    if (rc != ABS_OK) return rc;
+    if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
+    if ((o.flags & ~(uint32_t)(ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN)) || o._pad)
+        return ABS_ERR_FLAGS;
+    if (rows * cols == 0) return ABS_OK;
+    if (!in_bf16 || !out_bf16 || !tensor_scale_f32 || ((codes_u8 == nullptr) != (scales_e4m3 == nullptr))) return ABS_ERR_NULL;
+    if (!aligned16(in_bf16) || !aligned16(out_bf16) || !aligned16(codes_u8) || !aligned16(scales_e4m3) ||
+        ((uintptr_t)tensor_scale_f32 & 3u))
+        return ABS_ERR_ALIGN;
+    DeviceState* st = nullptr;
+    if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t ngroups = rows * cols / 16;
+    const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
+    const int grid = grid_waves(*st, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? ABS_OPT_ITERS : ABS_FAST_ITERS);
+    if (ngroups >= (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads) return ABS_ERR_SIZE;
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
+        unsigned long long* slot = nullptr;
+        uint32_t gen = 0;
+        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        const float denom = 6.0f * 448.0f;
+        rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+        if (rc != ABS_OK) return rc;
+        src.slot = slot;
+        src.gen = gen;
+        src.denom = denom;
+    }
+    const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
+    const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
+    const bool a32 = (reinterpret_cast<uintptr_t>(in_bf16) & 31u) == 0, o32 = (reinterpret_cast<uintptr_t>(out_bf16) & 31u) == 0;
+    const bool store = codes_u8 != nullptr;
+    cudaError_t e = cudaSuccess;
+#define ABS_LAUNCH_E3(I, R, S, SLOT)                                                                                \
+    e = launch_pdl(quantize4_opt_kernel<I, R, S, SLOT, true>, grid, kThreads, s, (const uint4*)in_bf16, (uint2*)codes_u8, \
+                   (uint8_t*)scales_e4m3, src, (int32_t)ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1, a32,        \
+                   (uint4*)out_bf16, o32, store)
+#define ABS_LAUNCH_E2(I, R, S)                                                                                      \
+    do {                                                                                                            \
+        if (src.slot) ABS_LAUNCH_E3(I, R, S, true);                                                                 \
+        else ABS_LAUNCH_E3(I, R, S, false);                                                                         \
+    } while (0)
+#define ABS_LAUNCH_E(I)                                                                                             \
+    do {                                                                                                            \
+        if (rht && sr) ABS_LAUNCH_E2(I, true, true);                                                                \
+        else if (rht) ABS_LAUNCH_E2(I, true, false);                                                                \
+        else if (sr) ABS_LAUNCH_E2(I, false, true);                                                                 \
+        else ABS_LAUNCH_E2(I, false, false);                                                                        \
+    } while (0)
+    if (fmt == ABS_FMT_IF4) ABS_LAUNCH_E(true);
+    else ABS_LAUNCH_E(false);
+#undef ABS_LAUNCH_E
+#undef ABS_LAUNCH_E2
+#undef ABS_LAUNCH_E3
+    return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
 
 abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,

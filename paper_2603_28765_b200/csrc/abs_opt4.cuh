@@ -159,16 +159,21 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
 }
 
 // Resident blocks of 256 threads per SM the kernel is compiled and launched for: the stochastic-rounding
-// instances need about 120 registers, the Hadamard-only ones run best with three blocks.
-constexpr int opt_blocks_per_sm(bool sr) { return sr ? 2 : 3; }
+// instances need about 120 registers, the Hadamard-only ones run best with three blocks, the plain
+// round-to-nearest instance (used by the emulation pass only) with four.
+constexpr int opt_blocks_per_sm(bool sr, bool rht = true) { return sr ? 2 : (rht ? 3 : 4); }
 
 // Persistent grid-stride kernel, one group of 16 per thread and iteration, next group's 32 bytes fetched
 // before the current one is encoded.  scale_mul is 17/16 with that option and 1 otherwise (times 1 is exact).
-template <bool HAS_INT, bool RHT, bool SR, bool FROM_SLOT>
-__global__ void __launch_bounds__(256, opt_blocks_per_sm(SR))
+// EMUL = true is the emulation pass of Sec. 4.1 (every format was emulated by dequantizing right after
+// quantizing): the group is decoded from the registers that hold its codes and scale, with the arithmetic of
+// the dequantize kernel, and written to `out` as bf16; codes and scale bytes are stored only when
+// `store_codes` is set.
+template <bool HAS_INT, bool RHT, bool SR, bool FROM_SLOT, bool EMUL>
+__global__ void __launch_bounds__(256, opt_blocks_per_sm(SR, RHT))
 quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
-                     uint32_t seed_hi, bool aligned32) {
+                     uint32_t seed_hi, bool aligned32, uint4* __restrict__ out, bool out_aligned32, bool store_codes) {
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
@@ -232,8 +237,22 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
                 encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
             }
         }
-        scales[g] = (uint8_t)sbyte;
-        codes[g] = make_uint2(c_lo, c_hi);
+        if (!EMUL || store_codes) {
+            scales[g] = (uint8_t)sbyte;
+            codes[g] = make_uint2(c_lo, c_hi);
+        }
+        if constexpr (EMUL) {
+            const bool is_int = HAS_INT && (sbyte & 0x80u);
+            const float dd = is_int ? __fmul_rn(d, __uint_as_float(0x3F5B6DB7u)) : d;        // d * fp32(6/7) for integer groups
+            const float addend = is_int ? -1032.0f : -0.0f;
+            const uint64_t D2 = pack2(dd, dd);
+            uint32_t lo[4], hi[4];
+            dequant_word4<HAS_INT>(c_lo, is_int, addend, D2, lo);
+            dequant_word4<HAS_INT>(c_hi, is_int, addend, D2, hi);
+            const uint32_t o[8] = {lo[0], lo[1], lo[2], lo[3], hi[0], hi[1], hi[2], hi[3]};
+            if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
+            else store32B<false>(out + 2 * (size_t)g, o);
+        }
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
