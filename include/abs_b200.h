@@ -83,6 +83,9 @@ enum {
                                        k * Delta * alpha WITHOUT the 6/7 de-scale.  Both halves are exact in bf16, so
                                        the MAC arithmetic of Sec. 5.2 (factors 1, 6/7, 36/49 applied in FP32 on the
                                        scale path) can be reproduced with four plain bf16 GEMMs                      */
+    ABS_F_GROUPS_DOWN_COLUMNS = 1u << 9, /* abs_quantize_dequantize only: groups are 16 consecutive ROWS of one column
+                                       (Sec. 4.1: the operands of the weight-gradient product are quantized along the
+                                       token dimension); needs rows % 16 == 0                                        */
     ABS_F_INDEX64 = 1u << 5         /* testing aid: run the kernel instances that index groups with 64-bit
                                        integers (otherwise chosen only beyond 2^31 groups); same results  */
 };
@@ -150,6 +153,9 @@ ABS_API abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16,
  *                    TRANSFORMED values; nothing inverts the transform, as in abs_dequantize)
  *   codes_u8, scales_e4m3   optional outputs as for abs_quantize; pass both or pass NULL for both
  *   tensor_scale_f32 device pointer to one float: out (alpha), or in with ABS_F_ALPHA_GIVEN
+ * With ABS_F_GROUPS_DOWN_COLUMNS the groups run down the columns, as in abs_quantize_transposed: out_bf16 is
+ * still [rows, cols] in the orientation of the input (element (r, c) is the dequantized value of input element
+ * (r, c)), while the optional codes and scales come in the transposed layout of abs_quantize_transposed.
  * Each group is decoded from the registers that hold its codes, so the codes are never read back.  All
  * pointers 16-byte aligned; in_bf16 and out_bf16 must not overlap.  Other formats: ABS_ERR_FMT; other flags:
  * ABS_ERR_FLAGS; more than about 2^31 groups: ABS_ERR_SIZE. */

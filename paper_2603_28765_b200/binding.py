@@ -25,6 +25,7 @@ ABS_F_ALPHA_GIVEN = 1 << 3
 ABS_F_OUT_FP32 = 1 << 4
 ABS_F_INDEX64 = 1 << 5
 ABS_F_SCALES_SWIZZLED = 1 << 6
+ABS_F_GROUPS_DOWN_COLUMNS = 1 << 9
 ABS_F_FP_GROUPS_ONLY = 1 << 7
 ABS_F_INT_GROUPS_RAW = 1 << 8
 

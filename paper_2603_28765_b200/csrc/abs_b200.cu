@@ -464,6 +464,10 @@ abs_status_t check_shape(abs_fmt_t fmt, int64_t rows, int64_t cols) {
 
 // ------------------------------------------------------------------------------------------ C ABI
 
+static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
+                                             void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
+                                             const abs_opts_t& o, void* stream, void* out_bf16, bool store_codes);
+
 extern "C" {
 
 size_t abs_codes_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
@@ -588,13 +592,21 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
-    if ((o.flags & ~(uint32_t)(ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN)) || o._pad)
+    if ((o.flags & ~(uint32_t)(ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN |
+                               ABS_F_GROUPS_DOWN_COLUMNS)) || o._pad)
         return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_GROUPS_DOWN_COLUMNS) && (rows % 16) != 0) return ABS_ERR_SHAPE;
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !out_bf16 || !tensor_scale_f32 || ((codes_u8 == nullptr) != (scales_e4m3 == nullptr))) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(out_bf16) || !aligned16(codes_u8) || !aligned16(scales_e4m3) ||
         ((uintptr_t)tensor_scale_f32 & 3u))
         return ABS_ERR_ALIGN;
+    if (o.flags & ABS_F_GROUPS_DOWN_COLUMNS) {
+        abs_opts_t ot = o;
+        ot.flags &= ~(uint32_t)ABS_F_GROUPS_DOWN_COLUMNS;
+        return quantize_transposed_impl(fmt, in_bf16, rows, cols, codes_u8, scales_e4m3, tensor_scale_f32, ot, stream,
+                                        out_bf16, codes_u8 != nullptr);
+    }
     DeviceState* st = nullptr;
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
@@ -662,6 +674,18 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     if (!in_bf16 || !codes_t_u8 || !scales_t_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(codes_t_u8) || !aligned16(scales_t_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
         return ABS_ERR_ALIGN;
+    return quantize_transposed_impl(fmt, in_bf16, rows, cols, codes_t_u8, scales_t_e4m3, tensor_scale_f32, o, stream,
+                                    nullptr, true);
+}
+
+}  // extern "C"
+
+// The transposed tile walk: plain transposed quantize (out == nullptr) or the emulation pass along the columns
+// (out = [rows, cols] bf16 in the original orientation; codes stored only when store_codes).  Arguments are
+// already validated.
+static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
+                                             void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
+                                             const abs_opts_t& o, void* stream, void* out_bf16, bool store_codes) {
     DeviceState* st = nullptr;
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
@@ -695,13 +719,18 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
     uint2* ct = (uint2*)codes_t_u8;
     uint8_t* stp = (uint8_t*)scales_t_e4m3;
     const uint32_t mask = o.had_sign_mask;
-#define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
+#define ABS_LAUNCH_TE(I, S, R, Q, M, E, SLOT, GEN)                                                                  \
     do {                                                                                                            \
-        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, Q, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, Q, M, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  kTransSmemBytes);                                                                  \
         if (e == cudaSuccess)                                                                                       \
-            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, Q, M>, in, ct, stp, src, rows, cols, mask, \
-                                   SLOT, GEN, mul, k0, k1);                                                         \
+            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, Q, M, E>, in, ct, stp, src, rows, cols, mask, \
+                                   SLOT, GEN, mul, k0, k1, (uint16_t*)out_bf16, store_codes);                       \
+    } while (0)
+#define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
+    do {                                                                                                            \
+        if (M == 0 && out_bf16) ABS_LAUNCH_TE(I, S, R, Q, 0, true, SLOT, GEN);                                      \
+        else ABS_LAUNCH_TE(I, S, R, Q, M, false, SLOT, GEN);                                                        \
     } while (0)
 
     const bool sr = o.flags & ABS_F_STOCHASTIC;
@@ -743,8 +772,11 @@ abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t
 #undef ABS_LAUNCH_T3
 #undef ABS_LAUNCH_T2
 #undef ABS_LAUNCH_T
+#undef ABS_LAUNCH_TE
     return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ABS_OK : ABS_ERR_CUDA;
 }
+
+extern "C" {
 
 abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                                   void* scales_e4m3, float* tensor_scale_f32, void* stream) {

@@ -66,14 +66,19 @@ __device__ __forceinline__ void hadamard16_pairs(float (&x)[16], uint32_t sign_m
 // the transposed path with the Hadamard option; publishes a tagged maximum like amax_kernel).
 // SR: stochastic rounding of both candidates (App. B); element indices, and so the Philox counters, are
 // those of the transposed matrix.  scale_mul is 17/16 with that option and 1 otherwise.
-template <bool HAS_INT, bool FROM_SLOT, bool RHT, bool SR, int MODE>
+// EMUL (MODE 0 only): the emulation pass of Sec. 4.1 along the columns.  Every group is decoded from the
+// registers that hold its codes and written back over its own input values in the shared-memory tile; the
+// finished tile then leaves with coalesced 16-byte stores to `out`, a [rows, cols] matrix in the ORIGINAL
+// orientation.  Codes and scales (transposed layout) are stored only when `store_codes` is set.
+template <bool HAS_INT, bool FROM_SLOT, bool RHT, bool SR, int MODE, bool EMUL = false>
 __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_t* __restrict__ in,
                                                                    uint2* __restrict__ codes_t,
                                                                    uint8_t* __restrict__ scales_t,
                                                                    const AlphaSrc alpha_src, int64_t rows, int64_t cols,
                                                                    uint32_t sign_mask, unsigned long long* amax_slot,
                                                                    uint32_t amax_gen, float scale_mul, uint32_t seed_lo,
-                                                                   uint32_t seed_hi) {
+                                                                   uint32_t seed_hi, uint16_t* __restrict__ out,
+                                                                   bool store_codes) {
     extern __shared__ __align__(16) uint16_t trans_smem[];
     pdl_launch_dependents();
     pdl_wait();
@@ -127,7 +132,7 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
         const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
         const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
         const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
-        const uint16_t* stage = trans_smem + s * kTransStageElems;
+        uint16_t* stage = trans_smem + s * kTransStageElems;
         const int c = threadIdx.x;
         if (c < ncols) {
             uint32_t cw[2 * kTransTileRowBlocks];
@@ -168,6 +173,25 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
                 } else {
                     encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
                 }
+                if constexpr (EMUL) {
+                    // decode the group from its codes (arithmetic of the dequantize kernel) over its own inputs
+                    const bool is_int = HAS_INT && (sbyte & 0x80u);
+                    const float dd = is_int ? __fmul_rn(d, __uint_as_float(0x3F5B6DB7u)) : d;
+                    const float addend = is_int ? -1032.0f : -0.0f;
+                    const uint64_t D2 = pack2(dd, dd);
+                    uint32_t lo[4], hi[4];
+                    dequant_word4<HAS_INT>(c_lo, is_int, addend, D2, lo);
+                    dequant_word4<HAS_INT>(c_hi, is_int, addend, D2, hi);
+                    uint16_t* colw = stage + 16 * k * kTransTileCols + c;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        colw[(2 * i) * kTransTileCols] = (uint16_t)lo[i];
+                        colw[(2 * i + 1) * kTransTileCols] = (uint16_t)(lo[i] >> 16);
+                        colw[(8 + 2 * i) * kTransTileCols] = (uint16_t)hi[i];
+                        colw[(9 + 2 * i) * kTransTileCols] = (uint16_t)(hi[i] >> 16);
+                    }
+                    if (!store_codes) continue;
+                }
                 if (vec_ok) {
                     // k is a runtime index: select the slot without dynamic register indexing
 #pragma unroll
@@ -179,10 +203,20 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
                     codes_t[g] = make_uint2(c_lo, c_hi);
                 }
             }
-            if (MODE == 0 && vec_ok) {
+            if (MODE == 0 && vec_ok && (!EMUL || store_codes)) {
                 const int64_t g0 = (c0 + c) * rblocks + rb0;
                 store32B<true>(codes_t + g0, reinterpret_cast<const uint32_t(&)[8]>(cw));
                 *reinterpret_cast<uint32_t*>(scales_t + g0) = sbytes;
+            }
+        }
+        if constexpr (EMUL) {
+            __syncthreads();                         // the whole tile now holds dequantized values
+            uint16_t* dst = out + rb0 * 16 * cols + c0;
+            const int chunks_per_row = ncols / 8;
+            for (int ch = threadIdx.x; ch < 16 * nrb * chunks_per_row; ch += blockDim.x) {
+                const int r = ch / chunks_per_row, q = ch - r * chunks_per_row;
+                *reinterpret_cast<uint4*>(dst + (int64_t)r * cols + q * 8) =
+                    *reinterpret_cast<const uint4*>(stage + r * kTransTileCols + q * 8);
             }
         }
         __syncthreads();                             // the stage may be overwritten by the next prefetch

@@ -528,6 +528,29 @@ def test_fused_quantize_dequantize_is_quantize_then_dequantize(B, oracle, fmt):
             assert_same("fused codes", codes.cpu().numpy()[:oc.size].reshape(oc.shape), oc)
             assert_same("fused scales", scales.cpu().numpy()[:osc.size].reshape(osc.shape), osc)
             assert bool((codes[oc.size:] == 0xA5).all()) and bool((scales[osc.size:] == 0xA5).all())
+    # groups down the columns (Sec. 4.1, weight-gradient operands): the output keeps the input's orientation
+    C_ = B.ABS_F_GROUPS_DOWN_COLUMNS
+    for flags in (0, H, H | S | S17, G):
+        for name, rows, cols in (("cfg2", 304, 1024), ("cfg4", 64, 2064), ("cfg5", 2048, 272), ("cfg1", 16, 16)):
+            xb = I.generate(name, rows, cols)
+            alpha = 0.004 if flags & G else None
+            ts = torch.tensor([alpha], dtype=torch.float32, device="cuda") if alpha is not None else None
+            oc, osc, oa = oracle.quantize(fmt, np.ascontiguousarray(xb.T), flags=flags, sign_mask=mask, sr_seed=77,
+                                          alpha=alpha, threads=THREADS)
+            od = np.ascontiguousarray(oracle.dequantize(fmt, oc, osc, oa, cols, rows, threads=THREADS).T)
+            codes = torch.full((oc.size + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            scales = torch.full((osc.size + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            out, a = B.abs_quantize_dequantize(fmt, to_dev(xb), codes=codes, scales=scales, tensor_scale=ts,
+                                               opts=B.make_opts(flags | C_, mask, 77))
+            out2, a2 = B.abs_quantize_dequantize(fmt, to_dev(xb), tensor_scale=ts.clone() if ts is not None else None,
+                                                 opts=B.make_opts(flags | C_, mask, 77))
+            torch.cuda.synchronize()
+            assert np.float32(a.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+            assert_same("column emulation out", out.view(torch.int16).cpu().numpy().view(np.uint16), od)
+            assert_same("column emulation out, no codes", out2.view(torch.int16).cpu().numpy().view(np.uint16), od)
+            assert_same("column emulation codes", codes.cpu().numpy()[:oc.size].reshape(oc.shape), oc)
+            assert_same("column emulation scales", scales.cpu().numpy()[:osc.size].reshape(osc.shape), osc)
+            assert bool((codes[oc.size:] == 0xA5).all()) and bool((scales[osc.size:] == 0xA5).all())
     # argument checks: other formats, unknown flags, one of the two optional outputs alone
     L = B.lib()
     x = to_dev(I.generate("cfg1", 16, 64))
@@ -541,6 +564,11 @@ def test_fused_quantize_dequantize_is_quantize_then_dequantize(B, oracle, fmt):
                                      ctypes.byref(bad), None) == 5
     assert L.abs_quantize_dequantize(fmt, x.data_ptr(), 16, 64, out.data_ptr(), buf.data_ptr(), None, ts.data_ptr(),
                                      None, None) == 1
+    col = B.make_opts(B.ABS_F_GROUPS_DOWN_COLUMNS)
+    assert L.abs_quantize_dequantize(fmt, x.data_ptr(), 8, 64, out.data_ptr(), None, None, ts.data_ptr(),
+                                     ctypes.byref(col), None) == 2          # rows must be a multiple of 16
+    assert L.abs_quantize_ex(fmt, x.data_ptr(), 16, 64, buf.data_ptr(), buf.data_ptr(), ts.data_ptr(),
+                             ctypes.byref(col), None) == 5                  # the flag belongs to the emulation call only
     torch.cuda.synchronize()
 
 
