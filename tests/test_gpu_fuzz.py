@@ -73,6 +73,12 @@ def test_random_cases_match_the_oracle(B, oracle, seed):
         assert np.array_equal(scales.cpu().numpy()[:osc.size].reshape(osc.shape), osc), where
         assert np.array_equal(out.view(torch.int16).cpu().numpy().view(np.uint16),
                               oracle.dequantize(fmt, oc, osc, oa, rows, cols)), where
+        if fmt in (0, 1):                   # the one-pass emulation gives the same dequantized bytes
+            od = oracle.dequantize(fmt, oc, osc, oa, rows, cols)
+            ts2 = torch.tensor([alpha], dtype=torch.float32, device="cuda") if alpha is not None else None
+            eo, _ = B.abs_quantize_dequantize(fmt, x, tensor_scale=ts2, opts=B.make_opts(flags, mask, sr_seed))
+            torch.cuda.synchronize()
+            assert np.array_equal(eo.view(torch.int16).cpu().numpy().view(np.uint16), od), where
         if fmt in (0, 1) and rows % 16 == 0:
             tf = flags & ~B.ABS_F_ALPHA_GIVEN
             ct, st, at = B.abs_quantize_transposed(fmt, x, opts=B.make_opts(tf, mask, sr_seed))
@@ -81,3 +87,7 @@ def test_random_cases_match_the_oracle(B, oracle, seed):
             assert np.float32(at.item()).view(np.uint32) == np.float32(oa).view(np.uint32), where
             assert np.array_equal(ct.cpu().numpy()[:oc.size].reshape(oc.shape), oc), where
             assert np.array_equal(st.cpu().numpy()[:osc.size].reshape(osc.shape), osc), where
+            eo, _ = B.abs_quantize_dequantize(fmt, x, opts=B.make_opts(tf | B.ABS_F_GROUPS_DOWN_COLUMNS, mask, sr_seed))
+            torch.cuda.synchronize()
+            odt = np.ascontiguousarray(oracle.dequantize(fmt, oc, osc, oa, cols, rows).T)
+            assert np.array_equal(eo.view(torch.int16).cpu().numpy().view(np.uint16), odt), where
