@@ -145,8 +145,9 @@ ABS_API abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16,
                                              const abs_opts_t* opts, void* stream);
 
 /* Quantize and dequantize in one pass: the emulation of Sec. 4.1 (every format studied was emulated by
- * dequantizing the quantized values back to BF16 before each matrix product).  Formats ABS_FMT_IF4 and
- * ABS_FMT_NVFP4; flags ABS_F_ALPHA_GIVEN, ABS_F_HADAMARD16, ABS_F_STOCHASTIC, ABS_F_SR_SCALE_17_16.
+ * dequantizing the quantized values back to BF16 before each matrix product).  Every format; flags
+ * ABS_F_ALPHA_GIVEN and ABS_F_SR_SCALE_17_16, and for ABS_FMT_IF4 / ABS_FMT_NVFP4 also ABS_F_HADAMARD16,
+ * ABS_F_STOCHASTIC and ABS_F_GROUPS_DOWN_COLUMNS.
  *   in_bf16          [rows, cols] bf16 (device), as for abs_quantize
  *   out_bf16         out, [rows, cols] bf16 (device): byte for byte what abs_dequantize gives for the result
  *                    of abs_quantize_ex with the same options (with the Hadamard option: the dequantized
@@ -157,7 +158,7 @@ ABS_API abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16,
  * still [rows, cols] in the orientation of the input (element (r, c) is the dequantized value of input element
  * (r, c)), while the optional codes and scales come in the transposed layout of abs_quantize_transposed.
  * Each group is decoded from the registers that hold its codes, so the codes are never read back.  All
- * pointers 16-byte aligned; in_bf16 and out_bf16 must not overlap.  Other formats: ABS_ERR_FMT; other flags:
+ * pointers 16-byte aligned; in_bf16 and out_bf16 must not overlap.  Flags the format does not take:
  * ABS_ERR_FLAGS; more than about 2^31 groups: ABS_ERR_SIZE. */
 ABS_API abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
                                              void* out_bf16, void* codes_u8, void* scales_e4m3, float* tensor_scale_f32,

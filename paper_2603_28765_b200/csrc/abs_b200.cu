@@ -176,14 +176,21 @@ abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const
 #endif
 
 template <int FMT>
+// emul_out != nullptr asks for the emulation pass (abs_quantize_dequantize) of the formats handled by the
+// kernels of abs_fastx.cuh: bf16 output, codes stored only when emul_store.  *handled tells the caller whether
+// a kernel with that ability exists for the format and options.
 abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
-                                 const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s, int64_t cols = 0) {
+                                 const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s, int64_t cols = 0,
+                                 void* emul_out = nullptr, bool emul_store = true, bool* handled = nullptr) {
+    if (handled) *handled = false;
+    const bool o32 = (reinterpret_cast<uintptr_t>(emul_out) & 31u) == 0;
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const int grid = grid_for(st, ngroups, 64);
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
+        if (emul_out) return ABS_ERR_FLAGS;      // the 4-bit emulation pass is launched by abs_quantize_dequantize
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
             const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(st, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(st, ngroups, 5, ABS_NV_ITERS);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
@@ -243,12 +250,15 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
         constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
         const int bgrid = grid_waves(st, ngroups, kInt ? 4 : 5, kInt ? ABS_IF6_ITERS : 5);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
+            if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const cudaError_t e =
-                alpha.slot ? launch_pdl(quantize4_bs8_kernel<kInt, true>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
-                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32)
-                           : launch_pdl(quantize4_bs8_kernel<kInt, false>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
-                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32);
+                alpha.slot ? (emul_out ? launch_pdl(quantize4_bs8_kernel<kInt, true, true>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize4_bs8_kernel<kInt, true, false>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true))
+                           : (emul_out ? launch_pdl(quantize4_bs8_kernel<kInt, false, true>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize4_bs8_kernel<kInt, false, false>, bgrid, kThreads, s, (const uint4*)in, (uint2*)codes,
+                                        (uint16_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true));
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
@@ -258,12 +268,15 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
         // 6-bit formats, round-to-nearest
         const int sgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
+            if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const cudaError_t e =
-                alpha.slot ? launch_pdl(quantize6_fast_kernel<FMT, true>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
-                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32)
-                           : launch_pdl(quantize6_fast_kernel<FMT, false>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
-                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32);
+                alpha.slot ? (emul_out ? launch_pdl(quantize6_fast_kernel<FMT, true, true>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize6_fast_kernel<FMT, true, false>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true))
+                           : (emul_out ? launch_pdl(quantize6_fast_kernel<FMT, false, true>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize6_fast_kernel<FMT, false, false>, sgrid, kThreads, s, (const uint4*)in, (uint32_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true));
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
@@ -274,17 +287,21 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
         constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
         const int tgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
+            if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const cudaError_t e =
-                alpha.slot ? launch_pdl(quantize3_fast_kernel<kG, true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
-                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32)
-                           : launch_pdl(quantize3_fast_kernel<kG, false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
-                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32);
+                alpha.slot ? (emul_out ? launch_pdl(quantize3_fast_kernel<kG, true, true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize3_fast_kernel<kG, true, false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true))
+                           : (emul_out ? launch_pdl(quantize3_fast_kernel<kG, false, true>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)emul_out, o32, emul_store) : launch_pdl(quantize3_fast_kernel<kG, false, false>, tgrid, kThreads, s, (const uint4*)in, (uint16_t*)codes,
+                                        (uint8_t*)scales, alpha, (int32_t)ngroups, mul, a32, (uint4*)nullptr, false, true));
             if (e != cudaSuccess) return ABS_ERR_CUDA;
             if (g_ev_quant_end) cudaEventRecord(g_ev_quant_end, s);
             return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
         }
     }
+    if (emul_out) return ABS_ERR_FLAGS;          // no emulation kernel for this format / option combination
     cudaError_t eq = cudaSuccess;
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
     eq = alpha.slot ? launch_pdl(quantize_kernel<FMT, R, S, true>, grid, kThreads, s, (const uint4*)in,         \
@@ -591,10 +608,12 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
-    if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
+    const bool four_bit = fmt == ABS_FMT_NVFP4 || fmt == ABS_FMT_IF4;
     if ((o.flags & ~(uint32_t)(ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN |
                                ABS_F_GROUPS_DOWN_COLUMNS)) || o._pad)
         return ABS_ERR_FLAGS;
+    // IF3, IF6 and the block-size-8 formats: round-to-nearest along the rows only
+    if (!four_bit && (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_GROUPS_DOWN_COLUMNS))) return ABS_ERR_FLAGS;
     if ((o.flags & ABS_F_GROUPS_DOWN_COLUMNS) && (rows % 16) != 0) return ABS_ERR_SHAPE;
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !out_bf16 || !tensor_scale_f32 || ((codes_u8 == nullptr) != (scales_e4m3 == nullptr))) return ABS_ERR_NULL;
@@ -613,23 +632,35 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     const int64_t ngroups = rows * cols / 16;
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
     const int grid = grid_waves(*st, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? ABS_OPT_ITERS : ABS_FAST_ITERS);
-    if (ngroups >= (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads) return ABS_ERR_SIZE;
+    if (ngroups >= (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads) return ABS_ERR_SIZE;    // 32-bit group indices only
     AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;
         uint32_t gen = 0;
         if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
-        const float denom = 6.0f * 448.0f;
+        const float denom = fmt_mfp((int)fmt) * 448.0f;
         rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
         if (rc != ABS_OK) return rc;
         src.slot = slot;
         src.gen = gen;
         src.denom = denom;
     }
+    const bool store = codes_u8 != nullptr;
+    if (!four_bit) {
+        bool handled = false;
+        switch (fmt) {
+            case ABS_FMT_IF3: rc = launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF6_E2M3: rc = launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF6_E3M2: rc = launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_NVFP4_BS8: rc = launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF4_BS8: rc = launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            default: rc = launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+        }
+        return (!handled && rc == ABS_ERR_FLAGS) ? ABS_ERR_SIZE : rc;
+    }
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     const bool a32 = (reinterpret_cast<uintptr_t>(in_bf16) & 31u) == 0, o32 = (reinterpret_cast<uintptr_t>(out_bf16) & 31u) == 0;
-    const bool store = codes_u8 != nullptr;
     cudaError_t e = cudaSuccess;
 #define ABS_LAUNCH_E3(I, R, S, SLOT)                                                                                \
     e = launch_pdl(quantize4_opt_kernel<I, R, S, SLOT, true>, grid, kThreads, s, (const uint4*)in_bf16, (uint2*)codes_u8, \

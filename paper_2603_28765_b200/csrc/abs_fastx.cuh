@@ -7,6 +7,70 @@
 
 namespace absq {
 
+// ----------------------------------------------------------------------------- decode helpers
+
+// Eight 3-bit fields of a 24-bit chunk (field j at bit 3j) spread to the low three bits of eight nibbles:
+// 12-bit halves to 16-bit halves, 6-bit pairs to bytes, 3-bit fields to nibbles, each step one mask and
+// one multiply-add (moving a part left by s bits adds (2^s - 1) times that part).
+__device__ __forceinline__ uint32_t spread3to4(uint32_t x) {
+    const uint32_t y = x + (x >> 12) * 0xF000u;
+    const uint32_t z = y + (y & 0x0FC00FC0u) * 3u;
+    return z + (z & 0x38383838u);
+}
+
+// Eight 3-bit codes (a 24-bit chunk) -> eight products value * d as four packed bf16 pairs, through the 4-bit
+// decoder: an E2M0 code s|ee is the E2M1 code s|ee|0 (values 0, 1, 2, 4 are the E2M1 codes with a zero mantissa
+// bit), and a 3-bit two's-complement integer sign-extends to a nibble.  d already holds the 4/3 factor of
+// integer groups.
+__device__ __forceinline__ void decode3x8(uint32_t chunk, bool is_int, float d, uint32_t (&r)[4]) {
+    const uint32_t u = spread3to4(chunk);
+    const uint32_t w = is_int ? (u + (u & 0x44444444u) * 2u) : (u << 1);
+    dequant_word4<true>(w, is_int, is_int ? -1032.0f : -0.0f, pack2(d, d), r);
+}
+
+// Four 6-bit fields of a 24-bit chunk (field j at bit 6j) spread to one field per byte: the inverse of
+// squeeze6x4 (below), again one mask and one multiply-add per step.
+__device__ __forceinline__ uint32_t spread6to8(uint32_t c) {
+    const uint32_t t = c + (c >> 12) * 0xF000u;
+    return t + (t & 0x0FC00FC0u) * 3u;
+}
+
+// Sixteen 6-bit codes (three words) -> sixteen products value * d as eight packed bf16 pairs.  Branch-free like
+// the 4-bit decoder: the FP decode is the hardware convert to f16 pairs, the integer decode places the field
+// k + 32 (field xor 32) in the mantissa of the f16 constant 1024, so the half is 1056 + k; one shared tail adds
+// -0 or -1056 in FP32, multiplies by the group scale (which already holds the de-scale factor of integer
+// groups) and rounds to bf16 pairs.
+template <ElemKind EK>
+__device__ __forceinline__ void decode6x16(uint32_t w0, uint32_t w1, uint32_t w2, bool is_int, float d, uint32_t (&o)[8]) {
+    const float addend = is_int ? -1056.0f : -0.0f;
+    const uint64_t D2 = pack2(d, d);
+    const uint32_t chunk[4] = {w0 & 0xFFFFFFu, (w0 >> 24) | ((w1 & 0xFFFFu) << 8), (w1 >> 16) | ((w2 & 0xFFu) << 16), w2 >> 8};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t bytes = spread6to8(chunk[q]);                       // codes 4q .. 4q+3, one per byte
+        uint32_t h0, h1;
+        if constexpr (EK == EK_E2M3) {
+            asm("{ .reg .b16 lo, hi;\n"
+                "  mov.b32 {lo, hi}, %2;\n"
+                "  cvt.rn.f16x2.e2m3x2 %0, lo;\n"
+                "  cvt.rn.f16x2.e2m3x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
+        } else {
+            asm("{ .reg .b16 lo, hi;\n"
+                "  mov.b32 {lo, hi}, %2;\n"
+                "  cvt.rn.f16x2.e3m2x2 %0, lo;\n"
+                "  cvt.rn.f16x2.e3m2x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
+        }
+        const uint32_t r0 = __byte_perm(bytes, 0u, 0x4140) ^ 0x64206420u;  // halves 1056 + k of codes 4q, 4q+1
+        const uint32_t r1 = __byte_perm(bytes, 0u, 0x4342) ^ 0x64206420u;  // ... of codes 4q+2, 4q+3
+        const uint32_t s0 = is_int ? r0 : h0, s1 = is_int ? r1 : h1;
+        float p0, p1, p2, p3;
+        unpack2(mul2(pack2(half_plus_f32(s0, false, addend), half_plus_f32(s0, true, addend)), D2), p0, p1);
+        unpack2(mul2(pack2(half_plus_f32(s1, false, addend), half_plus_f32(s1, true, addend)), D2), p2, p3);
+        o[2 * q] = bf16x2_rn(p0, p1);
+        o[2 * q + 1] = bf16x2_rn(p2, p3);
+    }
+}
+
 // ----------------------------------------------------------------------------- 4-bit, one scale per 8 values
 
 // Steps 3-10 of Fig. 3a for one group of EIGHT values (one 32-bit word of codes).  The error sums of a
@@ -71,10 +135,14 @@ __device__ __forceinline__ void encode_half4(const float* x, uint32_t sb, float 
 
 // One thread per aligned block of 16 values = two groups of 8: two scales, one 64-bit store of codes and
 // one 16-bit store of scale bytes.  scale_mul is 17/16 with that option and 1 otherwise.
-template <bool HAS_INT, bool FROM_SLOT>
+// EMUL (all kernels of this file): the emulation pass of Sec. 4.1, as in quantize4_opt_kernel: the group is decoded
+// from the registers that hold its codes and scale and written to `out` as bf16; codes and scale bytes are
+// stored only when `store_codes` is set.
+template <bool HAS_INT, bool FROM_SLOT, bool EMUL = false>
 __global__ void __launch_bounds__(256, HAS_INT ? 4 : 5)
 quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint16_t* __restrict__ scales,
-                     const AlphaSrc alpha_src, int32_t nblocks16, float scale_mul, bool aligned32) {
+                     const AlphaSrc alpha_src, int32_t nblocks16, float scale_mul, bool aligned32,
+                     uint4* __restrict__ out = nullptr, bool out_aligned32 = false, bool store_codes = true) {
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
@@ -101,7 +169,7 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
             x[2 * i] = __uint_as_float(w[i] << 16);
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
-        uint32_t cw[2], sbytes = 0u;
+        uint32_t cw[2], sbytes = 0u, o[8];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const float* xs = x + 8 * h;
@@ -118,9 +186,22 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
             }
             cw[h] = c;
             sbytes |= sbyte << (8 * h);
+            if constexpr (EMUL) {
+                const bool is_int = HAS_INT && (sbyte & 0x80u);
+                const float dd = is_int ? __fmul_rn(d, __uint_as_float(0x3F5B6DB7u)) : d;
+                uint32_t rr[4];
+                dequant_word4<HAS_INT>(c, is_int, is_int ? -1032.0f : -0.0f, pack2(dd, dd), rr);
+                o[4 * h] = rr[0]; o[4 * h + 1] = rr[1]; o[4 * h + 2] = rr[2]; o[4 * h + 3] = rr[3];
+            }
         }
-        scales[g] = (uint16_t)sbytes;
-        codes[g] = make_uint2(cw[0], cw[1]);
+        if (!EMUL || store_codes) {
+            scales[g] = (uint16_t)sbytes;
+            codes[g] = make_uint2(cw[0], cw[1]);
+        }
+        if constexpr (EMUL) {
+            if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
+            else store32B<false>(out + 2 * (size_t)g, o);
+        }
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
@@ -228,10 +309,11 @@ __device__ __forceinline__ void encode_body6(const float (&x)[16], uint32_t sb, 
     sbyte = sb | (flag ? 0x80u : 0u);                                           // S3
 }
 
-template <int FMT, bool FROM_SLOT>
+template <int FMT, bool FROM_SLOT, bool EMUL = false>
 __global__ void __launch_bounds__(256, 3)
 quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32) {
+                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32,
+                      uint4* __restrict__ out = nullptr, bool out_aligned32 = false, bool store_codes = true) {
     using F = Fmt<FMT>;
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
@@ -270,9 +352,18 @@ quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
         const float r = __frcp_rn(d);
         uint32_t sbyte = 0u, cw[3] = {0u, 0u, 0u};
         if (sb != 0u) encode_body6<F::EK>(x, sb, d, r, c_pre, c_post, sbyte, cw);   // G4: zero scale -> zeros
-        scales[g] = (uint8_t)sbyte;
-        uint32_t* cp = codes + 3 * (size_t)g;
-        cp[0] = cw[0]; cp[1] = cw[1]; cp[2] = cw[2];
+        if (!EMUL || store_codes) {
+            scales[g] = (uint8_t)sbyte;
+            uint32_t* cp = codes + 3 * (size_t)g;
+            cp[0] = cw[0]; cp[1] = cw[1]; cp[2] = cw[2];
+        }
+        if constexpr (EMUL) {
+            const bool is_int = sbyte & 0x80u;
+            uint32_t o[8];
+            decode6x16<F::EK>(cw[0], cw[1], cw[2], is_int, is_int ? __fmul_rn(d, c_post) : d, o);
+            if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
+            else store32B<false>(out + 2 * (size_t)g, o);
+        }
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
@@ -388,10 +479,11 @@ __device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_
 }
 
 // G = 16: one scale per thread's 16 values.  G = 8 (IF3-BS8): each half has its own scale and selection.
-template <int G, bool FROM_SLOT>
+template <int G, bool FROM_SLOT, bool EMUL = false>
 __global__ void __launch_bounds__(256, 3)
 quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32) {
+                      const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32,
+                      uint4* __restrict__ out = nullptr, bool out_aligned32 = false, bool store_codes = true) {
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
@@ -418,7 +510,8 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
             x[2 * i] = __uint_as_float(w[i] << 16);
             x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
         }
-        uint32_t c_lo = 0u, c_hi = 0u;
+        uint32_t c_lo = 0u, c_hi = 0u, o[8];
+        const float c_post3 = __fdiv_rn(4.0f, 3.0f);
         if constexpr (G == 16) {
             const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);                    // G1
             const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
@@ -434,7 +527,16 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
             } else {
                 encode_body3<false>(x, w, sb, d, r, sbyte, c_lo, c_hi);
             }
-            scales[g] = (uint8_t)sbyte;
+            if (!EMUL || store_codes) scales[g] = (uint8_t)sbyte;
+            if constexpr (EMUL) {
+                const bool is_int = sbyte & 0x80u;
+                const float dd = is_int ? __fmul_rn(d, c_post3) : d;
+                uint32_t r0[4], r1[4];
+                decode3x8(c_lo & 0xFFFFFFu, is_int, dd, r0);
+                decode3x8((c_lo >> 24) | (c_hi << 8), is_int, dd, r1);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { o[j] = r0[j]; o[4 + j] = r1[j]; }
+            }
         } else {
             uint32_t chunk[2] = {0u, 0u}, sbytes = 0u;
 #pragma unroll
@@ -454,14 +556,29 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
                     const bool flag = __fadd_rn(i0, i1) < __fadd_rn(f0, f1);  // a group of 8: S0 + S1
                     chunk[h] = flag ? ic : fc;
                     sbytes |= (sb | (flag ? 0x80u : 0u)) << (8 * h);
+                    if constexpr (EMUL) {
+                        uint32_t rr[4];
+                        decode3x8(chunk[h], flag, flag ? __fmul_rn(d, c_post3) : d, rr);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) o[4 * h + j] = rr[j];
+                    }
+                } else if constexpr (EMUL) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o[4 * h + j] = 0u;           // zero scale: the group decodes to +0
                 }
             }
             c_lo = chunk[0] | (chunk[1] << 24);
             c_hi = chunk[1] >> 8;
-            reinterpret_cast<uint16_t*>(scales)[g] = (uint16_t)sbytes;
+            if (!EMUL || store_codes) reinterpret_cast<uint16_t*>(scales)[g] = (uint16_t)sbytes;
         }
-        uint16_t* cp = codes + 3 * (size_t)g;                                // 6 bytes per block of 16
-        cp[0] = (uint16_t)c_lo; cp[1] = (uint16_t)(c_lo >> 16); cp[2] = (uint16_t)c_hi;
+        if (!EMUL || store_codes) {
+            uint16_t* cp = codes + 3 * (size_t)g;                            // 6 bytes per block of 16
+            cp[0] = (uint16_t)c_lo; cp[1] = (uint16_t)(c_lo >> 16); cp[2] = (uint16_t)c_hi;
+        }
+        if constexpr (EMUL) {
+            if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
+            else store32B<false>(out + 2 * (size_t)g, o);
+        }
         if (!more) break;
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = wn[i];
@@ -471,18 +588,8 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
 
 // ----------------------------------------------------------------------------- 3-bit dequantize
 
-// Eight 3-bit fields of a 24-bit chunk (field j at bit 3j) spread to the low three bits of eight nibbles:
-// 12-bit halves to 16-bit halves, 6-bit pairs to bytes, 3-bit fields to nibbles, each step one mask and
-// one multiply-add (moving a part left by s bits adds (2^s - 1) times that part).
-__device__ __forceinline__ uint32_t spread3to4(uint32_t x) {
-    const uint32_t y = x + (x >> 12) * 0xF000u;
-    const uint32_t z = y + (y & 0x0FC00FC0u) * 3u;
-    return z + (z & 0x38383838u);
-}
-
-// IF3 / IF3-BS8 dequantize through the 4-bit decoder: an E2M0 code s|ee is the E2M1 code s|ee|0 (values
-// 0, 1, 2, 4 are the E2M1 codes with a zero mantissa bit), and a 3-bit two's-complement integer sign-extends
-// to a nibble.  One thread per aligned block of 16 values; G = 8 gives each word of eight codes its own scale.
+// IF3 / IF3-BS8 dequantize (decode3x8).  One thread per aligned block of 16 values; G = 8 gives each word of
+// eight codes its own scale.
 template <int G, bool ALIGNED32>
 __global__ void __launch_bounds__(256) dequantize3_fast_kernel(const uint16_t* __restrict__ codes,
                                                                const uint8_t* __restrict__ scales,
@@ -514,10 +621,8 @@ __global__ void __launch_bounds__(256) dequantize3_fast_kernel(const uint16_t* _
             if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);        // E4M3 NaN propagates
             float d = __fmul_rn(Delta, alpha);
             if (is_int) d = __fmul_rn(d, c_post);                          // de-scale integer groups (Sec. 3)
-            const uint32_t u = spread3to4(chunk[h]);
-            const uint32_t w = is_int ? (u + (u & 0x44444444u) * 2u) : (u << 1);
             uint32_t r[4];
-            dequant_word4<true>(w, is_int, is_int ? -1032.0f : -0.0f, pack2(d, d), r);
+            decode3x8(chunk[h], is_int, d, r);
             o[4 * h] = r[0]; o[4 * h + 1] = r[1]; o[4 * h + 2] = r[2]; o[4 * h + 3] = r[3];
         }
         store32B<ALIGNED32>(out + 2 * (size_t)g, o);
@@ -561,17 +666,7 @@ __global__ void __launch_bounds__(256) dequantize4_bs8_kernel(const uint2* __res
 
 // ----------------------------------------------------------------------------- 6-bit dequantize
 
-// Four 6-bit fields of a 24-bit chunk (field j at bit 6j) spread to one field per byte: the inverse of
-// squeeze6x4, again one mask and one multiply-add per step.
-__device__ __forceinline__ uint32_t spread6to8(uint32_t c) {
-    const uint32_t t = c + (c >> 12) * 0xF000u;
-    return t + (t & 0x0FC00FC0u) * 3u;
-}
-
-// IF6 dequantize: one thread per group of 16 (three words of codes in, 32 bytes of bf16 out).  Branch-free
-// like the 4-bit kernel: the FP decode is the hardware convert to f16 pairs, the integer decode places the
-// field k + 32 (field xor 32) in the mantissa of the f16 constant 1024, so the half is 1056 + k; one shared
-// tail adds -0 or -1056 in FP32, multiplies by the group scale and rounds to bf16 pairs.
+// IF6 dequantize (decode6x16): one thread per group of 16 (three words of codes in, 32 bytes of bf16 out).
 template <ElemKind EK, bool ALIGNED32>
 __global__ void __launch_bounds__(256) dequantize6_fast_kernel(const uint32_t* __restrict__ codes,
                                                                const uint8_t* __restrict__ scales,
@@ -591,34 +686,8 @@ __global__ void __launch_bounds__(256) dequantize6_fast_kernel(const uint32_t* _
         if (mag == 0x7Fu) Delta = __uint_as_float(0x7FC00000u);            // E4M3 NaN propagates
         float d = __fmul_rn(Delta, alpha);
         if (is_int) d = __fmul_rn(d, c_post);                              // de-scale integer groups (Sec. 3)
-        const float addend = is_int ? -1056.0f : -0.0f;
-        const uint64_t D2 = pack2(d, d);
-        const uint32_t chunk[4] = {w0 & 0xFFFFFFu, (w0 >> 24) | ((w1 & 0xFFFFu) << 8), (w1 >> 16) | ((w2 & 0xFFu) << 16), w2 >> 8};
         uint32_t o[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t bytes = spread6to8(chunk[q]);                   // codes 4q .. 4q+3, one per byte
-            uint32_t h0, h1;
-            if constexpr (EK == EK_E2M3) {
-                asm("{ .reg .b16 lo, hi;\n"
-                    "  mov.b32 {lo, hi}, %2;\n"
-                    "  cvt.rn.f16x2.e2m3x2 %0, lo;\n"
-                    "  cvt.rn.f16x2.e2m3x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
-            } else {
-                asm("{ .reg .b16 lo, hi;\n"
-                    "  mov.b32 {lo, hi}, %2;\n"
-                    "  cvt.rn.f16x2.e3m2x2 %0, lo;\n"
-                    "  cvt.rn.f16x2.e3m2x2 %1, hi; }" : "=&r"(h0), "=&r"(h1) : "r"(bytes));
-            }
-            const uint32_t r0 = __byte_perm(bytes, 0u, 0x4140) ^ 0x64206420u;   // halves 1056 + k of codes 4q, 4q+1
-            const uint32_t r1 = __byte_perm(bytes, 0u, 0x4342) ^ 0x64206420u;   // ... of codes 4q+2, 4q+3
-            const uint32_t s0 = is_int ? r0 : h0, s1 = is_int ? r1 : h1;
-            float p0, p1, p2, p3;
-            unpack2(mul2(pack2(half_plus_f32(s0, false, addend), half_plus_f32(s0, true, addend)), D2), p0, p1);
-            unpack2(mul2(pack2(half_plus_f32(s1, false, addend), half_plus_f32(s1, true, addend)), D2), p2, p3);
-            o[2 * q] = bf16x2_rn(p0, p1);
-            o[2 * q + 1] = bf16x2_rn(p2, p3);
-        }
+        decode6x16<EK>(w0, w1, w2, is_int, d, o);
         store32B<ALIGNED32>(out + 2 * (size_t)g, o);
     }
 }

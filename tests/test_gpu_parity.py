@@ -552,12 +552,15 @@ def test_fused_quantize_dequantize_is_quantize_then_dequantize(B, oracle, fmt):
             assert_same("column emulation scales", scales.cpu().numpy()[:osc.size].reshape(osc.shape), osc)
             assert bool((codes[oc.size:] == 0xA5).all()) and bool((scales[osc.size:] == 0xA5).all())
     # argument checks: other formats, unknown flags, one of the two optional outputs alone
+    import ctypes
     L = B.lib()
     x = to_dev(I.generate("cfg1", 16, 64))
     out = torch.empty_like(x)
     ts = torch.zeros(1, dtype=torch.float32, device="cuda")
     buf = torch.empty(1024, dtype=torch.uint8, device="cuda")
-    assert L.abs_quantize_dequantize(3, x.data_ptr(), 16, 64, out.data_ptr(), None, None, ts.data_ptr(), None, None) == 4
+    hopt = B.make_opts(B.ABS_F_HADAMARD16)
+    assert L.abs_quantize_dequantize(3, x.data_ptr(), 16, 64, out.data_ptr(), None, None, ts.data_ptr(),
+                                     ctypes.byref(hopt), None) == 5         # options exist for the 4-bit formats only
     import ctypes
     bad = B.make_opts(B.ABS_F_SCALES_SWIZZLED)
     assert L.abs_quantize_dequantize(fmt, x.data_ptr(), 16, 64, out.data_ptr(), None, None, ts.data_ptr(),
@@ -570,6 +573,34 @@ def test_fused_quantize_dequantize_is_quantize_then_dequantize(B, oracle, fmt):
     assert L.abs_quantize_ex(fmt, x.data_ptr(), 16, 64, buf.data_ptr(), buf.data_ptr(), ts.data_ptr(),
                              ctypes.byref(col), None) == 5                  # the flag belongs to the emulation call only
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("fmt", [2, 3, 4, 5, 6, 7])
+def test_fused_quantize_dequantize_other_formats(B, oracle, fmt):
+    """The emulation pass of IF3, IF6 and the block-size-8 formats (round-to-nearest, optional 17/16 factor and
+    given alpha) against the oracle's quantize followed by its dequantize."""
+    S17, G = B.ABS_F_SR_SCALE_17_16, B.ABS_F_ALPHA_GIVEN
+    for flags in (0, S17, G):
+        for name, rows, cols in (("cfg5", 300, 1024), ("cfg2", 64, 2064), ("cfg1", 1, 16)):
+            xb = I.generate(name, rows, cols)
+            alpha = 0.004 if flags & G else None
+            ts = torch.tensor([alpha], dtype=torch.float32, device="cuda") if alpha is not None else None
+            oc, osc, oa = oracle.quantize(fmt, xb, flags=flags, alpha=alpha)
+            od = oracle.dequantize(fmt, oc, osc, oa, rows, cols)
+            codes = torch.full((oc.size + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            scales = torch.full((osc.size + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            out, a = B.abs_quantize_dequantize(fmt, to_dev(xb), codes=codes, scales=scales, tensor_scale=ts,
+                                               opts=B.make_opts(flags))
+            out2, a2 = B.abs_quantize_dequantize(fmt, to_dev(xb), tensor_scale=ts.clone() if ts is not None else None,
+                                                 opts=B.make_opts(flags))
+            torch.cuda.synchronize()
+            assert np.float32(a.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+            assert np.float32(a2.item()).view(np.uint32) == np.float32(oa).view(np.uint32)
+            assert_same("fused out", out.view(torch.int16).cpu().numpy().view(np.uint16), od)
+            assert_same("fused out, no codes", out2.view(torch.int16).cpu().numpy().view(np.uint16), od)
+            assert_same("fused codes", codes.cpu().numpy()[:oc.size].reshape(oc.shape), oc)
+            assert_same("fused scales", scales.cpu().numpy()[:osc.size].reshape(osc.shape), osc)
+            assert bool((codes[oc.size:] == 0xA5).all()) and bool((scales[osc.size:] == 0xA5).all())
 
 
 @pytest.mark.parametrize("fmt", [0, 1])
