@@ -604,6 +604,44 @@ def test_fused_quantize_dequantize_other_formats(B, oracle, fmt):
 
 
 @pytest.mark.parametrize("fmt", [0, 1])
+def test_linear_layer_recipe(B, oracle, fmt):
+    """Sec. 4.1: forward, dgrad and wgrad of an emulated quantized linear layer.  The operands the layer feeds to
+    its GEMMs are rebuilt with the oracle (which dimension, which options, which seeds), the products in float64;
+    the bf16 GEMM results must agree to bf16 accuracy, and the Hadamard transform must cancel in wgrad."""
+    from paper_2603_28765_b200 import linear
+    T, din, dout = 256, 192, 160
+    rng = np.random.default_rng(3)
+    xb = I.f32_to_bf16_bits(rng.standard_normal((T, din)).astype(np.float32))
+    wb = I.f32_to_bf16_bits((rng.standard_normal((dout, din)) * 0.05).astype(np.float32))
+    gb = I.f32_to_bf16_bits((rng.standard_normal((T, dout)) * 1e-3).astype(np.float32))
+    x, w, dy = to_dev(xb), to_dev(wb), to_dev(gb)
+    mask, seed = 0x5A3C, 11
+    H, S, S17 = oracle.F_HADAMARD16, oracle.F_STOCHASTIC, oracle.F_SR_SCALE_17_16
+
+    def oq(bits, flags=0, columns=False, sr_seed=0):
+        src = np.ascontiguousarray(bits.T) if columns else bits
+        c, s, a = oracle.quantize(fmt, src, flags=flags, sign_mask=mask, sr_seed=sr_seed)
+        d = I.bf16_bits_to_f32(oracle.dequantize(fmt, c, s, a, *src.shape)).astype(np.float64)
+        return d.T if columns else d
+
+    def close(got, want):
+        got = got.float().cpu().numpy().astype(np.float64)
+        scale = np.abs(want).max()
+        assert np.abs(got - want).max() <= 2.0 ** -7 * scale, np.abs(got - want).max() / scale
+
+    y = linear.forward(x, w, fmt)
+    close(y, oq(xb) @ oq(wb).T)
+    dx, dw = linear.backward(x, w, dy, fmt, sign_mask=mask, seed=seed)
+    close(dx, oq(gb, S | S17, sr_seed=seed) @ oq(wb, columns=True))
+    gq, xq = oq(gb, H | S | S17, columns=True, sr_seed=seed + 1), oq(xb, H, columns=True)
+    close(dw, gq.T @ xq)
+    # the transform cancels: the emulated wgrad approximates dY^T X of the untransformed tensors
+    exact = I.bf16_bits_to_f32(gb).astype(np.float64).T @ I.bf16_bits_to_f32(xb).astype(np.float64)
+    rel = np.linalg.norm(dw.float().cpu().numpy() - exact) / np.linalg.norm(exact)
+    assert rel < 0.25, rel
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
 def test_swizzled_scale_layout(B, oracle, fmt):
     """ABS_F_SCALES_SWIZZLED: same codes and alpha, scale bytes permuted into the 128x4-tile layout (the
     oracle builds that layout by reshapes from the row-major scales); padding bytes stay untouched; the
