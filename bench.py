@@ -322,6 +322,22 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": quant_kernel_bytes(n),
                 "traffic": (NCU_QUANT_TRAFFIC_BYTES_PER_ELEM * n) if NCU_QUANT_TRAFFIC_BYTES_PER_ELEM else None}
 
+    # ---- for information: the same result through the one-pass emulation call (amax pass + one kernel that
+    # quantizes and decodes from registers, writing codes, scales and the bf16 output); not part of `value`.
+    eargs = [(FMT_IF4, xs[k].data_ptr(), rows, cols, outs[k].data_ptr(), codes[k].data_ptr(), scales[k].data_ptr(),
+              alphas[k].data_ptr(), None, sp) for k in range(n_sets)]
+    for i in range(3):
+        L.abs_quantize_dequantize(*eargs[i % n_sets])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(n_q):
+        L.abs_quantize_dequantize(*eargs[i % n_sets])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    one_pass = {"us_per_call": round(e0.elapsed_time(e1) / n_q * 1e3, 2), "calls_timed": n_q,
+                "api": "abs_quantize_dequantize with code outputs (same outputs as one step, 2 kernels instead of 3)"}
+
     # ---- end to end through the host-buffer C-ABI calls (pinned host memory, copies in the timed region)
     e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
     ws = torch.empty(B.abs_host_workspace_bytes(FMT_IF4, rows, cols), dtype=torch.uint8, device=dev)
@@ -361,7 +377,7 @@ def run_cuda(args):
                        "bytes_per_step": step_bytes(n), "elements_per_s": round(world * n / (ms_per_step * 1e-3), 0),
                        "l2": f"cold: steps rotate over {n_sets} buffer sets ({n_sets * set_bytes >> 20} MiB > 4x L2)",
                        "sharding": "one independent tensor per rank, no collective"},
-            "roofline": roofline, "e2e": e2e, "gpu_launches": 3 * args.steps,
+            "roofline": roofline, "e2e": e2e, "one_pass": one_pass, "gpu_launches": 3 * args.steps,
             "clocks": sampler.summary(clock_note),
         }
         if world == 1 and not args.no_cpu_baseline:
