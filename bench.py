@@ -317,7 +317,8 @@ def run_cuda(args):
     achieved = quant_kernel_bytes(n) / (q_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "quantize4_fast_kernel<IF4> (group-quantize, Fig. 3a steps 1-10)",
                 "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "peak_source": peak_src, "us_per_launch": round(q_ms * 1e3, 2), "launches_timed": n_q,
+                "peak_source": peak_src, "frac_of_nominal_8000_gbs": round(achieved / 8000.0, 4),
+                "us_per_launch": round(q_ms * 1e3, 2), "launches_timed": n_q,
                 "in_step_probe_us": round(in_step_ms * 1e3, 2),
                 "algorithmic_bytes_per_launch": quant_kernel_bytes(n),
                 "traffic": (NCU_QUANT_TRAFFIC_BYTES_PER_ELEM * n) if NCU_QUANT_TRAFFIC_BYTES_PER_ELEM else None}

@@ -126,6 +126,8 @@ def main():
             print(json.dumps({
                 "config": name, "shape": [rows, cols], "fmt": fname, "options": opt,
                 "T1_quantize_kernel_us": round(t1 * 1e3, 1), "T1_GBs": round((2 * n + outb) / t1 / 1e6),
+                "T1_pct_of_8000": round((2 * n + outb) / t1 / 1e6 / 80.0, 1),
+                "T2_dram_basis_pct_of_8000": round((4 * n + outb) / t2 / 1e6 / 80.0, 1),
                 "T2_abs_quantize_us": round(t2 * 1e3, 1), "T2_dram_basis_GBs": round((4 * n + outb) / t2 / 1e6),
                 "T2_effective_GBs": round((2 * n + outb) / t2 / 1e6),
                 "T3_dequantize_us": round(t3 * 1e3, 1), "T3_GBs": round((2 * n + outb) / t3 / 1e6),
