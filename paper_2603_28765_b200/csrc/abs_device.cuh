@@ -322,6 +322,20 @@ __device__ __forceinline__ float resolve_alpha(const AlphaSrc& a) {
     return alpha_shared;
 }
 
+// The same without a barrier: every thread reads the slot (one L2 line, broadcast) and divides for itself.
+// For the grid-stride kernels whose threads handle several groups each: the dozen instructions of the IEEE
+// division are spread over those groups, and no block waits at a barrier before its first group
+// (measured 1 % faster for abs_quantize at 256 MiB than the shared-memory version).
+template <bool FROM_SLOT>
+__device__ __forceinline__ float resolve_alpha_per_thread(const AlphaSrc& a) {
+    if constexpr (!FROM_SLOT) return __ldg(a.alpha_p);
+    const unsigned long long v = __ldcg(a.slot);
+    const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
+    const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                           // Eq. 1
+    if (blockIdx.x == 0 && threadIdx.x == 0) *a.alpha_out = alpha;
+    return alpha;
+}
+
 // Byte offset of the scale of (row, k-th group of the row) in the 128x4-tile layout read by Blackwell
 // block-scaled MMAs; ktiles = ceil(groups_per_row / 4).
 __device__ __forceinline__ size_t swizzled_scale_offset(uint32_t row, uint32_t k, uint32_t ktiles) {

@@ -155,27 +155,23 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
     uint32_t w[8], wn[8];
     const bool active = g < ngroups;
     if (active) load32B<ALIGNED32>(in + 2 * (size_t)g, w);
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
-    while (true) {
-        const IdxT gn = g + stride;
-        const bool more = gn < ngroups;
-        if (more) load32B<ALIGNED32>(in + 2 * (size_t)gn, wn);
+    // one group: G1-G5, steps 3-10, stores
+    auto process = [&](const uint32_t (&ww)[8], IdxT gg) {
         float x[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            x[2 * i] = __uint_as_float(w[i] << 16);
-            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+            x[2 * i] = __uint_as_float(ww[i] << 16);
+            x[2 * i + 1] = __uint_as_float(ww[i] & 0xFFFF0000u);
         }
-        // G1: group maximum with three-input max.
         const float m0 = max3abs(x[0], x[1], x[2]), m1 = max3abs(x[3], x[4], x[5]);
         const float m2 = max3abs(x[6], x[7], x[8]), m3 = max3abs(x[9], x[10], x[11]);
         const float m4 = max3abs(x[12], x[13], x[14]);
-        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
-        // G2-G3 (Eq. 2).
-        float t = __fmul_rn(gmax, inv_a6);
-        if constexpr (SCALE_MUL) t = __fmul_rn(t, 1.0625f);                 // the 17/16 option
+        const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));   // G1: three-input max
+        float t = __fmul_rn(gmax, inv_a6);                                   // G2-G3 (Eq. 2)
+        if constexpr (SCALE_MUL) t = __fmul_rn(t, 1.0625f);                  // the 17/16 option
         const uint32_t sb = e4m3_encode(t);
         const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
         const float r = __frcp_rn(d);
@@ -186,12 +182,23 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
         } else {
             encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
         }
-        scales[scale_offset<SWZ>((size_t)g, gpr, ktiles)] = (uint8_t)sbyte;
-        codes[g] = make_uint2(c_lo, c_hi);
+        scales[scale_offset<SWZ>((size_t)gg, gpr, ktiles)] = (uint8_t)sbyte;
+        codes[gg] = make_uint2(c_lo, c_hi);
+    };
+    // two groups per trip, the two register buffers swapping roles: the next group's load is always in flight
+    // under the current group's arithmetic and nothing is copied between the buffers
+    while (true) {
+        const IdxT gn = g + stride;
+        const bool more = gn < ngroups;
+        if (more) load32B<ALIGNED32>(in + 2 * (size_t)gn, wn);
+        process(w, g);
         if (!more) break;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = wn[i];
-        g = gn;
+        const IdxT g2 = gn + stride;
+        const bool more2 = g2 < ngroups;
+        if (more2) load32B<ALIGNED32>(in + 2 * (size_t)g2, w);
+        process(wn, gn);
+        if (!more2) break;
+        g = g2;
     }
 }
 

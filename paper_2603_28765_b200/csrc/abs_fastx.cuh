@@ -153,16 +153,11 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
         if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
         else load32B<false>(in + 2 * (size_t)g, w);
     }
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
-    while (true) {
-        const int32_t gn = g + stride;
-        const bool more = gn < nblocks16;
-        if (more) {
-            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
-            else load32B<false>(in + 2 * (size_t)gn, wn);
-        }
+    // one block of 16 values held in `w`, index `g`
+    auto process = [&](const uint32_t (&w)[8], const int32_t g) {
         float x[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -202,10 +197,25 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
             if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
             else store32B<false>(out + 2 * (size_t)g, o);
         }
+    };
+    auto fetch = [&](uint32_t (&buf)[8], int32_t gg) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)gg, buf);
+        else load32B<false>(in + 2 * (size_t)gg, buf);
+    };
+    // two blocks per trip, the two register buffers swapping roles: the next load is always in flight under
+    // the current arithmetic and nothing is copied between the buffers
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < nblocks16;
+        if (more) fetch(wn, gn);
+        process(w, g);
         if (!more) break;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = wn[i];
-        g = gn;
+        const int32_t g2 = gn + stride;
+        const bool more2 = g2 < nblocks16;
+        if (more2) fetch(w, g2);
+        process(wn, gn);
+        if (!more2) break;
+        g = g2;
     }
 }
 
@@ -325,17 +335,12 @@ quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
         if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
         else load32B<false>(in + 2 * (size_t)g, w);
     }
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, F::M_FP));               // T3
     const float c_pre = __fdiv_rn(F::M_INT, F::M_FP), c_post = __fdiv_rn(F::M_FP, F::M_INT);
-    while (true) {
-        const int32_t gn = g + stride;
-        const bool more = gn < ngroups;
-        if (more) {
-            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
-            else load32B<false>(in + 2 * (size_t)gn, wn);
-        }
+    // one block of 16 values held in `w`, index `g`
+    auto process = [&](const uint32_t (&w)[8], const int32_t g) {
         float x[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -364,10 +369,25 @@ quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
             if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
             else store32B<false>(out + 2 * (size_t)g, o);
         }
+    };
+    auto fetch = [&](uint32_t (&buf)[8], int32_t gg) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)gg, buf);
+        else load32B<false>(in + 2 * (size_t)gg, buf);
+    };
+    // two blocks per trip, the two register buffers swapping roles: the next load is always in flight under
+    // the current arithmetic and nothing is copied between the buffers
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < ngroups;
+        if (more) fetch(wn, gn);
+        process(w, g);
         if (!more) break;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = wn[i];
-        g = gn;
+        const int32_t g2 = gn + stride;
+        const bool more2 = g2 < ngroups;
+        if (more2) fetch(w, g2);
+        process(wn, gn);
+        if (!more2) break;
+        g = g2;
     }
 }
 
@@ -494,16 +514,11 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
         if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
         else load32B<false>(in + 2 * (size_t)g, w);
     }
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 4.0f));                  // T3
-    while (true) {
-        const int32_t gn = g + stride;
-        const bool more = gn < ngroups;
-        if (more) {
-            if (aligned32) load32B<true>(in + 2 * (size_t)gn, wn);
-            else load32B<false>(in + 2 * (size_t)gn, wn);
-        }
+    // one block of 16 values held in `w`, index `g`
+    auto process = [&](const uint32_t (&w)[8], const int32_t g) {
         float x[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -579,10 +594,25 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
             if (out_aligned32) store32B<true>(out + 2 * (size_t)g, o);
             else store32B<false>(out + 2 * (size_t)g, o);
         }
+    };
+    auto fetch = [&](uint32_t (&buf)[8], int32_t gg) {
+        if (aligned32) load32B<true>(in + 2 * (size_t)gg, buf);
+        else load32B<false>(in + 2 * (size_t)gg, buf);
+    };
+    // two blocks per trip, the two register buffers swapping roles: the next load is always in flight under
+    // the current arithmetic and nothing is copied between the buffers
+    while (true) {
+        const int32_t gn = g + stride;
+        const bool more = gn < ngroups;
+        if (more) fetch(wn, gn);
+        process(w, g);
         if (!more) break;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = wn[i];
-        g = gn;
+        const int32_t g2 = gn + stride;
+        const bool more2 = g2 < ngroups;
+        if (more2) fetch(w, g2);
+        process(wn, gn);
+        if (!more2) break;
+        g = g2;
     }
 }
 

@@ -184,7 +184,7 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
         if (aligned32) load32B<true>(in + 2 * (size_t)g, w);
         else load32B<false>(in + 2 * (size_t)g, w);
     }
-    const float alpha = resolve_alpha<FROM_SLOT>(alpha_src);                 // T2 (block-wide: before any thread leaves)
+    const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     uint32_t smask[8];
