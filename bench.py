@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the group-quantize kernel per element, from the ncu capture summarised in
 # profiles/quantize4_fast_if4_cfg2.md: (dram__bytes_read.sum + dram__bytes_write.sum) per launch / N
-# = (67.12 MB + 3.08 MB) / 33 554 432 elements, captured on this same workload.
-NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = 70.20e6 / 33554432
+# = (67.13 MB + 3.30 MB) / 33 554 432 elements, captured on this same workload.
+NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = 70.43e6 / 33554432
 
 
 def step_bytes(n_elems: int) -> float:

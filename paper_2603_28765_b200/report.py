@@ -10,7 +10,7 @@ that rotate over enough buffer sets to defeat L2 reuse between calls:
   T1  the group-quantize kernel alone (alpha given)          bytes = 2N + codes + scales
   T2  abs_quantize end to end (amax pass + group-quantize)   bytes = 4N + codes + scales (DRAM basis)
   T3  abs_dequantize                                         bytes = codes + scales + 2N
-  T4  abs_quantize_dequantize (4-bit formats; amax pass + one-pass emulation, no code outputs)
+  T4  abs_quantize_dequantize (amax pass + one-pass emulation, no code outputs)
 and prints one JSON line per row.  With ``--transposed`` it times abs_quantize_transposed instead (the kernel
 alone, alpha given; the same bytes move), for IF4 and NVFP4 with and without the gradient options.  Inputs are random bf16 tensors of the configuration's shape
 (timing does not depend on the values beyond the INT/FP mix); parity is the test suite's job.
@@ -117,7 +117,7 @@ def main():
             t2 = loop_time(lambda i: L.abs_quantize_ex(*fa[i % k]))
             t3 = loop_time(lambda i: L.abs_dequantize(*da[i % k]))
             t4 = None
-            if fmt in (B.ABS_FMT_NVFP4, B.ABS_FMT_IF4):
+            if fmt in (B.ABS_FMT_NVFP4, B.ABS_FMT_IF4) or not (flags & (H | S)):
                 ea = [(fmt, xs[i].data_ptr(), rows, cols, outs[i % len(outs)].data_ptr(), None, None, ts[i].data_ptr(),
                        C.byref(o_full), sp) for i in range(k)]
                 t4 = loop_time(lambda i: L.abs_quantize_dequantize(*ea[i % k]))
