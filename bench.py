@@ -339,6 +339,35 @@ def run_cuda(args):
     one_pass = {"us_per_call": round(e0.elapsed_time(e1) / n_q * 1e3, 2), "calls_timed": n_q,
                 "api": "abs_quantize_dequantize with code outputs (same outputs as one step, 2 kernels instead of 3)"}
 
+    # ---- for information: the same steps issued alternately on two streams, so the bandwidth-bound amax /
+    # dequantize kernels of one tensor overlap the issue-bound group-quantize kernel of another (independent
+    # tensors, as in a layer with several operands to quantize); not part of `value`.
+    s2 = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    sp2 = [C.c_void_p(s.cuda_stream) for s in s2]
+
+    def step2(i):
+        k, p = i % n_sets, sp2[i & 1]
+        L.abs_quantize(*qargs[k][:-1], p)
+        L.abs_dequantize(*dargs[k][:-1], p)
+
+    n_t = max(8, min(args.steps, 400)) & ~1
+    for i in range(4):
+        step2(i)
+    torch.cuda.synchronize()
+    t0e, t1e, j = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), torch.cuda.Event())
+    t0e.record(s2[0])
+    s2[1].wait_event(t0e)
+    for i in range(n_t):
+        step2(i)
+    j.record(s2[1])
+    s2[0].wait_event(j)
+    t1e.record(s2[0])
+    torch.cuda.synchronize()
+    t_us = t0e.elapsed_time(t1e) / n_t * 1e3
+    two_streams = {"us_per_step": round(t_us, 2), "value": round(step_bytes(n) / (t_us * 1e-6) / 1e9, 1),
+                   "unit": UNIT, "steps_timed": n_t,
+                   "note": "steps alternate over two streams; per-rank figure, informational"}
+
     # ---- end to end through the host-buffer C-ABI calls (pinned host memory, copies in the timed region)
     e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
     ws = torch.empty(B.abs_host_workspace_bytes(FMT_IF4, rows, cols), dtype=torch.uint8, device=dev)
@@ -378,7 +407,8 @@ def run_cuda(args):
                        "bytes_per_step": step_bytes(n), "elements_per_s": round(world * n / (ms_per_step * 1e-3), 0),
                        "l2": f"cold: steps rotate over {n_sets} buffer sets ({n_sets * set_bytes >> 20} MiB > 4x L2)",
                        "sharding": "one independent tensor per rank, no collective"},
-            "roofline": roofline, "e2e": e2e, "one_pass": one_pass, "gpu_launches": 3 * args.steps,
+            "roofline": roofline, "e2e": e2e, "one_pass": one_pass, "two_streams": two_streams,
+            "gpu_launches": 3 * args.steps,
             "clocks": sampler.summary(clock_note),
         }
         if world == 1 and not args.no_cpu_baseline:
