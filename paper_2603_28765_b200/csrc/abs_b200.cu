@@ -3,8 +3,10 @@
 //
 // Path (paper Sec. 3): amax_kernel (Eq. 1, grid-wide max) -> group-quantize kernel (Eq. 2 and Fig. 3a
 // steps 1-10 per 16-value group, flag in the scale's sign bit, packed codes); the dequantize kernels are
-// the inverse (Sec. 3, Sec. 4.1).  Kernels: abs_generic.cuh (amax, every format and option),
-// abs_fast4.cuh (the 4-bit round-to-nearest fast paths, transposed quantize), abs_device.cuh (building blocks).
+// the inverse (Sec. 3, Sec. 4.1).  Kernels: abs_generic.cuh (amax; every format and option, element by
+// element), abs_fast4.cuh (4-bit round-to-nearest quantize and dequantize), abs_opt4.cuh (4-bit with the
+// Hadamard / stochastic-rounding options, one-pass emulation), abs_fastx.cuh (IF3, IF6, block size 8),
+// abs_trans4.cuh (groups down the columns), abs_device.cuh (building blocks).
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
 #include "abs_fast4.cuh"
@@ -962,11 +964,15 @@ abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const
     if (rows >= 16 * kHostChunks && !(opts && (opts->flags & ABS_F_SCALES_SWIZZLED)) && device_state(&st) == ABS_OK) {
         std::lock_guard<std::mutex> lock(st->host_mu);
         if (!st->d2h_stream) {
-            bool ok = cudaStreamCreateWithFlags(&st->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+            // created once per device; the stream pointer is published last, so a failed attempt is retried
+            cudaStream_t ns = nullptr;
+            bool ok = true;
             for (int i = 0; ok && i < kHostChunks; ++i)
-                ok = cudaEventCreateWithFlags(&st->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
-            ok = ok && cudaEventCreateWithFlags(&st->d2h_done, cudaEventDisableTiming) == cudaSuccess;
+                if (!st->chunk_done[i]) ok = cudaEventCreateWithFlags(&st->chunk_done[i], cudaEventDisableTiming) == cudaSuccess;
+            if (ok && !st->d2h_done) ok = cudaEventCreateWithFlags(&st->d2h_done, cudaEventDisableTiming) == cudaSuccess;
+            ok = ok && cudaStreamCreateWithFlags(&ns, cudaStreamNonBlocking) == cudaSuccess;
             if (!ok) return ABS_ERR_CUDA;
+            st->d2h_stream = ns;
         }
         if (cudaMemcpyAsync(d_alpha, tensor_scale_f32_host, 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return ABS_ERR_CUDA;
         const size_t out_row = (size_t)cols * (fp32 ? 4 : 2);
