@@ -411,7 +411,7 @@ __device__ __forceinline__ uint32_t sign_bits3x8(uint32_t w0, uint32_t w1, uint3
 // Candidates of EIGHT values of IF3 (E2M0 magnitudes {0, 1, 2, 4} or INT3), steps 3-9 of Fig. 3a: the
 // 24-bit chunks of FP and integer codes and the two error chains (even / odd elements) of each candidate.
 // E2M0 has no hardware convert.  Round-to-nearest-even onto {0, 1, 2, 4} of a = min(|y|, 4) is the sum of
-// two exact integer roundings, RNE(min(a, 2)) + 2 * RNE(max(a - 2, 0) / 2): the first covers 0..2 (ties
+// two exact integer roundings, RNE(min(a, 2)) + 2 * RNE((max(a, 2) - 2) / 2): the first covers 0..2 (ties
 // 0.5 -> 0, 1.5 -> 2), the second the step from 2 to 4 (tie 3 -> 2); the code index is the sum of the two
 // rounded integers.  FP errors are taken on magnitudes (|x| and |v| carry the same sign, so the squares
 // agree).  CLAMP as in the 4-bit kernel: only subnormal or saturated scale bytes let |y * 3/4| pass 3.5.
@@ -422,10 +422,13 @@ __device__ __forceinline__ void candidates3x8(const float* x, const uint32_t* w,
     const float c_pre = 0.75f, c_post = __fdiv_rn(4.0f, 3.0f);
     const float d_int = __fmul_rn(d, c_post);
     const uint64_t R2 = pack2(r, r), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
-    const uint64_t MG = pack2(kMagic0, kMagic0), NMG = pack2(-kMagic0, -kMagic0);
+    const uint64_t MG = pack2(kMagic0, kMagic0);
     const uint64_t MG4 = pack2(kMagic4, kMagic4), NMG4 = pack2(-kMagic4, -kMagic4);
-    const uint64_t NTWO = pack2(-2.0f, -2.0f), HALF = pack2(0.5f, 0.5f), TWO = pack2(2.0f, 2.0f);
-    uint64_t accI = 0;
+    // 1.5 * 2^24 has ulp 2: adding it rounds to even integers, i.e. 2 * RNE(. / 2), with the rounded integer in the
+    // low mantissa bits.  kStep - 2 folds the "- 2" of max(a, 2) - 2 into the same add; kBoth removes both magics.
+    constexpr float kStep = 25165824.0f;                                     // 1.5 * 2^24
+    const uint64_t STEP = pack2(kStep - 2.0f, kStep - 2.0f), NBOTH = pack2(-(kStep + kMagic0), -(kStep + kMagic0));
+    uint64_t accI = 0, accF = 0;
     uint32_t ib[8], kb[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -433,23 +436,25 @@ __device__ __forceinline__ void candidates3x8(const float* x, const uint32_t* w,
         const uint64_t Y = mul2(X, R2);                                      // E1 (step 3)
         float y0, y1;
         unpack2(Y, y0, y1);
-        // E2 (step 4): E2M0 index and value of the magnitude
-        const float a0 = fminf(fabsf(y0), 4.0f), a1 = fminf(fabsf(y1), 4.0f);
-        float u0, u1;
-        unpack2(add2(pack2(a0, a1), NTWO), u0, u1);                          // a - 2: exact for a in [2, 4], unused below 2
+        // E2 (step 4): E2M0 index and value of the magnitude.  Without CLAMP |y| <= 4 * 17/16, which rounds like 4
+        // (max(a, 2) / 2 - 1 <= 1.13), so the saturation at 4 is only needed for the rare scale bytes.
+        float a0 = fabsf(y0), a1 = fabsf(y1);
+        if constexpr (CLAMP) {
+            a0 = fminf(a0, 4.0f);
+            a1 = fminf(a1, 4.0f);
+        }
         const uint64_t M1 = add2(pack2(fminf(a0, 2.0f), fminf(a1, 2.0f)), MG);                // RNE(min(a, 2)) + magic
-        const uint64_t M2 = fma2(pack2(fmaxf(u0, 0.0f), fmaxf(u1, 0.0f)), HALF, MG);          // RNE(max(a - 2, 0) / 2) + magic
+        const uint64_t M2 = add2(pack2(fmaxf(a0, 2.0f), fmaxf(a1, 2.0f)), STEP);              // 2 * RNE((max(a, 2) - 2) / 2) + kStep
         float m10, m11, m20, m21;
         unpack2(M1, m10, m11);
         unpack2(M2, m20, m21);
-        ib[2 * i] = __float_as_uint(m10) + __float_as_uint(m20);             // 2 * kMagic0Bits + index
+        ib[2 * i] = __float_as_uint(m10) + __float_as_uint(m20);             // kMagic0Bits + kStepBits + index
         ib[2 * i + 1] = __float_as_uint(m11) + __float_as_uint(m21);
         float v0, v1;
-        unpack2(fma2(add2(M2, NMG), TWO, add2(M1, NMG)), v0, v1);            // the E2M0 magnitude: r1 + 2 * r2
+        unpack2(add2(add2(M2, NBOTH), M1), v0, v1);                          // the E2M0 magnitude r1 + 2 * r2 (both adds exact)
         // E3 (steps 5-6) on magnitudes
-        const float e0 = __fmaf_rn(v0, -d, fabsf(x[2 * i])), e1 = __fmaf_rn(v1, -d, fabsf(x[2 * i + 1]));
-        f0 = (i == 0) ? __fmul_rn(e0, e0) : __fmaf_rn(e0, e0, f0);
-        f1 = (i == 0) ? __fmul_rn(e1, e1) : __fmaf_rn(e1, e1, f1);
+        const uint64_t E = pack2(__fmaf_rn(v0, -d, fabsf(x[2 * i])), __fmaf_rn(v1, -d, fabsf(x[2 * i + 1])));
+        accF = (i == 0) ? mul2(E, E) : fma2(E, E, accF);
         // E4-E5 (steps 7-9): integer candidate, signed
         uint64_t KZ = fma2(Y, CP2, MG4);
         if constexpr (CLAMP) {
@@ -467,9 +472,10 @@ __device__ __forceinline__ void candidates3x8(const float* x, const uint32_t* w,
         kb[2 * i + 1] = __float_as_uint(kz1);
     }
     unpack2(accI, i0, i1);
+    unpack2(accF, f0, f1);
     // eight 3-bit fields by Horner on the raw sums; the constant parts are removed afterwards
     constexpr uint32_t kS8 = 0x249249u;                                      // 1 + 8 + ... + 8^7
-    constexpr uint32_t kConstF = 2u * kMagic0Bits * kS8;                     // leaves the indices 0..3
+    constexpr uint32_t kConstF = (kMagic0Bits + 0x4BC00000u) * kS8;          // bits of 1.5 * 2^23 and 1.5 * 2^24: leaves the indices 0..3
     constexpr uint32_t kConstI = (kMagic4Bits - 4u) * kS8;                   // leaves the fields k + 4
     uint32_t fc = ib[7], ic = kb[7];
 #pragma unroll
