@@ -287,7 +287,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // IF3 and its block-size-8 variant, round-to-nearest
         constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
-        const int tgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
+        const int tgrid = grid_waves(st, ngroups, ABS_IF3_MINB, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
