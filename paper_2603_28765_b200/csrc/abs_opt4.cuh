@@ -51,15 +51,16 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
     const uint64_t R2 = pack2(r, r);
     const uint64_t TWO = pack2(2.0f, 2.0f), HALF = pack2(0.5f, 0.5f), FOUR = pack2(4.0f, 4.0f);
     const uint64_t MG = pack2(kMagic, kMagic), NMG = pack2(-kMagic, -kMagic);
-    const uint64_t NSC16 = pack2(-1.0f / 65536.0f, -1.0f / 65536.0f), P128 = pack2(128.0f, 128.0f);
-    const uint64_t NH17 = pack2(-1.0f / 131072.0f, -1.0f / 131072.0f);
+    const uint64_t NSC16 = pack2(-1.0f / 65536.0f, -1.0f / 65536.0f);
+    const uint64_t P128MH = pack2(128.0f - 1.0f / 131072.0f, 128.0f - 1.0f / 131072.0f);   // 128 - 2^-17, 24 bits
 
     const float c_pre = __uint_as_float(0x3F955555u);    // fp32(7/6)
     const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
     const float d_int = __fmul_rn(d, c_post);
     const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
     const uint64_t MG8 = pack2(kMagic8, kMagic8);
-    const uint64_t NTWO = pack2(-2.0f, -2.0f), NEIGHT = pack2(-8.0f, -8.0f);
+    const uint64_t NMGH = pack2(-0.5f * kMagic, -0.5f * kMagic), NMG2 = pack2(-(kMagic + 2.0f), -(kMagic + 2.0f));
+    const uint64_t NMG8 = pack2(-(2.0f * kMagic + 8.0f), -(2.0f * kMagic + 8.0f));
 
     uint64_t accF[2], accI[2];
     uint32_t fw[2], kb[16], ib[16];
@@ -74,11 +75,12 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
             float y0, y1;
             unpack2(Y, y0, y1);
             ys[2 * i] = y0; ys[2 * i + 1] = y1;
-            // -u = -(h + 1/2) * 2^-16 from the 16-bit fields, exact: 2^23 + h as a float first
+            // -u = -(h + 1/2) * 2^-16 from the 16-bit fields: 2^23 + h as a float, then one multiply-add whose exact
+            // result -(2^23 + h) * 2^-16 + 128 - 2^-17 has 17 significant bits, so nothing is rounded
             const uint32_t rw = rnd[e >> 1];
             const float m0 = __uint_as_float((rw & 0xFFFFu) | 0x4B000000u);
             const float m1 = __uint_as_float(__byte_perm(rw, 0x4B00u, 0x5432));
-            const uint64_t NU = add2(fma2(pack2(m0, m1), NSC16, P128), NH17);
+            const uint64_t NU = fma2(pack2(m0, m1), NSC16, P128MH);
             // E2 under stochastic rounding: index = ceil(phi(a) - u)
             const float a0 = fminf(fabsf(y0), 6.0f), a1 = fminf(fabsf(y1), 6.0f);
             const uint64_t A = pack2(a0, a1);
@@ -93,11 +95,12 @@ __device__ __forceinline__ void encode_body4_sr(const float (&x)[16], const uint
             ib[e] = __float_as_uint(im0);
             ib[e + 1] = __float_as_uint(im1);
             if constexpr (HAS_INT) {
-                const uint64_t I = add2(IM, NMG);                              // the index as a float
+                // value of the index i = IM - kMagic: max(i/2, i - 2, 2i - 8), each piece formed from IM in one
+                // exact operation (kMagic / 2, kMagic + 2 and 2 * kMagic + 8 are all FP32 numbers)
                 float q00, q01, q10, q11, q20, q21;
-                unpack2(mul2(I, HALF), q00, q01);
-                unpack2(add2(I, NTWO), q10, q11);
-                unpack2(fma2(I, TWO, NEIGHT), q20, q21);
+                unpack2(fma2(IM, HALF, NMGH), q00, q01);
+                unpack2(add2(IM, NMG2), q10, q11);
+                unpack2(fma2(IM, TWO, NMG8), q20, q21);
                 const float v0 = max3f(q00, q10, q20), v1 = max3f(q01, q11, q21);          // value of the index
                 const float vs0 = __uint_as_float((__float_as_uint(v0) & 0x7FFFFFFFu) | sign_of(y0));
                 const float vs1 = __uint_as_float((__float_as_uint(v1) & 0x7FFFFFFFu) | sign_of(y1));
