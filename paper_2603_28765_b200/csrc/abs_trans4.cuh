@@ -96,16 +96,26 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
     const bool vec_ok = (rblocks % kTransTileRowBlocks) == 0 &&
                         ((reinterpret_cast<uintptr_t>(codes_t) & 31u) == 0) && ((reinterpret_cast<uintptr_t>(scales_t) & 3u) == 0);
 
-    // issue the asynchronous copies of tile t into stage s (one commit group per call, possibly empty)
+    // issue the asynchronous copies of tile t into stage s (one commit group per call, possibly empty).
+    // Tile counts fit 32 bits (a tile is 16384 elements), so the tile coordinates use 32-bit division.
     auto issue = [&](int64_t t, int s) {
         if (t < ntiles) {
-            const int64_t ty = t / ntx, tx = t - ty * ntx;
-            const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
+            const uint32_t ty = (uint32_t)t / (uint32_t)ntx, tx = (uint32_t)t - ty * (uint32_t)ntx;
+            const int64_t rb0 = (int64_t)ty * kTransTileRowBlocks, c0 = (int64_t)tx * kTransTileCols;
             const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
             const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
             uint16_t* stage = trans_smem + s * kTransStageElems;
             const uint16_t* src = in + rb0 * 16 * cols + c0;
-            if (ncols == kTransTileCols) {               // full-width tile: 32 chunks of 16 bytes per row
+            if (ncols == kTransTileCols && nrb == kTransTileRowBlocks) {
+                // complete tile: 2048 chunks of 16 bytes, chunk ch = thread + 256 j lands at stage + 8 ch and comes
+                // from row (thread / 32) + 8 j, columns 8 (thread % 32) ...
+                uint16_t* dst = stage + 8 * threadIdx.x;
+                const uint16_t* from = src + (int64_t)(threadIdx.x >> 5) * cols + 8 * (threadIdx.x & 31);
+                const int64_t step = 8 * cols;
+#pragma unroll
+                for (int j = 0; j < 16 * kTransTileRowBlocks * (kTransTileCols / 8) / 256; ++j)
+                    cp_async16(dst + j * 8 * 256, from + j * step);
+            } else if (ncols == kTransTileCols) {        // full-width tile: 32 chunks of 16 bytes per row
                 for (int ch = threadIdx.x; ch < 16 * nrb * (kTransTileCols / 8); ch += blockDim.x) {
                     const int r = ch >> 5, q = ch & 31;
                     cp_async16(stage + r * kTransTileCols + q * 8, src + (int64_t)r * cols + q * 8);
@@ -128,8 +138,8 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
         issue(t + gridDim.x, s ^ 1);                 // prefetch the block's next tile into the other stage
         cp_async_wait_all_but_one();                 // this thread's copies of tile t have landed
         __syncthreads();                             // ... and everybody else's
-        const int64_t ty = t / ntx, tx = t - ty * ntx;
-        const int64_t rb0 = ty * kTransTileRowBlocks, c0 = tx * kTransTileCols;
+        const uint32_t ty = (uint32_t)t / (uint32_t)ntx, tx = (uint32_t)t - ty * (uint32_t)ntx;
+        const int64_t rb0 = (int64_t)ty * kTransTileRowBlocks, c0 = (int64_t)tx * kTransTileCols;
         const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
         const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
         uint16_t* stage = trans_smem + s * kTransStageElems;
