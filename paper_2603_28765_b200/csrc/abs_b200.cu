@@ -728,10 +728,11 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
     const int64_t ntiles = ((cols + kTransTileCols - 1) / kTransTileCols) *
                            ((rblocks + kTransTileRowBlocks - 1) / kTransTileRowBlocks);
     if (ntiles > (int64_t)0x7FFFFFFF) return ABS_ERR_SIZE;      // the kernel indexes tiles with 32 bits
-    // 64 KiB of shared memory per block: 3 blocks per SM.  The arithmetic-bound variants (IF4, options) run
-    // best as several waves with about four tiles per block; plain NVFP4 as one wave of persistent blocks.
+    // 64 KiB of shared memory per block: 3 blocks per SM.  The arithmetic-bound variants (IF4, options) and the
+    // emulation pass run best as several waves with about four tiles per block; plain NVFP4 as one wave of
+    // persistent blocks.
     const int64_t resident = (int64_t)st->sm_count * 3;
-    const bool heavy = fmt == ABS_FMT_IF4 || (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC));
+    const bool heavy = fmt == ABS_FMT_IF4 || (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC)) || out_bf16 != nullptr;
     int64_t tgrid = ntiles < resident ? ntiles : resident;
     if (heavy && ntiles > resident) {
         int64_t waves = (ntiles + 2 * resident) / (4 * resident);
