@@ -96,11 +96,9 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
     const bool vec_ok = (rblocks % kTransTileRowBlocks) == 0 &&
                         ((reinterpret_cast<uintptr_t>(codes_t) & 31u) == 0) && ((reinterpret_cast<uintptr_t>(scales_t) & 3u) == 0);
 
-    // issue the asynchronous copies of tile t into stage s (one commit group per call, possibly empty).
-    // Tile counts fit 32 bits (a tile is 16384 elements), so the tile coordinates use 32-bit division.
-    auto issue = [&](int64_t t, int s) {
+    // issue the asynchronous copies of tile t = (ty, tx) into stage s (one commit group per call, possibly empty).
+    auto issue = [&](int64_t t, uint32_t ty, uint32_t tx, int s) {
         if (t < ntiles) {
-            const uint32_t ty = (uint32_t)t / (uint32_t)ntx, tx = (uint32_t)t - ty * (uint32_t)ntx;
             const int64_t rb0 = (int64_t)ty * kTransTileRowBlocks, c0 = (int64_t)tx * kTransTileCols;
             const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
             const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
@@ -132,13 +130,18 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
     };
 
     int s = 0;
+    // Tile counts fit 32 bits (a tile is 16384 elements).  The block's tiles are t, t + grid, ...: their
+    // coordinates advance by (grid / ntx, grid % ntx) with one carry, so only the first needs a division.
     int64_t t = blockIdx.x;
-    issue(t, 0);
+    const uint32_t ntx32 = (uint32_t)ntx, step_y = gridDim.x / ntx32, step_x = gridDim.x - step_y * ntx32;
+    uint32_t ty = blockIdx.x / ntx32, tx = blockIdx.x - ty * ntx32;
+    issue(t, ty, tx, 0);
     for (; t < ntiles; t += gridDim.x, s ^= 1) {
-        issue(t + gridDim.x, s ^ 1);                 // prefetch the block's next tile into the other stage
+        uint32_t ty_next = ty + step_y, tx_next = tx + step_x;
+        if (tx_next >= ntx32) { tx_next -= ntx32; ++ty_next; }
+        issue(t + gridDim.x, ty_next, tx_next, s ^ 1);   // prefetch the block's next tile into the other stage
         cp_async_wait_all_but_one();                 // this thread's copies of tile t have landed
         __syncthreads();                             // ... and everybody else's
-        const uint32_t ty = (uint32_t)t / (uint32_t)ntx, tx = (uint32_t)t - ty * (uint32_t)ntx;
         const int64_t rb0 = (int64_t)ty * kTransTileRowBlocks, c0 = (int64_t)tx * kTransTileCols;
         const int nrb = (int)min((int64_t)kTransTileRowBlocks, rblocks - rb0);
         const int ncols = (int)min((int64_t)kTransTileCols, cols - c0);
@@ -230,6 +233,8 @@ __global__ void __launch_bounds__(256) quantize4_transposed_kernel(const uint16_
             }
         }
         __syncthreads();                             // the stage may be overwritten by the next prefetch
+        ty = ty_next;
+        tx = tx_next;
     }
     if constexpr (MODE == 1) {
         __shared__ uint32_t warp_max[8];
