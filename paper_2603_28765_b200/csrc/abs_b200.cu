@@ -756,10 +756,10 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
     const uint32_t mask = o.had_sign_mask;
 #define ABS_LAUNCH_TE(I, S, R, Q, M, E, SLOT, GEN)                                                                  \
     do {                                                                                                            \
-        e = cudaFuncSetAttribute(quantize4_transposed_kernel<I, S, R, Q, M, E>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+        e = cudaFuncSetAttribute(transposed_kernel<I, S, R, Q, M, E>(), cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  kTransSmemBytes);                                                                  \
         if (e == cudaSuccess)                                                                                       \
-            e = cudaLaunchKernelEx(&cfg, quantize4_transposed_kernel<I, S, R, Q, M, E>, in, ct, stp, src, rows, cols, mask, \
+            e = cudaLaunchKernelEx(&cfg, transposed_kernel<I, S, R, Q, M, E>(), in, ct, stp, src, rows, cols, mask, \
                                    SLOT, GEN, mul, k0, k1, (uint16_t*)out_bf16, store_codes);                       \
     } while (0)
 #define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
