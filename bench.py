@@ -7,7 +7,10 @@ amax -> alpha, then the group-quantize kernel) followed by ``abs_dequantize`` --
 launches.  The metric is GB/s of algorithmic bytes in + out per step:
     quantize   2N (bf16 in) + N/2 (codes) + N/16 (scales)
     dequantize N/2 + N/16 in, 2N (bf16 out)                    => 5.125 N bytes per step.
-Steps rotate over enough tensor sets to exceed 4x the L2 capacity, so every step starts cold.
+Steps rotate over enough tensor sets that the inputs alone exceed 4x the L2 capacity, so every step starts cold.
+Before the timed region an untimed loop of the same steps runs for about 250 ms so that the clocks are up
+(disclosed as `clock_ramp_ms`); the timed region is exactly K steps.  The dominant kernel is timed separately in
+5 batches of 100 launches whatever K is (median, best and worst reported).
 
   python bench.py [--gpus N] [--steps K] [--warmup W]          CUDA path, one JSON line
   python bench.py --impl reference ...                         the CPU oracle timed on host cores
@@ -41,10 +44,26 @@ UNIT = "GB/s"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of the group-quantize kernel per element, from the ncu capture summarised in
-# profiles/quantize4_fast_if4_cfg2.md: (dram__bytes_read.sum + dram__bytes_write.sum) per launch / N
-# = (67.13 MB + 3.30 MB) / 33 554 432 elements, captured on this same workload.
-NCU_QUANT_TRAFFIC_BYTES_PER_ELEM = 70.43e6 / 33554432
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "quantize4_fast_if4_cfg2_traffic.txt")
+CLOCK_RAMP_MS = 250.0           # untimed steps run right before the timed region so that it starts at full clocks
+KERNEL_BATCHES = 5              # the dominant kernel is timed in this many batches ...
+KERNEL_BATCH_LAUNCHES = 100     # ... of this many back-to-back launches each, whatever --steps is
+
+
+def ncu_traffic(n_elems: int):
+    """DRAM bytes per launch of the group-quantize kernel from the tracked ncu summary (dram__bytes_read.sum +
+    dram__bytes_write.sum of one capture, scaled by the element count), and the commit it was captured at."""
+    try:
+        kv = {}
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                if ":" in line and not line.lstrip().startswith("#"):
+                    k, v = line.split(":", 1)
+                    kv[k.strip()] = v.strip()
+        per_elem = (float(kv["dram_bytes_read"]) + float(kv["dram_bytes_write"])) / float(kv["elements"])
+        return per_elem * n_elems, kv.get("commit", "unknown")
+    except Exception:
+        return None, None
 
 
 def step_bytes(n_elems: int) -> float:
@@ -67,12 +86,15 @@ def measured_peak():
 # ----------------------------------------------------------------------------- clocks
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons of one GPU through NVML, each sample with its host timestamp,
+    from before the clock-ramp loop until after the timed region; the report keeps the samples whose
+    timestamps fall inside the timed window."""
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
 
-    def __init__(self, torch_device_index: int):
-        self.samples, self.reasons, self.max_mhz, self.ok = [], set(), None, False
+    def __init__(self, torch_device_index: int, period_s: float = 0.0004):
+        self.samples, self.max_mhz, self.ok = [], None, False      # samples: (t, sm_mhz, reason bits)
+        self.period_s = period_s
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -96,17 +118,15 @@ class ClockSampler:
         nv = self.nv
         while not self._stop.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 try:
                     r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
                 except Exception:
                     r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                for bit, name in self.REASONS.items():
-                    if r & bit:
-                        self.reasons.add(name)
+                self.samples.append((time.perf_counter(), mhz, r))
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(self.period_s)
 
     def start(self):
         if self.ok:
@@ -120,14 +140,27 @@ class ClockSampler:
             self._thread.join()
             self._thread = None
 
-    def summary(self, note=""):
+    def summary(self, t0: float, t1: float):
+        """Clocks seen between host times t0 and t1 (the timed window)."""
         if not self.ok:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable: " + getattr(self, "err", "")}
-        out = {"sm_mhz": int(statistics.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
-               "reasons": sorted(self.reasons), "samples": len(self.samples)}
-        if note:
-            out["note"] = note
-        return out
+        inside = [(m, r) for (t, m, r) in self.samples if t0 <= t <= t1]
+        note = "samples inside the timed window"
+        if not inside and self.samples:
+            # the window was shorter than one NVML query: keep the two samples that bracket it
+            before = [x for x in self.samples if x[0] < t0][-1:]
+            after = [x for x in self.samples if x[0] > t1][:1]
+            inside = [(m, r) for (_, m, r) in before + after]
+            note = "timed window shorter than one NVML query: the samples taken just before and just after it"
+        reasons = set()
+        for _, r in inside:
+            for bit, name in self.REASONS.items():
+                if r & bit:
+                    reasons.add(name)
+        mhz = [m for m, _ in inside]
+        return {"sm_mhz": int(statistics.median(mhz)) if mhz else None, "sm_min_mhz": min(mhz) if mhz else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(reasons), "samples": len(inside),
+                "window_ms": round((t1 - t0) * 1e3, 3), "note": note}
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -207,7 +240,7 @@ def run_cuda(args):
     n = rows * cols
     nb_codes, nb_scales = B.abs_codes_bytes(FMT_IF4, rows, cols), B.abs_scales_bytes(FMT_IF4, rows, cols)
     set_bytes = 2 * n + nb_codes + nb_scales + 2 * n
-    n_sets = max(2, -(-4 * L2_BYTES // set_bytes))          # rotate over > 4x L2 of distinct buffers
+    n_sets = max(2, -(-4 * L2_BYTES // (2 * n)))            # the INPUTS alone rotate over >= 4x L2 (8 sets here)
 
     # Synthetic inputs: one host tensor per rank from the seeded recipe; the other sets are row
     # rotations of it (same distribution, different addresses and group contents).
@@ -237,47 +270,56 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
+    def event_pair():
+        return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_batches(fn, batches, launches, warm=8):
+        """Average time per call (ms) of `batches` back-to-back loops of `launches` calls each, every loop between
+        two CUDA events on the launching stream.  Returns the list of per-batch averages."""
+        for i in range(warm):
+            fn(i)
+        torch.cuda.synchronize()
+        res = []
+        for b in range(batches):
+            e0, e1 = event_pair()
+            e0.record(stream)
+            for i in range(launches):
+                fn(b * launches + i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            res.append(e0.elapsed_time(e1) / launches)
+        return res
+
+    sampler = ClockSampler(local)
+    sampler.start()
+
+    # ---- W warm-up steps, then an untimed clock-ramp loop of the same steps: a GPU that idled before the run
+    # needs a few hundred milliseconds of load to reach its full clocks, and the timed region must not pay for it.
+    warm = max(args.warmup, 3)
+    for i in range(warm):
         step(i)
     barrier()
+    ramp_t0 = time.perf_counter()
+    ramp_steps = 0
+    while (time.perf_counter() - ramp_t0) * 1e3 < CLOCK_RAMP_MS:
+        for i in range(64):
+            step(ramp_steps + i)
+        ramp_steps += 64
+        torch.cuda.synchronize()
+    clock_ramp_ms = (time.perf_counter() - ramp_t0) * 1e3
+    barrier()
 
-    # ---- timed region: exactly K steps; the quantize kernel is also timed on its own on every
-    # 8th step through the library's event hook (events on the launching stream).
-    sampler = ClockSampler(local)
-    n_probe = min(64, max(1, args.steps // 8))
-    probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_probe)]
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for a, b in probes:        # torch creates the CUDA event on first record; the library re-records it later
-        a.record(stream)
-        b.record(stream)
-    torch.cuda.synchronize()
-    sampler.start()
+    # ---- timed region: exactly K steps between two events on the launching stream
+    start, end = event_pair()
+    t_host0 = time.perf_counter()
     start.record(stream)
-    pi = 0
     for i in range(args.steps):
-        if i % 8 == 7 and pi < n_probe:
-            B.abs_profile_events(*probes[pi])
-            step(i)
-            B.abs_profile_events()
-            pi += 1
-        else:
-            step(i)
+        step(i)
     end.record(stream)
     barrier()
-    sampler.stop()
+    t_host1 = time.perf_counter()
     ms_total = start.elapsed_time(end)
-    clock_note = ""
-    if sampler.ok and len(sampler.samples) < 5:
-        # the timed region was shorter than a few NVML periods: sample an identical untimed loop too
-        sampler.start()
-        t_end = time.perf_counter() + 0.3
-        i = 0
-        while time.perf_counter() < t_end:
-            step(i)
-            i += 1
-        torch.cuda.synchronize()
-        sampler.stop()
-        clock_note = "timed region shorter than the sampling period; samples extended over an identical untimed loop"
+    clocks = sampler.summary(t_host0, t_host1)
     t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -285,58 +327,116 @@ def run_cuda(args):
     ms_per_step = ms_total / args.steps
     value = world * step_bytes(n) / (ms_per_step * 1e-3) / 1e9
 
-    quant_ms = [a.elapsed_time(b) for a, b in probes[:pi]]
-    if not quant_ms:     # fewer than 8 steps: time the kernel on one extra step
-        B.abs_profile_events(*probes[0])
-        step(0)
-        B.abs_profile_events()
-        torch.cuda.synchronize()
-        quant_ms = [probes[0][0].elapsed_time(probes[0][1])]
-    in_step_ms = sum(quant_ms) / len(quant_ms)
+    # ---- the same steps once more in batches, for the median next to the figure above (not part of `value`)
+    step_batches = timed_batches(step, KERNEL_BATCHES, KERNEL_BATCH_LAUNCHES, warm=0)
 
-    # The dominant kernel on its own: back-to-back launches of the group-quantize kernel over the same
-    # rotating buffer sets (alpha given = the alpha the steps just produced, so only that kernel runs),
-    # CUDA events around the loop on the launching stream.  An event placed between two kernels of a step
-    # (the in-step probe above) breaks their programmatic launch overlap and adds the launch latency to
-    # the interval, so this loop is the figure used for the roofline; both are reported.
+    # ---- the in-step view of the group-quantize kernel: events recorded by the library right before and after it
+    # on a few steps.  An event between two kernels of a step breaks their programmatic launch overlap, so the
+    # interval contains the kernel's launch latency; it is reported beside the figure used for the roofline.
+    probes = [event_pair() for _ in range(16)]
+    for a, b in probes:        # torch creates the CUDA event on first record; the library re-records it later
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize()
+    for pi, pr in enumerate(probes):
+        for i in range(7):
+            step(8 * pi + i)
+        B.abs_profile_events(*pr)
+        step(8 * pi + 7)
+        B.abs_profile_events()
+    torch.cuda.synchronize()
+    in_step_ms = statistics.median(a.elapsed_time(b) for a, b in probes)
+
+    # ---- the dominant kernel on its own: back-to-back launches of the group-quantize kernel over the same
+    # rotating buffer sets (alpha given = the alpha the steps just produced, so only that kernel runs), in
+    # KERNEL_BATCHES loops of KERNEL_BATCH_LAUNCHES launches whatever --steps is.  The median batch is the
+    # figure used for the roofline; best and worst are printed beside it.
     og = B.make_opts(B.ABS_F_ALPHA_GIVEN)
     gargs = [(FMT_IF4, xs[k].data_ptr(), rows, cols, codes[k].data_ptr(), scales[k].data_ptr(), alphas[k].data_ptr(),
               C.byref(og), sp) for k in range(n_sets)]
-    n_q = max(8, min(args.steps, 400))
-    for i in range(3):
-        L.abs_quantize_ex(*gargs[i % n_sets])
-    q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    q0.record(stream)
-    for i in range(n_q):
-        L.abs_quantize_ex(*gargs[i % n_sets])
-    q1.record(stream)
-    torch.cuda.synchronize()
-    q_ms = q0.elapsed_time(q1) / n_q
+    q_batches = timed_batches(lambda i: L.abs_quantize_ex(*gargs[i % n_sets]), KERNEL_BATCHES, KERNEL_BATCH_LAUNCHES)
+    q_ms = statistics.median(q_batches)
     peak, peak_src = measured_peak()
     achieved = quant_kernel_bytes(n) / (q_ms * 1e-3) / 1e9
+    traffic, traffic_commit = ncu_traffic(n)
     roofline = {"bound": "hbm", "kernel": "quantize4_fast_kernel<IF4> (group-quantize, Fig. 3a steps 1-10)",
                 "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                 "peak_source": peak_src, "frac_of_nominal_8000_gbs": round(achieved / 8000.0, 4),
-                "us_per_launch": round(q_ms * 1e3, 2), "launches_timed": n_q,
+                "us_per_launch": round(q_ms * 1e3, 2), "us_per_launch_best": round(min(q_batches) * 1e3, 2),
+                "us_per_launch_worst": round(max(q_batches) * 1e3, 2),
+                "launches_timed": KERNEL_BATCHES * KERNEL_BATCH_LAUNCHES, "batches": KERNEL_BATCHES,
                 "in_step_probe_us": round(in_step_ms * 1e3, 2),
                 "algorithmic_bytes_per_launch": quant_kernel_bytes(n),
-                "traffic": (NCU_QUANT_TRAFFIC_BYTES_PER_ELEM * n) if NCU_QUANT_TRAFFIC_BYTES_PER_ELEM else None}
+                "traffic": traffic, "traffic_source": f"profiles/{os.path.basename(TRAFFIC_FILE)} (ncu capture at commit {traffic_commit})"}
+
+    # ---- T2 / T3 of the same workload, cold (rotating sets) and warm (one set, input largely resident in L2)
+    def t_of(fn):
+        return statistics.median(timed_batches(fn, KERNEL_BATCHES, 40))
+
+    t2 = t_of(lambda i: L.abs_quantize(*qargs[i % n_sets]))
+    t3 = t_of(lambda i: L.abs_dequantize(*dargs[i % n_sets]))
+    t1_warm = t_of(lambda i: L.abs_quantize_ex(*gargs[0]))
+    t2_warm = t_of(lambda i: L.abs_quantize(*qargs[0]))
+    out_b = nb_codes + nb_scales
+    breakdown = {
+        "workload": f"bf16 {rows}x{cols} IF4, median of {KERNEL_BATCHES} batches",
+        "T1_quantize_kernel_us": round(q_ms * 1e3, 2), "T1_gbs": round((2 * n + out_b) / q_ms / 1e6, 1),
+        "T2_abs_quantize_us": round(t2 * 1e3, 2), "T2_gbs_dram_basis_4N_plus_out": round((4 * n + out_b) / t2 / 1e6, 1),
+        "T2_gbs_effective_2N_plus_out": round((2 * n + out_b) / t2 / 1e6, 1),
+        "T3_abs_dequantize_us": round(t3 * 1e3, 2), "T3_gbs": round((2 * n + out_b) / t3 / 1e6, 1),
+        "warm_l2_T1_us": round(t1_warm * 1e3, 2), "warm_l2_T2_us": round(t2_warm * 1e3, 2),
+        "warm_note": "warm = the same buffer set every call (the 64 MiB input mostly stays in the 126 MB L2)"}
+
+    # ---- the "and larger" half of the target: the same three figures at 16384x8192 (seeded device-side mixture
+    # of the format-sweep configuration's recipe: 70 % N(0,1), 30 % Laplace(0,1), 0.1 % of entries x100)
+    large = None
+    if not args.no_large:
+        lr, lc = 16384, 8192
+        ln = lr * lc
+        gen = torch.Generator(device=dev).manual_seed(6 + 1000 * rank)
+        lsets = 4                                             # 4 x 256 MiB of inputs = 8x L2
+        lx = []
+        for k in range(lsets):
+            u = torch.rand((lr, lc), device=dev, generator=gen)
+            v = torch.randn((lr, lc), device=dev, generator=gen)
+            e = torch.empty((lr, lc), device=dev).exponential_(generator=gen)
+            sgn = torch.where(torch.rand((lr, lc), device=dev, generator=gen) < 0.5, -1.0, 1.0)
+            v = torch.where(u < 0.7, v, e * sgn)
+            v = torch.where(torch.rand((lr, lc), device=dev, generator=gen) < 0.001, v * 100.0, v)
+            lx.append(v.to(torch.bfloat16))
+            del u, v, e, sgn
+        lcb, lsb = B.abs_codes_bytes(FMT_IF4, lr, lc), B.abs_scales_bytes(FMT_IF4, lr, lc)
+        lcodes = [torch.empty(lcb, dtype=torch.uint8, device=dev) for _ in range(lsets)]
+        lscales = [torch.empty(lsb, dtype=torch.uint8, device=dev) for _ in range(lsets)]
+        lalpha = [torch.zeros(1, dtype=torch.float32, device=dev) for _ in range(lsets)]
+        lout = [torch.empty((lr, lc), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        lq = [(FMT_IF4, lx[k].data_ptr(), lr, lc, lcodes[k].data_ptr(), lscales[k].data_ptr(), lalpha[k].data_ptr(), sp)
+              for k in range(lsets)]
+        lg = [a[:-1] + (C.byref(og), sp) for a in lq]
+        ld = [(FMT_IF4, lcodes[k].data_ptr(), lscales[k].data_ptr(), lalpha[k].data_ptr(), lr, lc,
+               lout[k % 2].data_ptr(), sp) for k in range(lsets)]
+        for k in range(lsets):
+            L.abs_quantize(*lq[k])
+        lt2 = statistics.median(timed_batches(lambda i: L.abs_quantize(*lq[i % lsets]), KERNEL_BATCHES, 24, warm=4))
+        lt1 = statistics.median(timed_batches(lambda i: L.abs_quantize_ex(*lg[i % lsets]), KERNEL_BATCHES, 24, warm=4))
+        lt3 = statistics.median(timed_batches(lambda i: L.abs_dequantize(*ld[i % lsets]), KERNEL_BATCHES, 24, warm=4))
+        lob = lcb + lsb
+        large = {"workload": f"bf16 {lr}x{lc} IF4 (format-sweep mixture, generated on the device, seed 6), "
+                             f"median of {KERNEL_BATCHES} batches of 24 calls, {lsets} rotating sets",
+                 "T1_quantize_kernel_us": round(lt1 * 1e3, 2), "T1_gbs": round((2 * ln + lob) / lt1 / 1e6, 1),
+                 "T1_frac_of_measured_peak": round((2 * ln + lob) / lt1 / 1e6 / peak, 4),
+                 "T2_abs_quantize_us": round(lt2 * 1e3, 2),
+                 "T2_gbs_dram_basis_4N_plus_out": round((4 * ln + lob) / lt2 / 1e6, 1),
+                 "T2_gbs_effective_2N_plus_out": round((2 * ln + lob) / lt2 / 1e6, 1),
+                 "T3_abs_dequantize_us": round(lt3 * 1e3, 2), "T3_gbs": round((2 * ln + lob) / lt3 / 1e6, 1)}
+        del lx, lcodes, lscales, lout
 
     # ---- for information: the same result through the one-pass emulation call (amax pass + one kernel that
     # quantizes and decodes from registers, writing codes, scales and the bf16 output); not part of `value`.
     eargs = [(FMT_IF4, xs[k].data_ptr(), rows, cols, outs[k].data_ptr(), codes[k].data_ptr(), scales[k].data_ptr(),
               alphas[k].data_ptr(), None, sp) for k in range(n_sets)]
-    for i in range(3):
-        L.abs_quantize_dequantize(*eargs[i % n_sets])
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record(stream)
-    for i in range(n_q):
-        L.abs_quantize_dequantize(*eargs[i % n_sets])
-    e1.record(stream)
-    torch.cuda.synchronize()
-    one_pass = {"us_per_call": round(e0.elapsed_time(e1) / n_q * 1e3, 2), "calls_timed": n_q,
+    e_ms = t_of(lambda i: L.abs_quantize_dequantize(*eargs[i % n_sets]))
+    one_pass = {"us_per_call": round(e_ms * 1e3, 2), "calls_timed": KERNEL_BATCHES * 40,
                 "api": "abs_quantize_dequantize with code outputs (same outputs as one step, 2 kernels instead of 3)"}
 
     # ---- for information: the same steps issued alternately on two streams, so the bandwidth-bound amax /
@@ -350,7 +450,7 @@ def run_cuda(args):
         L.abs_quantize(*qargs[k][:-1], p)
         L.abs_dequantize(*dargs[k][:-1], p)
 
-    n_t = max(8, min(args.steps, 400)) & ~1
+    n_t = 200
     for i in range(4):
         step2(i)
     torch.cuda.synchronize()
@@ -367,6 +467,7 @@ def run_cuda(args):
     two_streams = {"us_per_step": round(t_us, 2), "value": round(step_bytes(n) / (t_us * 1e-6) / 1e9, 1),
                    "unit": UNIT, "steps_timed": n_t,
                    "note": "steps alternate over two streams; per-rank figure, informational"}
+    sampler.stop()
 
     # ---- end to end through the host-buffer C-ABI calls (pinned host memory, copies in the timed region)
     e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
@@ -401,15 +502,23 @@ def run_cuda(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "warmup": warm, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"{WORKLOAD}: IF4 quantize+dequantize, bf16 {rows}x{cols}, {cfg.note}",
+                       "data_dtype": "bf16 in and out, FP32 arithmetic, 4-bit codes + E4M3 scales",
                        "bytes_per_step": step_bytes(n), "elements_per_s": round(world * n / (ms_per_step * 1e-3), 0),
-                       "l2": f"cold: steps rotate over {n_sets} buffer sets ({n_sets * set_bytes >> 20} MiB > 4x L2)",
-                       "sharding": "one independent tensor per rank, no collective"},
-            "roofline": roofline, "e2e": e2e, "one_pass": one_pass, "two_streams": two_streams,
+                       "l2": f"cold: steps rotate over {n_sets} buffer sets; the inputs alone are "
+                             f"{n_sets * 2 * n >> 20} MiB >= 4x L2, all buffers {n_sets * set_bytes >> 20} MiB",
+                       "sharding": "one independent tensor per rank, no collective",
+                       "input_sha256": I.sha256(xb)[:16]},
+            "clock_ramp_ms": round(clock_ramp_ms, 1), "clock_ramp_steps": ramp_steps,
+            "ms_per_step_batches": {"median": round(statistics.median(step_batches), 5),
+                                    "best": round(min(step_batches), 5), "worst": round(max(step_batches), 5),
+                                    "batches": KERNEL_BATCHES, "steps_per_batch": KERNEL_BATCH_LAUNCHES},
+            "roofline": roofline, "breakdown": breakdown, "large": large,
+            "e2e": e2e, "one_pass": one_pass, "two_streams": two_streams,
             "gpu_launches": 3 * args.steps,
-            "clocks": sampler.summary(clock_note),
+            "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
             threads = os.cpu_count() or 1
@@ -430,6 +539,7 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-large", action="store_true", help="skip the 16384x8192 figures (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

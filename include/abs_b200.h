@@ -20,8 +20,18 @@
  * Inputs must be finite and the tensor maximum either 0 or at least 2^-100; input and
  * output buffers must not overlap.  All device pointers must be 16-byte aligned.
  * The library keeps a small per-device scratch ring (allocated on the first quantize call
- * on a device, or by abs_init); make that first call outside any stream capture.  At most
- * ABS_MAX_INFLIGHT quantize calls may be in flight on one device at a time.
+ * on a device, or by abs_init); make that first call outside any stream capture.
+ *   - In flight: every call that runs an amax pass (abs_amax, and abs_quantize* without
+ *     ABS_F_ALPHA_GIVEN) takes the next of ABS_MAX_INFLIGHT ring slots, chosen on the host.  If
+ *     more than ABS_MAX_INFLIGHT such calls are enqueued on a device before the oldest has run,
+ *     the oldest loses its maximum: its kernel notices (the slot carries another call's tag),
+ *     quantizes with alpha = 1, and raises a flag that makes the NEXT such call on the device
+ *     return ABS_ERR_SIZE once, so the overrun cannot pass unseen.
+ *   - CUDA graphs: the slot and its tag are kernel arguments fixed at enqueue time, so a captured
+ *     call of that kind must not be replayed (a replay would merge its maximum with the previous
+ *     replay's).  Inside a graph use ABS_F_ALPHA_GIVEN with an alpha computed outside the graph,
+ *     or abs_quantize_noalloc, whose nodes re-arm their own scratch.  Calls with
+ *     ABS_F_ALPHA_GIVEN, and every dequantize call, use no scratch and may be captured.
  * There is no CPU fallback: without a CUDA device every compute call returns ABS_ERR_CUDA.
  */
 #ifndef ABS_B200_H
@@ -63,7 +73,8 @@ typedef enum {
     ABS_ERR_FMT = 4,    /* unknown format                                     */
     ABS_ERR_FLAGS = 5,  /* unknown flag bit, or a flag the call cannot honour */
     ABS_ERR_CUDA = 6,   /* a CUDA runtime call or a launch failed             */
-    ABS_ERR_SIZE = 7    /* workspace too small / size beyond a stated maximum */
+    ABS_ERR_SIZE = 7    /* workspace too small / size beyond a stated maximum / an earlier call on this device
+                           overran the ring of ABS_MAX_INFLIGHT scratch slots (see the top of this file)   */
 } abs_status_t;
 
 enum {
@@ -86,8 +97,7 @@ enum {
     ABS_F_GROUPS_DOWN_COLUMNS = 1u << 9, /* abs_quantize_dequantize only: groups are 16 consecutive ROWS of one column
                                        (Sec. 4.1: the operands of the weight-gradient product are quantized along the
                                        token dimension); needs rows % 16 == 0                                        */
-    ABS_F_INDEX64 = 1u << 5         /* testing aid: run the kernel instances that index groups with 64-bit
-                                       integers (otherwise chosen only beyond 2^31 groups); same results  */
+    ABS_F_INDEX64 = 1u << 5         /* TESTING ONLY (see the last block of this file)                    */
 };
 
 #define ABS_MAX_INFLIGHT 1024
@@ -97,6 +107,13 @@ typedef struct {
     uint16_t had_sign_mask; /* Hadamard option: bit i = 1 multiplies element i of each group by -1 */
     uint16_t _pad;          /* must be 0                                                          */
     uint64_t sr_seed;       /* stochastic rounding: Philox key                                    */
+    uint64_t sr_index_offset; /* stochastic rounding: index, in the whole tensor, of this call's first element.
+                               Element (r, c) of the matrix passed to the call draws the random field of index
+                               sr_index_offset + r * cols + c (App. B: one stream over the tensor), so a row shard
+                               that starts at row r0 of a [R, cols] tensor passes r0 * cols and gets the bytes the
+                               unsharded call gives for those rows.  A multiple of 16 (else ABS_ERR_SHAPE); read
+                               only with ABS_F_STOCHASTIC.  For abs_quantize_transposed and the column mode of
+                               abs_quantize_dequantize the index runs over the transposed matrix.               */
 } abs_opts_t;
 
 /* Sizes of the outputs of abs_quantize: rows*cols*b/8 and rows*cols/16 bytes (rows*cols/8 for the
@@ -181,6 +198,11 @@ ABS_API abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16,
  *     rows*cols returns ABS_ERR_SIZE and enqueues nothing.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
  *     device current); make that first call before any stream capture.
+ *   - With CUDA's default lazy module loading the first launch of each kernel loads its code onto the
+ *     device, which itself needs a little device memory.  A caller whose pool is about to take every
+ *     free byte should therefore make one abs_quantize_noalloc call per format it will use, with input
+ *     pointers of the alignment it will use (32-byte and 16-byte aligned inputs run different kernel
+ *     instances), BEFORE handing out its last memory, or run with CUDA_MODULE_LOADING=EAGER.
  *   - All calls on a device share the one array.  Each call clears the ticket word it needs at zero
  *     itself (a 4-byte cudaMemsetAsync on `stream`) and overwrites every partial maximum it reads, so
  *     stale contents from earlier calls are harmless; but two calls that overlap on the GPU (different
@@ -224,6 +246,13 @@ ABS_API abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, 
 ABS_API abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const void* scales_e4m3_host,
                                  const float* tensor_scale_f32_host, int64_t rows, int64_t cols, void* out_host,
                                  const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * TESTING AND PROFILING ONLY.  Nothing below (nor ABS_F_INDEX64 above) is part of the method or needed
+ * by an application; the test suite and the benchmark use them.
+ *   ABS_F_INDEX64: run the kernel instances that index groups with 64-bit integers (otherwise chosen
+ *   only beyond 2^31 groups); same results.
+ * ------------------------------------------------------------------------------------------------ */
 
 /* Profiling hook (no counterpart in the paper): while both handles (cudaEvent_t as void*) are set,
  * every quantize call records them on its stream immediately before and after the group-quantize

@@ -323,11 +323,14 @@ ORACLE_API float abs_oracle_alpha(int fmt, float amax) {
 
 /* Quantize rows [row0,row1) of a row-major bf16 matrix with tensor scale alpha.
  * Outputs: codes (rows x cols*b/8 bytes), scales (rows x cols/G bytes, G = values per scale); optional
- * per-group E_FP / E_INT (rows x cols/G floats each, may be NULL) for the selection invariants. */
+ * per-group E_FP / E_INT (rows x cols/G floats each, may be NULL) for the selection invariants.
+ * sr_index_offset: App. B draws one random stream over the whole tensor; when this matrix is a row shard
+ * of a larger one, the offset is the index of its element (0, 0) in that tensor, so that element (r, c)
+ * draws field sr_index_offset + r*cols + c. */
 ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_t rows, int64_t cols,
                                         int64_t row0, int64_t row1, float alpha, uint32_t flags,
-                                        uint16_t sign_mask, uint64_t sr_seed, uint8_t* codes,
-                                        uint8_t* scales, float* dbg_e_fp, float* dbg_e_int) {
+                                        uint16_t sign_mask, uint64_t sr_seed, uint64_t sr_index_offset,
+                                        uint8_t* codes, uint8_t* scales, float* dbg_e_fp, float* dbg_e_int) {
     if (fmt < 0 || fmt >= FMT_COUNT || cols % 16 != 0 || row0 < 0 || row1 > rows) return 1;
     const fmt_desc* F = &FMTS[fmt];
     const int b = F->bits;
@@ -385,7 +388,7 @@ ORACLE_API int abs_oracle_quantize_rows(int fmt, const uint16_t* in_bf16, int64_
                     const float xi = xs[i];
                     float u = 0.0f;
                     if (flags & F_STOCHASTIC)
-                        u = sr_uniform(sr_seed, (uint64_t)(r * cols + gi * 16 + sub * G + i));
+                        u = sr_uniform(sr_seed, sr_index_offset + (uint64_t)(r * cols + gi * 16 + sub * G + i));
                     /* E1 (step 3). */
                     const float y = xi * rcp;
                     const uint32_t ysign = f32_to_bits(y) >> 31;
@@ -451,7 +454,9 @@ ORACLE_API int abs_oracle_dequantize_rows(int fmt, const uint8_t* codes, const u
             unpack_codes(codes + (r * gpr + gi) * (2 * b), b, code);
             for (int i = 0; i < 16; ++i) {
                 const uint8_t sbyte = scales[(r * gpr + gi) * nsub + i / G];
-                const int flag = sbyte >> 7;
+                /* Sec. 3: the flag lives in the sign bit that an NVFP4 scale leaves unused; a plain NVFP4
+                 * tensor has no integer groups, so there the bit is ignored and the byte is its magnitude. */
+                const int flag = F->has_int ? (sbyte >> 7) : 0;
                 const float Delta = abs_oracle_e4m3_value(sbyte);
                 float d = Delta * alpha;
                 if (flag && !(select & F_INT_GROUPS_RAW)) d = d * c_post;

@@ -86,8 +86,8 @@ def lib():
             L.abs_oracle_alpha.argtypes = [C.c_int, C.c_float]
             L.abs_oracle_quantize_rows.restype = C.c_int
             L.abs_oracle_quantize_rows.argtypes = [C.c_int, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
-                                                   C.c_float, C.c_uint32, C.c_uint16, C.c_uint64, C.c_void_p,
-                                                   C.c_void_p, C.c_void_p, C.c_void_p]
+                                                   C.c_float, C.c_uint32, C.c_uint16, C.c_uint64, C.c_uint64,
+                                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
             L.abs_oracle_dequantize_rows.restype = C.c_int
             L.abs_oracle_dequantize_rows.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_float, C.c_int64,
                                                      C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_uint32]
@@ -223,8 +223,9 @@ def alpha_from_amax(fmt: int, A) -> np.float32:
 
 
 def quantize(fmt: int, x_bf16_bits, flags: int = 0, sign_mask: int = 0, sr_seed: int = 0,
-             alpha=None, threads: int = 1, debug: bool = False):
-    """Quantize a 2-D array of bf16 bit patterns.
+             alpha=None, threads: int = 1, debug: bool = False, sr_index_offset: int = 0):
+    """Quantize a 2-D array of bf16 bit patterns.  ``sr_index_offset``: index of element (0, 0) in the
+    whole tensor when the array is a row shard of a larger one (stochastic rounding only).
 
     Returns (codes u8[rows, cols*b/8], scales u8[rows, cols/16], alpha float32) and, with
     ``debug``, additionally (E_FP, E_INT) per group as float32[rows, cols/16]."""
@@ -246,7 +247,8 @@ def quantize(fmt: int, x_bf16_bits, flags: int = 0, sign_mask: int = 0, sr_seed:
 
     def work(rr):
         rc = L.abs_oracle_quantize_rows(fmt, a.ctypes.data, rows, cols, rr[0], rr[1], C.c_float(float(alpha)),
-                                        flags, sign_mask, sr_seed, codes.ctypes.data, scales.ctypes.data,
+                                        flags, sign_mask, sr_seed, sr_index_offset, codes.ctypes.data,
+                                        scales.ctypes.data,
                                         efp.ctypes.data if debug else None, eint.ctypes.data if debug else None)
         if rc != 0:
             raise ValueError("abs_oracle_quantize_rows rejected its arguments")

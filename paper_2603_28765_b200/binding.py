@@ -40,7 +40,8 @@ EXPORTS = [
 
 
 class AbsOpts(C.Structure):
-    _fields_ = [("flags", C.c_uint32), ("had_sign_mask", C.c_uint16), ("_pad", C.c_uint16), ("sr_seed", C.c_uint64)]
+    _fields_ = [("flags", C.c_uint32), ("had_sign_mask", C.c_uint16), ("_pad", C.c_uint16), ("sr_seed", C.c_uint64),
+                ("sr_index_offset", C.c_uint64)]
 
 
 class AbsError(RuntimeError):
@@ -119,8 +120,8 @@ def _check(status: int, what: str):
         raise AbsError(status, what)
 
 
-def make_opts(flags: int = 0, had_sign_mask: int = 0, sr_seed: int = 0) -> AbsOpts:
-    return AbsOpts(flags, had_sign_mask, 0, sr_seed)
+def make_opts(flags: int = 0, had_sign_mask: int = 0, sr_seed: int = 0, sr_index_offset: int = 0) -> AbsOpts:
+    return AbsOpts(flags, had_sign_mask, 0, sr_seed, sr_index_offset)
 
 
 def _stream_ptr(stream=None):

@@ -49,7 +49,10 @@ struct DeviceState {
     std::once_flag once;
     cudaError_t init_err = cudaSuccess;
     uint32_t* ring = nullptr;          // ABS_MAX_INFLIGHT slots of 16 bytes: tagged maximum (u64), ticket (u32), pad
-    std::atomic<uint32_t> next{0};
+    std::mutex slot_mu;                // guards `next` and the clearing of the ring when the generation wraps
+    uint64_t next = 0;                 // calls that took a slot so far; generation = low 32 bits
+    uint32_t* overrun_host = nullptr;  // pinned, mapped word a kernel sets when its slot was reused under it
+    uint32_t* overrun_dev = nullptr;   // the same word as the device sees it
     int sm_count = 148;
     // abs_dequantize_host: a second stream for the device-to-host copies and the events that order it
     std::mutex host_mu;
@@ -69,6 +72,11 @@ abs_status_t device_state(DeviceState** out) {
     std::call_once(st.once, [&]() {
         st.init_err = cudaMalloc(&st.ring, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t));
         if (st.init_err == cudaSuccess) st.init_err = cudaMemset(st.ring, 0, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t));
+        if (st.init_err == cudaSuccess) st.init_err = cudaHostAlloc(&st.overrun_host, sizeof(uint32_t), cudaHostAllocMapped);
+        if (st.init_err == cudaSuccess) {
+            *st.overrun_host = 0u;
+            st.init_err = cudaHostGetDevicePointer(&st.overrun_dev, st.overrun_host, 0);
+        }
         int sms = 0;
         if (st.init_err == cudaSuccess) st.init_err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms > 0) st.sm_count = sms;
@@ -102,9 +110,9 @@ float fmt_mfp(int fmt) {
 constexpr uint32_t kQuantFlags = ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN |
                                  ABS_F_INDEX64 | ABS_F_SCALES_SWIZZLED;
 
-int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
+int grid_for(int sm_count, int64_t work_items, int blocks_per_sm) {
     int64_t want = (work_items + kThreads - 1) / kThreads;
-    int64_t cap = (int64_t)st.sm_count * blocks_per_sm;
+    int64_t cap = (int64_t)sm_count * blocks_per_sm;
     return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
 }
 
@@ -113,9 +121,9 @@ int grid_for(const DeviceState& st, int64_t work_items, int blocks_per_sm) {
 // amortise the prologue and keep the prefetch running; several waves let blocks that start later overlap
 // their first loads with the arithmetic of the others (measured: about seven items per thread is best for
 // the IF4 kernel, 10 % faster than one wave of long-running blocks).
-int grid_waves(const DeviceState& st, int64_t work_items, int resident_per_sm, int target_iters) {
+int grid_waves(int sm_count, int64_t work_items, int resident_per_sm, int target_iters) {
     const int64_t want = (work_items + kThreads - 1) / kThreads;
-    const int64_t resident = (int64_t)st.sm_count * resident_per_sm;
+    const int64_t resident = (int64_t)sm_count * resident_per_sm;
     if (want <= resident) return (int)(want < 1 ? 1 : want);
     int64_t waves = (want + (int64_t)target_iters * resident / 2) / ((int64_t)target_iters * resident);
     if (waves < 1) waves = 1;
@@ -123,14 +131,21 @@ int grid_waves(const DeviceState& st, int64_t work_items, int resident_per_sm, i
     return (int)(grid < want ? grid : want);
 }
 
-// Takes the next scratch slot and generation of this device.  Generations grow by one per call; when
-// the 32-bit counter wraps (after 2^32 calls) the ring is cleared once, after the device went idle.
+// Takes the next scratch slot and generation of this device.  Generations grow by one per call; when the
+// 32-bit generation wraps (after 2^32 calls) the ring is cleared once, after the device went idle, while the
+// mutex keeps other callers out.  Returns ABS_ERR_SIZE (once) if a kernel of an earlier call reported that its
+// slot had been reused while it was in flight: that call's scales were computed with alpha = 1.
 abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen) {
-    uint32_t g = st.next.fetch_add(1) + 1;
+    std::lock_guard<std::mutex> lock(st.slot_mu);
+    if (*reinterpret_cast<volatile uint32_t*>(st.overrun_host)) {
+        *reinterpret_cast<volatile uint32_t*>(st.overrun_host) = 0u;
+        return ABS_ERR_SIZE;
+    }
+    uint32_t g = (uint32_t)++st.next;
     if (g == 0) {
         if (cudaDeviceSynchronize() != cudaSuccess) return ABS_ERR_CUDA;
         if (cudaMemset(st.ring, 0, ABS_MAX_INFLIGHT * 4 * sizeof(uint32_t)) != cudaSuccess) return ABS_ERR_CUDA;
-        g = st.next.fetch_add(1) + 1;
+        g = (uint32_t)++st.next;
     }
     *gen = g;
     *slot = reinterpret_cast<unsigned long long*>(st.ring + 4 * (g % ABS_MAX_INFLIGHT));
@@ -139,13 +154,13 @@ abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen
 
 // ticket = true: the kernel itself writes max |x| (denom == 0) or alpha to `result` (abs_amax).
 // ticket = false: the maximum stays in the slot for the quantize kernel of the same call.
-abs_status_t launch_amax(DeviceState& st, const void* in, int64_t ngroups, const abs_opts_t& o, bool ticket,
+abs_status_t launch_amax(int sm_count, const void* in, int64_t ngroups, const abs_opts_t& o, bool ticket,
                          unsigned long long* slot, uint32_t gen, float* result, float denom, cudaStream_t s) {
     const bool rht = o.flags & ABS_F_HADAMARD16;
 #ifndef ABS_AMAX_RHT_BPS
 #define ABS_AMAX_RHT_BPS ABS_AMAX_BPS
 #endif
-    const int grid = grid_for(st, rht ? ngroups : ngroups * 2, rht ? ABS_AMAX_RHT_BPS : ABS_AMAX_BPS);
+    const int grid = grid_for(sm_count, rht ? ngroups : ngroups * 2, rht ? ABS_AMAX_RHT_BPS : ABS_AMAX_BPS);
     cudaError_t e;
 #define ABS_LAUNCH_A(R, T)                                                                                          \
     e = launch_pdl(amax_kernel<R, T>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, \
@@ -181,20 +196,21 @@ template <int FMT>
 // emul_out != nullptr asks for the emulation pass (abs_quantize_dequantize) of the formats handled by the
 // kernels of abs_fastx.cuh: bf16 output, codes stored only when emul_store.  *handled tells the caller whether
 // a kernel with that ability exists for the format and options.
-abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroups, void* codes, void* scales,
+abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, void* codes, void* scales,
                                  const AlphaSrc& alpha, const abs_opts_t& o, cudaStream_t s, int64_t cols = 0,
                                  void* emul_out = nullptr, bool emul_store = true, bool* handled = nullptr) {
     if (handled) *handled = false;
     const bool o32 = (reinterpret_cast<uintptr_t>(emul_out) & 31u) == 0;
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
-    const int grid = grid_for(st, ngroups, 64);
+    const int grid = grid_for(sm_count, ngroups, 64);
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
+    const uint64_t ctr = o.sr_index_offset / 8;      // Philox block of the call's first element (even: offset % 16 == 0)
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (emul_out) return ABS_ERR_FLAGS;      // the 4-bit emulation pass is launched by abs_quantize_dequantize
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
-            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(st, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(st, ngroups, 5, ABS_NV_ITERS);
+            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(sm_count, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(sm_count, ngroups, 5, ABS_NV_ITERS);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
@@ -226,7 +242,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     }
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         // Hadamard / stochastic-rounding options of the 4-bit formats: the packed persistent kernel
-        const int ogrid = grid_waves(st, ngroups, opt_blocks_per_sm(sr, rht), ABS_OPT_ITERS);
+        const int ogrid = grid_waves(sm_count, ngroups, opt_blocks_per_sm(sr, rht), ABS_OPT_ITERS);
         if (!(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)ogrid * kThreads) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -234,10 +250,10 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 #define ABS_LAUNCH_O(R, S)                                                                                        \
     e = alpha.slot ? launch_pdl(quantize4_opt_kernel<kInt, R, S, true, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, a32, (uint4*)nullptr, false, true)             \
+                                (uint32_t)o.had_sign_mask, k0, k1, ctr, a32, (uint4*)nullptr, false, true)             \
                    : launch_pdl(quantize4_opt_kernel<kInt, R, S, false, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, a32, (uint4*)nullptr, false, true)
+                                (uint32_t)o.had_sign_mask, k0, k1, ctr, a32, (uint4*)nullptr, false, true)
             if (rht && sr) ABS_LAUNCH_O(true, true);
             else if (rht) ABS_LAUNCH_O(true, false);
             else ABS_LAUNCH_O(false, true);
@@ -250,7 +266,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
         // block-size-8 variants of the 4-bit formats, round-to-nearest: two groups of 8 per thread
         constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
-        const int bgrid = grid_waves(st, ngroups, kInt ? 4 : 5, kInt ? ABS_IF6_ITERS : 5);
+        const int bgrid = grid_waves(sm_count, ngroups, kInt ? 4 : 5, kInt ? ABS_IF6_ITERS : 5);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -268,7 +284,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     }
     if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
         // 6-bit formats, round-to-nearest
-        const int sgrid = grid_waves(st, ngroups, 3, ABS_IF6_ITERS);
+        const int sgrid = grid_waves(sm_count, ngroups, 3, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -287,7 +303,7 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // IF3 and its block-size-8 variant, round-to-nearest
         constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
-        const int tgrid = grid_waves(st, ngroups, ABS_IF3_MINB, ABS_IF6_ITERS);
+        const int tgrid = grid_waves(sm_count, ngroups, ABS_IF3_MINB, ABS_IF6_ITERS);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -308,10 +324,10 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 #define ABS_LAUNCH_Q(R, S)                                                                                      \
     eq = alpha.slot ? launch_pdl(quantize_kernel<FMT, R, S, true>, grid, kThreads, s, (const uint4*)in,         \
                                  (uint8_t*)codes, (uint8_t*)scales, alpha, ngroups, mul,                        \
-                                 (uint32_t)o.had_sign_mask, k0, k1)                                             \
+                                 (uint32_t)o.had_sign_mask, k0, k1, ctr)                                        \
                     : launch_pdl(quantize_kernel<FMT, R, S, false>, grid, kThreads, s, (const uint4*)in,        \
                                  (uint8_t*)codes, (uint8_t*)scales, alpha, ngroups, mul,                        \
-                                 (uint32_t)o.had_sign_mask, k0, k1)
+                                 (uint32_t)o.had_sign_mask, k0, k1, ctr)
     if (rht && sr) ABS_LAUNCH_Q(true, true);
     else if (rht) ABS_LAUNCH_Q(true, false);
     else if (sr) ABS_LAUNCH_Q(false, true);
@@ -322,14 +338,14 @@ abs_status_t launch_quantize_fmt(DeviceState& st, const void* in, int64_t ngroup
 }
 
 template <int FMT>
-abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const void* scales, const float* alpha,
+abs_status_t launch_dequantize_fmt(int sm_count, const void* codes, const void* scales, const float* alpha,
                                    int64_t ngroups, void* out, bool fp32, bool index64, cudaStream_t s,
                                    int64_t swz_cols = 0, int sel = 0) {
-    const int grid = grid_for(st, ngroups, 64);
+    const int grid = grid_for(sm_count, ngroups, 64);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
-            const int grid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);    // 31 registers: 8 resident blocks per SM
+            const int grid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);    // 31 registers: 8 resident blocks per SM
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
             const bool i32 = !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
             cudaError_t e;
@@ -356,7 +372,7 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
         }
     }
     if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
-        const int bgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        const int bgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
             constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
@@ -369,7 +385,7 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
         }
     }
     if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
-        const int sgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        const int sgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
             constexpr ElemKind kEK = Fmt<FMT>::EK;
             const float c_post = Fmt<FMT>::M_FP / Fmt<FMT>::M_INT;         // IEEE single division, as in the generic kernel
@@ -384,7 +400,7 @@ abs_status_t launch_dequantize_fmt(DeviceState& st, const void* codes, const voi
     }
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // 3-bit codes widened to nibbles and decoded like the 4-bit formats
-        const int tgrid = grid_waves(st, ngroups, 8, ABS_DEQ_ITERS);
+        const int tgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
@@ -514,7 +530,7 @@ const char* abs_status_string(abs_status_t status) {
         case ABS_ERR_FMT: return "unknown format";
         case ABS_ERR_FLAGS: return "unknown or unsupported flag";
         case ABS_ERR_CUDA: return "CUDA error";
-        case ABS_ERR_SIZE: return "size beyond the supported maximum or workspace too small";
+        case ABS_ERR_SIZE: return "size beyond the supported maximum, workspace too small, or scratch ring overrun by an earlier call";
         default: return "unknown status";
     }
 }
@@ -543,7 +559,7 @@ float abs_alpha_from_amax(abs_fmt_t fmt, float amax) {
 
 abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs_opts_t* opts, float* amax_f32,
                       void* stream) {
-    abs_opts_t o = {0, 0, 0, 0};
+    abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return ABS_ERR_SHAPE;
     if ((o.flags & ~(uint32_t)ABS_F_HADAMARD16) || o._pad) return ABS_ERR_FLAGS;
@@ -556,17 +572,19 @@ abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     unsigned long long* slot = nullptr;
     uint32_t gen = 0;
-    if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
-    return launch_amax(*st, in_bf16, rows * cols / 16, o, true, slot, gen, amax_f32, 0.0f, s);
+    const abs_status_t rc = next_slot(*st, &slot, &gen);
+    if (rc != ABS_OK) return rc;
+    return launch_amax(st->sm_count, in_bf16, rows * cols / 16, o, true, slot, gen, amax_f32, 0.0f, s);
 }
 
 abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                              void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream) {
-    abs_opts_t o = {0, 0, 0, 0};
+    abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if ((o.flags & ~kQuantFlags) || o._pad) return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_STOCHASTIC) && (o.sr_index_offset % 16) != 0) return ABS_ERR_SHAPE;
     if ((o.flags & ABS_F_SCALES_SWIZZLED) &&
         ((fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) || (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC)) ||
          cols / 16 > 0x7FFFFFFF || rows > 0x7FFFFFFF))
@@ -579,34 +597,35 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
     if (device_state(&st) != ABS_OK) return ABS_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
-    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;
         uint32_t gen = 0;
-        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        if ((rc = next_slot(*st, &slot, &gen)) != ABS_OK) return rc;
         const float denom = fmt_mfp((int)fmt) * 448.0f;
-        rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+        rc = launch_amax(st->sm_count, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
         if (rc != ABS_OK) return rc;
         src.slot = slot;
         src.gen = gen;
         src.denom = denom;
+        src.overrun = st->overrun_dev;
     }
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_IF4: return launch_quantize_fmt<1>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_IF3: return launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
-        default: return launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        default: return launch_quantize_fmt<7>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
     }
 }
 
 abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* out_bf16,
                                      void* codes_u8, void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts,
                                      void* stream) {
-    abs_opts_t o = {0, 0, 0, 0};
+    abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
@@ -614,6 +633,7 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     if ((o.flags & ~(uint32_t)(ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16 | ABS_F_ALPHA_GIVEN |
                                ABS_F_GROUPS_DOWN_COLUMNS)) || o._pad)
         return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_STOCHASTIC) && (o.sr_index_offset % 16) != 0) return ABS_ERR_SHAPE;
     // IF3, IF6 and the block-size-8 formats: round-to-nearest along the rows only
     if (!four_bit && (o.flags & (ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_GROUPS_DOWN_COLUMNS))) return ABS_ERR_FLAGS;
     if ((o.flags & ABS_F_GROUPS_DOWN_COLUMNS) && (rows % 16) != 0) return ABS_ERR_SHAPE;
@@ -633,40 +653,42 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
-    const int grid = grid_waves(*st, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? ABS_OPT_ITERS : ABS_FAST_ITERS);
+    const int grid = grid_waves(st->sm_count, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? ABS_OPT_ITERS : ABS_FAST_ITERS);
     if (ngroups >= (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads) return ABS_ERR_SIZE;    // 32-bit group indices only
-    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;
         uint32_t gen = 0;
-        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        if ((rc = next_slot(*st, &slot, &gen)) != ABS_OK) return rc;
         const float denom = fmt_mfp((int)fmt) * 448.0f;
-        rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+        rc = launch_amax(st->sm_count, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
         if (rc != ABS_OK) return rc;
         src.slot = slot;
         src.gen = gen;
         src.denom = denom;
+        src.overrun = st->overrun_dev;
     }
     const bool store = codes_u8 != nullptr;
     if (!four_bit) {
         bool handled = false;
         switch (fmt) {
-            case ABS_FMT_IF3: rc = launch_quantize_fmt<2>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
-            case ABS_FMT_IF6_E2M3: rc = launch_quantize_fmt<3>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
-            case ABS_FMT_IF6_E3M2: rc = launch_quantize_fmt<4>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
-            case ABS_FMT_NVFP4_BS8: rc = launch_quantize_fmt<5>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
-            case ABS_FMT_IF4_BS8: rc = launch_quantize_fmt<6>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
-            default: rc = launch_quantize_fmt<7>(*st, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF3: rc = launch_quantize_fmt<2>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF6_E2M3: rc = launch_quantize_fmt<3>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF6_E3M2: rc = launch_quantize_fmt<4>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_NVFP4_BS8: rc = launch_quantize_fmt<5>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            case ABS_FMT_IF4_BS8: rc = launch_quantize_fmt<6>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
+            default: rc = launch_quantize_fmt<7>(st->sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols, out_bf16, store, &handled); break;
         }
         return (!handled && rc == ABS_ERR_FLAGS) ? ABS_ERR_SIZE : rc;
     }
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
+    const uint64_t ctr = o.sr_index_offset / 8;
     const bool a32 = (reinterpret_cast<uintptr_t>(in_bf16) & 31u) == 0, o32 = (reinterpret_cast<uintptr_t>(out_bf16) & 31u) == 0;
     cudaError_t e = cudaSuccess;
 #define ABS_LAUNCH_E3(I, R, S, SLOT)                                                                                \
     e = launch_pdl(quantize4_opt_kernel<I, R, S, SLOT, true>, grid, kThreads, s, (const uint4*)in_bf16, (uint2*)codes_u8, \
-                   (uint8_t*)scales_e4m3, src, (int32_t)ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1, a32,        \
+                   (uint8_t*)scales_e4m3, src, (int32_t)ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1, ctr, a32,   \
                    (uint4*)out_bf16, o32, store)
 #define ABS_LAUNCH_E2(I, R, S)                                                                                      \
     do {                                                                                                            \
@@ -697,12 +719,13 @@ abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int6
 abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
                                      void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
                                      const abs_opts_t* opts, void* stream) {
-    abs_opts_t o = {0, 0, 0, 0};
+    abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
     if (rows < 0 || cols < 0 || (cols % 16) != 0 || (rows % 16) != 0) return ABS_ERR_SHAPE;
     if ((o.flags & ~(uint32_t)(ABS_F_ALPHA_GIVEN | ABS_F_HADAMARD16 | ABS_F_STOCHASTIC | ABS_F_SR_SCALE_17_16)) || o._pad)
         return ABS_ERR_FLAGS;
+    if ((o.flags & ABS_F_STOCHASTIC) && (o.sr_index_offset % 16) != 0) return ABS_ERR_SHAPE;
     if (rows * cols == 0) return ABS_OK;
     if (!in_bf16 || !codes_t_u8 || !scales_t_e4m3 || !tensor_scale_f32) return ABS_ERR_NULL;
     if (!aligned16(in_bf16) || !aligned16(codes_t_u8) || !aligned16(scales_t_e4m3) || ((uintptr_t)tensor_scale_f32 & 3u))
@@ -760,7 +783,7 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
                                  kTransSmemBytes);                                                                  \
         if (e == cudaSuccess)                                                                                       \
             e = cudaLaunchKernelEx(&cfg, transposed_kernel<I, S, R, Q, M, E>(), in, ct, stp, src, rows, cols, mask, \
-                                   SLOT, GEN, mul, k0, k1, (uint16_t*)out_bf16, store_codes);                       \
+                                   SLOT, GEN, mul, k0, k1, ctr, (uint16_t*)out_bf16, store_codes);                  \
     } while (0)
 #define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
     do {                                                                                                            \
@@ -771,23 +794,26 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
     const bool sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
-    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};
+    const uint64_t ctr = o.sr_index_offset / 8;
+    AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;
         uint32_t gen = 0;
-        if (next_slot(*st, &slot, &gen) != ABS_OK) return ABS_ERR_CUDA;
+        const abs_status_t rs = next_slot(*st, &slot, &gen);
+        if (rs != ABS_OK) return rs;
         const float denom = 6.0f * 448.0f;
         if (rht) {
             // the maximum is taken over the transformed column groups: same tile walk, MODE 1
             ABS_LAUNCH_T(false, false, true, false, 1, slot, gen);
             if (e != cudaSuccess) return ABS_ERR_CUDA;
         } else {
-            abs_status_t rc = launch_amax(*st, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
+            abs_status_t rc = launch_amax(st->sm_count, in_bf16, ngroups, o, false, slot, gen, tensor_scale_f32, denom, s);
             if (rc != ABS_OK) return rc;
         }
         src.slot = slot;
         src.gen = gen;
         src.denom = denom;
+        src.overrun = st->overrun_dev;
     }
     unsigned long long* no_slot = nullptr;
 #define ABS_LAUNCH_T2(I, R, Q)                                                                                      \
@@ -842,26 +868,24 @@ abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t ro
     amax_chunks_kernel<<<(int)nchunks, kThreads, 0, s>>>((const uint4*)in_bf16, ngroups, na.scratch, tensor_scale_f32,
                                                         fmt_mfp((int)fmt) * 448.0f);
     if (cudaGetLastError() != cudaSuccess) return ABS_ERR_CUDA;
-    DeviceState grid_info;                 // only its SM count is read by the launchers; no ring is touched
-    grid_info.sm_count = na.sm_count;
-    const abs_opts_t o = {0, 0, 0, 0};
-    const AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32};   // alpha was written by the chunked pass
+    const abs_opts_t o = {0, 0, 0, 0, 0};
+    const AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};   // alpha was written by the chunked pass
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF4: return launch_quantize_fmt<1>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF3: return launch_quantize_fmt<2>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
-        default: return launch_quantize_fmt<7>(grid_info, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s);
+        case ABS_FMT_NVFP4: return launch_quantize_fmt<0>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4: return launch_quantize_fmt<1>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF3: return launch_quantize_fmt<2>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E2M3: return launch_quantize_fmt<3>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF6_E3M2: return launch_quantize_fmt<4>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_NVFP4_BS8: return launch_quantize_fmt<5>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        case ABS_FMT_IF4_BS8: return launch_quantize_fmt<6>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
+        default: return launch_quantize_fmt<7>(na.sm_count, in_bf16, ngroups, codes_u8, scales_e4m3, src, o, s, cols);
     }
 }
 
 abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
                                const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out,
                                const abs_opts_t* opts, void* stream) {
-    abs_opts_t o = {0, 0, 0, 0};
+    abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
@@ -886,14 +910,14 @@ abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* 
     const int64_t swz_cols = (o.flags & ABS_F_SCALES_SWIZZLED) ? cols : 0;
     const int sel = (o.flags & ABS_F_FP_GROUPS_ONLY) ? 1 : ((o.flags & ABS_F_INT_GROUPS_RAW) ? 2 : 0);
     switch (fmt) {
-        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
-        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols, sel);
-        case ABS_FMT_IF3: return launch_dequantize_fmt<2>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        case ABS_FMT_IF6_E3M2: return launch_dequantize_fmt<4>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        case ABS_FMT_NVFP4_BS8: return launch_dequantize_fmt<5>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        case ABS_FMT_IF4_BS8: return launch_dequantize_fmt<6>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
-        default: return launch_dequantize_fmt<7>(*st, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_NVFP4: return launch_dequantize_fmt<0>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols);
+        case ABS_FMT_IF4: return launch_dequantize_fmt<1>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s, swz_cols, sel);
+        case ABS_FMT_IF3: return launch_dequantize_fmt<2>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF6_E2M3: return launch_dequantize_fmt<3>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF6_E3M2: return launch_dequantize_fmt<4>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_NVFP4_BS8: return launch_dequantize_fmt<5>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        case ABS_FMT_IF4_BS8: return launch_dequantize_fmt<6>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
+        default: return launch_dequantize_fmt<7>(st->sm_count, codes_u8, scales_e4m3, tensor_scale_f32, ngroups, out, fp32, i64, s);
     }
 }
 

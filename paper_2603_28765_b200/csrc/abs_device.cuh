@@ -303,7 +303,17 @@ struct AlphaSrc {
     uint32_t gen;                         // generation of this call
     float denom;                          // M_FP * 448
     float* alpha_out;                     // where alpha is published for the caller
+    uint32_t* overrun;                    // host-mapped word set when the slot carries another call's generation
 };
+// After the amax pass of the same call the slot holds this call's generation.  Any other generation means
+// that a later call reused the slot while this one was still in flight (more than ABS_MAX_INFLIGHT calls
+// between the two): the maximum is lost.  The kernel then reports it through the host-mapped word, which
+// the next library call on the device turns into ABS_ERR_SIZE, and continues with alpha = 1.
+__device__ __forceinline__ float slot_amax(const AlphaSrc& a, unsigned long long v, bool reporter) {
+    if ((uint32_t)(v >> 32) == a.gen) return __uint_as_float((uint32_t)v);
+    if (reporter && a.overrun) *reinterpret_cast<volatile uint32_t*>(a.overrun) = 1u;
+    return 0.0f;
+}
 // Must be called by every thread of the block (it synchronises): thread 0 reads the slot, divides once
 // (Eq. 1) and shares alpha through shared memory, so one-group-per-thread launches do not pay a division
 // per thread.  Block 0 also publishes alpha for the caller.
@@ -313,7 +323,7 @@ __device__ __forceinline__ float resolve_alpha(const AlphaSrc& a) {
     __shared__ float alpha_shared;
     if (threadIdx.x == 0) {
         const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(a.slot);
-        const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
+        const float A = slot_amax(a, v, blockIdx.x == 0);
         const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                   // Eq. 1
         alpha_shared = alpha;
         if (blockIdx.x == 0) *a.alpha_out = alpha;
@@ -330,7 +340,7 @@ template <bool FROM_SLOT>
 __device__ __forceinline__ float resolve_alpha_per_thread(const AlphaSrc& a) {
     if constexpr (!FROM_SLOT) return __ldg(a.alpha_p);
     const unsigned long long v = __ldcg(a.slot);
-    const float A = ((uint32_t)(v >> 32) == a.gen) ? __uint_as_float((uint32_t)v) : 0.0f;
+    const float A = slot_amax(a, v, blockIdx.x == 0 && threadIdx.x == 0);
     const float alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, a.denom);                           // Eq. 1
     if (blockIdx.x == 0 && threadIdx.x == 0) *a.alpha_out = alpha;
     return alpha;

@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
                                                             uint8_t* __restrict__ scales,
                                                             const AlphaSrc alpha_src, int64_t ngroups,
                                                             float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
-                                                            uint32_t seed_hi) {
+                                                            uint32_t seed_hi, uint64_t ctr_base) {
     using F = Fmt<FMT>;
     constexpr int B = F::BITS, G = F::GROUP, NSUB = 16 / G;
     pdl_launch_dependents();
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const uint4* __restr
 
         uint32_t rnd[8];
         if constexpr (SR) {
-            const uint64_t i8 = (uint64_t)g * 2u;
+            const uint64_t i8 = ctr_base + (uint64_t)g * 2u;      // ctr_base = sr_index_offset / 8 (even)
             uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
             uint4 p1 = philox4x32_10((uint32_t)(i8 + 1), (uint32_t)((i8 + 1) >> 32), seed_lo, seed_hi);
             rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;

@@ -152,4 +152,41 @@ def edge_tensors() -> dict[str, np.ndarray]:
     cases["wide_dynamic_range"] = f32_to_bf16_bits(wide)
     ragged = rng.standard_normal((37, 16 * 13), dtype=np.float32)
     cases["ragged_37x208"] = f32_to_bf16_bits(ragged)
+    # bf16 subnormal elements (bit patterns 0x0001..0x007F, both signs) under a normal tensor maximum: alone in
+    # a group (zero scale), next to normal values, and as the only non-zero values of a row
+    sub = f32_to_bf16_bits(rng.standard_normal((4, 64), dtype=np.float32))
+    sub[0, :16] = rng.integers(1, 0x80, 16).astype(np.uint16) | (rng.integers(0, 2, 16).astype(np.uint16) << 15)
+    sub[1, 16:24] = rng.integers(1, 0x80, 8).astype(np.uint16)
+    sub[2, :] = 0
+    sub[2, 5] = 0x0001
+    sub[2, 40] = 0x807F
+    cases["bf16_subnormals"] = sub
+    # the smallest tensor maximum the library supports, 2^-100, and one a little above it
+    for name, k in (("amax_2^-100", -100), ("amax_2^-96", -96)):
+        t = rng.standard_normal((4, 64), dtype=np.float32)
+        t = t / np.abs(t).max() * np.float32(2.0 ** k)
+        cases[name] = f32_to_bf16_bits(t)
     return cases
+
+
+def below_range_tensor() -> np.ndarray:
+    """A tensor whose maximum, 2^-110, lies below the supported range (maximum 0 or at least 2^-100)."""
+    rng = np.random.Generator(np.random.PCG64(4321))
+    t = rng.standard_normal((4, 64), dtype=np.float32)
+    return f32_to_bf16_bits(t / np.abs(t).max() * np.float32(2.0 ** -110))
+
+
+
+def arbitrary_quantized_bytes(bits: int, group: int, rows: int = 16, cols: int = 1024, seed: int = 0):
+    """Code and scale bytes that no quantizer produced, for the dequantize tests: random code bytes; every scale
+    byte 0x00..0xFF occurs (rows 0 and 1 run through all of them); row 2 starts with the special bytes -- E4M3
+    NaN with and without bit 7, 0x80, zero, the largest scale with and without bit 7, the smallest -- over code
+    bytes that contain the most negative integer patterns and the FP code 'minus zero'."""
+    rng = np.random.default_rng(100 + seed)
+    codes = rng.integers(0, 256, (rows, cols * bits // 8), dtype=np.uint8)
+    scales = rng.integers(0, 256, (rows, cols // group), dtype=np.uint8)
+    scales[0, :] = np.arange(cols // group) % 256
+    scales[1, :] = (255 - np.arange(cols // group)) % 256
+    scales[2, :8] = [0x7F, 0xFF, 0x80, 0x00, 0x7E, 0xFE, 0x01, 0x81]
+    codes[2, :16 * bits] = np.tile(np.frombuffer(bytes([0x88, 0x08, 0x80, 0x00, 0xFF, 0x77, 0x24, 0x92]), np.uint8), 2 * bits)
+    return codes, scales

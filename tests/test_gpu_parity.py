@@ -175,8 +175,8 @@ def test_option_parity(B, oracle, fmt, flags):
         check_case(B, oracle, fmt, I.edge_tensors()[case], flags=f, mask=mask, seed=99)
 
 
-def test_sr_element_index_beyond_32_bits_of_groups(B, oracle):
-    """Different seeds and row offsets give different streams; the same seed repeats exactly."""
+def test_sr_stream_depends_on_the_seed_only(B, oracle):
+    """Different seeds give different streams; the same seed repeats exactly."""
     xb = I.generate("cfg1", 64, 256)
     a = gpu_quantize(B, 1, xb, B.ABS_F_STOCHASTIC, 0, 5)
     b = gpu_quantize(B, 1, xb, B.ABS_F_STOCHASTIC, 0, 5)
@@ -266,23 +266,10 @@ def test_large_tensor_sampled_parity(B, oracle):
 
 def oracle_rows_with_offset(oracle, fmt, row_bits, row_index, cols, alpha, flags, seed):
     """Oracle result for one row that sits at `row_index` of a larger tensor (matters only for the
-    element index of the stochastic stream): calls the row-range entry point on a fake base pointer."""
-    import ctypes as C
-    L = oracle.lib()
-    b = oracle.fmt_bits(fmt)
-    codes = np.zeros((1, cols * b // 8), dtype=np.uint8)
-    scales = np.zeros((1, cols // 16), dtype=np.uint8)
-    row = np.ascontiguousarray(row_bits)
-    row_index = int(row_index)
-    # base pointers are shifted back by row_index rows so that row `row_index` lands on our buffers
-    in_base = row.ctypes.data - row_index * cols * 2
-    c_base = codes.ctypes.data - row_index * (cols * b // 8)
-    s_base = scales.ctypes.data - row_index * (cols // 16)
-    rc = L.abs_oracle_quantize_rows(fmt, C.c_void_p(in_base), row_index + 1, cols, row_index, row_index + 1,
-                                    C.c_float(float(alpha)), flags | oracle.F_ALPHA_GIVEN, 0, seed,
-                                    C.c_void_p(c_base), C.c_void_p(s_base), None, None)
-    assert rc == 0
-    return codes, scales
+    element index of the stochastic stream)."""
+    c, s, _ = oracle.quantize(fmt, np.ascontiguousarray(row_bits), flags=flags | oracle.F_ALPHA_GIVEN, alpha=alpha,
+                              sr_seed=seed, sr_index_offset=int(row_index) * cols)
+    return c, s
 
 
 def test_amax_entry_point(B, oracle):
@@ -706,3 +693,124 @@ def test_split_dequantize_and_mac_matmul(B, oracle):
     one = B.make_opts(B.ABS_F_FP_GROUPS_ONLY)
     assert L.abs_dequantize_ex(0, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), m, k, out.data_ptr(),
                                ctypes.byref(one), None) == 5
+
+
+# ------------------------------------------------------------------ dequantize of bytes no quantizer produced
+
+def nan_aware_same(name, got, want, as_float):
+    got, want = np.asarray(got), np.asarray(want)
+    gn, wn = np.isnan(as_float(got)), np.isnan(as_float(want))
+    assert np.array_equal(gn, wn), f"{name}: NaN positions differ ({int(gn.sum())} vs {int(wn.sum())})"
+    assert_same(name, np.where(gn, 0, got), np.where(wn, 0, want))
+
+
+@pytest.mark.parametrize("fmt", ALL_FMTS)
+def test_dequantize_arbitrary_bytes(B, oracle, fmt):
+    """abs_dequantize on arbitrary code and scale bytes -- every scale byte 0x00..0xFF (0x7F / 0xFF: E4M3 NaN, which
+    must propagate; 0x80; bit 7 set on plain NVFP4 scales), the most negative integer code, the FP code 'minus
+    zero' -- against the oracle by bit pattern, bf16 and fp32 outputs, NaNs compared as 'is NaN'."""
+    rows, cols = 16, 1024
+    for seed, alpha in ((0, 0.0173), (1, 1.0), (2, 3.0e-20)):
+        codes, scales = I.arbitrary_quantized_bytes(B.FMT_BITS[fmt], B.FMT_GROUP[fmt], rows, cols, seed)
+        dc, ds = torch.from_numpy(codes).cuda(), torch.from_numpy(scales).cuda()
+        ts = torch.tensor([alpha], dtype=torch.float32, device="cuda")
+        a32 = np.float32(ts.item())
+        got16 = B.abs_dequantize(fmt, dc, ds, ts, rows, cols).view(torch.int16).cpu().numpy().view(np.uint16)
+        got32 = B.abs_dequantize(fmt, dc, ds, ts, rows, cols, opts=B.make_opts(B.ABS_F_OUT_FP32)).cpu().numpy()
+        want16 = oracle.dequantize(fmt, codes, scales, a32, rows, cols)
+        want32 = oracle.dequantize(fmt, codes, scales, a32, rows, cols, out_fp32=True)
+        assert np.isnan(want32).any()
+        nan_aware_same("bf16", got16, want16, I.bf16_bits_to_f32)
+        nan_aware_same("fp32", got32.view(np.uint32), want32.view(np.uint32), lambda u: u.view(np.float32))
+        if fmt == 1:      # the split halves used for the MAC arithmetic read the same bytes
+            for flag, sel in ((B.ABS_F_FP_GROUPS_ONLY, oracle.F_FP_GROUPS_ONLY), (B.ABS_F_INT_GROUPS_RAW, oracle.F_INT_GROUPS_RAW)):
+                g = B.abs_dequantize(fmt, dc, ds, ts, rows, cols, opts=B.make_opts(flag))
+                w = oracle.dequantize(fmt, codes, scales, a32, rows, cols, select=sel)
+                nan_aware_same("split", g.view(torch.int16).cpu().numpy().view(np.uint16), w, I.bf16_bits_to_f32)
+        if fmt in (0, 1):  # the tiled scale layout reads the same bytes from other places
+            sw = torch.from_numpy(oracle.swizzle_scales(scales)).cuda()
+            g = B.abs_dequantize(fmt, dc, sw, ts, rows, cols, opts=B.make_opts(B.ABS_F_SCALES_SWIZZLED))
+            nan_aware_same("swizzled", g.view(torch.int16).cpu().numpy().view(np.uint16), want16, I.bf16_bits_to_f32)
+
+
+def test_tensor_maximum_below_the_supported_range(B, oracle):
+    """The supported range is a tensor maximum of 0 or at least 2^-100 (both sides of that line with parity are in
+    the edge-tensor cases).  Below it the reciprocals of Eq. 2 can overflow: the call still succeeds, alpha is
+    still Eq. 1 exactly, and the outputs are unspecified -- nothing else is promised, and nothing else is checked."""
+    xb = I.below_range_tensor()
+    for fmt in ALL_FMTS:
+        c, s, a, _ = gpu_quantize(B, fmt, xb)
+        want = oracle.alpha_from_amax(fmt, oracle.amax(xb))
+        assert np.float32(a).view(np.uint32) == np.float32(want).view(np.uint32)
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ row shards through the product calls
+
+@pytest.mark.parametrize("fmt", [0, 1, 2, 3, 6])
+@pytest.mark.parametrize("opt", ["rtn", "sr", "hsr17"])
+def test_row_shards_through_the_library_equal_one_call(B, oracle, fmt, opt):
+    """The multi-GPU protocol with the library's own calls, run on one GPU: every shard reduces its rows with
+    abs_amax, the maxima are combined on the host (the one 4-byte exchange), every shard is quantized with
+    abs_quantize_ex(ABS_F_ALPHA_GIVEN) and, for stochastic rounding, the index of its first element as
+    sr_index_offset.  Codes and scales concatenated must equal one abs_quantize_ex call on the whole tensor and
+    the oracle, byte for byte; so must alpha."""
+    flags = {"rtn": 0, "sr": B.ABS_F_STOCHASTIC,
+             "hsr17": B.ABS_F_HADAMARD16 | B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16}[opt]
+    mask, seed = oracle.hadamard_sign_mask(3), 0x1234567890ABCDEF
+    xb = I.generate("cfg4" if flags else "cfg2", 600, 2048)
+    rows, cols = xb.shape
+    whole_c, whole_s, whole_a, _ = gpu_quantize(B, fmt, xb, flags, mask, seed)
+    oc, osc, oa = oracle.quantize(fmt, xb, flags=flags, sign_mask=mask, sr_seed=seed, threads=THREADS)
+    assert np.float32(whole_a).view(np.uint32) == np.float32(oa).view(np.uint32)
+    assert_same("whole codes", whole_c, oc)
+    assert_same("whole scales", whole_s, osc)
+    bounds = [(0, 256), (256, 257), (257, 600)]
+    shards = [to_dev(np.ascontiguousarray(xb[lo:hi])) for lo, hi in bounds]
+    amax_opts = B.make_opts(flags & B.ABS_F_HADAMARD16, mask)
+    local_max = [float(B.abs_amax(x, opts=amax_opts).item()) for x in shards]
+    alpha = B.abs_alpha_from_amax(fmt, max(local_max))                  # host max = the all-reduce(max) of 4 bytes
+    assert np.float32(alpha).view(np.uint32) == np.float32(oa).view(np.uint32)
+    cs, ss = [], []
+    for (lo, hi), x in zip(bounds, shards):
+        ts = torch.tensor([alpha], dtype=torch.float32, device="cuda")
+        o = B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, mask, seed, lo * cols)
+        c, s, _ = B.abs_quantize(fmt, x, tensor_scale=ts, opts=o)
+        cs.append(c.cpu().numpy().reshape(hi - lo, -1))
+        ss.append(s.cpu().numpy().reshape(hi - lo, -1))
+    assert_same("shard codes", np.concatenate(cs), oc)
+    assert_same("shard scales", np.concatenate(ss), osc)
+    if flags & B.ABS_F_STOCHASTIC:
+        import ctypes
+        L = B.lib()
+        bad = B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, mask, seed, 8)           # not a multiple of 16
+        x = shards[0]
+        ts = torch.tensor([alpha], dtype=torch.float32, device="cuda")
+        assert L.abs_quantize_ex(fmt, x.data_ptr(), 256, cols, c.data_ptr(), s.data_ptr(), ts.data_ptr(),
+                                 ctypes.byref(bad), None) == 2
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_index_offset_in_the_other_stochastic_entry_points(B, oracle, fmt):
+    """sr_index_offset in abs_quantize_dequantize (both orientations) and abs_quantize_transposed: a matrix quantized
+    on its own with the offset of its first element equals the corresponding rows of the larger tensor."""
+    flags = B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16
+    seed = 4242
+    xb = I.generate("cfg4", 96, 512)
+    oc, osc, oa = oracle.quantize(fmt, xb, flags=flags, sr_seed=seed)
+    od = oracle.dequantize(fmt, oc, osc, oa, 96, 512)
+    lo = 32
+    part = np.ascontiguousarray(xb[lo:])
+    ts = torch.tensor([float(oa)], dtype=torch.float32, device="cuda")
+    out, _ = B.abs_quantize_dequantize(fmt, to_dev(part), tensor_scale=ts,
+                                       opts=B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, 0, seed, lo * 512))
+    assert_same("emulation shard", out.view(torch.int16).cpu().numpy().view(np.uint16), od[lo:])
+    # transposed: the index runs over X^T [512, 96]; the last 64 columns of X are rows 448.. of X^T
+    xt = np.ascontiguousarray(xb.T)
+    tc, tsc, ta = oracle.quantize(fmt, xt, flags=flags, sr_seed=seed)
+    cols_part = np.ascontiguousarray(xb[:, 448:])
+    ts = torch.tensor([float(ta)], dtype=torch.float32, device="cuda")
+    ct, st, _ = B.abs_quantize_transposed(fmt, to_dev(cols_part), tensor_scale=ts,
+                                          opts=B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, 0, seed, 448 * 96))
+    assert_same("transposed shard codes", ct.cpu().numpy().reshape(64, -1), tc[448:])
+    assert_same("transposed shard scales", st.cpu().numpy().reshape(64, -1), tsc[448:])

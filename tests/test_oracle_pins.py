@@ -95,13 +95,13 @@ def test_table1_mse_normal(oracle):
         c, s, a = oracle.quantize(fmt, xb, threads=4)
         d = oracle.dequantize(fmt, c, s, a, 1024, 1024, out_fp32=True, threads=4).astype(np.float64)
         mse = np.mean((d - xf) ** 2) * 1e3
-        assert abs(mse - float(g[name][0])) < 0.12, (name, mse)
+        assert abs(mse - float(g[name][0])) < 0.1, (name, mse)
     # the per-group error sums of the two candidates (steps 5-6 and 8-9 of Fig. 3a), before selection: the FP
     # candidate alone is NVFP4, the integer candidate alone is NVINT4 up to where the E4M3 rounding falls
     c, s, a, e_fp, e_int = oracle.quantize(1, xb, threads=4, debug=True)
-    assert abs(e_fp.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVFP4"][0])) < 0.12
-    assert abs(e_int.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVINT4"][0])) < 0.12
-    assert abs(np.minimum(e_fp, e_int).astype(np.float64).sum() / xb.size * 1e3 - float(g["IF4"][0])) < 0.12
+    assert abs(e_fp.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVFP4"][0])) < 0.1
+    assert abs(e_int.astype(np.float64).sum() / xb.size * 1e3 - float(g["NVINT4"][0])) < 0.1
+    assert abs(np.minimum(e_fp, e_int).astype(np.float64).sum() / xb.size * 1e3 - float(g["IF4"][0])) < 0.1
 
 
 def test_format_facts(oracle):
@@ -284,7 +284,6 @@ def test_selection_invariants(oracle, fmt, case):
     flag = (s >> 7).astype(bool)
     # chosen error <= other error; integer only if strictly smaller (step 10)
     assert np.all(eint[flag] < efp[flag])
-    assert np.all(efp[~flag] <= eint[~flag]) or np.all(np.isfinite(eint[~flag]) | True)
     assert np.all(~(eint[~flag] < efp[~flag]))
     # the byte 0x80 ("minus zero scale") never appears; zero scale means all-zero codes
     assert not np.any(s == 0x80)
@@ -799,3 +798,151 @@ def test_mac_constants_and_reference(oracle):
     da = oracle.dequantize(1, *qa, 32, 256, out_fp32=True).astype(np.float64)
     db = oracle.dequantize(1, *qb, 48, 256, out_fp32=True).astype(np.float64)
     assert np.abs(ref - da @ db.T).max() <= 1e-5 * np.abs(ref).max()    # cancellation: compare on the result's scale
+
+
+# --------------------------------------------------------------------------- dequantize on arbitrary bytes
+
+BASE_FMT = {0: 0, 1: 1, 2: 2, 3: 3, 4: 4, 5: 0, 6: 1, 7: 2}       # block-size-8 variants share their sibling's element format
+
+
+def dequantize_by_definition(oracle, fmt, codes, scales, alpha, rows, cols):
+    """Sec. 3 and Sec. 4.1 written out with numpy and library casts, for ANY byte values:
+    element = value(code) * Delta * alpha, times M_FP / M_INT for an integer group, product in FP32, then BF16.
+      - Delta: torch's float8_e4m3fn decode of the scale byte's low seven bits (0x7F is NaN by that format);
+      - the group is an integer group iff the format has an integer alternative and bit 7 of the byte is set
+        (Sec. 3: the flag sits in the sign bit an NVFP4 scale leaves unused, so plain NVFP4 ignores it);
+      - FP codes: sign | index into the format's magnitude grid; integer codes: two's complement in b bits
+        (Sec. 3 footnote: the most negative pattern is given up by the encoder, the decoder still reads it);
+      - BF16 rounding: torch's cast."""
+    torch = pytest.importorskip("torch")
+    base = BASE_FMT[fmt]
+    b, G = oracle.fmt_bits(fmt), oracle.fmt_group(fmt)
+    has_int = base != 0
+    e4 = torch.arange(128, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+    grid = np.array(fp_grid(base), dtype=np.float32)
+    code = np.stack([unpack_bitstream(row, b) for row in np.asarray(codes).reshape(rows * cols // 16, 2 * b)])
+    code = code.reshape(rows, cols).astype(np.int64)
+    sb = np.repeat(np.asarray(scales, dtype=np.uint8).reshape(rows, cols // G), G, axis=1).astype(np.int64)
+    flag = (sb >> 7).astype(bool) if has_int else np.zeros_like(sb, dtype=bool)
+    with np.errstate(invalid="ignore"):
+        d = e4[sb & 0x7F] * np.float32(alpha)
+        if has_int:
+            c_post = np.float32(oracle.m_fp(fmt)) / np.float32(oracle.m_int(fmt))
+            d = np.where(flag, d * c_post, d).astype(np.float32)
+        v_fp = grid[code & ((1 << (b - 1)) - 1)] * np.where(code >> (b - 1), np.float32(-1), np.float32(1))
+        v_int = np.where(code >= (1 << (b - 1)), code - (1 << b), code).astype(np.float32)
+        out32 = (np.where(flag, v_int, v_fp).astype(np.float32) * d).astype(np.float32)
+    bf = torch.from_numpy(out32.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    return out32, bf
+
+
+def same_bits_or_both_nan(got, want, as_float):
+    g, w = np.asarray(got), np.asarray(want)
+    gn, wn = np.isnan(as_float(g)), np.isnan(as_float(w))
+    return np.array_equal(gn, wn) and np.array_equal(g[~gn], w[~wn])
+
+
+@pytest.mark.parametrize("fmt", [0, 1, 2, 3, 4, 5, 6, 7])
+def test_dequantize_arbitrary_bytes_against_definition(oracle, fmt):
+    """Bytes the quantizer never produces decode as the formats define them: scale 0x7F / 0xFF is the E4M3 NaN
+    and propagates, 0x80 is a zero scale with the flag set, the most negative integer code is plain two's
+    complement, the FP code 'minus zero' gives -0, and plain NVFP4 ignores bit 7 of its scale bytes."""
+    rows, cols, alpha = 16, 1024, np.float32(0.0173)
+    codes, scales = I.arbitrary_quantized_bytes(oracle.fmt_bits(fmt), oracle.fmt_group(fmt), rows, cols)
+    want32, want16 = dequantize_by_definition(oracle, fmt, codes, scales, alpha, rows, cols)
+    got32 = oracle.dequantize(fmt, codes, scales, alpha, rows, cols, out_fp32=True)
+    got16 = oracle.dequantize(fmt, codes, scales, alpha, rows, cols)
+    assert np.isnan(want32).any() and (want32 == 0).any()
+    assert same_bits_or_both_nan(got32.view(np.uint32), want32.view(np.uint32), lambda u: u.view(np.float32))
+    assert same_bits_or_both_nan(got16, want16, I.bf16_bits_to_f32)
+    # the named cases, one by one (IF4): most negative code under an integer flag, -0 under an FP flag
+    if fmt == 1:
+        c = np.zeros((1, 8), np.uint8)
+        c[0, 0] = 0x88                                              # nibbles 8, 8
+        out = oracle.dequantize(1, c, np.array([[0xC8]], np.uint8), 1.0, 1, 16, out_fp32=True)   # flag | E4M3(4.0)
+        assert out[0, 0] == np.float32(-8) * (np.float32(4) * (np.float32(6) / np.float32(7)))
+        out = oracle.dequantize(1, c, np.array([[0x48]], np.uint8), 1.0, 1, 16, out_fp32=True)   # same byte, FP group
+        assert out[0, 0] == 0 and np.signbit(out[0, 0])
+        assert np.isnan(oracle.dequantize(1, c, np.array([[0xFF]], np.uint8), 1.0, 1, 16, out_fp32=True)).all()
+
+
+# --------------------------------------------------------------------------- order of the error sums
+
+def _round_to_f32(q):
+    """Exact rational -> nearest binary32 (ties to even, subnormals kept) by integer arithmetic."""
+    from fractions import Fraction
+    if q == 0:
+        return Fraction(0)
+    sign, a = (-1 if q < 0 else 1), abs(q)
+    e = a.numerator.bit_length() - a.denominator.bit_length()        # 2^(e-1) <= a < 2^(e+1)
+    if Fraction(2) ** e > a:
+        e -= 1                                                        # now 2^e <= a < 2^(e+1)
+    ulp = Fraction(2) ** (max(e, -126) - 23)
+    n, rem = divmod(a, ulp)
+    if rem * 2 > ulp or (rem * 2 == ulp and n % 2 == 1):
+        n += 1
+    return sign * n * ulp
+
+
+def test_error_sum_order_is_four_fused_chains(oracle):
+    """The selection compares SUM16 of the squared errors.  Its order -- four fused multiply-add chains over the
+    elements {0,2,4,6}, {1,3,5,7}, {8,..,14}, {9,..,15}, then (S0 + S1) + (S2 + S3) -- is recomputed here in exact
+    rational arithmetic with one explicit rounding per operation, from the stored codes of each group, and must equal
+    the error the oracle reports for the chosen candidate bit for bit.  A plain left-to-right sum differs on many of
+    the same groups, so this test fails for a sequential implementation."""
+    from fractions import Fraction as Fr
+    xb = I.generate("cfg1", 8, 256)
+    rows, cols = xb.shape
+    c, s, a, efp, eint = oracle.quantize(1, xb, debug=True)
+    x = I.bf16_bits_to_f32(xb)
+    e4, grid = e4m3_grid(), fp_grid(1)
+    c_post = np.float32(6) / np.float32(7)
+    differs_from_sequential = 0
+    for r in range(rows):
+        for g in range(cols // 16):
+            sb = int(s[r, g])
+            if (sb & 0x7F) == 0:
+                continue
+            flag = sb >> 7
+            d = np.float32(e4[sb & 0x7F]) * np.float32(a)
+            if flag:
+                d = np.float32(d * c_post)
+            codes = unpack_bitstream(c[r, 8 * g: 8 * g + 8], 4)
+            errs = []
+            for j in range(16):
+                k = int(codes[j])
+                v = (k - 16 if k >= 8 else k) if flag else (-1 if k & 8 else 1) * grid[k & 7]
+                errs.append(_round_to_f32(Fr(v) * Fr(float(d)) - Fr(float(x[r, 16 * g + j]))))     # one fused rounding
+            chains = []
+            for first in (0, 1, 8, 9):
+                acc = Fr(0)
+                for j in range(first, first + 8, 2):
+                    acc = _round_to_f32(errs[j] * errs[j] + acc)
+                chains.append(acc)
+            total = _round_to_f32(_round_to_f32(chains[0] + chains[1]) + _round_to_f32(chains[2] + chains[3]))
+            reported = (eint if flag else efp)[r, g]
+            assert Fr(float(reported)) == total, (r, g, float(reported), float(total))
+            seq = Fr(0)
+            for j in range(16):
+                seq = _round_to_f32(errs[j] * errs[j] + seq)
+            differs_from_sequential += seq != total
+    assert differs_from_sequential > 20
+
+
+# --------------------------------------------------------------------------- row shards and the random stream
+
+def test_row_shards_with_index_offset_equal_the_whole_tensor(oracle):
+    """App. B's random stream runs over the whole tensor.  Quantizing row shards on their own, each with the index
+    of its first element as offset and the shared alpha, gives the bytes of the unsharded call."""
+    xb = I.generate("cfg4", 48, 256)
+    flags = oracle.F_STOCHASTIC | oracle.F_HADAMARD16 | oracle.F_SR_SCALE_17_16
+    for fmt in (0, 1, 2, 3, 6):
+        c, s, a = oracle.quantize(fmt, xb, flags=flags, sign_mask=0x1234, sr_seed=77)
+        parts = [oracle.quantize(fmt, np.ascontiguousarray(xb[lo:hi]), flags=flags | oracle.F_ALPHA_GIVEN, alpha=a,
+                                 sign_mask=0x1234, sr_seed=77, sr_index_offset=lo * 256)
+                 for lo, hi in ((0, 16), (16, 17), (17, 48))]
+        assert np.array_equal(np.concatenate([p[0] for p in parts]), c)
+        assert np.array_equal(np.concatenate([p[1] for p in parts]), s)
+        wrong = oracle.quantize(fmt, np.ascontiguousarray(xb[16:48]), flags=flags | oracle.F_ALPHA_GIVEN, alpha=a,
+                                sign_mask=0x1234, sr_seed=77)
+        assert not np.array_equal(wrong[0], c[16:48])                 # without the offset the stream restarts
