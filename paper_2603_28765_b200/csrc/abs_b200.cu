@@ -213,15 +213,19 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
             const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(sm_count, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(sm_count, ngroups, 5, ABS_NV_ITERS);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
-            const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)pgrid * kThreads;
+            // the kernel looks three grid strides past the current group (next group, and its L2 prefetch)
+            const bool i32 = !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - 3 * (int64_t)pgrid * kThreads;
             cudaError_t e;
             const bool swz = o.flags & ABS_F_SCALES_SWIZZLED;
             const uint32_t gpr = swz ? (uint32_t)(cols / 16) : 0u, ktiles = (gpr + 3u) / 4u;
+            // L2 prefetch ahead of the loads unless the amax pass of this call has just streamed an input that
+            // fits the L2 (about 100 MB of the 126 MB stay resident behind a streaming read)
+            const bool pf = !alpha.slot || ngroups * 32 > (int64_t)96 << 20;
 #define ABS_LAUNCH_F3(IDX, A32, SLOT, MUL)                                                                           \
     e = swz ? launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL, true>, pgrid, kThreads, s,                  \
-                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles)         \
+                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles, pf)     \
             : launch_pdl(quantize4_fast_kernel<kInt, IDX, A32, SLOT, MUL, false>, pgrid, kThreads, s,                 \
-                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles)
+                         (const uint4*)in, (uint2*)codes, (uint8_t*)scales, alpha, (IDX)ngroups, gpr, ktiles, pf)
 #define ABS_LAUNCH_F(IDX, A32)                                                                                       \
     do {                                                                                                             \
         if (alpha.slot && mul != 1.0f) ABS_LAUNCH_F3(IDX, A32, true, true);                                          \

@@ -146,6 +146,7 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (g < nblocks16) prefetch_l2(in + 2 * (size_t)g);                  // before the wait: see prefetch_l2
     pdl_wait();
     uint32_t w[8], wn[8];
     const bool active = g < nblocks16;
@@ -328,6 +329,7 @@ quantize6_fast_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (g < ngroups) prefetch_l2(in + 2 * (size_t)g);                  // before the wait: see prefetch_l2
     pdl_wait();
     uint32_t w[8], wn[8];
     const bool active = g < ngroups;
@@ -517,6 +519,7 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (g < ngroups) prefetch_l2(in + 2 * (size_t)g);                  // before the wait: see prefetch_l2
     pdl_wait();
     uint32_t w[8], wn[8];
     const bool active = g < ngroups;
@@ -639,6 +642,8 @@ __global__ void __launch_bounds__(256) dequantize3_fast_kernel(const uint16_t* _
     pdl_launch_dependents();
     const float c_post = __fdiv_rn(4.0f, 3.0f);
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    if ((int32_t)(blockIdx.x * blockDim.x + threadIdx.x) < nblocks16)        // before the wait: see prefetch_l2
+        prefetch_l2(codes + 3 * (size_t)(blockIdx.x * blockDim.x + threadIdx.x));
     pdl_wait();
     const float alpha = __ldg(alpha_p);
     for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < nblocks16; g += stride) {
@@ -680,6 +685,8 @@ __global__ void __launch_bounds__(256) dequantize4_bs8_kernel(const uint2* __res
     pdl_launch_dependents();
     const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    if ((int32_t)(blockIdx.x * blockDim.x + threadIdx.x) < nblocks16)        // before the wait: see prefetch_l2
+        prefetch_l2(codes + (size_t)(blockIdx.x * blockDim.x + threadIdx.x));
     pdl_wait();
     const float alpha = __ldg(alpha_p);
     for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < nblocks16; g += stride) {
@@ -714,6 +721,8 @@ __global__ void __launch_bounds__(256) dequantize6_fast_kernel(const uint32_t* _
                                                                uint4* __restrict__ out, float c_post) {
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
+    if ((int32_t)(blockIdx.x * blockDim.x + threadIdx.x) < ngroups)          // before the wait: see prefetch_l2
+        prefetch_l2(codes + 3 * (size_t)(blockIdx.x * blockDim.x + threadIdx.x));
     pdl_wait();
     const float alpha = __ldg(alpha_p);
     for (int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x); g < ngroups; g += stride) {

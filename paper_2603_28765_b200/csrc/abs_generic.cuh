@@ -33,6 +33,11 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
     pdl_launch_dependents();
     uint32_t local = 0u;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    {   // before the wait (see prefetch_l2): the thread's first two 32-byte pieces
+        const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        if (first < ngroups) prefetch_l2(in + 2 * first);
+        if (first + stride < ngroups) prefetch_l2(in + 2 * (first + stride));
+    }
     pdl_wait();
     if constexpr (!RHT) {
         // |x| and max on packed bf16 pairs

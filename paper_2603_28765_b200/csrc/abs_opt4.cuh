@@ -181,6 +181,7 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
     int32_t g = (int32_t)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (g < ngroups) prefetch_l2(in + 2 * (size_t)g);                  // before the wait: see prefetch_l2
     pdl_wait();
     uint32_t w[8], wn[8];
     const bool active = g < ngroups;
