@@ -320,6 +320,8 @@ def mac_matmul_reference(fmt: int, qa, qb, m: int, n: int, k: int) -> np.ndarray
         it = dequantize(fmt, codes, scales, 1.0, rows, k, out_fp32=True, select=F_INT_GROUPS_RAW).astype(np.float64)
         parts.append((fp, it, float(alpha)))
     (af, ai, aa), (bf, bi, ab) = parts
+    if float(m_int(fmt)) == 0.0:                      # plain NVFP4: there are no integer groups
+        return (af @ bf.T) * (aa * ab)
     c67 = float(m_fp(fmt)) / float(m_int(fmt))
     c = af @ bf.T + c67 * (af @ bi.T + ai @ bf.T) + (c67 * c67) * (ai @ bi.T)
     return c * (aa * ab)

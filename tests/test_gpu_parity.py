@@ -814,3 +814,34 @@ def test_index_offset_in_the_other_stochastic_entry_points(B, oracle, fmt):
                                           opts=B.make_opts(flags | B.ABS_F_ALPHA_GIVEN, 0, seed, 448 * 96))
     assert_same("transposed shard codes", ct.cpu().numpy().reshape(64, -1), tc[448:])
     assert_same("transposed shard scales", st.cpu().numpy().reshape(64, -1), tsc[448:])
+
+
+def test_tensor_core_consumer_reads_codes_and_swizzled_scales(B, oracle):
+    """Sec. 3: a group stored as FP4 is an NVFP4 group, so a plain-NVFP4 tensor from this library -- packed codes,
+    E4M3 scales in the 128x4-tile layout (ABS_F_SCALES_SWIZZLED), FP32 tensor scale -- must be directly usable as an
+    operand of Blackwell's block-scaled FP4 tensor-core product.  The consumer here is the block-scaled matrix
+    product that PyTorch exposes (a library kernel, operands in this GPU's memory): it is given the library's
+    buffers as they are, and its FP32 result is compared with the float64 product of the oracle's dequantized
+    operands.  Every product of two codes and two scales is exact and the sums are accumulated in FP32, so the
+    tolerance is that of an FP32 sum over K terms."""
+    F = torch.nn.functional
+    if not (hasattr(F, "scaled_mm") and hasattr(torch, "float4_e2m1fn_x2")):
+        pytest.skip("this PyTorch has no block-scaled FP4 matrix product")
+    for (m, n, k) in ((256, 384, 1024), (128, 128, 64), (640, 256, 4096)):
+        a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+        sw = B.make_opts(B.ABS_F_SCALES_SWIZZLED)
+        ca, sa, aa = B.abs_quantize(0, to_dev(a), opts=sw)
+        cb, sb, ab = B.abs_quantize(0, to_dev(b), opts=sw)
+        torch.cuda.synchronize()
+        qa, qb = oracle.quantize(0, a, threads=THREADS), oracle.quantize(0, b, threads=THREADS)
+        ref = oracle.mac_matmul_reference(0, qa, qb, m, n, k)
+        a4 = ca.view(m, k // 2).view(torch.float4_e2m1fn_x2)
+        b4 = cb.view(n, k // 2).view(torch.float4_e2m1fn_x2)
+        block, tensor = F.ScalingType.BlockWise1x16, F.ScalingType.TensorWise
+        tiled, plain = F.SwizzleType.SWIZZLE_32_4_4, F.SwizzleType.NO_SWIZZLE
+        c = F.scaled_mm(a4, b4.t(), scale_a=[sa.view(torch.float8_e4m3fn), aa], scale_recipe_a=[block, tensor],
+                        scale_b=[sb.view(torch.float8_e4m3fn), ab], scale_recipe_b=[block, tensor],
+                        swizzle_a=[tiled, plain], swizzle_b=[tiled, plain], output_dtype=torch.float32)
+        torch.cuda.synchronize()
+        err = np.abs(c.double().cpu().numpy() - ref).max() / np.abs(ref).max()
+        assert err < 2e-6, (m, n, k, err)
