@@ -232,6 +232,29 @@ ABS_API abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, c
 /* Host arithmetic of Eq. 1: amax / (M_FP * 448) in IEEE single precision; 1.0f when amax == 0. */
 ABS_API float abs_alpha_from_amax(abs_fmt_t fmt, float amax);
 
+/* Matrix product of two quantized operands on the tensor cores, C = A B^T, with the arithmetic of the paper's MAC
+ * unit (Sec. 5.2): the decoded codes of a pair of groups are multiplied and summed exactly, the sum is scaled by
+ * Delta_a * Delta_b, and the FP32 factor 1, 6/7 or 36/49 is applied on the scale path when none, one or both of
+ * the groups are stored as integers; alpha_a * alpha_b multiplies the result.  FP groups are NVFP4 groups (Sec. 3)
+ * and go to the block-scaled FP4 MMA (tcgen05.mma kind::mxf4nvf4) unchanged; an integer code k in -7..7 is the sum
+ * of two E2M1 values (5 = 4 + 1, 7 = 6 + 1), so each operand is first split into three NVFP4 planes in the
+ * workspace and the three kinds of group pairs accumulate in three FP32 accumulators that meet in the epilogue.
+ *   fmt                ABS_FMT_IF4 or ABS_FMT_NVFP4 (both operands)
+ *   a_codes, a_scales  A as abs_quantize wrote it: [m, k] quantized along k, scales row-major [m, k/16]; a_alpha its alpha
+ *   b_codes, b_scales  B likewise: [n, k]
+ *   c_f32              out, [m, n] float, row-major
+ *   workspace          device memory, 1024-byte aligned, at least abs_matmul_workspace_bytes(fmt, m, n, k) bytes
+ * m and n must be multiples of 128, k a multiple of 256 (ABS_ERR_SHAPE otherwise; abs_matmul_workspace_bytes
+ * returns 0).  Asynchronous like the other calls.  Every wait inside the kernel is bounded; if one runs out (it
+ * never should) the kernel stops and leaves a non-zero word at the start of the workspace, which
+ * abs_matmul_check(workspace, stream) reads back (it synchronises the stream): ABS_OK, or ABS_ERR_CUDA.
+ * Single GPU: the tensor maps cover the caller's workspace on the current device only. */
+ABS_API size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k);
+ABS_API abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
+                                const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n,
+                                int64_t k, float* c_f32, void* workspace, size_t workspace_bytes, void* stream);
+ABS_API abs_status_t abs_matmul_check(const void* workspace, void* stream);
+
 /* Host-buffer variants: `*_host` pointers are HOST memory (pinned memory makes the copies
  * asynchronous), `d_workspace` is a device buffer of at least abs_host_workspace_bytes() bytes.
  * Each call copies its inputs to the device, runs the same kernels as above, copies the results

@@ -36,6 +36,7 @@ EXPORTS = [
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
     "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled", "abs_quantize_dequantize",
+    "abs_matmul_workspace_bytes", "abs_matmul", "abs_matmul_check",
 ]
 
 
@@ -103,6 +104,12 @@ def lib():
             L.abs_quantize_host.argtypes = [C.c_int, vp, i64, i64, vp, vp, vp, op, vp, sz, vp]
             L.abs_dequantize_host.restype = C.c_int
             L.abs_dequantize_host.argtypes = [C.c_int, vp, vp, vp, i64, i64, vp, op, vp, sz, vp]
+            L.abs_matmul_workspace_bytes.restype = sz
+            L.abs_matmul_workspace_bytes.argtypes = [C.c_int, i64, i64, i64]
+            L.abs_matmul.restype = C.c_int
+            L.abs_matmul.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+            L.abs_matmul_check.restype = C.c_int
+            L.abs_matmul_check.argtypes = [vp, vp]
             L.abs_profile_events.restype = None
             L.abs_profile_events.argtypes = [vp, vp]
             L.abs_selftest_convert.restype = C.c_int
@@ -242,6 +249,30 @@ def abs_dequantize(fmt: int, codes, scales, tensor_scale, rows: int, cols: int, 
         rc = lib().abs_dequantize_ex(fmt, codes.data_ptr(), scales.data_ptr(), tensor_scale.data_ptr(), rows, cols,
                                      out.data_ptr(), C.byref(opts) if opts is not None else None, _stream_ptr(stream))
     _check(rc, "abs_dequantize")
+    return out
+
+
+def abs_matmul(fmt: int, qa, qb, m: int, n: int, k: int, out=None, workspace=None, stream=None, check: bool = False):
+    """C = A B^T on the tensor cores for two quantized operands ``qa`` = (codes, scales, alpha) of A [m, k] and
+    ``qb`` of B [n, k] (row-major scales), with the MAC arithmetic of Sec. 5.2.  Returns C as float32 [m, n].
+    ``check`` synchronises and raises if a wait inside the kernel ran out."""
+    import torch
+    L = lib()
+    need = L.abs_matmul_workspace_bytes(fmt, m, n, k)
+    if need == 0:
+        raise AbsError(2, "abs_matmul: m, n multiples of 128 and k a multiple of 256; IF4 or NVFP4")
+    if workspace is None:
+        workspace = torch.empty(need + 1024, dtype=torch.uint8, device=qa[0].device)
+    off = (-workspace.data_ptr()) % 1024
+    if out is None:
+        out = torch.empty((m, n), dtype=torch.float32, device=qa[0].device)
+    with torch.cuda.device(qa[0].device):
+        sp = _stream_ptr(stream)
+        rc = L.abs_matmul(fmt, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), qb[0].data_ptr(), qb[1].data_ptr(),
+                          qb[2].data_ptr(), m, n, k, out.data_ptr(), workspace.data_ptr() + off, workspace.numel() - off, sp)
+        _check(rc, "abs_matmul")
+        if check:
+            _check(L.abs_matmul_check(workspace.data_ptr() + off, sp), "abs_matmul (a wait inside the kernel ran out)")
     return out
 
 

@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libabs_b200.so")
-SOURCES = [os.path.join(CSRC, "abs_b200.cu")]
+SOURCES = [os.path.join(CSRC, "abs_b200.cu"), os.path.join(CSRC, "abs_gemm.cu")]
 HEADERS = [os.path.join(CSRC, "abs_device.cuh"), os.path.join(CSRC, "abs_fast4.cuh"), os.path.join(CSRC, "abs_opt4.cuh"), os.path.join(CSRC, "abs_fastx.cuh"), os.path.join(CSRC, "abs_trans4.cuh"), os.path.join(CSRC, "abs_generic.cuh"), os.path.join(os.path.dirname(_HERE), "include", "abs_b200.h")]
 
 NVCC_FLAGS = [

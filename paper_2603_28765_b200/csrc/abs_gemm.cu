@@ -1,0 +1,425 @@
+// IF4 matrix product on the Blackwell tensor cores (tcgen05): C = A B^T for two IF4 (or NVFP4) operands with the
+// arithmetic of the paper's MAC unit (Sec. 5.2): inside a pair of groups the decoded codes are multiplied and
+// summed exactly, the sum is scaled by Delta_a * Delta_b, and the factors 1, 6/7 or 36/49 -- none, one or both
+// groups stored as integers -- are applied in FP32 on the scale path, here in the epilogue.
+//
+// How integer groups reach an FP4 tensor core.  An FP4 group is an NVFP4 group (Sec. 3) and goes to
+// tcgen05.mma kind::mxf4nvf4 as it is.  An integer code k in -7..7 is not an E2M1 value, but it is the sum of
+// two: k = h + l with h in {0, 1, 2, 3, 4, 6} and l in {0, 1} (5 = 4 + 1, 7 = 6 + 1), signs equal.  So every
+// operand is split once into three NVFP4 "planes" that share the group scales:
+//     F: the codes of the FP groups (integer groups zero)     H, L: the two parts of the integer groups
+// and the product is  F_a F_b  +  6/7 (F_a (H_b + L_b) + (H_a + L_a) F_b)  +  36/49 (H_a + L_a)(H_b + L_b),
+// nine block-scaled MMAs per K-step into three FP32 accumulators that live in tensor memory side by side
+// (3 x 128 columns) and meet only in the epilogue.  Every product and partial sum is exact in the tensor core's
+// FP32 accumulation up to its rounding of the running sum, which is what the float64 reference is compared to.
+//
+// Kernel: one 128 x 128 tile of C per block.  One thread feeds the pipeline with TMA (cp.async.bulk.tensor.2d,
+// 128-byte swizzle, no multicast; the scale tiles with plain bulk copies), one thread copies the scales to tensor
+// memory (tcgen05.cp) and issues the MMAs, four warps read the accumulators back (tcgen05.ld) and write C.
+// Every mbarrier wait is bounded: when a wait runs out the block raises an error word, stops issuing, frees its
+// tensor memory and returns.
+#include "../../include/abs_b200.h"
+#include "abs_device.cuh"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <mutex>
+
+namespace absq {
+
+constexpr int kTileM = 128, kTileN = 128;
+constexpr int kStageK = 256;                       // elements of K per pipeline stage: 128 bytes of packed codes per row
+constexpr int kMmaK = 64;                          // K of one tcgen05.mma kind::mxf4nvf4
+constexpr int kStages = 2;
+constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one plane of one operand in one stage
+constexpr int kSfBytes = (kStageK / kMmaK) * 512;  // 2 KiB: scale tiles (128 rows x 4 scales) of one operand in one stage
+constexpr int kStageBytes = 6 * kPlaneBytes + 2 * kSfBytes;
+constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint32_t kWaitLimit = 1u << 22;          // polls of one mbarrier wait before the block gives up
+
+// ----------------------------------------------------------------------------- operand split
+
+// Splits the 16 codes of one group (two words) into the planes F, H, L and writes the magnitude of its scale byte
+// into the 128x4-tile layout the tensor core reads.  FP groups: F = codes.  Integer groups (two's complement
+// nibbles): sign s, magnitude m = |k|; H = s | e2m1(m - (m is 5 or 7)), L = s | e2m1(1) where m is 5 or 7.
+// E2M1 codes of the integers 0, 1, 2, 3, 4, 6 are 0, 2, 4, 5, 6, 7.
+__device__ __forceinline__ void split_word(uint32_t w, bool is_int, uint32_t& f, uint32_t& h, uint32_t& l) {
+    if (!is_int) { f = w; h = 0u; l = 0u; return; }
+    f = 0u; h = 0u; l = 0u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int k = (int)((w >> (4 * j)) << 28) >> 28;             // sign-extended nibble
+        const uint32_t m = (uint32_t)(k < 0 ? -k : k), s = k < 0 ? 8u : 0u;
+        const bool odd57 = (m == 5u) || (m >= 7u);                    // m = 8 (never produced) is treated as 7 + 1
+        const uint32_t mh = odd57 ? m - 1u : m;                       // 0, 1, 2, 3, 4, 6
+        const uint32_t ch = mh <= 1u ? 2u * mh : (mh <= 4u ? mh + 2u : 7u);
+        h |= ((m ? s : 0u) | ch) << (4 * j);
+        l |= (odd57 ? (s | 2u) : 0u) << (4 * j);
+    }
+}
+
+__global__ void __launch_bounds__(256) if4_split_kernel(const uint2* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                        int64_t ngroups, uint32_t gpr, uint32_t ktiles, bool has_int,
+                                                        uint2* __restrict__ plane_f, uint2* __restrict__ plane_h,
+                                                        uint2* __restrict__ plane_l, uint8_t* __restrict__ sf_tiled) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+        const uint2 c = __ldg(codes + g);
+        const uint32_t sb = __ldg(scales + g);
+        const bool is_int = has_int && (sb & 0x80u);
+        uint32_t f0, h0, l0, f1, h1, l1;
+        split_word(c.x, is_int, f0, h0, l0);
+        split_word(c.y, is_int, f1, h1, l1);
+        plane_f[g] = make_uint2(f0, f1);
+        plane_h[g] = make_uint2(h0, h1);
+        plane_l[g] = make_uint2(l0, l1);
+        const uint32_t row = (uint32_t)(g / gpr), k = (uint32_t)(g - (int64_t)row * gpr);
+        sf_tiled[swizzled_scale_offset(row, k, ktiles)] = (uint8_t)(sb & 0x7Fu);
+    }
+}
+
+// ----------------------------------------------------------------------------- PTX building blocks
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        uint32_t done;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// One 2-D tile (inner coordinate x in bytes, outer coordinate y in rows) from a tensor map into shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Contiguous bytes (multiple of 16, both addresses 16-byte aligned) into shared memory.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t columns) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_result), "r"(columns) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_free(uint32_t addr, uint32_t columns) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(addr), "r"(columns) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Arrives on the mbarrier once every tcgen05 operation this thread issued before has completed.
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+// Scale tile (32 rows x 16 bytes in shared memory = the scales of 128 rows x 4 groups) into four columns of tensor
+// memory, replicated over the four 32-lane quarters.
+__device__ __forceinline__ void tc_copy_scales(uint32_t tmem_addr, uint64_t smem_desc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" :: "r"(tmem_addr), "l"(smem_desc) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 64, E2M1 operands, one UE4M3 scale per 16 elements read from tensor memory.
+__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem) {
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
+                 "  tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p; }"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                 : "memory");
+}
+// 32 lanes x 32 columns of 32 bits: thread t of the warp gets columns c .. c+31 of lane (warp % 4) * 32 + t.
+__device__ __forceinline__ void tmem_load32(uint32_t addr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (64 bits): start address, leading / stride byte offsets (all in 16-byte units),
+// descriptor version 1 (Blackwell) in bits 46-47, swizzle mode in bits 61-63.
+//   operand tiles: K-major rows of 128 bytes, 128-byte swizzle (mode 2), 8-row groups 1024 bytes apart
+//   scale tiles:   32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t scale_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
+}
+// Instruction descriptor of kind::mxf4nvf4: A and B E2M1 (format 1, bits 7-9 and 10-12), both K-major, N / 8 in bits
+// 17-22, scale format UE4M3 (bit 23 = 0), M / 16 in bits 24-28, dense, K = 64 (bit 31 = 0), scale ids 0.
+constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+
+// ----------------------------------------------------------------------------- the product kernel
+
+// Tensor memory columns (512 allocated): three accumulators of 128 columns, then per stage 16 columns of A scales
+// and 16 of B scales (four per K-step of 64).
+constexpr uint32_t kTmemCols = 512, kTmemSf = 3 * kTileN;
+
+struct GemmMaps {
+    CUtensorMap a[3], b[3];        // planes F, H, L of A [M, K/2 bytes] and B [N, K/2 bytes], boxes of 128 bytes x 128 rows
+};
+
+// planes = 3: IF4 operands (nine MMAs per K-step); planes = 1: plain NVFP4 (one).  error: device word set to a
+// non-zero code when a wait ran out.
+__global__ void __launch_bounds__(128, 1)
+if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
+                const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t n_cols,
+                int32_t k_iters, int32_t planes, int* __restrict__ error) {
+    extern __shared__ uint8_t gemm_smem_raw[];
+    const uint32_t raw = smem_u32(gemm_smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                    // 128-byte swizzle wants 1024-byte aligned tiles
+    const uint32_t bars = base + kStages * kStageBytes;              // full[2], empty[2], acc_done, tmem address word
+    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 64);
+    const uint32_t full0 = bars, empty0 = bars + 16, acc_done = bars + 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile_m = blockIdx.y, tile_n = blockIdx.x;
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(acc_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) { tmem_alloc(smem_u32(tmem_word), kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_word;
+    pdl_wait();
+
+    if (warp == 0 && lane == 0) {
+        // ---- producer: TMA loads of the operand planes and bulk copies of the scale tiles
+        const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes + 2u * kSfBytes;
+        const int32_t ktiles = k_iters * (kStageK / kMmaK);
+        for (int32_t it = 0; it < k_iters; ++it) {
+            const int s = it % kStages;
+            if (!mbar_wait(empty0 + 8 * s, ((it / kStages) & 1) ^ 1)) { atomicExch(error, 1); break; }
+            const uint32_t st = base + s * kStageBytes, bar = full0 + 8 * s;
+            mbar_expect_tx(bar, bytes);
+            for (int p = 0; p < planes; ++p) {
+                tma_load_2d(st + p * kPlaneBytes, &maps.a[p], it * (kStageK / 2), tile_m * kTileM, bar);
+                tma_load_2d(st + (3 + p) * kPlaneBytes, &maps.b[p], it * (kStageK / 2), tile_n * kTileN, bar);
+            }
+            bulk_load(st + 6 * kPlaneBytes, sfa + ((size_t)tile_m * ktiles + (size_t)it * (kStageK / kMmaK)) * 512, kSfBytes, bar);
+            bulk_load(st + 6 * kPlaneBytes + kSfBytes, sfb + ((size_t)tile_n * ktiles + (size_t)it * (kStageK / kMmaK)) * 512, kSfBytes, bar);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- scale copies and MMAs
+        bool ok = true;
+        for (int32_t it = 0; it < k_iters && ok; ++it) {
+            const int s = it % kStages;
+            if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1)) { atomicExch(error, 2); ok = false; break; }
+            tc_fence_after();
+            const uint32_t st = base + s * kStageBytes;
+            const uint32_t tsfa = tmem + kTmemSf + s * 32, tsfb = tsfa + 16;
+#pragma unroll
+            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                tc_copy_scales(tsfa + 4 * kb, scale_desc(st + 6 * kPlaneBytes + kb * 512));
+                tc_copy_scales(tsfb + 4 * kb, scale_desc(st + 6 * kPlaneBytes + kSfBytes + kb * 512));
+            }
+#pragma unroll
+            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                const bool first = it == 0 && kb == 0;
+                uint64_t da[3], db[3];
+#pragma unroll
+                for (int p = 0; p < 3; ++p) {
+                    da[p] = operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2));
+                    db[p] = operand_desc(st + (3 + p) * kPlaneBytes + kb * (kMmaK / 2));
+                }
+                const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
+                tc_mma_nvf4(tmem, da[0], db[0], kInstrDesc, !first, fa, fb);                       // F F
+                if (planes == 3) {
+                    tc_mma_nvf4(tmem + kTileN, da[0], db[1], kInstrDesc, !first, fa, fb);          // F H
+                    tc_mma_nvf4(tmem + kTileN, da[0], db[2], kInstrDesc, true, fa, fb);            // F L
+                    tc_mma_nvf4(tmem + kTileN, da[1], db[0], kInstrDesc, true, fa, fb);            // H F
+                    tc_mma_nvf4(tmem + kTileN, da[2], db[0], kInstrDesc, true, fa, fb);            // L F
+                    tc_mma_nvf4(tmem + 2 * kTileN, da[1], db[1], kInstrDesc, !first, fa, fb);      // H H
+                    tc_mma_nvf4(tmem + 2 * kTileN, da[1], db[2], kInstrDesc, true, fa, fb);        // H L
+                    tc_mma_nvf4(tmem + 2 * kTileN, da[2], db[1], kInstrDesc, true, fa, fb);        // L H
+                    tc_mma_nvf4(tmem + 2 * kTileN, da[2], db[2], kInstrDesc, true, fa, fb);        // L L
+                }
+            }
+            tc_commit(empty0 + 8 * s);              // the stage's shared memory is free once these MMAs have run
+        }
+        if (ok) tc_commit(acc_done);
+    }
+    __syncwarp();
+
+    // ---- epilogue: all four warps; warp w owns lanes (rows) 32 w .. 32 w + 31 of the accumulators
+    bool have = mbar_wait(acc_done, 0);
+    if (!have && lane == 0) atomicExch(error, 3);
+    have = __all_sync(0xFFFFFFFFu, have);
+    tc_fence_after();
+    if (have) {
+        const float scale = __fmul_rn(__ldg(alpha_a), __ldg(alpha_b));
+        const float c1 = __uint_as_float(0x3F5B6DB7u);                 // fp32(6/7)
+        const float c2 = __fdiv_rn(36.0f, 49.0f);
+        float* out = c + ((size_t)tile_m * kTileM + warp * 32 + lane) * (size_t)n_cols + (size_t)tile_n * kTileN;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
+            uint32_t r0[32], r1[32], r2[32];
+            tmem_load32(lane_base + chunk * 32, r0);
+            if (planes == 3) {
+                tmem_load32(lane_base + kTileN + chunk * 32, r1);
+                tmem_load32(lane_base + 2 * kTileN + chunk * 32, r2);
+            }
+            tmem_load_wait();
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                float acc = __uint_as_float(r0[j]);
+                if (planes == 3) acc = __fmaf_rn(c2, __uint_as_float(r2[j]), __fmaf_rn(c1, __uint_as_float(r1[j]), acc));
+                v[j] = __fmul_rn(acc, scale);
+            }
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(out + chunk * 32 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_free(tmem, kTmemCols);
+}
+
+}  // namespace absq
+
+// ----------------------------------------------------------------------------- host side
+
+namespace {
+
+using namespace absq;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda).
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, []() {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Tensor map of one plane: bytes [rows, row_bytes], box 128 bytes x 128 rows, 128-byte swizzle.  The map covers
+// this GPU's own workspace only.
+bool plane_map(CUtensorMap* map, void* base, uint64_t rows, uint64_t row_bytes) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {row_bytes, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {128, 128}, elem[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t round1k(size_t n) { return (n + 1023) & ~(size_t)1023; }
+
+struct GemmLayout {
+    size_t plane_a, plane_b, sf_a, sf_b;       // sizes
+    size_t off_a, off_b, off_sfa, off_sfb, total;
+};
+GemmLayout gemm_layout(int64_t m, int64_t n, int64_t k) {
+    GemmLayout L;
+    L.plane_a = round1k((size_t)m * k / 2);
+    L.plane_b = round1k((size_t)n * k / 2);
+    L.sf_a = round1k((size_t)m * k / 16);
+    L.sf_b = round1k((size_t)n * k / 16);
+    L.off_a = 1024;
+    L.off_b = L.off_a + 3 * L.plane_a;
+    L.off_sfa = L.off_b + 3 * L.plane_b;
+    L.off_sfb = L.off_sfa + L.sf_a;
+    L.total = L.off_sfb + L.sf_b;
+    return L;
+}
+
+bool gemm_shape_ok(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k) {
+    return (fmt == ABS_FMT_IF4 || fmt == ABS_FMT_NVFP4) && m > 0 && n > 0 && k > 0 && m % kTileM == 0 && n % kTileN == 0 &&
+           k % kStageK == 0 && m < ((int64_t)1 << 30) && n < ((int64_t)1 << 30) && k < ((int64_t)1 << 30);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k) {
+    if (!gemm_shape_ok(fmt, m, n, k)) return 0;
+    return gemm_layout(m, n, k).total;
+}
+
+abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
+                        const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (fmt != ABS_FMT_IF4 && fmt != ABS_FMT_NVFP4) return ABS_ERR_FMT;
+    if (!gemm_shape_ok(fmt, m, n, k)) return ABS_ERR_SHAPE;
+    if (!a_codes || !a_scales || !a_alpha || !b_codes || !b_scales || !b_alpha || !c_f32 || !workspace) return ABS_ERR_NULL;
+    const uintptr_t all = (uintptr_t)a_codes | (uintptr_t)a_scales | (uintptr_t)b_codes | (uintptr_t)b_scales | (uintptr_t)c_f32;
+    if ((all & 15u) || ((uintptr_t)workspace & 1023u)) return ABS_ERR_ALIGN;
+    const GemmLayout L = gemm_layout(m, n, k);
+    if (workspace_bytes < L.total) return ABS_ERR_SIZE;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    const bool has_int = fmt == ABS_FMT_IF4;
+    const int planes = has_int ? 3 : 1;
+
+    GemmMaps maps;
+    for (int p = 0; p < 3; ++p) {
+        if (!plane_map(&maps.a[p], ws + L.off_a + p * L.plane_a, (uint64_t)m, (uint64_t)k / 2) ||
+            !plane_map(&maps.b[p], ws + L.off_b + p * L.plane_b, (uint64_t)n, (uint64_t)k / 2))
+            return ABS_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(ws, 0, 1024, s) != cudaSuccess) return ABS_ERR_CUDA;          // the error word
+    const uint32_t gpr = (uint32_t)(k / 16), ktiles = (gpr + 3u) / 4u;
+    for (int op = 0; op < 2; ++op) {
+        const int64_t rows = op ? n : m;
+        const int64_t ngroups = rows * (k / 16);
+        const size_t off = op ? L.off_b : L.off_a, plane = op ? L.plane_b : L.plane_a;
+        int64_t blocks = (ngroups + 255) / 256;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        if4_split_kernel<<<(int)blocks, 256, 0, s>>>((const uint2*)(op ? b_codes : a_codes), (const uint8_t*)(op ? b_scales : a_scales),
+                                                    ngroups, gpr, ktiles, has_int, (uint2*)(ws + off), (uint2*)(ws + off + plane),
+                                                    (uint2*)(ws + off + 2 * plane), ws + (op ? L.off_sfb : L.off_sfa));
+        if (cudaGetLastError() != cudaSuccess) return ABS_ERR_CUDA;
+    }
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, []() {
+        attr_err = cudaFuncSetAttribute(if4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return ABS_ERR_CUDA;
+    const dim3 grid((unsigned)(n / kTileN), (unsigned)(m / kTileM));
+    if4_gemm_kernel<<<grid, 128, kGemmSmemBytes, s>>>(maps, ws + L.off_sfa, ws + L.off_sfb, a_alpha, b_alpha, c_f32, (int32_t)n,
+                                                      (int32_t)(k / kStageK), planes, (int*)ws);
+    return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+abs_status_t abs_matmul_check(const void* workspace, void* stream) {
+    if (!workspace) return ABS_ERR_NULL;
+    int word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess ||
+        cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess)
+        return ABS_ERR_CUDA;
+    return word == 0 ? ABS_OK : ABS_ERR_CUDA;
+}
+
+}  // extern "C"

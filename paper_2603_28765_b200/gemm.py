@@ -8,14 +8,18 @@ Both take operands quantized along K: A as [M, K], B as [N, K] (codes, scales, a
 ``matmul_mac``       the arithmetic of the paper's IF4 MAC unit (Sec. 5.2): inside a pair of groups the
                      decoded 4-bit values are multiplied and summed, and the pair's scale product gets the
                      factor 1, 6/7 or 36/49 (none, one, both groups stored as integers) in FP32 on the
-                     scale path.  Here: the library's split dequantize produces, for each operand, the
+                     scale path.  This is the library's own tensor-core kernel (``abs_matmul``: block-scaled
+                     FP4 MMAs on the codes themselves, three accumulators, factors in the FP32 epilogue)
+                     whenever M and N are multiples of 128 and K of 256.
+``matmul_mac_split`` the same arithmetic for any shape, and the cross-check of the kernel above, from parts
+                     that are exact in BF16: the library's split dequantize produces, for each operand, the
                      FP-group part and the raw integer-group part -- each a 4-bit code times an E4M3 scale,
                      hence EXACT in BF16 -- and four plain BF16 tensor-core GEMMs (FP32 accumulation, every
                      product exact) are combined with the FP32 factors:
                          C = A_F B_F^T + 6/7 (A_F B_I^T + A_I B_F^T) + 36/49 A_I B_I^T,  times alpha_a alpha_b.
 
-The GEMMs themselves are plain library calls (torch.matmul -> cuBLAS); everything format-specific runs in
-this library's kernels.
+In ``matmul_emulated`` and ``matmul_mac_split`` the GEMMs are plain library calls (torch.mm -> cuBLAS);
+``matmul_mac`` contracts in this library's own kernel.
 """
 from __future__ import annotations
 
@@ -41,6 +45,13 @@ def matmul_emulated(qa, qb, m: int, n: int, k: int):
 
 
 def matmul_mac(qa, qb, m: int, n: int, k: int):
+    """Sec. 5.2 MAC arithmetic: the library's tcgen05 kernel where the shape allows, else the BF16 split."""
+    if m % 128 == 0 and n % 128 == 0 and k % 256 == 0:
+        return B.abs_matmul(FMT, qa, qb, m, n, k)
+    return matmul_mac_split(qa, qb, m, n, k)
+
+
+def matmul_mac_split(qa, qb, m: int, n: int, k: int):
     """Sec. 5.2 MAC arithmetic via the exact BF16 split (see the module docstring)."""
     import torch
     a_f = _deq(qa, m, k, B.ABS_F_FP_GROUPS_ONLY, unit_alpha=True)

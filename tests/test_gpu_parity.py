@@ -845,3 +845,31 @@ def test_tensor_core_consumer_reads_codes_and_swizzled_scales(B, oracle):
         torch.cuda.synchronize()
         err = np.abs(c.double().cpu().numpy() - ref).max() / np.abs(ref).max()
         assert err < 2e-6, (m, n, k, err)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_tensor_core_matmul_matches_mac_reference(B, oracle, fmt):
+    """abs_matmul (hand-written tcgen05 kernel: TMA-fed block-scaled FP4 MMAs, three accumulators for the FP x FP,
+    mixed and INT x INT group pairs, factors 1, 6/7, 36/49 in the FP32 epilogue) against the float64 reference of the
+    MAC arithmetic of Sec. 5.2.  Every code product is exact; the difference is the FP32 accumulation of the tensor
+    core over K terms, so the tolerance is that of an FP32 sum (2e-5 of the largest |C| is ample up to K = 4096)."""
+    for (m, n, k) in ((128, 128, 256), (256, 384, 1024), (128, 256, 4096), (640, 128, 512)):
+        a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+        qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
+        oa, ob = oracle.quantize(fmt, a, threads=THREADS), oracle.quantize(fmt, b, threads=THREADS)
+        ref = oracle.mac_matmul_reference(fmt, oa, ob, m, n, k)
+        c = B.abs_matmul(fmt, qa, qb, m, n, k, check=True).double().cpu().numpy()
+        err = np.abs(c - ref).max() / np.abs(ref).max()
+        assert err < 2e-5, (fmt, m, n, k, err)
+        if fmt == 1:
+            assert 0.05 < float((oa[1] >> 7).mean()) < 0.95     # both kinds of groups take part
+    # shapes the kernel does not take, and other formats
+    L = B.lib()
+    assert L.abs_matmul_workspace_bytes(fmt, 100, 128, 256) == 0 and L.abs_matmul_workspace_bytes(fmt, 128, 128, 128) == 0
+    assert L.abs_matmul_workspace_bytes(2, 128, 128, 256) == 0
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    out = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    args = (qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), qb[0].data_ptr(), qb[1].data_ptr(), qb[2].data_ptr())
+    assert L.abs_matmul(fmt, *args, 128, 128, 192, out.data_ptr(), ws.data_ptr(), 4096, None) == 2      # k % 256
+    assert L.abs_matmul(3, *args, 128, 128, 256, out.data_ptr(), ws.data_ptr(), 4096, None) == 4        # format
+    assert L.abs_matmul(fmt, *args, 128, 128, 256, out.data_ptr(), ws.data_ptr(), 4096, None) in (3, 7)  # alignment or size
