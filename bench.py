@@ -301,7 +301,7 @@ def run_cuda(args):
     barrier()
     ramp_t0 = time.perf_counter()
     ramp_steps = 0
-    while (time.perf_counter() - ramp_t0) * 1e3 < CLOCK_RAMP_MS:
+    while not args.no_ramp and (time.perf_counter() - ramp_t0) * 1e3 < CLOCK_RAMP_MS:
         for i in range(64):
             step(ramp_steps + i)
         ramp_steps += 64
@@ -539,6 +539,7 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-ramp", action="store_true", help="skip the clock-ramp loop (profiling runs only: fewer launches)")
     ap.add_argument("--no-large", action="store_true", help="skip the 16384x8192 figures (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":

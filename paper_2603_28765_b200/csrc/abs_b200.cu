@@ -157,10 +157,8 @@ abs_status_t next_slot(DeviceState& st, unsigned long long** slot, uint32_t* gen
 abs_status_t launch_amax(int sm_count, const void* in, int64_t ngroups, const abs_opts_t& o, bool ticket,
                          unsigned long long* slot, uint32_t gen, float* result, float denom, cudaStream_t s) {
     const bool rht = o.flags & ABS_F_HADAMARD16;
-#ifndef ABS_AMAX_RHT_BPS
-#define ABS_AMAX_RHT_BPS ABS_AMAX_BPS
-#endif
-    const int grid = grid_for(sm_count, rht ? ngroups : ngroups * 2, rht ? ABS_AMAX_RHT_BPS : ABS_AMAX_BPS);
+constexpr int kAmaxRhtBlocksPerSm = kAmaxBlocksPerSm;
+    const int grid = grid_for(sm_count, rht ? ngroups : ngroups * 2, rht ? kAmaxRhtBlocksPerSm : kAmaxBlocksPerSm);
     cudaError_t e;
 #define ABS_LAUNCH_A(R, T)                                                                                          \
     e = launch_pdl(amax_kernel<R, T>, grid, kThreads, s, (const uint4*)in, ngroups, (uint32_t)o.had_sign_mask, slot, \
@@ -176,21 +174,11 @@ abs_status_t launch_amax(int sm_count, const void* in, int64_t ngroups, const ab
 
 // Groups per thread the grid-stride kernels are launched for (see grid_waves); measured optima, all flat
 // within a few per cent around the value.
-#ifndef ABS_IF6_ITERS
-#define ABS_IF6_ITERS 7           // IF6, IF3 and the integer-bearing block-size-8 round-to-nearest kernels
-#endif
-#ifndef ABS_NV_ITERS
-#define ABS_NV_ITERS 5            // groups per thread of the NVFP4 round-to-nearest kernel (5 resident blocks per SM)
-#endif
-#ifndef ABS_DEQ_ITERS
-#define ABS_DEQ_ITERS 2           // groups per thread of the 4-bit dequantize kernel
-#endif
-#ifndef ABS_FAST_ITERS
-#define ABS_FAST_ITERS 7          // groups per thread the IF4 round-to-nearest kernel is launched for
-#endif
-#ifndef ABS_OPT_ITERS
-#define ABS_OPT_ITERS 12          // same for the Hadamard / stochastic-rounding kernel
-#endif
+constexpr int kIf6Iters = 7;   // IF6, IF3 and the integer-bearing block-size-8 round-to-nearest kernels
+constexpr int kNvIters = 5;   // groups per thread of the NVFP4 round-to-nearest kernel (5 resident blocks per SM)
+constexpr int kDeqIters = 2;   // groups per thread of the 4-bit dequantize kernel
+constexpr int kFastIters = 7;   // groups per thread the IF4 round-to-nearest kernel is launched for
+constexpr int kOptIters = 12;   // same for the Hadamard / stochastic-rounding kernel
 
 template <int FMT>
 // emul_out != nullptr asks for the emulation pass (abs_quantize_dequantize) of the formats handled by the
@@ -210,7 +198,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (emul_out) return ABS_ERR_FLAGS;      // the 4-bit emulation pass is launched by abs_quantize_dequantize
         if (!rht && !sr) {   // the 4-bit round-to-nearest fast path
-            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(sm_count, ngroups, ABS_FAST_MINB, ABS_FAST_ITERS) : grid_waves(sm_count, ngroups, 5, ABS_NV_ITERS);
+            const int pgrid = FMT == ABS_FMT_IF4 ? grid_waves(sm_count, ngroups, kFastMinBlocks, kFastIters) : grid_waves(sm_count, ngroups, 5, kNvIters);
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
             // the kernel looks three grid strides past the current group (next group, and its L2 prefetch)
@@ -246,7 +234,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     }
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         // Hadamard / stochastic-rounding options of the 4-bit formats: the packed persistent kernel
-        const int ogrid = grid_waves(sm_count, ngroups, opt_blocks_per_sm(sr, rht), ABS_OPT_ITERS);
+        const int ogrid = grid_waves(sm_count, ngroups, opt_blocks_per_sm(sr, rht), kOptIters);
         if (!(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)ogrid * kThreads) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -270,7 +258,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
         // block-size-8 variants of the 4-bit formats, round-to-nearest: two groups of 8 per thread
         constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
-        const int bgrid = grid_waves(sm_count, ngroups, kInt ? 4 : 5, kInt ? ABS_IF6_ITERS : 5);
+        const int bgrid = grid_waves(sm_count, ngroups, kInt ? 4 : 5, kInt ? kIf6Iters : 5);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -288,7 +276,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     }
     if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
         // 6-bit formats, round-to-nearest
-        const int sgrid = grid_waves(sm_count, ngroups, 3, ABS_IF6_ITERS);
+        const int sgrid = grid_waves(sm_count, ngroups, 3, kIf6Iters);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -307,7 +295,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // IF3 and its block-size-8 variant, round-to-nearest
         constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
-        const int tgrid = grid_waves(sm_count, ngroups, ABS_IF3_MINB, ABS_IF6_ITERS);
+        const int tgrid = grid_waves(sm_count, ngroups, kIf3MinBlocks, kIf6Iters);
         if (!rht && !sr && !(o.flags & ABS_F_INDEX64) && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             if (handled) *handled = true;
             const bool a32 = (reinterpret_cast<uintptr_t>(in) & 31u) == 0;
@@ -349,7 +337,7 @@ abs_status_t launch_dequantize_fmt(int sm_count, const void* codes, const void* 
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (!fp32) {
             constexpr bool kInt = FMT == ABS_FMT_IF4;
-            const int grid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);    // 31 registers: 8 resident blocks per SM
+            const int grid = grid_waves(sm_count, ngroups, 8, kDeqIters);    // 31 registers: 8 resident blocks per SM
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
             const bool i32 = !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads;
             cudaError_t e;
@@ -376,7 +364,7 @@ abs_status_t launch_dequantize_fmt(int sm_count, const void* codes, const void* 
         }
     }
     if constexpr (FMT == ABS_FMT_NVFP4_BS8 || FMT == ABS_FMT_IF4_BS8) {
-        const int bgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
+        const int bgrid = grid_waves(sm_count, ngroups, 8, kDeqIters);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)bgrid * kThreads) {
             constexpr bool kInt = FMT == ABS_FMT_IF4_BS8;
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
@@ -389,7 +377,7 @@ abs_status_t launch_dequantize_fmt(int sm_count, const void* codes, const void* 
         }
     }
     if constexpr (FMT == ABS_FMT_IF6_E2M3 || FMT == ABS_FMT_IF6_E3M2) {
-        const int sgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
+        const int sgrid = grid_waves(sm_count, ngroups, 8, kDeqIters);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)sgrid * kThreads) {
             constexpr ElemKind kEK = Fmt<FMT>::EK;
             const float c_post = Fmt<FMT>::M_FP / Fmt<FMT>::M_INT;         // IEEE single division, as in the generic kernel
@@ -404,7 +392,7 @@ abs_status_t launch_dequantize_fmt(int sm_count, const void* codes, const void* 
     }
     if constexpr (FMT == ABS_FMT_IF3 || FMT == ABS_FMT_IF3_BS8) {
         // 3-bit codes widened to nibbles and decoded like the 4-bit formats
-        const int tgrid = grid_waves(sm_count, ngroups, 8, ABS_DEQ_ITERS);
+        const int tgrid = grid_waves(sm_count, ngroups, 8, kDeqIters);
         if (!fp32 && !index64 && ngroups < (int64_t)0x7FFFFFFF - (int64_t)tgrid * kThreads) {
             constexpr int kG = FMT == ABS_FMT_IF3 ? 16 : 8;
             const bool a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
@@ -563,6 +551,7 @@ float abs_alpha_from_amax(abs_fmt_t fmt, float amax) {
 
 abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs_opts_t* opts, float* amax_f32,
                       void* stream) {
+    const CallRange range("abs_amax");
     abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return ABS_ERR_SHAPE;
@@ -583,6 +572,7 @@ abs_status_t abs_amax(const void* in_bf16, int64_t rows, int64_t cols, const abs
 
 abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                              void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts, void* stream) {
+    const CallRange range("abs_quantize_ex");
     abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
@@ -629,6 +619,7 @@ abs_status_t abs_quantize_ex(abs_fmt_t fmt, const void* in_bf16, int64_t rows, i
 abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* out_bf16,
                                      void* codes_u8, void* scales_e4m3, float* tensor_scale_f32, const abs_opts_t* opts,
                                      void* stream) {
+    const CallRange range("abs_quantize_dequantize");
     abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
@@ -657,7 +648,7 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
     cudaStream_t s = (cudaStream_t)stream;
     const int64_t ngroups = rows * cols / 16;
     const bool rht = o.flags & ABS_F_HADAMARD16, sr = o.flags & ABS_F_STOCHASTIC;
-    const int grid = grid_waves(st->sm_count, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? ABS_OPT_ITERS : ABS_FAST_ITERS);
+    const int grid = grid_waves(st->sm_count, ngroups, opt_blocks_per_sm(sr, rht), (rht || sr) ? kOptIters : kFastIters);
     if (ngroups >= (int64_t)0x7FFFFFFF - (int64_t)grid * kThreads) return ABS_ERR_SIZE;    // 32-bit group indices only
     AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
@@ -723,6 +714,7 @@ abs_status_t abs_quantize(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int6
 abs_status_t abs_quantize_transposed(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols,
                                      void* codes_t_u8, void* scales_t_e4m3, float* tensor_scale_f32,
                                      const abs_opts_t* opts, void* stream) {
+    const CallRange range("abs_quantize_transposed");
     abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (fmt != ABS_FMT_NVFP4 && fmt != ABS_FMT_IF4) return ABS_ERR_FMT;
@@ -845,6 +837,7 @@ extern "C" {
 
 abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t rows, int64_t cols, void* codes_u8,
                                   void* scales_e4m3, float* tensor_scale_f32, void* stream) {
+    const CallRange range("abs_quantize_noalloc");
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if (rows * cols == 0) return ABS_OK;
@@ -889,6 +882,7 @@ abs_status_t abs_quantize_noalloc(abs_fmt_t fmt, const void* in_bf16, int64_t ro
 abs_status_t abs_dequantize_ex(abs_fmt_t fmt, const void* codes_u8, const void* scales_e4m3,
                                const float* tensor_scale_f32, int64_t rows, int64_t cols, void* out,
                                const abs_opts_t* opts, void* stream) {
+    const CallRange range("abs_dequantize_ex");
     abs_opts_t o = {0, 0, 0, 0, 0};
     if (opts) o = *opts;
     abs_status_t rc = check_shape(fmt, rows, cols);
@@ -943,6 +937,7 @@ size_t abs_host_workspace_bytes(abs_fmt_t fmt, int64_t rows, int64_t cols) {
 abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t rows, int64_t cols,
                                void* codes_u8_host, void* scales_e4m3_host, float* tensor_scale_f32_host,
                                const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream) {
+    const CallRange range("abs_quantize_host");
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if (rows * cols == 0) return ABS_OK;
@@ -971,6 +966,7 @@ abs_status_t abs_quantize_host(abs_fmt_t fmt, const void* in_bf16_host, int64_t 
 abs_status_t abs_dequantize_host(abs_fmt_t fmt, const void* codes_u8_host, const void* scales_e4m3_host,
                                  const float* tensor_scale_f32_host, int64_t rows, int64_t cols, void* out_host,
                                  const abs_opts_t* opts, void* d_workspace, size_t workspace_bytes, void* stream) {
+    const CallRange range("abs_dequantize_host");
     abs_status_t rc = check_shape(fmt, rows, cols);
     if (rc != ABS_OK) return rc;
     if (rows * cols == 0) return ABS_OK;

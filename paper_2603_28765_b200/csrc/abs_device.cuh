@@ -8,8 +8,18 @@
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <nvtx3/nvToolsExt.h>
 
 namespace absq {
+
+// Host-side NVTX range around the enqueue work of one library call, so that a timeline tool shows which call
+// launched which kernels.  Header-only NVTX: without a tool attached a push / pop is one load and a branch.
+struct CallRange {
+    explicit CallRange(const char* name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+    CallRange(const CallRange&) = delete;
+    CallRange& operator=(const CallRange&) = delete;
+};
 
 enum ElemKind { EK_E2M1 = 0, EK_E2M0 = 1, EK_E2M3 = 2, EK_E3M2 = 3 };
 

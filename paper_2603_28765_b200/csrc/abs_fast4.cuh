@@ -135,16 +135,14 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
     }
 }
 
-#ifndef ABS_FAST_MINB
-#define ABS_FAST_MINB 4          // resident blocks of 256 threads per SM the IF4 instance is compiled for
-#endif
+constexpr int kFastMinBlocks = 4;   // resident blocks of 256 threads per SM the IF4 instance is compiled for
 
 // Grid-stride kernel: every thread encodes groups g, g + stride, ... (a handful of them: the host sizes the
 // grid as a few waves of resident blocks) and fetches the next group's 32 bytes before it works on the
 // current one, so loads stay in flight under the math.
 // IdxT is int32_t whenever the group count allows it (shorter address arithmetic).
 template <bool HAS_INT, typename IdxT, bool ALIGNED32, bool FROM_SLOT, bool SCALE_MUL, bool SWZ>
-__global__ void __launch_bounds__(256, HAS_INT ? ABS_FAST_MINB : 5)
+__global__ void __launch_bounds__(256, HAS_INT ? kFastMinBlocks : 5)
 quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
                       const AlphaSrc alpha_src, IdxT ngroups, uint32_t gpr, uint32_t ktiles, bool l2_prefetch) {
     pdl_launch_dependents();

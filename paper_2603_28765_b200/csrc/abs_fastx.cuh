@@ -506,13 +506,11 @@ __device__ __forceinline__ void encode_body3(const float (&x)[16], const uint32_
     sbyte = sb | (flag ? 0x80u : 0u);                                        // S3
 }
 
-#ifndef ABS_IF3_MINB
-#define ABS_IF3_MINB 3           // resident blocks of 256 threads per SM the IF3 kernel is compiled for
-#endif
+constexpr int kIf3MinBlocks = 3;   // resident blocks of 256 threads per SM the IF3 kernel is compiled for
 
 // G = 16: one scale per thread's 16 values.  G = 8 (IF3-BS8): each half has its own scale and selection.
 template <int G, bool FROM_SLOT, bool EMUL = false>
-__global__ void __launch_bounds__(256, ABS_IF3_MINB)
+__global__ void __launch_bounds__(256, kIf3MinBlocks)
 quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes, uint8_t* __restrict__ scales,
                       const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, bool aligned32,
                       uint4* __restrict__ out = nullptr, bool out_aligned32 = false, bool store_codes = true) {

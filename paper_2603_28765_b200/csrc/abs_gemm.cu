@@ -370,6 +370,7 @@ size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k
 abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
                         const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
                         void* workspace, size_t workspace_bytes, void* stream) {
+    const absq::CallRange range("abs_matmul");
     if (fmt != ABS_FMT_IF4 && fmt != ABS_FMT_NVFP4) return ABS_ERR_FMT;
     if (!gemm_shape_ok(fmt, m, n, k)) return ABS_ERR_SHAPE;
     if (!a_codes || !a_scales || !a_alpha || !b_codes || !b_scales || !b_alpha || !c_f32 || !workspace) return ABS_ERR_NULL;

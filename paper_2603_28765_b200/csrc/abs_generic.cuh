@@ -8,15 +8,9 @@ namespace absq {
 
 constexpr int kThreads = 256;
 
-#ifndef ABS_AMAX_UNROLL
-#define ABS_AMAX_UNROLL 4        // 128-bit loads in flight per thread in the amax pass (input not 32-byte aligned)
-#endif
-#ifndef ABS_AMAX_V8
-#define ABS_AMAX_V8 2            // 256-bit loads in flight per thread when the input is 32-byte aligned
-#endif
-#ifndef ABS_AMAX_BPS
-#define ABS_AMAX_BPS 4           // blocks of 256 threads per SM in the amax pass
-#endif
+constexpr int kAmaxUnroll = 4;   // 128-bit loads in flight per thread in the amax pass (input not 32-byte aligned)
+constexpr int kAmaxV8 = 2;   // 256-bit loads in flight per thread when the input is 32-byte aligned
+constexpr int kAmaxBlocksPerSm = 4;   // blocks of 256 threads per SM in the amax pass
 
 // ------------------------------------------------------------------------------------------ amax
 
@@ -45,13 +39,13 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
         uint32_t m0 = 0u, m1 = 0u;
         int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
         if ((reinterpret_cast<uintptr_t>(in) & 31u) == 0) {
-            // 256-bit loads: one group of 16 values per load, ABS_AMAX_V8 loads in flight per thread
-            for (; i + (ABS_AMAX_V8 - 1) * stride < ngroups; i += ABS_AMAX_V8 * stride) {
-                uint32_t w[ABS_AMAX_V8][8];
+            // 256-bit loads: one group of 16 values per load, kAmaxV8 loads in flight per thread
+            for (; i + (kAmaxV8 - 1) * stride < ngroups; i += kAmaxV8 * stride) {
+                uint32_t w[kAmaxV8][8];
 #pragma unroll
-                for (int k = 0; k < ABS_AMAX_V8; ++k) load32B<true>(in + 2 * (i + k * stride), w[k]);
+                for (int k = 0; k < kAmaxV8; ++k) load32B<true>(in + 2 * (i + k * stride), w[k]);
 #pragma unroll
-                for (int k = 0; k < ABS_AMAX_V8; ++k) {
+                for (int k = 0; k < kAmaxV8; ++k) {
                     m0 = __vmaxu2(m0, __vmaxu2(__vmaxu2(w[k][0] & 0x7FFF7FFFu, w[k][1] & 0x7FFF7FFFu),
                                                __vmaxu2(w[k][2] & 0x7FFF7FFFu, w[k][3] & 0x7FFF7FFFu)));
                     m1 = __vmaxu2(m1, __vmaxu2(__vmaxu2(w[k][4] & 0x7FFF7FFFu, w[k][5] & 0x7FFF7FFFu),
@@ -68,12 +62,12 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const uint4* __restrict_
             }
             i = nvec;
         }
-        for (; i + (ABS_AMAX_UNROLL - 1) * stride < nvec; i += ABS_AMAX_UNROLL * stride) {
-            uint4 v[ABS_AMAX_UNROLL];
+        for (; i + (kAmaxUnroll - 1) * stride < nvec; i += kAmaxUnroll * stride) {
+            uint4 v[kAmaxUnroll];
 #pragma unroll
-            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) v[k] = __ldg(in + i + k * stride);
+            for (int k = 0; k < kAmaxUnroll; ++k) v[k] = __ldg(in + i + k * stride);
 #pragma unroll
-            for (int k = 0; k < ABS_AMAX_UNROLL; ++k) {
+            for (int k = 0; k < kAmaxUnroll; ++k) {
                 m0 = __vmaxu2(m0, __vmaxu2(v[k].x & 0x7FFF7FFFu, v[k].y & 0x7FFF7FFFu));
                 m1 = __vmaxu2(m1, __vmaxu2(v[k].z & 0x7FFF7FFFu, v[k].w & 0x7FFF7FFFu));
             }

@@ -19,10 +19,7 @@ namespace absq {
 // the four groups of 16 rows; those are neighbours in the transposed output, so their codes leave as one
 // 256-bit store and their scale bytes as one 32-bit store whenever the tile is complete and the output
 // addresses allow it.
-#ifndef ABS_TRANS_UNROLL
-#define ABS_TRANS_UNROLL 4
-#endif
-constexpr int kTransUnroll = ABS_TRANS_UNROLL;
+constexpr int kTransUnroll = 4;
 constexpr int kTransTileCols = 256;
 constexpr int kTransTileRowBlocks = 4;
 constexpr int kTransStageElems = 16 * kTransTileRowBlocks * kTransTileCols;        // bf16 elements per stage

@@ -1,6 +1,6 @@
 """Per-configuration throughput table of the library's kernels (run on a B200 machine).
 
-    python -m paper_2603_28765_b200.report [--quick] [--only CFG[:FMT]] [--rows R] [--transposed]
+    python -m paper_2603_28765_b200.report [--quick] [--only CFG[:FMT]] [--rows R] [--transposed] [--matmul]
 
 ``--only cfg4:if4 --rows 4096 --quick`` restricts the run to one configuration (and format) at a reduced
 row count: the small case to put under a profiler.
@@ -11,7 +11,8 @@ that rotate over enough buffer sets to defeat L2 reuse between calls:
   T2  abs_quantize end to end (amax pass + group-quantize)   bytes = 4N + codes + scales (DRAM basis)
   T3  abs_dequantize                                         bytes = codes + scales + 2N
   T4  abs_quantize_dequantize (amax pass + one-pass emulation, no code outputs)
-and prints one JSON line per row.  With ``--transposed`` it times abs_quantize_transposed instead (the kernel
+and prints one JSON line per row, with the same three figures for a warm L2 (one buffer set reused) and the
+first 16 hex digits of the SHA-256 of the first input set and of its codes and scale bytes.  With ``--transposed`` it times abs_quantize_transposed instead (the kernel
 alone, alpha given; the same bytes move), for IF4 and NVFP4 with and without the gradient options.  Inputs are random bf16 tensors of the configuration's shape
 (timing does not depend on the values beyond the INT/FP mix); parity is the test suite's job.
 """
@@ -31,6 +32,7 @@ def main():
     ap.add_argument("--only", default="", help="one configuration, optionally one format: cfg4 or cfg4:if4")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (smaller case for profiling)")
     ap.add_argument("--transposed", action="store_true", help="time abs_quantize_transposed (groups down the columns)")
+    ap.add_argument("--matmul", action="store_true", help="time abs_matmul (square sizes; --rows picks one size)")
     args = ap.parse_args()
     L = B.lib()
     reps = 10 if args.quick else 40
@@ -47,6 +49,10 @@ def main():
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
+    def digest(t):
+        import hashlib
+        return hashlib.sha256(t.cpu().numpy().tobytes()).hexdigest()[:16]
+
     H, S, S17 = B.ABS_F_HADAMARD16, B.ABS_F_STOCHASTIC, B.ABS_F_SR_SCALE_17_16
     rows_cfg = [
         ("cfg2", 8192, 4096, [("if4", 0)]),
@@ -58,6 +64,31 @@ def main():
     ]
     sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
     only_cfg, _, only_fmt = args.only.partition(":")
+    if args.matmul:
+        # abs_matmul (tcgen05 kernel, Sec. 5.2 arithmetic) against the split path built from cuBLAS GEMMs and the
+        # BF16 emulation of Sec. 4.1; operands N(0,1) and N(0, 0.02^2)
+        from . import gemm
+        for size in ([args.rows] if args.rows else [2048, 4096, 8192]):
+            m = n = kk = size
+            x = torch.randn(m, kk, device="cuda").to(torch.bfloat16)
+            w = (torch.randn(n, kk, device="cuda") * 0.02).to(torch.bfloat16)
+            for fname in ("if4", "nvfp4"):
+                fmt = B.FMT_NAMES[fname]
+                qa, qb = B.abs_quantize(fmt, x), B.abs_quantize(fmt, w)
+                ws = torch.empty(L.abs_matmul_workspace_bytes(fmt, m, n, kk) + 1024, dtype=torch.uint8, device="cuda")
+                out = torch.empty((m, n), dtype=torch.float32, device="cuda")
+                t = loop_time(lambda i: B.abs_matmul(fmt, qa, qb, m, n, kk, out=out, workspace=ws))
+                B.abs_matmul(fmt, qa, qb, m, n, kk, out=out, workspace=ws, check=True)
+                row = {"matmul": [m, n, kk], "fmt": fname, "abs_matmul_ms": round(t, 4),
+                       "useful_TFLOPs": round(2.0 * m * n * kk / t / 1e9, 1),
+                       "mma_TFLOPs": round((9 if fname == "if4" else 1) * 2.0 * m * n * kk / t / 1e9, 1)}
+                if fname == "if4":
+                    row["split_path_cublas_ms"] = round(loop_time(lambda i: gemm.matmul_mac_split(qa, qb, m, n, kk)), 4)
+                    row["bf16_emulation_ms"] = round(loop_time(lambda i: gemm.matmul_emulated(qa, qb, m, n, kk)), 4)
+                    ref = gemm.matmul_mac_split(qa, qb, m, n, kk)
+                    row["max_diff_vs_split_path"] = float((out - ref).abs().max() / ref.abs().max())
+                print(json.dumps(row), flush=True)
+        return
     if args.transposed:
         for name, rows, cols in (("cfg2", 8192, 4096), ("cfg4", 16384, 8192)):
             if only_cfg and name != only_cfg:
@@ -116,6 +147,14 @@ def main():
             t1 = loop_time(lambda i: L.abs_quantize_ex(*qa[i % k]))
             t2 = loop_time(lambda i: L.abs_quantize_ex(*fa[i % k]))
             t3 = loop_time(lambda i: L.abs_dequantize(*da[i % k]))
+            # warm L2: the same buffer set every call (tensors up to about 100 MB stay in the 126 MB L2)
+            t1w = loop_time(lambda i: L.abs_quantize_ex(*qa[0]))
+            t2w = loop_time(lambda i: L.abs_quantize_ex(*fa[0]))
+            t3w = loop_time(lambda i: L.abs_dequantize(*da[0]))
+            # fingerprints of what was timed: SHA-256 of the first input set and of its outputs
+            L.abs_quantize_ex(*fa[0])
+            torch.cuda.synchronize()
+            sha = {"input": digest(xs[0].view(torch.int16)), "codes": digest(codes[0]), "scales": digest(scales[0])}
             t4 = None
             if fmt in (B.ABS_FMT_NVFP4, B.ABS_FMT_IF4) or not (flags & (H | S)):
                 ea = [(fmt, xs[i].data_ptr(), rows, cols, outs[i % len(outs)].data_ptr(), None, None, ts[i].data_ptr(),
@@ -133,6 +172,8 @@ def main():
                 "T3_dequantize_us": round(t3 * 1e3, 1), "T3_GBs": round((2 * n + outb) / t3 / 1e6),
                 "T4_quantize_dequantize_us": round(t4 * 1e3, 1) if t4 else None,
                 "elements_per_s_T2": round(n / (t2 * 1e-3)),
+                "warm_l2_us": {"T1": round(t1w * 1e3, 1), "T2": round(t2w * 1e3, 1), "T3": round(t3w * 1e3, 1)},
+                "sha256_16": sha,
             }), flush=True)
             del codes, scales, outs
         del xs
