@@ -194,6 +194,7 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
     const int grid = grid_for(sm_count, ngroups, 64);
     const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     const uint64_t ctr = o.sr_index_offset / 8;      // Philox block of the call's first element (even: offset % 16 == 0)
+    const PhiloxKeys pk = philox_keys(o.sr_seed);
     if (g_ev_quant_begin) cudaEventRecord(g_ev_quant_begin, s);
     if constexpr (FMT == ABS_FMT_NVFP4 || FMT == ABS_FMT_IF4) {
         if (emul_out) return ABS_ERR_FLAGS;      // the 4-bit emulation pass is launched by abs_quantize_dequantize
@@ -242,10 +243,10 @@ abs_status_t launch_quantize_fmt(int sm_count, const void* in, int64_t ngroups, 
 #define ABS_LAUNCH_O(R, S)                                                                                        \
     e = alpha.slot ? launch_pdl(quantize4_opt_kernel<kInt, R, S, true, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, ctr, a32, (uint4*)nullptr, false, true)             \
+                                (uint32_t)o.had_sign_mask, pk, ctr, a32, (uint4*)nullptr, false, true)             \
                    : launch_pdl(quantize4_opt_kernel<kInt, R, S, false, false>, ogrid, kThreads, s, (const uint4*)in, \
                                 (uint2*)codes, (uint8_t*)scales, alpha, (int32_t)ngroups, mul,                    \
-                                (uint32_t)o.had_sign_mask, k0, k1, ctr, a32, (uint4*)nullptr, false, true)
+                                (uint32_t)o.had_sign_mask, pk, ctr, a32, (uint4*)nullptr, false, true)
             if (rht && sr) ABS_LAUNCH_O(true, true);
             else if (rht) ABS_LAUNCH_O(true, false);
             else ABS_LAUNCH_O(false, true);
@@ -677,13 +678,13 @@ abs_status_t abs_quantize_dequantize(abs_fmt_t fmt, const void* in_bf16, int64_t
         return (!handled && rc == ABS_ERR_FLAGS) ? ABS_ERR_SIZE : rc;
     }
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
-    const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     const uint64_t ctr = o.sr_index_offset / 8;
+    const PhiloxKeys pk = philox_keys(o.sr_seed);
     const bool a32 = (reinterpret_cast<uintptr_t>(in_bf16) & 31u) == 0, o32 = (reinterpret_cast<uintptr_t>(out_bf16) & 31u) == 0;
     cudaError_t e = cudaSuccess;
 #define ABS_LAUNCH_E3(I, R, S, SLOT)                                                                                \
     e = launch_pdl(quantize4_opt_kernel<I, R, S, SLOT, true>, grid, kThreads, s, (const uint4*)in_bf16, (uint2*)codes_u8, \
-                   (uint8_t*)scales_e4m3, src, (int32_t)ngroups, mul, (uint32_t)o.had_sign_mask, k0, k1, ctr, a32,   \
+                   (uint8_t*)scales_e4m3, src, (int32_t)ngroups, mul, (uint32_t)o.had_sign_mask, pk, ctr, a32,       \
                    (uint4*)out_bf16, o32, store)
 #define ABS_LAUNCH_E2(I, R, S)                                                                                      \
     do {                                                                                                            \
@@ -779,7 +780,7 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
                                  kTransSmemBytes);                                                                  \
         if (e == cudaSuccess)                                                                                       \
             e = cudaLaunchKernelEx(&cfg, transposed_kernel<I, S, R, Q, M, E>(), in, ct, stp, src, rows, cols, mask, \
-                                   SLOT, GEN, mul, k0, k1, ctr, (uint16_t*)out_bf16, store_codes);                  \
+                                   SLOT, GEN, mul, pk, ctr, (uint16_t*)out_bf16, store_codes);                      \
     } while (0)
 #define ABS_LAUNCH_T(I, S, R, Q, M, SLOT, GEN)                                                                      \
     do {                                                                                                            \
@@ -789,8 +790,8 @@ static abs_status_t quantize_transposed_impl(abs_fmt_t fmt, const void* in_bf16,
 
     const bool sr = o.flags & ABS_F_STOCHASTIC;
     const float mul = (o.flags & ABS_F_SR_SCALE_17_16) ? 1.0625f : 1.0f;
-    const uint32_t k0 = (uint32_t)o.sr_seed, k1 = (uint32_t)(o.sr_seed >> 32);
     const uint64_t ctr = o.sr_index_offset / 8;
+    const PhiloxKeys pk = philox_keys(o.sr_seed);
     AlphaSrc src = {tensor_scale_f32, nullptr, 0u, 0.0f, tensor_scale_f32, nullptr};
     if (!(o.flags & ABS_F_ALPHA_GIVEN)) {
         unsigned long long* slot = nullptr;

@@ -175,8 +175,8 @@ constexpr int opt_blocks_per_sm(bool sr, bool rht = true) { return sr ? 2 : (rht
 template <bool HAS_INT, bool RHT, bool SR, bool FROM_SLOT, bool EMUL>
 __global__ void __launch_bounds__(256, opt_blocks_per_sm(SR, RHT))
 quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                     const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, uint32_t sign_mask, uint32_t seed_lo,
-                     uint32_t seed_hi, uint64_t ctr_base, bool aligned32, uint4* __restrict__ out, bool out_aligned32,
+                     const AlphaSrc alpha_src, int32_t ngroups, float scale_mul, uint32_t sign_mask,
+                     const PhiloxKeys keys, uint64_t ctr_base, bool aligned32, uint4* __restrict__ out, bool out_aligned32,
                      bool store_codes) {
     pdl_launch_dependents();
     const int32_t stride = (int32_t)(gridDim.x * blockDim.x);
@@ -218,8 +218,8 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
             // Philox blocks 2g and 2g+1 hold the sixteen 16-bit fields of elements 16g .. 16g+15; ctr_base (even)
             // is the block index of the call's first element in the whole tensor (sr_index_offset / 8)
             const uint64_t i8 = ctr_base + (uint64_t)(uint32_t)g * 2u;
-            const uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
-            const uint4 p1 = philox4x32_10((uint32_t)i8 + 1u, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
+            const uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), keys);
+            const uint4 p1 = philox4x32_10((uint32_t)i8 + 1u, (uint32_t)(i8 >> 32), keys);
             rnd[0] = p0.x; rnd[1] = p0.y; rnd[2] = p0.z; rnd[3] = p0.w;
             rnd[4] = p1.x; rnd[5] = p1.y; rnd[6] = p1.z; rnd[7] = p1.w;
         }

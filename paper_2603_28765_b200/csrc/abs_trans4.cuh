@@ -73,7 +73,7 @@ __device__ __forceinline__ void quantize4_transposed_body(const uint16_t* __rest
                                                           uint8_t* __restrict__ scales_t, const AlphaSrc alpha_src,
                                                           int64_t rows, int64_t cols, uint32_t sign_mask,
                                                           unsigned long long* amax_slot, uint32_t amax_gen,
-                                                          float scale_mul, uint32_t seed_lo, uint32_t seed_hi,
+                                                          float scale_mul, const PhiloxKeys& keys,
                                                           uint64_t ctr_base, uint16_t* __restrict__ out,
                                                           bool store_codes) {
     extern __shared__ __align__(16) uint16_t trans_smem[];
@@ -179,8 +179,8 @@ __device__ __forceinline__ void quantize4_transposed_body(const uint16_t* __rest
                 if constexpr (SR) {
                     if (sb != 0u) {
                         const uint64_t i8 = ctr_base + (uint64_t)g * 2u;   // Philox blocks 2g, 2g+1: elements 16g .. 16g+15
-                        const uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
-                        const uint4 p1 = philox4x32_10((uint32_t)i8 + 1u, (uint32_t)(i8 >> 32), seed_lo, seed_hi);
+                        const uint4 p0 = philox4x32_10((uint32_t)i8, (uint32_t)(i8 >> 32), keys);
+                        const uint4 p1 = philox4x32_10((uint32_t)i8 + 1u, (uint32_t)(i8 >> 32), keys);
                         const uint32_t rnd[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
                         encode_body4_sr<HAS_INT>(x, rnd, sb, d, r, sbyte, c_lo, c_hi);
                     }
@@ -258,10 +258,10 @@ __device__ __forceinline__ void quantize4_transposed_body(const uint16_t* __rest
 #define ABS_TRANS_PARAMS                                                                                              \
     const uint16_t *__restrict__ in, uint2 *__restrict__ codes_t, uint8_t *__restrict__ scales_t,                     \
         const AlphaSrc alpha_src, int64_t rows, int64_t cols, uint32_t sign_mask, unsigned long long *amax_slot,      \
-        uint32_t amax_gen, float scale_mul, uint32_t seed_lo, uint32_t seed_hi, uint64_t ctr_base,                    \
+        uint32_t amax_gen, float scale_mul, const PhiloxKeys keys, uint64_t ctr_base,                                   \
         uint16_t *__restrict__ out, bool store_codes
 #define ABS_TRANS_ARGS                                                                                                \
-    in, codes_t, scales_t, alpha_src, rows, cols, sign_mask, amax_slot, amax_gen, scale_mul, seed_lo, seed_hi,        \
+    in, codes_t, scales_t, alpha_src, rows, cols, sign_mask, amax_slot, amax_gen, scale_mul, keys,                    \
         ctr_base, out, store_codes
 
 // Round-to-nearest and Hadamard instances are held to the registers of three blocks per SM (what the shared
