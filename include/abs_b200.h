@@ -29,9 +29,8 @@
  *     return ABS_ERR_SIZE once, so the overrun cannot pass unseen.
  *   - CUDA graphs: the slot and its tag are kernel arguments fixed at enqueue time, so a captured
  *     call of that kind must not be replayed (a replay would merge its maximum with the previous
- *     replay's).  Inside a graph use ABS_F_ALPHA_GIVEN with an alpha computed outside the graph,
- *     or abs_quantize_noalloc, whose nodes re-arm their own scratch.  Calls with
- *     ABS_F_ALPHA_GIVEN, and every dequantize call, use no scratch and may be captured.
+ *     replay's).  Inside a graph use ABS_F_ALPHA_GIVEN with an alpha computed outside the graph.
+ *     Calls with ABS_F_ALPHA_GIVEN, and every dequantize call, use no scratch and may be captured.
  * There is no CPU fallback: without a CUDA device every compute call returns ABS_ERR_CUDA.
  */
 #ifndef ABS_B200_H

@@ -402,12 +402,15 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
                                                     (uint2*)(ws + off + 2 * plane), ws + (op ? L.off_sfb : L.off_sfa));
         if (cudaGetLastError() != cudaSuccess) return ABS_ERR_CUDA;
     }
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, []() {
-        attr_err = cudaFuncSetAttribute(if4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    // the opt-in to more than 48 KiB of dynamic shared memory is per device
+    static std::once_flag attr_once[64];
+    static cudaError_t attr_err[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ABS_ERR_CUDA;
+    std::call_once(attr_once[dev], [dev]() {
+        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     });
-    if (attr_err != cudaSuccess) return ABS_ERR_CUDA;
+    if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
     const dim3 grid((unsigned)(n / kTileN), (unsigned)(m / kTileM));
     if4_gemm_kernel<<<grid, 128, kGemmSmemBytes, s>>>(maps, ws + L.off_sfa, ws + L.off_sfb, a_alpha, b_alpha, c_f32, (int32_t)n,
                                                       (int32_t)(k / kStageK), planes, (int*)ws);

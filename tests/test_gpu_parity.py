@@ -873,3 +873,35 @@ def test_tensor_core_matmul_matches_mac_reference(B, oracle, fmt):
     assert L.abs_matmul(fmt, *args, 128, 128, 192, out.data_ptr(), ws.data_ptr(), 4096, None) == 2      # k % 256
     assert L.abs_matmul(3, *args, 128, 128, 256, out.data_ptr(), ws.data_ptr(), 4096, None) == 4        # format
     assert L.abs_matmul(fmt, *args, 128, 128, 256, out.data_ptr(), ws.data_ptr(), 4096, None) in (3, 7)  # alignment or size
+
+
+def test_calls_without_scratch_replay_from_a_cuda_graph(B, oracle):
+    """The header allows capturing the calls that use no scratch: abs_quantize_ex with ABS_F_ALPHA_GIVEN and
+    abs_dequantize.  Captured once, replayed on two different tensors copied into the same input buffer, the
+    outputs must be the oracle's both times."""
+    rows, cols = 96, 1024
+    xs = [I.generate("cfg1", rows, cols, seed=s) for s in (3, 4)]
+    alpha = 0.0042
+    x = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    ts = torch.tensor([alpha], dtype=torch.float32, device="cuda")
+    codes = torch.empty(rows * cols // 2, dtype=torch.uint8, device="cuda")
+    scales = torch.empty(rows * cols // 16, dtype=torch.uint8, device="cuda")
+    out = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    opts = B.make_opts(B.ABS_F_ALPHA_GIVEN)
+    B.abs_quantize(1, x, codes, scales, ts, opts=opts)            # first call on the device happens outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            B.abs_quantize(1, x, codes, scales, ts, opts=opts, stream=s)
+            B.abs_dequantize(1, codes, scales, ts, rows, cols, out=out, stream=s)
+    for xb in xs:
+        x.copy_(to_dev(xb))
+        g.replay()
+        torch.cuda.synchronize()
+        oc, osc, oa = oracle.quantize(1, xb, flags=oracle.F_ALPHA_GIVEN, alpha=alpha)
+        assert_same("graph codes", codes.cpu().numpy().reshape(rows, -1), oc)
+        assert_same("graph scales", scales.cpu().numpy().reshape(rows, -1), osc)
+        assert_same("graph dequant", out.view(torch.int16).cpu().numpy().view(np.uint16),
+                    oracle.dequantize(1, oc, osc, oa, rows, cols))
