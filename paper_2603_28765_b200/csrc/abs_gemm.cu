@@ -41,8 +41,9 @@ constexpr uint32_t kWaitLimit = 1u << 22;          // polls of one mbarrier wait
 
 // Splits the 16 codes of one group (two words) into the planes F, H, L and writes the magnitude of its scale byte
 // into the 128x4-tile layout the tensor core reads.  FP groups: F = codes.  Integer groups (two's complement
-// nibbles): sign s, magnitude m = |k|; H = s | e2m1(m - (m is 5 or 7)), L = s | e2m1(1) where m is 5 or 7.
-// E2M1 codes of the integers 0, 1, 2, 3, 4, 6 are 0, 2, 4, 5, 6, 7.
+// nibbles): sign s, magnitude m = |k|; H = s | e2m1(h), L = s | e2m1(l) with m = h + l, h in {0, 1, 2, 3, 4, 6} and
+// l = 1 for m = 5 or 7, l = 2 for m = 8 (the most negative code, which no quantizer writes but dequantize reads as
+// -8), else 0.  E2M1 codes of the integers 0, 1, 2, 3, 4, 6 are 0, 2, 4, 5, 6, 7.
 __device__ __forceinline__ void split_word(uint32_t w, bool is_int, uint32_t& f, uint32_t& h, uint32_t& l) {
     if (!is_int) { f = w; h = 0u; l = 0u; return; }
     f = 0u; h = 0u; l = 0u;
@@ -50,11 +51,11 @@ __device__ __forceinline__ void split_word(uint32_t w, bool is_int, uint32_t& f,
     for (int j = 0; j < 8; ++j) {
         const int k = (int)((w >> (4 * j)) << 28) >> 28;             // sign-extended nibble
         const uint32_t m = (uint32_t)(k < 0 ? -k : k), s = k < 0 ? 8u : 0u;
-        const bool odd57 = (m == 5u) || (m >= 7u);                    // m = 8 (never produced) is treated as 7 + 1
-        const uint32_t mh = odd57 ? m - 1u : m;                       // 0, 1, 2, 3, 4, 6
+        const uint32_t ml = (m == 5u || m == 7u) ? 1u : (m == 8u ? 2u : 0u);
+        const uint32_t mh = m - ml;                                   // 0, 1, 2, 3, 4, 6
         const uint32_t ch = mh <= 1u ? 2u * mh : (mh <= 4u ? mh + 2u : 7u);
         h |= ((m ? s : 0u) | ch) << (4 * j);
-        l |= (odd57 ? (s | 2u) : 0u) << (4 * j);
+        l |= (ml ? (s | (2u * ml)) : 0u) << (4 * j);
     }
 }
 

@@ -905,3 +905,30 @@ def test_calls_without_scratch_replay_from_a_cuda_graph(B, oracle):
         assert_same("graph scales", scales.cpu().numpy().reshape(rows, -1), osc)
         assert_same("graph dequant", out.view(torch.int16).cpu().numpy().view(np.uint16),
                     oracle.dequantize(1, oc, osc, oa, rows, cols))
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_tensor_core_matmul_on_arbitrary_bytes(B, oracle, fmt):
+    """abs_matmul on operands that no quantizer produced: random code bytes (every nibble, the most negative integer
+    code and FP minus zero included) and random finite scale bytes with and without bit 7 -- all-FP tensors, all-integer
+    tensors and mixtures, so each of the three accumulators is exercised alone and together -- against the float64
+    reference built from the oracle's dequantize.  Plain NVFP4 must ignore bit 7 of its scale bytes."""
+    m, n, k = 128, 256, 512
+    rng = np.random.default_rng(5)
+    for a_flags, b_flags in (("mixed", "mixed"), ("fp", "fp"), ("int", "int"), ("fp", "int"), ("int", "mixed")):
+        ops = []
+        for rows, kind in ((m, a_flags), (n, b_flags)):
+            codes = rng.integers(0, 256, (rows, k // 2), dtype=np.uint8)
+            mag = rng.integers(0x20, 0x50, (rows, k // 16), dtype=np.uint8)       # scales 2^-3 .. 2^3: sums stay moderate
+            bit7 = {"fp": 0, "int": 0x80}.get(kind)
+            if bit7 is None:
+                bit7 = (rng.integers(0, 2, mag.shape, dtype=np.uint8) << 7).astype(np.uint8)
+            scales = (mag | bit7).astype(np.uint8)
+            scales[rows // 2, :4] = [0x00, 0x80, 0x01, 0x7E]                       # zero scale, flagged zero, smallest, largest
+            ops.append((codes, scales, np.float32(0.75 if rows == m else 1.5)))
+        ref = oracle.mac_matmul_reference(fmt, ops[0], ops[1], m, n, k)
+        dev = [(torch.from_numpy(c).cuda(), torch.from_numpy(s).cuda(), torch.tensor([a], dtype=torch.float32, device="cuda"))
+               for c, s, a in ops]
+        c = B.abs_matmul(fmt, dev[0], dev[1], m, n, k, check=True).double().cpu().numpy()
+        err = np.abs(c - ref).max() / np.abs(ref).max()
+        assert err < 2e-5, (fmt, a_flags, b_flags, err)
