@@ -55,9 +55,10 @@ __device__ __forceinline__ uint32_t e2m1x8_encode(const float (&y)[8]) {
 // CLAMP is the rare variant for scale bytes that are subnormal (1..7) or saturated (0x7E): there
 // |y * 7/6| can exceed 7.5, so the integer candidate must be clamped to +-7; for every other scale
 // byte |y| <= 6 * 17/16 and the rounded integer is within +-7 by construction.
-template <bool HAS_INT, bool CLAMP>
+// D_INT_GIVEN: the caller also passes d * fp32(6/7) (from the block's table) instead of having it computed here.
+template <bool HAS_INT, bool CLAMP, bool D_INT_GIVEN = false>
 __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, float d, float r, uint32_t& sbyte,
-                                             uint32_t& c_lo, uint32_t& c_hi) {
+                                             uint32_t& c_lo, uint32_t& c_hi, float d_int_given = 0.0f) {
     const uint64_t R2 = pack2(r, r);
     if constexpr (!HAS_INT) {
 #pragma unroll
@@ -72,7 +73,7 @@ __device__ __forceinline__ void encode_body4(const float (&x)[16], uint32_t sb, 
     } else {
         const float c_pre = __uint_as_float(0x3F955555u);    // fp32(7/6)
         const float c_post = __uint_as_float(0x3F5B6DB7u);   // fp32(6/7)
-        const float d_int = __fmul_rn(d, c_post);
+        const float d_int = D_INT_GIVEN ? d_int_given : __fmul_rn(d, c_post);
         const uint64_t ND2 = pack2(-d, -d), NDI2 = pack2(-d_int, -d_int), CP2 = pack2(c_pre, c_pre);
         const uint64_t MG2 = pack2(kMagic8, kMagic8);
         uint64_t accF[2], accI[2];                                           // (S0,S1) and (S2,S3) chains
@@ -160,6 +161,13 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
     auto at = [&](IdxT gg) -> IdxT { return (FROM_SLOT && !HAS_INT) ? (IdxT)(ngroups - 1 - gg) : gg; };
     if (active) load32B<ALIGNED32>(in + 2 * (size_t)at(g), w);
     const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
+    // G5 once per block for every scale byte 0x00..0x7E: d = Delta * alpha, 1 / d, d * 6/7 (8192x4096: 16.68 -> 16.56 us)
+    __shared__ float4 scale_lut[128];
+    if (threadIdx.x < 127) {
+        const float dd = __fmul_rn(e4m3_value(threadIdx.x), alpha);
+        scale_lut[threadIdx.x] = make_float4(dd, __frcp_rn(dd), __fmul_rn(dd, __uint_as_float(0x3F5B6DB7u)), 0.0f);
+    }
+    __syncthreads();
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     // one group: G1-G5, steps 3-10, stores
@@ -177,14 +185,16 @@ quantize4_fast_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, u
         float t = __fmul_rn(gmax, inv_a6);                                   // G2-G3 (Eq. 2)
         if constexpr (SCALE_MUL) t = __fmul_rn(t, 1.0625f);                  // the 17/16 option
         const uint32_t sb = e4m3_encode(t);
-        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
-        const float r = __frcp_rn(d);
         uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
+        // G5 from the block's table (d = Delta * alpha, 1 / d, d * 6/7: the same three roundings, done once per scale
+        // byte and block instead of once per group)
+        const float4 e = scale_lut[sb];
+        const float d = e.x, r = e.y;
         if ((sb - 8u) >= 118u) {
             // rare path: zero scale (G4: all codes 0), subnormal scale bytes 1..7 and the saturated 0x7E
-            if (sb != 0u) encode_body4<HAS_INT, HAS_INT>(x, sb, d, r, sbyte, c_lo, c_hi);
+            if (sb != 0u) encode_body4<HAS_INT, HAS_INT, true>(x, sb, d, r, sbyte, c_lo, c_hi, e.z);
         } else {
-            encode_body4<HAS_INT, false>(x, sb, d, r, sbyte, c_lo, c_hi);
+            encode_body4<HAS_INT, false, true>(x, sb, d, r, sbyte, c_lo, c_hi, e.z);
         }
         scales[scale_offset<SWZ>((size_t)gg, gpr, ktiles)] = (uint8_t)sbyte;
         codes[gg] = make_uint2(c_lo, c_hi);
