@@ -14,7 +14,7 @@
 // FP32 accumulation up to its rounding of the running sum, which is what the float64 reference is compared to.
 //
 // Kernel: one 128 x 128 tile of C per block.  One thread feeds the pipeline with TMA (cp.async.bulk.tensor.2d,
-// 128-byte swizzle, no multicast; the scale tiles with plain bulk copies), one thread copies the scales to tensor
+// 128-byte swizzle, each load for this CTA alone; the scale tiles with plain bulk copies), one thread copies the scales to tensor
 // memory (tcgen05.cp) and issues the MMAs, four warps read the accumulators back (tcgen05.ld) and write C.
 // Every mbarrier wait is bounded: when a wait runs out the block raises an error word, stops issuing, frees its
 // tensor memory and returns.
