@@ -932,3 +932,52 @@ def test_tensor_core_matmul_on_arbitrary_bytes(B, oracle, fmt):
         c = B.abs_matmul(fmt, dev[0], dev[1], m, n, k, check=True).double().cpu().numpy()
         err = np.abs(c - ref).max() / np.abs(ref).max()
         assert err < 2e-5, (fmt, a_flags, b_flags, err)
+
+
+def test_scratch_ring_overrun_is_reported(B, oracle):
+    """More than ABS_MAX_INFLIGHT amax-carrying calls enqueued between the two kernels of one call: that call loses
+    its maximum.  Provoked without any fault: stream A first runs a bounded delay kernel, then one abs_quantize;
+    while A is delayed, stream B runs 1100 abs_quantize calls, which wraps the ring of 1024 slots past A's slot.
+    A's group-quantize kernel then finds another call's tag in its slot and raises the flag: the next call that
+    takes a slot returns ABS_ERR_SIZE (7) exactly once, and the library works normally afterwards."""
+    import ctypes
+    L = B.lib()
+    xb = I.generate("cfg1", 64, 256)
+    x = to_dev(xb)
+    a, b = torch.cuda.Stream(), torch.cuda.Stream()
+    outs_b = B.abs_quantize(1, x)                      # buffers reused by every call on stream B
+    codes_a, scales_a, ts_a = B.abs_quantize(1, x)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(a):
+        torch.cuda._sleep(400_000_000)                  # about 0.2 s at 2 GHz: a bounded busy-wait, nothing else
+        B.abs_quantize(1, x, codes_a, scales_a, ts_a, stream=a)
+    for _ in range(1100):
+        B.abs_quantize(1, x, outs_b[0], outs_b[1], outs_b[2], stream=b)
+    torch.cuda.synchronize()
+    sp = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    args = (1, x.data_ptr(), 64, 256, outs_b[0].data_ptr(), outs_b[1].data_ptr(), outs_b[2].data_ptr(), sp)
+    assert L.abs_quantize(*args) == 7                   # the overrun of the delayed call is reported here ...
+    assert L.abs_quantize(*args) == 0                   # ... once
+    torch.cuda.synchronize()
+    assert float(ts_a.item()) == 1.0                    # the overrun call fell back to alpha = 1, visibly
+    check_case(B, oracle, 1, xb)                        # and everything is back to normal
+
+
+def test_tensor_core_matmul_full_size_sampled(B, oracle):
+    """abs_matmul at 4096 x 4096 x 4096 (the size its timing is quoted on): 48 sampled rows of A against 48 sampled
+    rows of B give a 48 x 48 sample of C that the float64 reference can compute; first and last rows included."""
+    m = n = k = 4096
+    a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+    qa, qb = B.abs_quantize(1, to_dev(a)), B.abs_quantize(1, to_dev(b))
+    c = B.abs_matmul(1, qa, qb, m, n, k, check=True)
+    rng = np.random.default_rng(17)
+    ra = np.array(sorted(set([0, m - 1] + [int(v) for v in rng.integers(0, m, 46)])))
+    rb = np.array(sorted(set([0, n - 1] + [int(v) for v in rng.integers(0, n, 46)])))
+    alpha_a, alpha_b = np.float32(qa[2].item()), np.float32(qb[2].item())
+    oa = oracle.quantize(1, np.ascontiguousarray(a[ra]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_a)
+    ob = oracle.quantize(1, np.ascontiguousarray(b[rb]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_b)
+    assert np.array_equal(qa[0].view(m, k // 2)[torch.from_numpy(ra).cuda()].cpu().numpy(), oa[0])     # same operands
+    ref = oracle.mac_matmul_reference(1, oa, ob, len(ra), len(rb), k)
+    got = c[torch.from_numpy(ra).cuda()][:, torch.from_numpy(rb).cuda()].double().cpu().numpy()
+    scale = float(c.abs().max().item())
+    assert np.abs(got - ref).max() <= 2e-5 * scale, np.abs(got - ref).max() / scale

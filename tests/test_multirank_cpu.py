@@ -40,6 +40,12 @@ def _shard_worker(rank, world, port, out_dir):
     dist.all_reduce(a, op=dist.ReduceOp.MAX)                       # the only exchange: 4 bytes
     alpha = O.alpha_from_amax(O.FMT_IF4, np.float32(a.item()))
     c, s, _ = O.quantize(O.FMT_IF4, local, flags=O.F_ALPHA_GIVEN, alpha=alpha)
+    # the same shard with stochastic rounding: App. B's stream runs over the whole tensor, so the shard passes the
+    # index of its first element
+    cs, ss, _ = O.quantize(O.FMT_IF4, local, flags=O.F_ALPHA_GIVEN | O.F_STOCHASTIC, alpha=alpha, sr_seed=31,
+                           sr_index_offset=lo * xb.shape[1])
+    np.save(os.path.join(out_dir, f"sr_codes{rank}.npy"), cs)
+    np.save(os.path.join(out_dir, f"sr_scales{rank}.npy"), ss)
     np.save(os.path.join(out_dir, f"codes{rank}.npy"), c)
     np.save(os.path.join(out_dir, f"scales{rank}.npy"), s)
     np.save(os.path.join(out_dir, f"alpha{rank}.npy"), np.array([alpha], np.float32))
@@ -60,6 +66,9 @@ def test_row_sharded_protocol_matches_single_process(tmp_path):
     assert np.array_equal(codes, c) and np.array_equal(scales, s)
     for r in range(world):
         assert np.load(tmp_path / f"alpha{r}.npy")[0] == a
+    cs, ss, _ = O.quantize(O.FMT_IF4, xb, flags=O.F_STOCHASTIC, sr_seed=31)
+    assert np.array_equal(np.concatenate([np.load(tmp_path / f"sr_codes{r}.npy") for r in range(world)]), cs)
+    assert np.array_equal(np.concatenate([np.load(tmp_path / f"sr_scales{r}.npy") for r in range(world)]), ss)
 
 
 def test_reference_arm_prints_once_under_two_ranks():
