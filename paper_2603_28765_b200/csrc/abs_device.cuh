@@ -387,6 +387,18 @@ __device__ __forceinline__ float resolve_alpha_per_thread(const AlphaSrc& a) {
     return alpha;
 }
 
+// Per-block table of G5 for every scale byte 0x00..0x7E: d = Delta * alpha and its IEEE reciprocal depend only on
+// the byte, so a block computes the 127 pairs once and a group reads its pair with one 8-byte load instead of a
+// multiply, a multiply and a reciprocal (same operations, same bits).  Every thread of the block must call this
+// (it ends with a barrier); entry 0 (d = 0) is never read.
+__device__ __forceinline__ void fill_scale_table(float2* table, float alpha) {
+    if (threadIdx.x < 127) {
+        const float d = __fmul_rn(e4m3_value(threadIdx.x), alpha);
+        table[threadIdx.x] = make_float2(d, __frcp_rn(d));
+    }
+    __syncthreads();
+}
+
 // Byte offset of the scale of (row, k-th group of the row) in the 128x4-tile layout read by Blackwell
 // block-scaled MMAs; ktiles = ceil(groups_per_row / 4).
 __device__ __forceinline__ size_t swizzled_scale_offset(uint32_t row, uint32_t k, uint32_t ktiles) {

@@ -155,6 +155,8 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
         else load32B<false>(in + 2 * (size_t)g, w);
     }
     const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
+    __shared__ float2 scale_table[128];
+    fill_scale_table(scale_table, alpha);                                    // G5 for every scale byte, once per block
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     // one block of 16 values held in `w`, index `g`
@@ -172,8 +174,8 @@ quantize4_bs8_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
             const float gmax = max3abs(max3abs(xs[0], xs[1], xs[2]), max3abs(xs[3], xs[4], xs[5]), fmaxf(fabsf(xs[6]), fabsf(xs[7])));   // G1
             const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);   // G2
             const uint32_t sb = e4m3_encode(t);                              // G3
-            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
-            const float r = __frcp_rn(d);
+            const float2 dr = scale_table[sb];                                 // G5: d = Delta * alpha and 1 / d
+            const float d = dr.x, r = dr.y;
             uint32_t sbyte = 0u, c = 0u;
             if ((sb - 8u) >= 118u) {
                 if (sb != 0u) encode_half4<HAS_INT, HAS_INT>(xs, sb, d, r, sbyte, c);      // G4: zero scale -> zeros
@@ -545,7 +547,7 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
             const float gmax = fmaxf(max3abs(m0, m1, m2), max3abs(m3, m4, x[15]));
             const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);   // G2
             const uint32_t sb = e4m3_encode(t);                              // G3
-            const float d = __fmul_rn(e4m3_value(sb), alpha);                // G5
+            const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
             const float r = __frcp_rn(d);
             uint32_t sbyte = 0u;
             if ((sb - 8u) >= 118u) {
@@ -572,7 +574,7 @@ quantize3_fast_kernel(const uint4* __restrict__ in, uint16_t* __restrict__ codes
                                            fmaxf(fabsf(xs[6]), fabsf(xs[7])));              // G1
                 const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
                 const uint32_t sb = e4m3_encode(t);
-                const float d = __fmul_rn(e4m3_value(sb), alpha);
+                const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
                 const float r = __frcp_rn(d);
                 if (sb != 0u) {
                     uint32_t fc, ic;

@@ -190,6 +190,8 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
         else load32B<false>(in + 2 * (size_t)g, w);
     }
     const float alpha = resolve_alpha_per_thread<FROM_SLOT>(alpha_src);      // T2
+    __shared__ float2 scale_table[128];
+    fill_scale_table(scale_table, alpha);                                    // G5 for every scale byte, once per block
     if (!active) return;
     const float inv_a6 = __frcp_rn(__fmul_rn(alpha, 6.0f));                  // T3
     uint32_t smask[8];
@@ -231,8 +233,8 @@ quantize4_opt_kernel(const uint4* __restrict__ in, uint2* __restrict__ codes, ui
         // G2-G3 (Eq. 2), with the 17/16 option folded into scale_mul.
         const float t = __fmul_rn(__fmul_rn(gmax, inv_a6), scale_mul);
         const uint32_t sb = e4m3_encode(t);
-        const float d = __fmul_rn(e4m3_value(sb), alpha);                    // G5
-        const float r = __frcp_rn(d);
+        const float2 dr = scale_table[sb];                                 // G5: d = Delta * alpha and 1 / d
+        const float d = dr.x, r = dr.y;
         uint32_t sbyte = 0u, c_lo = 0u, c_hi = 0u;
         if constexpr (SR) {
             if (sb != 0u) encode_body4_sr<HAS_INT>(x, rnd, sb, d, r, sbyte, c_lo, c_hi);      // G4: zero scale -> zeros
