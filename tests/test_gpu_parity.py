@@ -981,3 +981,25 @@ def test_tensor_core_matmul_full_size_sampled(B, oracle):
     got = c[torch.from_numpy(ra).cuda()][:, torch.from_numpy(rb).cuda()].double().cpu().numpy()
     scale = float(c.abs().max().item())
     assert np.abs(got - ref).max() <= 2e-5 * scale, np.abs(got - ref).max() / scale
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_weight_gradient_product_from_transposed_quantize(B, oracle, fmt):
+    """Sec. 4.1: for the weight-gradient product dW = dY^T X both operands are quantized along the token dimension.
+    abs_quantize_transposed writes exactly the K-major codes and scales abs_matmul reads (K = tokens), so the two
+    calls compose without any layout step: dW from the library against the float64 MAC reference on the oracle's
+    quantization of the transposed operands."""
+    tokens, d_out, d_in = 512, 256, 128
+    rng = np.random.default_rng(23)
+    dy = I.f32_to_bf16_bits((rng.standard_normal((tokens, d_out)) * 1e-3).astype(np.float32))
+    x = I.f32_to_bf16_bits(rng.standard_normal((tokens, d_in)).astype(np.float32))
+    q_dy = B.abs_quantize_transposed(fmt, to_dev(dy))          # dY^T [d_out, tokens], groups along the tokens
+    q_x = B.abs_quantize_transposed(fmt, to_dev(x))            # X^T  [d_in,  tokens]
+    dw = B.abs_matmul(fmt, q_dy, q_x, d_out, d_in, tokens, check=True).double().cpu().numpy()
+    o_dy = oracle.quantize(fmt, np.ascontiguousarray(dy.T), threads=THREADS)
+    o_x = oracle.quantize(fmt, np.ascontiguousarray(x.T), threads=THREADS)
+    ref = oracle.mac_matmul_reference(fmt, o_dy, o_x, d_out, d_in, tokens)
+    assert np.abs(dw - ref).max() <= 2e-5 * np.abs(ref).max()
+    exact = I.bf16_bits_to_f32(dy).astype(np.float64).T @ I.bf16_bits_to_f32(x).astype(np.float64)
+    rel = np.linalg.norm(dw - exact) / np.linalg.norm(exact)
+    assert rel < 0.2, rel                                        # and it is the weight gradient, up to the quantization error
