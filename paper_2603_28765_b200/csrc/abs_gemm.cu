@@ -39,45 +39,77 @@ constexpr uint32_t kWaitLimit = 1u << 22;          // polls of one mbarrier wait
 
 // ----------------------------------------------------------------------------- operand split
 
-// Splits the 16 codes of one group (two words) into the planes F, H, L and writes the magnitude of its scale byte
-// into the 128x4-tile layout the tensor core reads.  FP groups: F = codes.  Integer groups (two's complement
-// nibbles): sign s, magnitude m = |k|; H = s | e2m1(h), L = s | e2m1(l) with m = h + l, h in {0, 1, 2, 3, 4, 6} and
-// l = 1 for m = 5 or 7, l = 2 for m = 8 (the most negative code, which no quantizer writes but dequantize reads as
-// -8), else 0.  E2M1 codes of the integers 0, 1, 2, 3, 4, 6 are 0, 2, 4, 5, 6, 7.
-__device__ __forceinline__ void split_word(uint32_t w, bool is_int, uint32_t& f, uint32_t& h, uint32_t& l) {
-    if (!is_int) { f = w; h = 0u; l = 0u; return; }
-    f = 0u; h = 0u; l = 0u;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int k = (int)((w >> (4 * j)) << 28) >> 28;             // sign-extended nibble
-        const uint32_t m = (uint32_t)(k < 0 ? -k : k), s = k < 0 ? 8u : 0u;
-        const uint32_t ml = (m == 5u || m == 7u) ? 1u : (m == 8u ? 2u : 0u);
-        const uint32_t mh = m - ml;                                   // 0, 1, 2, 3, 4, 6
-        const uint32_t ch = mh <= 1u ? 2u * mh : (mh <= 4u ? mh + 2u : 7u);
-        h |= ((m ? s : 0u) | ch) << (4 * j);
-        l |= (ml ? (s | (2u * ml)) : 0u) << (4 * j);
-    }
+// Splits eight integer codes (two's complement nibbles of one word) into the planes H and L, all nibbles at once:
+// sign s, magnitude m = |k|; H = s | e2m1(h), L = s | e2m1(l) with m = h + l, h in {0, 1, 2, 3, 4, 6} and l = 1 for
+// m = 5 or 7, l = 2 for m = 8 (the most negative code, which no quantizer writes but dequantize reads as -8), else
+// 0.  E2M1 codes of the integers 0, 1, 2, 3, 4, 6 are 0, 2, 4, 5, 6, 7.  No step carries from one nibble into the next.
+__device__ __forceinline__ void split_int_word(uint32_t w, uint32_t& h, uint32_t& l) {
+    constexpr uint32_t kOnes = 0x11111111u;
+    const uint32_t s = w & 0x88888888u, neg = s >> 3;
+    const uint32_t m = (w ^ (neg * 15u)) + neg;                      // |k| per nibble, 0 .. 8
+    const uint32_t l1 = (m >> 2) & m & kOnes;                         // m = 5 or 7
+    const uint32_t l2 = (m >> 3) & kOnes;                             // m = 8
+    const uint32_t mh = m - (l1 | (l2 << 1));                         // 0, 1, 2, 3, 4, 6
+    const uint32_t c0 = mh & kOnes, c1 = (mh >> 1) & kOnes, c2 = (mh >> 2) & kOnes;
+    h = s | ((c2 | c1) << 2) | ((c2 | (c0 & ~c1)) << 1) | (c1 & (c0 | c2));
+    l = (((l1 | l2) << 3) & s) | (l1 << 1) | (l2 << 2);
 }
 
-__global__ void __launch_bounds__(256) if4_split_kernel(const uint2* __restrict__ codes, const uint8_t* __restrict__ scales,
-                                                        int64_t ngroups, uint32_t gpr, uint32_t ktiles, bool has_int,
-                                                        uint2* __restrict__ plane_f, uint2* __restrict__ plane_h,
-                                                        uint2* __restrict__ plane_l, uint8_t* __restrict__ sf_tiled) {
+// One operand of the product as the split kernel sees it.
+struct SplitOperand {
+    const uint4* codes;            // [rows, k / 2] bytes as abs_quantize wrote them
+    const uint8_t* scales;         // [rows, k / 16] row-major
+    uint4 *plane_f, *plane_h, *plane_l;
+    uint8_t* sf_tiled;             // magnitudes of the scales in the 128x4-tile layout
+    int64_t pairs;                 // rows * k / 32: pairs of groups (16 bytes of codes)
+    int64_t sf_items;              // rows / 128 * ktiles / 4 * 32: one item = 4 rows x 16 scales
+    uint32_t gpr, ktiles;          // groups per row (a multiple of 16), gpr / 4
+};
+
+// Prepares both operands in one launch.  Code items (IF4 only; an NVFP4 operand is read by the product kernel where
+// it lies): 32 codes = two groups -> 16 bytes of each of the planes F, H, L.  Scale items: thread i of a warp reads 16
+// scale bytes of each of the rows i, i + 32, i + 64, i + 96 of a 128-row block and writes, for each of four
+// consecutive 128x4 tiles, the 16 bytes that tile keeps for those four rows.  Also clears the error word.
+__global__ void __launch_bounds__(256) if4_split_kernel(const SplitOperand a, const SplitOperand b, bool has_int,
+                                                        int* __restrict__ error) {
     pdl_launch_dependents();
     pdl_wait();
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
-        const uint2 c = __ldg(codes + g);
-        const uint32_t sb = __ldg(scales + g);
-        const bool is_int = has_int && (sb & 0x80u);
-        uint32_t f0, h0, l0, f1, h1, l1;
-        split_word(c.x, is_int, f0, h0, l0);
-        split_word(c.y, is_int, f1, h1, l1);
-        plane_f[g] = make_uint2(f0, f1);
-        plane_h[g] = make_uint2(h0, h1);
-        plane_l[g] = make_uint2(l0, l1);
-        const uint32_t row = (uint32_t)(g / gpr), k = (uint32_t)(g - (int64_t)row * gpr);
-        sf_tiled[swizzled_scale_offset(row, k, ktiles)] = (uint8_t)(sb & 0x7Fu);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x, first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (first == 0) *error = 0;
+    const int64_t code_items = has_int ? a.pairs + b.pairs : 0;
+    for (int64_t i = first; i < code_items; i += stride) {
+        const SplitOperand& o = i < a.pairs ? a : b;
+        const int64_t p = i < a.pairs ? i : i - a.pairs;
+        const uint4 c = __ldg(o.codes + p);
+        const uint32_t sb = __ldg(reinterpret_cast<const uint16_t*>(o.scales) + p);
+        uint4 f = c, h = make_uint4(0u, 0u, 0u, 0u), l = h;
+        if (sb & 0x80u) { f.x = 0u; f.y = 0u; split_int_word(c.x, h.x, l.x); split_int_word(c.y, h.y, l.y); }
+        if (sb & 0x8000u) { f.z = 0u; f.w = 0u; split_int_word(c.z, h.z, l.z); split_int_word(c.w, h.w, l.w); }
+        o.plane_f[p] = f;
+        o.plane_h[p] = h;
+        o.plane_l[p] = l;
+    }
+    const int64_t sf_items = a.sf_items + b.sf_items;
+    for (int64_t i = first; i < sf_items; i += stride) {
+        const SplitOperand& o = i < a.sf_items ? a : b;
+        const int64_t j = i < a.sf_items ? i : i - a.sf_items;
+        const uint32_t lane = (uint32_t)(j & 31);
+        const int64_t t4 = j >> 5;                                    // (row block, group of four tiles)
+        const uint32_t quads = o.ktiles >> 2;
+        const int64_t rb = t4 / quads;
+        const uint32_t kq = (uint32_t)(t4 - rb * quads);
+        uint4 r[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int64_t row = rb * 128 + q * 32 + lane;
+            r[q] = __ldg(reinterpret_cast<const uint4*>(o.scales + row * o.gpr) + kq);
+        }
+        uint4* out = reinterpret_cast<uint4*>(o.sf_tiled + ((size_t)rb * o.ktiles + (size_t)kq * 4u) * 512u) + lane;
+        constexpr uint32_t kMag = 0x7F7F7F7Fu;
+        out[0] = make_uint4(r[0].x & kMag, r[1].x & kMag, r[2].x & kMag, r[3].x & kMag);
+        out[32] = make_uint4(r[0].y & kMag, r[1].y & kMag, r[2].y & kMag, r[3].y & kMag);
+        out[64] = make_uint4(r[0].z & kMag, r[1].z & kMag, r[2].z & kMag, r[3].z & kMag);
+        out[96] = make_uint4(r[0].w & kMag, r[1].w & kMag, r[2].w & kMag, r[3].w & kMag);
     }
 }
 
@@ -336,6 +368,23 @@ bool plane_map(CUtensorMap* map, void* base, uint64_t rows, uint64_t row_bytes) 
 
 size_t round1k(size_t n) { return (n + 1023) & ~(size_t)1023; }
 
+// Launch with programmatic stream serialization: the kernel may become resident while its predecessor in the stream
+// drains; both kernels here call pdl_wait() before their first global access.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 struct GemmLayout {
     size_t plane_a, plane_b, sf_a, sf_b;       // sizes
     size_t off_a, off_b, off_sfa, off_sfb, total;
@@ -386,22 +435,34 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
 
     GemmMaps maps;
     for (int p = 0; p < 3; ++p) {
-        if (!plane_map(&maps.a[p], ws + L.off_a + p * L.plane_a, (uint64_t)m, (uint64_t)k / 2) ||
-            !plane_map(&maps.b[p], ws + L.off_b + p * L.plane_b, (uint64_t)n, (uint64_t)k / 2))
+        // NVFP4 needs no split: its single plane is the caller's codes
+        void* pa = has_int ? (void*)(ws + L.off_a + p * L.plane_a) : const_cast<void*>(a_codes);
+        void* pb = has_int ? (void*)(ws + L.off_b + p * L.plane_b) : const_cast<void*>(b_codes);
+        if (!plane_map(&maps.a[p], pa, (uint64_t)m, (uint64_t)k / 2) || !plane_map(&maps.b[p], pb, (uint64_t)n, (uint64_t)k / 2))
             return ABS_ERR_CUDA;
     }
-    if (cudaMemsetAsync(ws, 0, 1024, s) != cudaSuccess) return ABS_ERR_CUDA;          // the error word
-    const uint32_t gpr = (uint32_t)(k / 16), ktiles = (gpr + 3u) / 4u;
+    const uint32_t gpr = (uint32_t)(k / 16), ktiles = gpr / 4u;
+    SplitOperand so[2];
     for (int op = 0; op < 2; ++op) {
         const int64_t rows = op ? n : m;
-        const int64_t ngroups = rows * (k / 16);
         const size_t off = op ? L.off_b : L.off_a, plane = op ? L.plane_b : L.plane_a;
-        int64_t blocks = (ngroups + 255) / 256;
-        if (blocks > 148 * 16) blocks = 148 * 16;
-        if4_split_kernel<<<(int)blocks, 256, 0, s>>>((const uint2*)(op ? b_codes : a_codes), (const uint8_t*)(op ? b_scales : a_scales),
-                                                    ngroups, gpr, ktiles, has_int, (uint2*)(ws + off), (uint2*)(ws + off + plane),
-                                                    (uint2*)(ws + off + 2 * plane), ws + (op ? L.off_sfb : L.off_sfa));
-        if (cudaGetLastError() != cudaSuccess) return ABS_ERR_CUDA;
+        so[op].codes = (const uint4*)(op ? b_codes : a_codes);
+        so[op].scales = (const uint8_t*)(op ? b_scales : a_scales);
+        so[op].plane_f = (uint4*)(ws + off);
+        so[op].plane_h = (uint4*)(ws + off + plane);
+        so[op].plane_l = (uint4*)(ws + off + 2 * plane);
+        so[op].sf_tiled = ws + (op ? L.off_sfb : L.off_sfa);
+        so[op].pairs = rows * (k / 32);
+        so[op].sf_items = rows / 128 * (int64_t)(ktiles / 4u) * 32;
+        so[op].gpr = gpr;
+        so[op].ktiles = ktiles;
+    }
+    {
+        const int64_t items = has_int ? so[0].pairs + so[1].pairs : so[0].sf_items + so[1].sf_items;
+        int64_t blocks = (items + 255) / 256;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        if (launch_pdl(if4_split_kernel, dim3((unsigned)blocks), 256, 0, s, so[0], so[1], has_int, (int*)ws) != cudaSuccess)
+            return ABS_ERR_CUDA;
     }
     // the opt-in to more than 48 KiB of dynamic shared memory is per device
     static std::once_flag attr_once[64];
@@ -413,8 +474,10 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
     });
     if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
     const dim3 grid((unsigned)(n / kTileN), (unsigned)(m / kTileM));
-    if4_gemm_kernel<<<grid, 128, kGemmSmemBytes, s>>>(maps, ws + L.off_sfa, ws + L.off_sfb, a_alpha, b_alpha, c_f32, (int32_t)n,
-                                                      (int32_t)(k / kStageK), planes, (int*)ws);
+    if (launch_pdl(if4_gemm_kernel, grid, 128, kGemmSmemBytes, s, maps, (const uint8_t*)(ws + L.off_sfa),
+                   (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, (int32_t)n, (int32_t)(k / kStageK), planes,
+                   (int*)ws) != cudaSuccess)
+        return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 
