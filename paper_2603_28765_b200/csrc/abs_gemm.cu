@@ -13,11 +13,15 @@
 // (3 x 128 columns) and meet only in the epilogue.  Every product and partial sum is exact in the tensor core's
 // FP32 accumulation up to its rounding of the running sum, which is what the float64 reference is compared to.
 //
-// Kernel: one 128 x 128 tile of C per block.  One thread feeds the pipeline with TMA (cp.async.bulk.tensor.2d,
-// 128-byte swizzle, each load for this CTA alone; the scale tiles with plain bulk copies), one thread copies the scales to tensor
-// memory (tcgen05.cp) and issues the MMAs, four warps read the accumulators back (tcgen05.ld) and write C.
-// Every mbarrier wait is bounded: when a wait runs out the block raises an error word, stops issuing, frees its
-// tensor memory and returns.
+// Kernel: persistent, one block per SM over the 128 x 128 tiles of C.  One thread feeds the pipeline with TMA
+// (cp.async.bulk.tensor.2d, 128-byte swizzle, each load for this CTA alone; the scale tiles with plain bulk copies)
+// and runs ahead into the next tile, one thread copies the scales to tensor memory (tcgen05.cp) and issues the MMAs,
+// four warps read the accumulators back (tcgen05.ld) and write C.  Every mbarrier wait is bounded in time: when a
+// wait runs out the block raises an error word, stops issuing, frees its tensor memory and returns.
+//
+// What bounds it: a 128 x 128 x 64 MMA reads 4 KiB of A and 4 KiB of B from shared memory in the 64 cycles it takes,
+// which is all a shared memory delivers, so the TMA writes of the next stage (100 KiB per nine-MMA K-step of 256)
+// come on top of the MMA time and do not hide under it.
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
 
@@ -30,12 +34,14 @@ namespace absq {
 constexpr int kTileM = 128, kTileN = 128;
 constexpr int kStageK = 256;                       // elements of K per pipeline stage: 128 bytes of packed codes per row
 constexpr int kMmaK = 64;                          // K of one tcgen05.mma kind::mxf4nvf4
-constexpr int kStages = 2;
 constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one plane of one operand in one stage
 constexpr int kSfBytes = (kStageK / kMmaK) * 512;  // 2 KiB: scale tiles (128 rows x 4 scales) of one operand in one stage
-constexpr int kStageBytes = 6 * kPlaneBytes + 2 * kSfBytes;
-constexpr int kGemmSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr uint32_t kWaitLimit = 1u << 22;          // polls of one mbarrier wait before the block gives up
+// One-SM kernel: a stage holds PLANES planes of A, PLANES of B and the two scale tiles.  IF4 (three planes, 100 KiB)
+// has room for two stages; plain NVFP4 (one plane, 36 KiB) is bound by load latency and takes six.
+template <int PLANES> constexpr int kStageBytes = 2 * PLANES * kPlaneBytes + 2 * kSfBytes;
+template <int PLANES> constexpr int kStages = PLANES == 3 ? 2 : 6;
+template <int PLANES> constexpr int kGemmSmemBytes = kStages<PLANES> * kStageBytes<PLANES> + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // one second: how long an mbarrier wait polls before the block gives up
 
 // ----------------------------------------------------------------------------- operand split
 
@@ -120,17 +126,31 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for the phase with the given parity, bounded in time (a try_wait may itself sleep for a while, so counting
+// polls would not bound it); false when the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        uint32_t done;
-        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-    }
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    do {
+        if (mbar_try_wait(bar, parity)) return true;
+    } while (global_timer_ns() - t0 < kWaitLimitNs);
     return false;
 }
 // One 2-D tile (inner coordinate x in bytes, outer coordinate y in rows) from a tensor map into shared memory.
@@ -198,33 +218,55 @@ constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3
 
 // ----------------------------------------------------------------------------- the product kernel
 
-// Tensor memory columns (512 allocated): three accumulators of 128 columns, then per stage 16 columns of A scales
-// and 16 of B scales (four per K-step of 64).
+// Tensor memory columns (512 allocated): three accumulators of 128 columns, then two slots (even and odd K-step) of
+// 16 columns of A scales and 16 of B scales (four per MMA of K = 64).  tcgen05.cp and tcgen05.mma of one thread
+// execute in issue order, so a slot is rewritten only after the MMAs that read it.
 constexpr uint32_t kTmemCols = 512, kTmemSf = 3 * kTileN;
 
 struct GemmMaps {
     CUtensorMap a[3], b[3];        // planes F, H, L of A [M, K/2 bytes] and B [N, K/2 bytes], boxes of 128 bytes x 128 rows
 };
 
-// planes = 3: IF4 operands (nine MMAs per K-step); planes = 1: plain NVFP4 (one).  error: device word set to a
+// Tile t of the (tiles_m x tiles_n) grid of 128 x 128 tiles, walked in bands of eight tile rows, column by column
+// inside a band, so that the blocks running at the same time share few rows of A and few of B (L2 reuse).
+__device__ __forceinline__ void tile_of(int32_t t, int32_t tiles_m, int32_t tiles_n, int32_t& tm, int32_t& tn) {
+    constexpr int32_t kBand = 8;
+    const int32_t per_band = kBand * tiles_n, band = t / per_band, in_band = t - band * per_band;
+    const int32_t first = band * kBand, rows = min(kBand, tiles_m - first);
+    tn = in_band / rows;
+    tm = first + (in_band - tn * rows);
+}
+
+// PLANES = 3: IF4 operands (nine MMAs per K-step); PLANES = 1: plain NVFP4 (one).  error: device word set to a
 // non-zero code when a wait ran out.
-__global__ void __launch_bounds__(128, 1)
+//
+// Persistent: one block per SM walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Six warps: warp 0 (one
+// thread) feeds the pipeline and runs ahead into the next tile while the current one is finished; warp 1 (one thread)
+// copies scales and issues MMAs; warps 2-5 are the epilogue (warp w reads the 32 accumulator lanes of tensor-memory
+// quarter w % 4).  The accumulators pass between MMA and epilogue through acc_full / acc_empty barriers; NVFP4, with
+// one accumulator of 128 columns, alternates between two of them so that a tile's epilogue overlaps the next tile's
+// MMAs, IF4 (3 x 128 columns) has room for one set and overlaps the epilogue only with the next tile's loads.
+template <int PLANES>
+__global__ void __launch_bounds__(192, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
-                const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t n_cols,
-                int32_t k_iters, int32_t planes, int* __restrict__ error) {
+                const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t tiles_m,
+                int32_t tiles_n, int32_t k_iters, int* __restrict__ error) {
+    constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
+    constexpr int kSfAt = 2 * PLANES * kPlaneBytes;                  // the scale tiles follow the planes
+    constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
     const uint32_t raw = smem_u32(gemm_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                    // 128-byte swizzle wants 1024-byte aligned tiles
-    const uint32_t bars = base + kStages * kStageBytes;              // full[2], empty[2], acc_done, tmem address word
-    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 64);
-    const uint32_t full0 = bars, empty0 = bars + 16, acc_done = bars + 32;
+    const uint32_t bars = base + kStages * kStageBytes;              // full[], empty[], acc_full[2], acc_empty[2], tmem word
+    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 192);
+    const uint32_t full0 = bars, empty0 = bars + 64, acc_full0 = bars + 128, acc_empty0 = bars + 144;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_m = blockIdx.y, tile_n = blockIdx.x;
+    const int32_t num_tiles = tiles_m * tiles_n, n_cols = tiles_n * kTileN;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(acc_done, 1);
+        for (int i = 0; i < kAccBufs; ++i) { mbar_init(acc_full0 + 8 * i, 1); mbar_init(acc_empty0 + 8 * i, 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) { tmem_alloc(smem_u32(tmem_word), kTmemCols); tmem_relinquish(); }
@@ -234,294 +276,125 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     const uint32_t tmem = *tmem_word;
     pdl_wait();
 
-    if (warp == 0 && lane == 0) {
-        // ---- producer: TMA loads of the operand planes and bulk copies of the scale tiles
-        const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes + 2u * kSfBytes;
-        const int32_t ktiles = k_iters * (kStageK / kMmaK);
-        for (int32_t it = 0; it < k_iters; ++it) {
-            const int s = it % kStages;
-            if (!mbar_wait(empty0 + 8 * s, ((it / kStages) & 1) ^ 1)) { atomicExch(error, 1); break; }
-            const uint32_t st = base + s * kStageBytes, bar = full0 + 8 * s;
-            mbar_expect_tx(bar, bytes);
-            for (int p = 0; p < planes; ++p) {
-                tma_load_2d(st + p * kPlaneBytes, &maps.a[p], it * (kStageK / 2), tile_m * kTileM, bar);
-                tma_load_2d(st + (3 + p) * kPlaneBytes, &maps.b[p], it * (kStageK / 2), tile_n * kTileN, bar);
-            }
-            bulk_load(st + 6 * kPlaneBytes, sfa + ((size_t)tile_m * ktiles + (size_t)it * (kStageK / kMmaK)) * 512, kSfBytes, bar);
-            bulk_load(st + 6 * kPlaneBytes + kSfBytes, sfb + ((size_t)tile_n * ktiles + (size_t)it * (kStageK / kMmaK)) * 512, kSfBytes, bar);
-        }
-    } else if (warp == 1 && lane == 0) {
-        // ---- scale copies and MMAs
-        bool ok = true;
-        for (int32_t it = 0; it < k_iters && ok; ++it) {
-            const int s = it % kStages;
-            if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1)) { atomicExch(error, 2); ok = false; break; }
-            tc_fence_after();
-            const uint32_t st = base + s * kStageBytes;
-            const uint32_t tsfa = tmem + kTmemSf + s * 32, tsfb = tsfa + 16;
-#pragma unroll
-            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                tc_copy_scales(tsfa + 4 * kb, scale_desc(st + 6 * kPlaneBytes + kb * 512));
-                tc_copy_scales(tsfb + 4 * kb, scale_desc(st + 6 * kPlaneBytes + kSfBytes + kb * 512));
-            }
-#pragma unroll
-            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                const bool first = it == 0 && kb == 0;
-                uint64_t da[3], db[3];
-#pragma unroll
-                for (int p = 0; p < 3; ++p) {
-                    da[p] = operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2));
-                    db[p] = operand_desc(st + (3 + p) * kPlaneBytes + kb * (kMmaK / 2));
-                }
-                const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
-                tc_mma_nvf4(tmem, da[0], db[0], kInstrDesc, !first, fa, fb);                       // F F
-                if (planes == 3) {
-                    tc_mma_nvf4(tmem + kTileN, da[0], db[1], kInstrDesc, !first, fa, fb);          // F H
-                    tc_mma_nvf4(tmem + kTileN, da[0], db[2], kInstrDesc, true, fa, fb);            // F L
-                    tc_mma_nvf4(tmem + kTileN, da[1], db[0], kInstrDesc, true, fa, fb);            // H F
-                    tc_mma_nvf4(tmem + kTileN, da[2], db[0], kInstrDesc, true, fa, fb);            // L F
-                    tc_mma_nvf4(tmem + 2 * kTileN, da[1], db[1], kInstrDesc, !first, fa, fb);      // H H
-                    tc_mma_nvf4(tmem + 2 * kTileN, da[1], db[2], kInstrDesc, true, fa, fb);        // H L
-                    tc_mma_nvf4(tmem + 2 * kTileN, da[2], db[1], kInstrDesc, true, fa, fb);        // L H
-                    tc_mma_nvf4(tmem + 2 * kTileN, da[2], db[2], kInstrDesc, true, fa, fb);        // L L
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- producer: TMA loads of the operand planes and bulk copies of the scale tiles
+            const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes + 2u * kSfBytes;
+            const int32_t ktiles = k_iters * (kStageK / kMmaK);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                int32_t tile_m, tile_n;
+                tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
+                for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
+                    const uint32_t s = it % kStages;
+                    if (!mbar_wait(empty0 + 8 * s, ((it / kStages) & 1u) ^ 1u)) { atomicExch(error, 1); ok = false; break; }
+                    const uint32_t st = base + s * kStageBytes, bar = full0 + 8 * s;
+                    mbar_expect_tx(bar, bytes);
+                    for (int p = 0; p < planes; ++p) {
+                        tma_load_2d(st + p * kPlaneBytes, &maps.a[p], kt * (kStageK / 2), tile_m * kTileM, bar);
+                        tma_load_2d(st + (PLANES + p) * kPlaneBytes, &maps.b[p], kt * (kStageK / 2), tile_n * kTileN, bar);
+                    }
+                    bulk_load(st + kSfAt, sfa + ((size_t)tile_m * ktiles + (size_t)kt * (kStageK / kMmaK)) * 512, kSfBytes, bar);
+                    bulk_load(st + kSfAt + kSfBytes, sfb + ((size_t)tile_n * ktiles + (size_t)kt * (kStageK / kMmaK)) * 512, kSfBytes, bar);
                 }
             }
-            tc_commit(empty0 + 8 * s);              // the stage's shared memory is free once these MMAs have run
         }
-        if (ok) tc_commit(acc_done);
-    }
-    __syncwarp();
-
-    // ---- epilogue: all four warps; warp w owns lanes (rows) 32 w .. 32 w + 31 of the accumulators
-    bool have = mbar_wait(acc_done, 0);
-    if (!have && lane == 0) atomicExch(error, 3);
-    have = __all_sync(0xFFFFFFFFu, have);
-    tc_fence_after();
-    if (have) {
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- scale copies and MMAs
+            uint32_t it = 0, j = 0;
+            bool ok = true;
+            for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++j) {
+                const uint32_t buf = j % kAccBufs, acc = tmem + buf * kTileN;
+                if (!mbar_wait(acc_empty0 + 8 * buf, ((j / kAccBufs) & 1u) ^ 1u)) { atomicExch(error, 4); ok = false; break; }
+                tc_fence_after();
+                for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
+                    const uint32_t s = it % kStages;
+                    if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1u)) { atomicExch(error, 2); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t st = base + s * kStageBytes;
+                    const uint32_t tsfa = tmem + kTmemSf + (it & 1u) * 32u, tsfb = tsfa + 16;
+#pragma unroll
+                    for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                        tc_copy_scales(tsfa + 4 * kb, scale_desc(st + kSfAt + kb * 512));
+                        tc_copy_scales(tsfb + 4 * kb, scale_desc(st + kSfAt + kSfBytes + kb * 512));
+                    }
+#pragma unroll
+                    for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                        const bool first = kt == 0 && kb == 0;
+                        uint64_t da[3], db[3];
+#pragma unroll
+                        for (int p = 0; p < 3; ++p) {
+                            da[p] = operand_desc(st + (p < PLANES ? p : 0) * kPlaneBytes + kb * (kMmaK / 2));
+                            db[p] = operand_desc(st + (PLANES + (p < PLANES ? p : 0)) * kPlaneBytes + kb * (kMmaK / 2));
+                        }
+                        const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
+                        tc_mma_nvf4(acc, da[0], db[0], kInstrDesc, !first, fa, fb);                       // F F
+                        if (planes == 3) {
+                            tc_mma_nvf4(acc + kTileN, da[0], db[1], kInstrDesc, !first, fa, fb);          // F H
+                            tc_mma_nvf4(acc + kTileN, da[0], db[2], kInstrDesc, true, fa, fb);            // F L
+                            tc_mma_nvf4(acc + kTileN, da[1], db[0], kInstrDesc, true, fa, fb);            // H F
+                            tc_mma_nvf4(acc + kTileN, da[2], db[0], kInstrDesc, true, fa, fb);            // L F
+                            tc_mma_nvf4(acc + 2 * kTileN, da[1], db[1], kInstrDesc, !first, fa, fb);      // H H
+                            tc_mma_nvf4(acc + 2 * kTileN, da[1], db[2], kInstrDesc, true, fa, fb);        // H L
+                            tc_mma_nvf4(acc + 2 * kTileN, da[2], db[1], kInstrDesc, true, fa, fb);        // L H
+                            tc_mma_nvf4(acc + 2 * kTileN, da[2], db[2], kInstrDesc, true, fa, fb);        // L L
+                        }
+                    }
+                    tc_commit(empty0 + 8 * s);          // the stage's shared memory is free once these MMAs have run
+                }
+                if (ok) tc_commit(acc_full0 + 8 * buf); // and the tile's accumulators are complete
+            }
+        }
+    } else {
+        // ---- epilogue: warp w owns the accumulator lanes (rows of the tile) 32 (w % 4) .. 32 (w % 4) + 31
+        const int quarter = warp & 3;
         const float scale = __fmul_rn(__ldg(alpha_a), __ldg(alpha_b));
         const float c1 = __uint_as_float(0x3F5B6DB7u);                 // fp32(6/7)
         const float c2 = __fdiv_rn(36.0f, 49.0f);
-        float* out = c + ((size_t)tile_m * kTileM + warp * 32 + lane) * (size_t)n_cols + (size_t)tile_n * kTileN;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
-            uint32_t r0[32], r1[32], r2[32];
-            tmem_load32(lane_base + chunk * 32, r0);
-            if (planes == 3) {
-                tmem_load32(lane_base + kTileN + chunk * 32, r1);
-                tmem_load32(lane_base + 2 * kTileN + chunk * 32, r2);
-            }
-            tmem_load_wait();
-            float v[32];
+        uint32_t j = 0;
+        for (int32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
+            int32_t tile_m, tile_n;
+            tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
+            const uint32_t buf = j % kAccBufs;
+            bool have = mbar_wait(acc_full0 + 8 * buf, (j / kAccBufs) & 1u);
+            if (!have && lane == 0) atomicExch(error, 3);
+            have = __all_sync(0xFFFFFFFFu, have);
+            if (!have) break;
+            tc_fence_after();
+            float* out = c + ((size_t)tile_m * kTileM + quarter * 32 + lane) * (size_t)n_cols + (size_t)tile_n * kTileN;
+            const uint32_t lane_base = tmem + buf * kTileN + ((uint32_t)(quarter * 32) << 16);
+            for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
+                uint32_t r0[32], r1[32], r2[32];
+                tmem_load32(lane_base + chunk * 32, r0);
+                if (planes == 3) {
+                    tmem_load32(lane_base + kTileN + chunk * 32, r1);
+                    tmem_load32(lane_base + 2 * kTileN + chunk * 32, r2);
+                }
+                tmem_load_wait();
+                if (chunk == kTileN / 32 - 1) {         // everything is in registers: the MMAs of the next tile may start
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+                }
+                float v[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float acc = __uint_as_float(r0[j]);
-                if (planes == 3) acc = __fmaf_rn(c2, __uint_as_float(r2[j]), __fmaf_rn(c1, __uint_as_float(r1[j]), acc));
-                v[j] = __fmul_rn(acc, scale);
-            }
+                for (int jj = 0; jj < 32; ++jj) {
+                    float acc = __uint_as_float(r0[jj]);
+                    if (planes == 3) acc = __fmaf_rn(c2, __uint_as_float(r2[jj]), __fmaf_rn(c1, __uint_as_float(r1[jj]), acc));
+                    v[jj] = __fmul_rn(acc, scale);
+                }
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(out + chunk * 32 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                for (int jj = 0; jj < 32; jj += 4)
+                    *reinterpret_cast<float4*>(out + chunk * 32 + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+            }
         }
     }
+    __syncwarp();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_free(tmem, kTmemCols);
-}
-
-
-// ----------------------------------------------------------------------------- the product kernel on pairs of SMs
-
-// The one-SM kernel above is bound by shared-memory bandwidth: every 128 x 128 x 64 MMA reads 4 KiB of A and 4 KiB of
-// B from shared memory in the 64 cycles it takes, which is all a shared memory delivers, and the TMA writes of the
-// next stage come on top.  Here two CTAs of a cluster (two SMs) compute a 256 x 128 tile together with
-// tcgen05.mma.cta_group::2: each CTA holds its own 128 rows of A and of the accumulators, and only HALF of the B tile
-// (64 of its 128 rows), which the pair shares -- 6 KiB read per MMA and SM instead of 8, 76 KiB written per stage
-// instead of 100.  Protocol (the roles as above, in both CTAs unless noted):
-//   producer       waits for its own CTA's `empty`, loads its own operand parts with cp.async.bulk.tensor
-//                  .cta_group::2 (no multicast); every load signals the `full` barrier of the LEADER (rank 0), on
-//                  which the leader's producer has announced the bytes of both CTAs
-//   MMA issuer     leader only: waits for `full`, copies the scales (tcgen05.cp.cta_group::2: each CTA from its own
-//                  shared memory into its own tensor memory) and issues the MMAs for the pair; tcgen05.commit with a
-//                  two-CTA mask releases the stage in both CTAs and, at the end, hands both their accumulators
-//   epilogue       each CTA reads its own 128 rows from its tensor memory
-// The scale tiles come through tensor maps too (a bulk copy could not signal the other CTA's barrier).
-constexpr int kPairPlaneB = kPlaneBytes / 2;                                    // 64 rows of B
-constexpr int kPairStageBytes = 3 * kPlaneBytes + 3 * kPairPlaneB + 2 * kSfBytes;  // 76 KiB
-constexpr int kPairStages = 2;
-constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 + 256;
-constexpr uint32_t kInstrDescPair = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)((2 * kTileM) >> 4) << 24);
-
-struct PairMaps {
-    CUtensorMap a[3], b[3];        // planes of A (boxes of 128 bytes x 128 rows) and of B (128 bytes x 64 rows)
-    CUtensorMap sfa, sfb;          // tiled scales as [tiles, 128 words]; boxes of 4 tiles = one stage
-};
-
-__device__ __forceinline__ uint32_t cluster_cta_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Address, in the cluster's shared window, of the same shared-memory offset in the CTA of the given rank.
-__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t leader_bar) {
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t columns) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_result), "r"(columns) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_free_pair(uint32_t addr, uint32_t columns) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(addr), "r"(columns) : "memory");
-}
-// Arrives, once every tcgen05 operation issued before has completed, on the barrier at this offset in both CTAs.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 :: "r"(bar), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void tc_copy_scales_pair(uint32_t tmem_addr, uint64_t smem_desc) {
-    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" :: "r"(tmem_addr), "l"(smem_desc) : "memory");
-}
-__device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate,
-                                                 uint32_t sfa_tmem, uint32_t sfb_tmem) {
-    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
-                 "  tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p; }"
-                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-                 : "memory");
-}
-
-// Grid (m / 128, n / 128) in clusters of (2, 1): blockIdx.x is this CTA's own block of 128 rows of A and C.
-__global__ void __launch_bounds__(128, 1)
-if4_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const float* __restrict__ alpha_a, const float* __restrict__ alpha_b,
-                     float* __restrict__ c, int32_t n_cols, int32_t k_iters, int32_t planes, int* __restrict__ error) {
-    extern __shared__ uint8_t gemm_smem_raw[];
-    const uint32_t raw = smem_u32(gemm_smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    const uint32_t bars = base + kPairStages * kPairStageBytes;      // full[2], empty[2], acc_done, tmem address word
-    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 64);
-    const uint32_t full0 = bars, empty0 = bars + 16, acc_done = bars + 32;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_m = blockIdx.x, tile_n = blockIdx.y;
-    const uint32_t rank = cluster_cta_rank();
-    const bool leader = rank == 0;
-
-    pdl_launch_dependents();
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(acc_done, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) { tmem_alloc_pair(smem_u32(tmem_word), kTmemCols); tmem_relinquish_pair(); }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                             // both CTAs' barriers exist before anything signals them
-    tc_fence_after();
-    const uint32_t tmem = *tmem_word;
-    pdl_wait();
-
-    if (warp == 0 && lane == 0) {
-        // ---- producer (both CTAs)
-        const uint32_t bytes = (uint32_t)planes * (kPlaneBytes + kPairPlaneB) + 2u * kSfBytes;
-        const int32_t ktiles = k_iters * (kStageK / kMmaK);
-        for (int32_t it = 0; it < k_iters; ++it) {
-            const int s = it % kPairStages;
-            if (!mbar_wait(empty0 + 8 * s, ((it / kPairStages) & 1) ^ 1)) { atomicExch(error, 1); break; }
-            const uint32_t st = base + s * kPairStageBytes;
-            if (leader) mbar_expect_tx(full0 + 8 * s, 2u * bytes);
-            const uint32_t bar = cluster_map(full0 + 8 * s, 0);
-            for (int p = 0; p < planes; ++p) {
-                tma_load_2d_pair(st + p * kPlaneBytes, &maps.a[p], it * (kStageK / 2), tile_m * kTileM, bar);
-                tma_load_2d_pair(st + 3 * kPlaneBytes + p * kPairPlaneB, &maps.b[p], it * (kStageK / 2),
-                                 tile_n * kTileN + (int32_t)rank * (kTileN / 2), bar);
-            }
-            const uint32_t sf = st + 3 * kPlaneBytes + 3 * kPairPlaneB;
-            tma_load_2d_pair(sf, &maps.sfa, 0, tile_m * ktiles + it * (kStageK / kMmaK), bar);
-            tma_load_2d_pair(sf + kSfBytes, &maps.sfb, 0, tile_n * ktiles + it * (kStageK / kMmaK), bar);
-        }
-    } else if (warp == 1 && lane == 0 && leader) {
-        // ---- scale copies and MMAs for the pair
-        bool ok = true;
-        for (int32_t it = 0; it < k_iters && ok; ++it) {
-            const int s = it % kPairStages;
-            if (!mbar_wait(full0 + 8 * s, (it / kPairStages) & 1)) { atomicExch(error, 2); ok = false; break; }
-            tc_fence_after();
-            const uint32_t st = base + s * kPairStageBytes, sf = st + 3 * kPlaneBytes + 3 * kPairPlaneB;
-            const uint32_t tsfa = tmem + kTmemSf + s * 32, tsfb = tsfa + 16;
-#pragma unroll
-            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                tc_copy_scales_pair(tsfa + 4 * kb, scale_desc(sf + kb * 512));
-                tc_copy_scales_pair(tsfb + 4 * kb, scale_desc(sf + kSfBytes + kb * 512));
-            }
-#pragma unroll
-            for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                const bool first = it == 0 && kb == 0;
-                uint64_t da[3], db[3];
-#pragma unroll
-                for (int p = 0; p < 3; ++p) {
-                    da[p] = operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2));
-                    db[p] = operand_desc(st + 3 * kPlaneBytes + p * kPairPlaneB + kb * (kMmaK / 2));
-                }
-                const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
-                tc_mma_nvf4_pair(tmem, da[0], db[0], kInstrDescPair, !first, fa, fb);                       // F F
-                if (planes == 3) {
-                    tc_mma_nvf4_pair(tmem + kTileN, da[0], db[1], kInstrDescPair, !first, fa, fb);          // F H
-                    tc_mma_nvf4_pair(tmem + kTileN, da[0], db[2], kInstrDescPair, true, fa, fb);            // F L
-                    tc_mma_nvf4_pair(tmem + kTileN, da[1], db[0], kInstrDescPair, true, fa, fb);            // H F
-                    tc_mma_nvf4_pair(tmem + kTileN, da[2], db[0], kInstrDescPair, true, fa, fb);            // L F
-                    tc_mma_nvf4_pair(tmem + 2 * kTileN, da[1], db[1], kInstrDescPair, !first, fa, fb);      // H H
-                    tc_mma_nvf4_pair(tmem + 2 * kTileN, da[1], db[2], kInstrDescPair, true, fa, fb);        // H L
-                    tc_mma_nvf4_pair(tmem + 2 * kTileN, da[2], db[1], kInstrDescPair, true, fa, fb);        // L H
-                    tc_mma_nvf4_pair(tmem + 2 * kTileN, da[2], db[2], kInstrDescPair, true, fa, fb);        // L L
-                }
-            }
-            tc_commit_pair(empty0 + 8 * s);
-        }
-        if (ok) tc_commit_pair(acc_done);
-    }
-    __syncwarp();
-
-    // ---- epilogue: each CTA its own 128 rows
-    bool have = mbar_wait(acc_done, 0);
-    if (!have && lane == 0) atomicExch(error, 3);
-    have = __all_sync(0xFFFFFFFFu, have);
-    tc_fence_after();
-    if (have) {
-        const float scale = __fmul_rn(__ldg(alpha_a), __ldg(alpha_b));
-        const float c1 = __uint_as_float(0x3F5B6DB7u);                 // fp32(6/7)
-        const float c2 = __fdiv_rn(36.0f, 49.0f);
-        float* out = c + ((size_t)tile_m * kTileM + warp * 32 + lane) * (size_t)n_cols + (size_t)tile_n * kTileN;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
-            uint32_t r0[32], r1[32], r2[32];
-            tmem_load32(lane_base + chunk * 32, r0);
-            if (planes == 3) {
-                tmem_load32(lane_base + kTileN + chunk * 32, r1);
-                tmem_load32(lane_base + 2 * kTileN + chunk * 32, r2);
-            }
-            tmem_load_wait();
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float acc = __uint_as_float(r0[j]);
-                if (planes == 3) acc = __fmaf_rn(c2, __uint_as_float(r2[j]), __fmaf_rn(c1, __uint_as_float(r1[j]), acc));
-                v[j] = __fmul_rn(acc, scale);
-            }
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(out + chunk * 32 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                             // neither CTA leaves while the other may still signal it
-    if (warp == 0) tmem_free_pair(tmem, kTmemCols);
 }
 
 }  // namespace absq
@@ -552,25 +425,14 @@ EncodeTiledFn encode_tiled_fn() {
 
 // Tensor map of one plane: bytes [rows, row_bytes], box 128 bytes x 128 rows, 128-byte swizzle.  The map covers
 // this GPU's own workspace only.
-bool plane_map(CUtensorMap* map, void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows = 128) {
+bool plane_map(CUtensorMap* map, void* base, uint64_t rows, uint64_t row_bytes) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const cuuint64_t dims[2] = {row_bytes, rows};
     const cuuint64_t strides[1] = {row_bytes};
-    const cuuint32_t box[2] = {128, box_rows}, elem[2] = {1, 1};
+    const cuuint32_t box[2] = {128, 128}, elem[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Tensor map of a tiled scale array: [tiles, 128] 32-bit words (512 bytes per 128x4 tile), boxes of four tiles.
-bool scale_map(CUtensorMap* map, void* base, uint64_t tiles) {
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return false;
-    const cuuint64_t dims[2] = {128, tiles};
-    const cuuint64_t strides[1] = {512};
-    const cuuint32_t box[2] = {128, (cuuint32_t)(kStageK / kMmaK)}, elem[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, base, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 size_t round1k(size_t n) { return (n + 1023) & ~(size_t)1023; }
@@ -591,26 +453,6 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, int block, size_t sm
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
-// The same in clusters of two CTAs along x.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, int block, size_t smem, cudaStream_t s, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3((unsigned)block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = 2;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 struct GemmLayout {
     size_t plane_a, plane_b, sf_a, sf_b;       // sizes
     size_t off_a, off_b, off_sfa, off_sfb, total;
@@ -657,26 +499,15 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
     cudaStream_t s = (cudaStream_t)stream;
     uint8_t* ws = (uint8_t*)workspace;
     const bool has_int = fmt == ABS_FMT_IF4;
-    const int planes = has_int ? 3 : 1;
 
-    // two SMs per 256 x 128 tile where m allows and the operands have three planes (measured: a gain of 3 to 5 per cent
-    // for IF4, a loss for plain NVFP4, which is bound by load latency and not by shared memory); else one SM per tile
-    const bool pairs = has_int && m % (2 * kTileM) == 0;
     GemmMaps maps;
-    PairMaps pmaps;
     for (int p = 0; p < 3; ++p) {
         // NVFP4 needs no split: its single plane is the caller's codes
         void* pa = has_int ? (void*)(ws + L.off_a + p * L.plane_a) : const_cast<void*>(a_codes);
         void* pb = has_int ? (void*)(ws + L.off_b + p * L.plane_b) : const_cast<void*>(b_codes);
-        const bool ok = pairs ? plane_map(&pmaps.a[p], pa, (uint64_t)m, (uint64_t)k / 2) &&
-                                    plane_map(&pmaps.b[p], pb, (uint64_t)n, (uint64_t)k / 2, kTileN / 2)
-                              : plane_map(&maps.a[p], pa, (uint64_t)m, (uint64_t)k / 2) &&
-                                    plane_map(&maps.b[p], pb, (uint64_t)n, (uint64_t)k / 2);
-        if (!ok) return ABS_ERR_CUDA;
+        if (!plane_map(&maps.a[p], pa, (uint64_t)m, (uint64_t)k / 2) || !plane_map(&maps.b[p], pb, (uint64_t)n, (uint64_t)k / 2))
+            return ABS_ERR_CUDA;
     }
-    if (pairs && (!scale_map(&pmaps.sfa, ws + L.off_sfa, (uint64_t)(m / 128) * (uint64_t)(k / 64)) ||
-                  !scale_map(&pmaps.sfb, ws + L.off_sfb, (uint64_t)(n / 128) * (uint64_t)(k / 64))))
-        return ABS_ERR_CUDA;
     const uint32_t gpr = (uint32_t)(k / 16), ktiles = gpr / 4u;
     SplitOperand so[2];
     for (int op = 0; op < 2; ++op) {
@@ -703,26 +534,28 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
     // the opt-in to more than 48 KiB of dynamic shared memory is per device
     static std::once_flag attr_once[64];
     static cudaError_t attr_err[64];
+    static int sm_count[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ABS_ERR_CUDA;
     std::call_once(attr_once[dev], [dev]() {
-        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+        if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count[dev] < 1)
+            sm_count[dev] = 1;
+        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
         if (attr_err[dev] == cudaSuccess)
-            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
     });
     if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
-    const dim3 grid((unsigned)(n / kTileN), (unsigned)(m / kTileM));
-    if (pairs) {
-        const dim3 pgrid((unsigned)(m / kTileM), (unsigned)(n / kTileN));
-        if (launch_pdl_pairs(if4_gemm_pair_kernel, pgrid, 128, kPairSmemBytes, s, pmaps, a_alpha, b_alpha, c_f32, (int32_t)n,
-                             (int32_t)(k / kStageK), planes, (int*)ws) != cudaSuccess)
-            return ABS_ERR_CUDA;
-        return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
-    }
-    if (launch_pdl(if4_gemm_kernel, grid, 128, kGemmSmemBytes, s, maps, (const uint8_t*)(ws + L.off_sfa),
-                   (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, (int32_t)n, (int32_t)(k / kStageK), planes,
-                   (int*)ws) != cudaSuccess)
-        return ABS_ERR_CUDA;
+    const int32_t tiles_m = (int32_t)(m / kTileM), tiles_n = (int32_t)(n / kTileN);
+    const int64_t num_tiles = (int64_t)tiles_m * tiles_n;
+    const dim3 pgrid((unsigned)(num_tiles < sm_count[dev] ? num_tiles : sm_count[dev]));
+    const cudaError_t e =
+        has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 192, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
+                             (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
+                             (int*)ws)
+                : launch_pdl(if4_gemm_kernel<1>, pgrid, 192, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
+                             (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
+                             (int*)ws);
+    if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
 

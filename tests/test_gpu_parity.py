@@ -963,24 +963,31 @@ def test_scratch_ring_overrun_is_reported(B, oracle):
     check_case(B, oracle, 1, xb)                        # and everything is back to normal
 
 
-def test_tensor_core_matmul_full_size_sampled(B, oracle):
-    """abs_matmul at 4096 x 4096 x 4096 (the size its timing is quoted on): 48 sampled rows of A against 48 sampled
-    rows of B give a 48 x 48 sample of C that the float64 reference can compute; first and last rows included."""
-    m = n = k = 4096
+@pytest.mark.parametrize("fmt,m,n,k", [(1, 4096, 4096, 4096), (0, 4096, 4096, 4096), (1, 1920, 2176, 1024), (0, 1920, 2176, 1024)])
+def test_tensor_core_matmul_full_size_sampled(B, oracle, fmt, m, n, k):
+    """abs_matmul at 4096 x 4096 x 4096 (the size its timing is quoted on) and at a size whose tile rows do not fill
+    the last band of the tile walk: every block of the persistent kernel computes several tiles here.  48 sampled rows
+    of A against 48 sampled rows of B give a 48 x 48 sample of C, spread over the tiles, that the float64 reference
+    can compute; first and last rows included."""
     a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
-    qa, qb = B.abs_quantize(1, to_dev(a)), B.abs_quantize(1, to_dev(b))
-    c = B.abs_matmul(1, qa, qb, m, n, k, check=True)
+    qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
+    c = B.abs_matmul(fmt, qa, qb, m, n, k, check=True)
     rng = np.random.default_rng(17)
     ra = np.array(sorted(set([0, m - 1] + [int(v) for v in rng.integers(0, m, 46)])))
     rb = np.array(sorted(set([0, n - 1] + [int(v) for v in rng.integers(0, n, 46)])))
     alpha_a, alpha_b = np.float32(qa[2].item()), np.float32(qb[2].item())
-    oa = oracle.quantize(1, np.ascontiguousarray(a[ra]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_a)
-    ob = oracle.quantize(1, np.ascontiguousarray(b[rb]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_b)
+    oa = oracle.quantize(fmt, np.ascontiguousarray(a[ra]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_a)
+    ob = oracle.quantize(fmt, np.ascontiguousarray(b[rb]), flags=oracle.F_ALPHA_GIVEN, alpha=alpha_b)
     assert np.array_equal(qa[0].view(m, k // 2)[torch.from_numpy(ra).cuda()].cpu().numpy(), oa[0])     # same operands
-    ref = oracle.mac_matmul_reference(1, oa, ob, len(ra), len(rb), k)
+    ref = oracle.mac_matmul_reference(fmt, oa, ob, len(ra), len(rb), k)
     got = c[torch.from_numpy(ra).cuda()][:, torch.from_numpy(rb).cuda()].double().cpu().numpy()
     scale = float(c.abs().max().item())
     assert np.abs(got - ref).max() <= 2e-5 * scale, np.abs(got - ref).max() / scale
+    # and every tile was written by the block that owns it: the whole of C against the split path (four cuBLAS GEMMs)
+    if fmt == 1:
+        from paper_2603_28765_b200 import gemm
+        other = gemm.matmul_mac_split(qa, qb, m, n, k).float()
+        assert float((c - other).abs().max().item()) <= 2e-6 * scale
 
 
 @pytest.mark.parametrize("fmt", [0, 1])
