@@ -35,10 +35,9 @@ constexpr int kTileM = 128, kTileN = 128;
 constexpr int kStageK = 256;                       // elements of K per pipeline stage: 128 bytes of packed codes per row
 constexpr int kMmaK = 64;                          // K of one tcgen05.mma kind::mxf4nvf4
 constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one plane of one operand in one stage
-constexpr int kSfBytes = (kStageK / kMmaK) * 512;  // 2 KiB: scale tiles (128 rows x 4 scales) of one operand in one stage
-// One-SM kernel: a stage holds PLANES planes of A, PLANES of B and the two scale tiles.  IF4 (three planes, 100 KiB)
-// has room for two stages; plain NVFP4 (one plane, 36 KiB) is bound by load latency and takes six.
-template <int PLANES> constexpr int kStageBytes = 2 * PLANES * kPlaneBytes + 2 * kSfBytes;
+// A stage holds PLANES planes of A and PLANES of B (the scales do not pass through shared memory).  IF4 (three
+// planes, 96 KiB) has room for two stages; plain NVFP4 (one plane, 32 KiB) is bound by load latency and takes six.
+template <int PLANES> constexpr int kStageBytes = 2 * PLANES * kPlaneBytes;
 template <int PLANES> constexpr int kStages = PLANES == 3 ? 2 : 6;
 template <int PLANES> constexpr int kGemmSmemBytes = kStages<PLANES> * kStageBytes<PLANES> + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // one second: how long an mbarrier wait polls before the block gives up
@@ -158,11 +157,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  :: "r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
-// Contiguous bytes (multiple of 16, both addresses 16-byte aligned) into shared memory.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t columns) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_result), "r"(columns) : "memory");
 }
@@ -175,11 +169,6 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 // Arrives on the mbarrier once every tcgen05 operation this thread issued before has completed.
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
-}
-// Scale tile (32 rows x 16 bytes in shared memory = the scales of 128 rows x 4 groups) into four columns of tensor
-// memory, replicated over the four 32-lane quarters.
-__device__ __forceinline__ void tc_copy_scales(uint32_t tmem_addr, uint64_t smem_desc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" :: "r"(tmem_addr), "l"(smem_desc) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 64, E2M1 operands, one UE4M3 scale per 16 elements read from tensor memory.
 __device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate,
@@ -200,17 +189,21 @@ __device__ __forceinline__ void tmem_load32(uint32_t addr, uint32_t (&r)[32]) {
                  : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 lanes x 16 columns of 32 bits: thread t of the warp writes columns c .. c+15 of lane (warp % 4) * 32 + t.
+__device__ __forceinline__ void tmem_store16(uint32_t addr, const uint4& a, const uint4& b, const uint4& c, const uint4& d) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 :: "r"(addr), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w), "r"(c.x), "r"(c.y),
+                    "r"(c.z), "r"(c.w), "r"(d.x), "r"(d.y), "r"(d.z), "r"(d.w)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptors (64 bits): start address, leading / stride byte offsets (all in 16-byte units),
 // descriptor version 1 (Blackwell) in bits 46-47, swizzle mode in bits 61-63.
 //   operand tiles: K-major rows of 128 bytes, 128-byte swizzle (mode 2), 8-row groups 1024 bytes apart
-//   scale tiles:   32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart
 __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
     return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ uint64_t scale_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
 }
 // Instruction descriptor of kind::mxf4nvf4: A and B E2M1 (format 1, bits 7-9 and 10-12), both K-major, N / 8 in bits
 // 17-22, scale format UE4M3 (bit 23 = 0), M / 16 in bits 24-28, dense, K = 64 (bit 31 = 0), scale ids 0.
@@ -240,26 +233,32 @@ __device__ __forceinline__ void tile_of(int32_t t, int32_t tiles_m, int32_t tile
 // PLANES = 3: IF4 operands (nine MMAs per K-step); PLANES = 1: plain NVFP4 (one).  error: device word set to a
 // non-zero code when a wait ran out.
 //
-// Persistent: one block per SM walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Six warps: warp 0 (one
+// Persistent: one block per SM walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Ten warps: warp 0 (one
 // thread) feeds the pipeline and runs ahead into the next tile while the current one is finished; warp 1 (one thread)
-// copies scales and issues MMAs; warps 2-5 are the epilogue (warp w reads the 32 accumulator lanes of tensor-memory
-// quarter w % 4).  The accumulators pass between MMA and epilogue through acc_full / acc_empty barriers; NVFP4, with
-// one accumulator of 128 columns, alternates between two of them so that a tile's epilogue overlaps the next tile's
-// MMAs, IF4 (3 x 128 columns) has room for one set and overlaps the epilogue only with the next tile's loads.
+// issues MMAs; warps 2-5 are the epilogue (warp w reads the 32 accumulator lanes of tensor-memory quarter w % 4);
+// warps 6-9 bring the scales: each loads the 128x4 scale tiles of a K-step from global memory into registers and
+// writes them to its quarter of tensor memory (tcgen05.st; every quarter holds the same four columns per MMA: rows
+// r, r+32, r+64, r+96 of the tile, which is the byte order of the 128x4 tile), two slots used alternately and handed
+// over through sf_full / sf_empty barriers -- a tcgen05.cp from shared memory by the MMA thread would stand in the
+// MMA queue for some 34 cycles per copy, 270 per K-step.  The accumulators pass between MMA and epilogue through
+// acc_full / acc_empty barriers; NVFP4, with one accumulator of 128 columns, alternates between two of them so that a
+// tile's epilogue overlaps the next tile's MMAs, IF4 (3 x 128 columns) has room for one set and overlaps the epilogue
+// only with the next tile's loads.
 template <int PLANES>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
                 const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t tiles_m,
                 int32_t tiles_n, int32_t k_iters, int* __restrict__ error) {
     constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
-    constexpr int kSfAt = 2 * PLANES * kPlaneBytes;                  // the scale tiles follow the planes
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
     const uint32_t raw = smem_u32(gemm_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                    // 128-byte swizzle wants 1024-byte aligned tiles
-    const uint32_t bars = base + kStages * kStageBytes;              // full[], empty[], acc_full[2], acc_empty[2], tmem word
+    // barriers: full[], empty[] (stages), acc_full[2], acc_empty[2], sf_full[2], sf_empty[2]; then the tmem address word
+    const uint32_t bars = base + kStages * kStageBytes;
     uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 192);
     const uint32_t full0 = bars, empty0 = bars + 64, acc_full0 = bars + 128, acc_empty0 = bars + 144;
+    const uint32_t sf_full0 = bars + 160, sf_empty0 = bars + 176;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int32_t num_tiles = tiles_m * tiles_n, n_cols = tiles_n * kTileN;
 
@@ -267,6 +266,7 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int i = 0; i < kAccBufs; ++i) { mbar_init(acc_full0 + 8 * i, 1); mbar_init(acc_empty0 + 8 * i, 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(sf_full0 + 8 * i, 4); mbar_init(sf_empty0 + 8 * i, 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) { tmem_alloc(smem_u32(tmem_word), kTmemCols); tmem_relinquish(); }
@@ -278,9 +278,8 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
 
     if (warp == 0) {
         if (lane == 0) {
-            // ---- producer: TMA loads of the operand planes and bulk copies of the scale tiles
-            const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes + 2u * kSfBytes;
-            const int32_t ktiles = k_iters * (kStageK / kMmaK);
+            // ---- producer: TMA loads of the operand planes
+            const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes;
             uint32_t it = 0;
             bool ok = true;
             for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -295,14 +294,12 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                         tma_load_2d(st + p * kPlaneBytes, &maps.a[p], kt * (kStageK / 2), tile_m * kTileM, bar);
                         tma_load_2d(st + (PLANES + p) * kPlaneBytes, &maps.b[p], kt * (kStageK / 2), tile_n * kTileN, bar);
                     }
-                    bulk_load(st + kSfAt, sfa + ((size_t)tile_m * ktiles + (size_t)kt * (kStageK / kMmaK)) * 512, kSfBytes, bar);
-                    bulk_load(st + kSfAt + kSfBytes, sfb + ((size_t)tile_n * ktiles + (size_t)kt * (kStageK / kMmaK)) * 512, kSfBytes, bar);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // ---- scale copies and MMAs
+            // ---- MMAs
             uint32_t it = 0, j = 0;
             bool ok = true;
             for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++j) {
@@ -311,15 +308,12 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                 tc_fence_after();
                 for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
                     const uint32_t s = it % kStages;
+                    const uint32_t slot = it & 1u;
                     if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1u)) { atomicExch(error, 2); ok = false; break; }
+                    if (!mbar_wait(sf_full0 + 8 * slot, (it >> 1) & 1u)) { atomicExch(error, 5); ok = false; break; }
                     tc_fence_after();
                     const uint32_t st = base + s * kStageBytes;
-                    const uint32_t tsfa = tmem + kTmemSf + (it & 1u) * 32u, tsfb = tsfa + 16;
-#pragma unroll
-                    for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                        tc_copy_scales(tsfa + 4 * kb, scale_desc(st + kSfAt + kb * 512));
-                        tc_copy_scales(tsfb + 4 * kb, scale_desc(st + kSfAt + kSfBytes + kb * 512));
-                    }
+                    const uint32_t tsfa = tmem + kTmemSf + slot * 32u, tsfb = tsfa + 16;
 #pragma unroll
                     for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
                         const bool first = kt == 0 && kb == 0;
@@ -343,8 +337,41 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                         }
                     }
                     tc_commit(empty0 + 8 * s);          // the stage's shared memory is free once these MMAs have run
+                    tc_commit(sf_empty0 + 8 * slot);    // and so is the slot of scales
                 }
                 if (ok) tc_commit(acc_full0 + 8 * buf); // and the tile's accumulators are complete
+            }
+        }
+    } else if (warp >= 6) {
+        // ---- scales: this warp's copy of every K-step's scale tiles, global memory -> registers -> tensor memory
+        const int32_t ktiles = k_iters * (kStageK / kMmaK);
+        const uint32_t lane_base = tmem + kTmemSf + ((uint32_t)((warp & 3) * 32) << 16);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            int32_t tile_m, tile_n;
+            tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
+            const uint4* pa = reinterpret_cast<const uint4*>(sfa + (size_t)tile_m * ktiles * 512) + lane;
+            const uint4* pb = reinterpret_cast<const uint4*>(sfb + (size_t)tile_n * ktiles * 512) + lane;
+            for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
+                uint4 a[4], b[4];                                   // tile kb of the step: 16 bytes per lane, tiles 512 bytes apart
+#pragma unroll
+                for (int kb = 0; kb < 4; ++kb) {
+                    a[kb] = __ldg(pa + (kt * 4 + kb) * 32);
+                    b[kb] = __ldg(pb + (kt * 4 + kb) * 32);
+                }
+                const uint32_t slot = it & 1u;
+                bool have = mbar_wait(sf_empty0 + 8 * slot, ((it >> 1) & 1u) ^ 1u);
+                if (!have && lane == 0) atomicExch(error, 6);
+                have = __all_sync(0xFFFFFFFFu, have);
+                if (!have) { ok = false; break; }
+                tc_fence_after();
+                tmem_store16(lane_base + slot * 32u, a[0], a[1], a[2], a[3]);
+                tmem_store16(lane_base + slot * 32u + 16u, b[0], b[1], b[2], b[3]);
+                tmem_store_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sf_full0 + 8 * slot);
             }
         }
     } else {
@@ -549,10 +576,10 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
     const int64_t num_tiles = (int64_t)tiles_m * tiles_n;
     const dim3 pgrid((unsigned)(num_tiles < sm_count[dev] ? num_tiles : sm_count[dev]));
     const cudaError_t e =
-        has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 192, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
+        has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 320, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
                              (int*)ws)
-                : launch_pdl(if4_gemm_kernel<1>, pgrid, 192, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
+                : launch_pdl(if4_gemm_kernel<1>, pgrid, 320, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
                              (int*)ws);
     if (e != cudaSuccess) return ABS_ERR_CUDA;
