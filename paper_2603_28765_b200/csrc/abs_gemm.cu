@@ -171,12 +171,23 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 64, E2M1 operands, one UE4M3 scale per 16 elements read from tensor memory.
+// What happens to the A operand in the tensor core's collector buffer: read from shared memory and dropped, read and
+// kept (kFill), taken from the buffer and kept (kUse), taken from the buffer and dropped (kLastUse).  An MMA that
+// takes A from the buffer reads only B from shared memory.
+enum Collector { kDiscard, kFill, kUse, kLastUse };
+template <Collector C = kDiscard>
 __device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate,
                                             uint32_t sfa_tmem, uint32_t sfb_tmem) {
-    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
-                 "  tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p; }"
-                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-                 : "memory");
+#define ABS_MMA_NVF4(USAGE)                                                                                              \
+    asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"                                                               \
+                 "  tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16" USAGE " [%0], %1, %2, %3, [%5], [%6], p; }" \
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(sfa_tmem), "r"(sfb_tmem) \
+                 : "memory")
+    if constexpr (C == kFill) ABS_MMA_NVF4(".collector::a::fill");
+    else if constexpr (C == kUse) ABS_MMA_NVF4(".collector::a::use");
+    else if constexpr (C == kLastUse) ABS_MMA_NVF4(".collector::a::lastuse");
+    else ABS_MMA_NVF4("");
+#undef ABS_MMA_NVF4
 }
 // 32 lanes x 32 columns of 32 bits: thread t of the warp gets columns c .. c+31 of lane (warp % 4) * 32 + t.
 __device__ __forceinline__ void tmem_load32(uint32_t addr, uint32_t (&r)[32]) {
@@ -314,26 +325,28 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     tc_fence_after();
                     const uint32_t st = base + s * kStageBytes;
                     const uint32_t tsfa = tmem + kTmemSf + slot * 32u, tsfb = tsfa + 16;
+                    // the MMAs of a step, one accumulator after the other (K order inside an accumulator is free)
+                    auto desc_a = [&](int p, int kb) { return operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2)); };
+                    auto desc_b = [&](int p, int kb) { return operand_desc(st + (PLANES + p) * kPlaneBytes + kb * (kMmaK / 2)); };
 #pragma unroll
-                    for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
-                        const bool first = kt == 0 && kb == 0;
-                        uint64_t da[3], db[3];
+                    for (int kb = 0; kb < kStageK / kMmaK; ++kb)
+                        tc_mma_nvf4(acc, desc_a(0, kb), desc_b(0, kb), kInstrDesc, !(kt == 0 && kb == 0), tsfa + 4 * kb, tsfb + 4 * kb);   // F F
+                    if constexpr (PLANES == 3) {
 #pragma unroll
-                        for (int p = 0; p < 3; ++p) {
-                            da[p] = operand_desc(st + (p < PLANES ? p : 0) * kPlaneBytes + kb * (kMmaK / 2));
-                            db[p] = operand_desc(st + (PLANES + (p < PLANES ? p : 0)) * kPlaneBytes + kb * (kMmaK / 2));
+                        for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                            const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
+                            tc_mma_nvf4<kFill>(acc + kTileN, desc_a(0, kb), desc_b(1, kb), kInstrDesc, !(kt == 0 && kb == 0), fa, fb);   // F H
+                            tc_mma_nvf4<kLastUse>(acc + kTileN, desc_a(0, kb), desc_b(2, kb), kInstrDesc, true, fa, fb);                 // F L
+                            tc_mma_nvf4(acc + kTileN, desc_a(1, kb), desc_b(0, kb), kInstrDesc, true, fa, fb);                           // H F
+                            tc_mma_nvf4(acc + kTileN, desc_a(2, kb), desc_b(0, kb), kInstrDesc, true, fa, fb);                           // L F
                         }
-                        const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
-                        tc_mma_nvf4(acc, da[0], db[0], kInstrDesc, !first, fa, fb);                       // F F
-                        if (planes == 3) {
-                            tc_mma_nvf4(acc + kTileN, da[0], db[1], kInstrDesc, !first, fa, fb);          // F H
-                            tc_mma_nvf4(acc + kTileN, da[0], db[2], kInstrDesc, true, fa, fb);            // F L
-                            tc_mma_nvf4(acc + kTileN, da[1], db[0], kInstrDesc, true, fa, fb);            // H F
-                            tc_mma_nvf4(acc + kTileN, da[2], db[0], kInstrDesc, true, fa, fb);            // L F
-                            tc_mma_nvf4(acc + 2 * kTileN, da[1], db[1], kInstrDesc, !first, fa, fb);      // H H
-                            tc_mma_nvf4(acc + 2 * kTileN, da[1], db[2], kInstrDesc, true, fa, fb);        // H L
-                            tc_mma_nvf4(acc + 2 * kTileN, da[2], db[1], kInstrDesc, true, fa, fb);        // L H
-                            tc_mma_nvf4(acc + 2 * kTileN, da[2], db[2], kInstrDesc, true, fa, fb);        // L L
+#pragma unroll
+                        for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                            const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
+                            tc_mma_nvf4<kFill>(acc + 2 * kTileN, desc_a(1, kb), desc_b(1, kb), kInstrDesc, !(kt == 0 && kb == 0), fa, fb);  // H H
+                            tc_mma_nvf4<kLastUse>(acc + 2 * kTileN, desc_a(1, kb), desc_b(2, kb), kInstrDesc, true, fa, fb);              // H L
+                            tc_mma_nvf4<kFill>(acc + 2 * kTileN, desc_a(2, kb), desc_b(1, kb), kInstrDesc, true, fa, fb);                 // L H
+                            tc_mma_nvf4<kLastUse>(acc + 2 * kTileN, desc_a(2, kb), desc_b(2, kb), kInstrDesc, true, fa, fb);              // L L
                         }
                     }
                     tc_commit(empty0 + 8 * s);          // the stage's shared memory is free once these MMAs have run
