@@ -83,6 +83,16 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+def bf16_tensor_peak():
+    """(TFLOP/s, source): the measured cuBLAS bf16 burst rate, else the recipe's fallback."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    except Exception:
+        return 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+
+
 # ----------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -431,6 +441,34 @@ def run_cuda(args):
                  "T3_abs_dequantize_us": round(lt3 * 1e3, 2), "T3_gbs": round((2 * ln + lob) / lt3 / 1e6, 1)}
         del lx, lcodes, lscales, lout
 
+    # ---- the matrix product of two IF4 operands with the MAC arithmetic of Sec. 5.2 (abs_matmul, tcgen05): the one
+    # dense contraction of the library, so its roofline is the tensor one.  Nine block-scaled FP4 MMAs are issued per
+    # useful one; `achieved` counts the MMAs issued.  No FP4 peak was measured on this machine: the denominator is the
+    # measured bf16 rate x 4 (the nominal FP4 : bf16 ratio).
+    matmul = None
+    if not args.no_matmul:
+        mm = 4096
+        gen = torch.Generator(device=dev).manual_seed(11 + 1000 * rank)
+        ma = torch.randn((mm, mm), device=dev, generator=gen).to(torch.bfloat16)
+        mb = (torch.randn((mm, mm), device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+        qa, qb = B.abs_quantize(FMT_IF4, ma), B.abs_quantize(FMT_IF4, mb)
+        mws = torch.empty(L.abs_matmul_workspace_bytes(FMT_IF4, mm, mm, mm) + 1024, dtype=torch.uint8, device=dev)
+        mout = torch.empty((mm, mm), dtype=torch.float32, device=dev)
+        B.abs_matmul(FMT_IF4, qa, qb, mm, mm, mm, out=mout, workspace=mws, check=True)
+        mt = statistics.median(timed_batches(lambda i: B.abs_matmul(FMT_IF4, qa, qb, mm, mm, mm, out=mout, workspace=mws),
+                                             KERNEL_BATCHES, 20, warm=4))
+        tpeak, tsrc = bf16_tensor_peak()
+        issued = 9 * 2 * mm ** 3 / (mt * 1e-3) / 1e12
+        matmul = {"workload": f"IF4 x IF4, {mm}^3, N(0,1) x N(0,0.02), operand split + product per call, "
+                              f"median of {KERNEL_BATCHES} batches of 20 calls",
+                  "ms_per_call": round(mt, 4), "useful_tflops": round(issued / 9, 1),
+                  "roofline": {"bound": "tensor", "achieved": round(issued, 1), "peak": round(4 * tpeak, 1),
+                               "unit": "TFLOP/s", "frac": round(issued / (4 * tpeak), 4),
+                               "peak_source": tsrc + " x 4 (nominal FP4 : bf16)",
+                               "frac_of_nominal_9000_tflops": round(issued / 9000.0, 4),
+                               "flops_counted": "the nine block-scaled FP4 MMAs issued per useful one"}}
+        del ma, mb, qa, qb, mws, mout
+
     # ---- for information: the same result through the one-pass emulation call (amax pass + one kernel that
     # quantizes and decodes from registers, writing codes, scales and the bf16 output); not part of `value`.
     eargs = [(FMT_IF4, xs[k].data_ptr(), rows, cols, outs[k].data_ptr(), codes[k].data_ptr(), scales[k].data_ptr(),
@@ -515,7 +553,7 @@ def run_cuda(args):
             "ms_per_step_batches": {"median": round(statistics.median(step_batches), 5),
                                     "best": round(min(step_batches), 5), "worst": round(max(step_batches), 5),
                                     "batches": KERNEL_BATCHES, "steps_per_batch": KERNEL_BATCH_LAUNCHES},
-            "roofline": roofline, "breakdown": breakdown, "large": large,
+            "roofline": roofline, "breakdown": breakdown, "large": large, "matmul": matmul,
             "e2e": e2e, "one_pass": one_pass, "two_streams": two_streams,
             "gpu_launches": 3 * args.steps,
             "clocks": clocks,
@@ -541,6 +579,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-ramp", action="store_true", help="skip the clock-ramp loop (profiling runs only: fewer launches)")
     ap.add_argument("--no-large", action="store_true", help="skip the 16384x8192 figures (profiling runs)")
+    ap.add_argument("--no-matmul", action="store_true", help="skip the abs_matmul figure (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
