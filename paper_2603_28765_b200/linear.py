@@ -16,6 +16,11 @@ rounding is applied to activation gradients only; the 16/17 factor of Sec. 4.1 g
 
 All format-specific work is one call of ``abs_quantize_dequantize`` per operand (the one-pass emulation, along
 rows or down the columns, output in the operand's own orientation); the GEMMs are plain library calls.
+
+``forward_tc`` / ``backward_tc`` compute the same three products without the BF16 detour: every operand is quantized
+once into codes and scales that are K-major for its product (``abs_quantize`` along the rows, ``abs_quantize_transposed``
+down the columns) and the products run on the tensor cores with the MAC arithmetic of Sec. 5.2 (``abs_matmul``:
+exact code products, FP32 scale path with the factors 6/7 and 36/49, FP32 accumulation and output).
 """
 from __future__ import annotations
 
@@ -51,4 +56,39 @@ def backward(x, w, dy, fmt: int = B.ABS_FMT_IF4, *, sign_mask: int = 0x5A3C, see
     dyq = emulate(dy, fmt, columns=True, hadamard=True, stochastic=True, sign_mask=sign_mask, seed=seed + 1)
     xq = emulate(x, fmt, columns=True, hadamard=True, sign_mask=sign_mask)
     dw = _mm(dyq.t(), xq)
+    return dx, dw
+
+
+# ----------------------------------------------------------------------------- the same layer on the tensor cores
+
+
+def _opts(*, hadamard: bool = False, stochastic: bool = False, sign_mask: int = 0, seed: int = 0):
+    flags = B.ABS_F_HADAMARD16 if hadamard else 0
+    if stochastic:
+        flags |= B.ABS_F_STOCHASTIC | B.ABS_F_SR_SCALE_17_16
+    return B.make_opts(flags, sign_mask, seed) if flags else None
+
+
+def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4):
+    """Y = q(X) q(W)^T as float32 [tokens, d_out]: both operands quantized along d_in, one ``abs_matmul``.
+    tokens and d_out must be multiples of 128, d_in of 256."""
+    tokens, d_in = x.shape
+    d_out = w.shape[0]
+    return B.abs_matmul(fmt, B.abs_quantize(fmt, x), B.abs_quantize(fmt, w), tokens, d_out, d_in)
+
+
+def backward_tc(x, w, dy, fmt: int = B.ABS_FMT_IF4, *, sign_mask: int = 0x5A3C, seed: int = 0):
+    """(dX float32 [tokens, d_in], dW float32 [d_out, d_in]) with the recipe of ``backward``:
+    dX = q(dY) q(W^T)^T contracts over d_out, dW = q(dY^T) q(X^T)^T over the tokens (Hadamard on both, stochastic
+    rounding and the 17/16 factor on the gradient).  The transposed operands come from ``abs_quantize_transposed``,
+    which writes them K-major without materialising a transpose.  All three sizes multiples of 256."""
+    tokens, d_in = x.shape
+    d_out = w.shape[0]
+    q_dy = B.abs_quantize(fmt, dy, opts=_opts(stochastic=True, seed=seed))                 # [tokens, d_out] along d_out
+    q_wt = B.abs_quantize_transposed(fmt, w)                                                # W^T [d_in, d_out] along d_out
+    dx = B.abs_matmul(fmt, q_dy, q_wt, tokens, d_in, d_out)
+    q_dyt = B.abs_quantize_transposed(fmt, dy, opts=_opts(hadamard=True, stochastic=True, sign_mask=sign_mask,
+                                                          seed=seed + 1))                  # dY^T [d_out, tokens]
+    q_xt = B.abs_quantize_transposed(fmt, x, opts=_opts(hadamard=True, sign_mask=sign_mask))  # X^T [d_in, tokens]
+    dw = B.abs_matmul(fmt, q_dyt, q_xt, d_out, d_in, tokens)
     return dx, dw

@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--only", default="", help="one configuration, optionally one format: cfg4 or cfg4:if4")
     ap.add_argument("--rows", type=int, default=0, help="override the row count (smaller case for profiling)")
     ap.add_argument("--transposed", action="store_true", help="time abs_quantize_transposed (groups down the columns)")
+    ap.add_argument("--linear", action="store_true", help="time the quantized linear layer (forward + backward), tensor-core and emulated routes")
     ap.add_argument("--matmul", action="store_true", help="time abs_matmul (square sizes; --rows picks one size)")
     args = ap.parse_args()
     L = B.lib()
@@ -88,6 +89,28 @@ def main():
                     ref = gemm.matmul_mac_split(qa, qb, m, n, kk)
                     row["max_diff_vs_split_path"] = float((out - ref).abs().max() / ref.abs().max())
                 print(json.dumps(row), flush=True)
+        return
+    if args.linear:
+        # the quantized linear layer of Sec. 4.1 (forward, dgrad, wgrad with the gradient options): tensor-core route
+        # (quantize to K-major codes + abs_matmul) against the emulated route (one-pass emulation + cuBLAS BF16 GEMMs)
+        from . import linear
+        tokens, d_in, d_out = (args.rows or 8192), 4096, 14336
+        x = torch.randn(tokens, d_in, device="cuda").to(torch.bfloat16)
+        w = (torch.randn(d_out, d_in, device="cuda") * 0.02).to(torch.bfloat16)
+        dy = (torch.randn(tokens, d_out, device="cuda") * 1e-3).to(torch.bfloat16)
+        for fname in ("if4", "nvfp4"):
+            fmt = B.FMT_NAMES[fname]
+            row = {"linear": {"tokens": tokens, "d_in": d_in, "d_out": d_out}, "fmt": fname,
+                   "forward_tc_ms": round(loop_time(lambda i: linear.forward_tc(x, w, fmt)), 4),
+                   "backward_tc_ms": round(loop_time(lambda i: linear.backward_tc(x, w, dy, fmt)), 4),
+                   "forward_emulated_ms": round(loop_time(lambda i: linear.forward(x, w, fmt)), 4),
+                   "backward_emulated_ms": round(loop_time(lambda i: linear.backward(x, w, dy, fmt)), 4),
+                   "bf16_gemms_alone_ms": round(loop_time(lambda i: (torch.matmul(x, w.t()), torch.matmul(dy, w),
+                                                                     torch.matmul(dy.t(), x))), 4),
+                   "gemm_flops": 6.0 * tokens * d_in * d_out}
+            y, ye = linear.forward_tc(x, w, fmt), linear.forward(x, w, fmt).float()
+            row["forward_tc_vs_emulated_rel"] = float((y - ye).norm() / y.norm())
+            print(json.dumps(row), flush=True)
         return
     if args.transposed:
         for name, rows, cols in (("cfg2", 8192, 4096), ("cfg4", 16384, 8192)):

@@ -1010,3 +1010,45 @@ def test_weight_gradient_product_from_transposed_quantize(B, oracle, fmt):
     exact = I.bf16_bits_to_f32(dy).astype(np.float64).T @ I.bf16_bits_to_f32(x).astype(np.float64)
     rel = np.linalg.norm(dw - exact) / np.linalg.norm(exact)
     assert rel < 0.2, rel                                        # and it is the weight gradient, up to the quantization error
+
+
+def test_linear_layer_on_the_tensor_cores(B, oracle):
+    """The quantized linear layer of Sec. 4.1 without the BF16 detour (linear.forward_tc / backward_tc): three
+    tensor-core products of operands quantized K-major by abs_quantize / abs_quantize_transposed, the gradient
+    operands with Hadamard, stochastic rounding and the 17/16 factor.  Each product is compared with the float64 MAC
+    reference on the oracle's quantization of the same operand with the same options (so this also pins that the
+    options and seeds reach the right operand), and with the exact product up to the quantization error."""
+    from paper_2603_28765_b200 import linear
+    tokens, d_in, d_out = 768, 256, 512        # each of them is the K of one product: multiples of 256
+    mask, seed = 0x5A3C, 77
+    rng = np.random.default_rng(31)
+    x = I.f32_to_bf16_bits(rng.standard_normal((tokens, d_in)).astype(np.float32))
+    w = I.f32_to_bf16_bits((rng.standard_normal((d_out, d_in)) * 0.05).astype(np.float32))
+    dy = I.f32_to_bf16_bits((rng.standard_normal((tokens, d_out)) * 1e-3).astype(np.float32))
+    xd, wd, dyd = to_dev(x), to_dev(w), to_dev(dy)
+    T = lambda a: np.ascontiguousarray(a.T)
+    SR = oracle.F_STOCHASTIC | oracle.F_SR_SCALE_17_16
+    tol = lambda ref: 2e-5 * np.abs(ref).max()
+
+    y = linear.forward_tc(xd, wd).double().cpu().numpy()
+    ref = oracle.mac_matmul_reference(1, oracle.quantize(1, x, threads=THREADS), oracle.quantize(1, w, threads=THREADS),
+                                      tokens, d_out, d_in)
+    assert np.abs(y - ref).max() <= tol(ref)
+
+    dx, dw = linear.backward_tc(xd, wd, dyd, sign_mask=mask, seed=seed)
+    dx, dw = dx.double().cpu().numpy(), dw.double().cpu().numpy()
+    ref_dx = oracle.mac_matmul_reference(1, oracle.quantize(1, dy, flags=SR, sr_seed=seed, threads=THREADS),
+                                         oracle.quantize(1, T(w), threads=THREADS), tokens, d_in, d_out)
+    assert np.abs(dx - ref_dx).max() <= tol(ref_dx)
+    H = oracle.F_HADAMARD16
+    ref_dw = oracle.mac_matmul_reference(1, oracle.quantize(1, T(dy), flags=H | SR, sign_mask=mask, sr_seed=seed + 1, threads=THREADS),
+                                         oracle.quantize(1, T(x), flags=H, sign_mask=mask, threads=THREADS), d_out, d_in, tokens)
+    assert np.abs(dw - ref_dw).max() <= tol(ref_dw)
+
+    f = lambda a: I.bf16_bits_to_f32(a).astype(np.float64)
+    for got, exact in ((y, f(x) @ f(w).T), (dx, f(dy) @ f(w)), (dw, f(dy).T @ f(x))):
+        rel = np.linalg.norm(got - exact) / np.linalg.norm(exact)
+        assert rel < 0.2, rel                       # the Hadamard transform of the two wgrad operands cancels in the product
+    # and the emulated layer (BF16 GEMMs on dequantized operands) gives the same products up to its BF16 roundings
+    y_e = linear.forward(xd, wd).double().cpu().numpy()
+    assert np.linalg.norm(y - y_e) / np.linalg.norm(y) < 1e-2
