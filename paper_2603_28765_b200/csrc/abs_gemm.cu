@@ -39,7 +39,11 @@ constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one plane of one o
 // planes, 96 KiB) has room for two stages; plain NVFP4 (one plane, 32 KiB) is bound by load latency and takes six.
 template <int PLANES> constexpr int kStageBytes = 2 * PLANES * kPlaneBytes;
 template <int PLANES> constexpr int kStages = PLANES == 3 ? 2 : 6;
-template <int PLANES> constexpr int kGemmSmemBytes = kStages<PLANES> * kStageBytes<PLANES> + 1024 /* alignment slack */ + 256 /* barriers */;
+// Epilogue staging: each of the four epilogue warps turns its 32 rows x 32 columns of a chunk through shared memory
+// (rows 36 floats apart: 16-byte aligned and free of bank conflicts for 128-bit accesses both ways).
+constexpr int kStagePitch = 36, kStagingBytes = 4 * 32 * kStagePitch * 4;
+template <int PLANES> constexpr int kGemmSmemBytes =
+    kStages<PLANES> * kStageBytes<PLANES> + 1024 /* alignment slack */ + 512 /* barriers */ + kStagingBytes;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // one second: how long an mbarrier wait polls before the block gives up
 
 // ----------------------------------------------------------------------------- operand split
@@ -222,10 +226,9 @@ constexpr uint32_t kInstrDesc = (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3
 
 // ----------------------------------------------------------------------------- the product kernel
 
-// Tensor memory columns (512 allocated): three accumulators of 128 columns, then two slots (even and odd K-step) of
-// 16 columns of A scales and 16 of B scales (four per MMA of K = 64).  tcgen05.cp and tcgen05.mma of one thread
-// execute in issue order, so a slot is rewritten only after the MMAs that read it.
-constexpr uint32_t kTmemCols = 512, kTmemSf = 3 * kTileN;
+// Tensor memory columns (512 allocated): the accumulators (IF4: three of 128 columns; NVFP4: two, used alternately),
+// then the scale slots: 16 columns of A scales and 16 of B scales each (four per MMA of K = 64).
+constexpr uint32_t kTmemCols = 512;
 
 struct GemmMaps {
     CUtensorMap a[3], b[3];        // planes F, H, L of A [M, K/2 bytes] and B [N, K/2 bytes], boxes of 128 bytes x 128 rows
@@ -265,11 +268,15 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     extern __shared__ uint8_t gemm_smem_raw[];
     const uint32_t raw = smem_u32(gemm_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                    // 128-byte swizzle wants 1024-byte aligned tiles
-    // barriers: full[], empty[] (stages), acc_full[2], acc_empty[2], sf_full[2], sf_empty[2]; then the tmem address word
+    // Scale slots in tensor memory: 32 columns each (16 of A scales, 16 of B scales).  IF4 has room for two behind its
+    // three accumulators; NVFP4, whose K-steps are only four MMAs long, takes eight behind its two accumulators so
+    // that the scale warps can run several steps ahead of the MMAs.
+    constexpr uint32_t kSfSlots = PLANES == 1 ? 8 : 2, kSfBase = PLANES == 1 ? 2 * kTileN : 3 * kTileN;
+    // barriers: full[], empty[] (stages), acc_full[2], acc_empty[2], sf_full[], sf_empty[] (slots); then the tmem address word
     const uint32_t bars = base + kStages * kStageBytes;
-    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 192);
+    uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 320);
     const uint32_t full0 = bars, empty0 = bars + 64, acc_full0 = bars + 128, acc_empty0 = bars + 144;
-    const uint32_t sf_full0 = bars + 160, sf_empty0 = bars + 176;
+    const uint32_t sf_full0 = bars + 192, sf_empty0 = bars + 256;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int32_t num_tiles = tiles_m * tiles_n, n_cols = tiles_n * kTileN;
 
@@ -277,7 +284,7 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int i = 0; i < kAccBufs; ++i) { mbar_init(acc_full0 + 8 * i, 1); mbar_init(acc_empty0 + 8 * i, 4); }
-        for (int i = 0; i < 2; ++i) { mbar_init(sf_full0 + 8 * i, 4); mbar_init(sf_empty0 + 8 * i, 1); }
+        for (int i = 0; i < (int)kSfSlots; ++i) { mbar_init(sf_full0 + 8 * i, 4); mbar_init(sf_empty0 + 8 * i, 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) { tmem_alloc(smem_u32(tmem_word), kTmemCols); tmem_relinquish(); }
@@ -319,12 +326,12 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                 tc_fence_after();
                 for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
                     const uint32_t s = it % kStages;
-                    const uint32_t slot = it & 1u;
+                    const uint32_t slot = it % kSfSlots;
                     if (!mbar_wait(full0 + 8 * s, (it / kStages) & 1u)) { atomicExch(error, 2); ok = false; break; }
-                    if (!mbar_wait(sf_full0 + 8 * slot, (it >> 1) & 1u)) { atomicExch(error, 5); ok = false; break; }
+                    if (!mbar_wait(sf_full0 + 8 * slot, (it / kSfSlots) & 1u)) { atomicExch(error, 5); ok = false; break; }
                     tc_fence_after();
                     const uint32_t st = base + s * kStageBytes;
-                    const uint32_t tsfa = tmem + kTmemSf + slot * 32u, tsfb = tsfa + 16;
+                    const uint32_t tsfa = tmem + kSfBase + slot * 32u, tsfb = tsfa + 16;
                     // the MMAs of a step, one accumulator after the other (K order inside an accumulator is free)
                     auto desc_a = [&](int p, int kb) { return operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2)); };
                     auto desc_b = [&](int p, int kb) { return operand_desc(st + (PLANES + p) * kPlaneBytes + kb * (kMmaK / 2)); };
@@ -357,39 +364,50 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
         }
     } else if (warp >= 6) {
         // ---- scales: this warp's copy of every K-step's scale tiles, global memory -> registers -> tensor memory
+        // The loads of step it + 1 are in flight while step it waits for its slot and is written.
         const int32_t ktiles = k_iters * (kStageK / kMmaK);
-        const uint32_t lane_base = tmem + kTmemSf + ((uint32_t)((warp & 3) * 32) << 16);
-        uint32_t it = 0;
-        bool ok = true;
-        for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-            int32_t tile_m, tile_n;
-            tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
-            const uint4* pa = reinterpret_cast<const uint4*>(sfa + (size_t)tile_m * ktiles * 512) + lane;
-            const uint4* pb = reinterpret_cast<const uint4*>(sfb + (size_t)tile_n * ktiles * 512) + lane;
-            for (int32_t kt = 0; kt < k_iters; ++kt, ++it) {
-                uint4 a[4], b[4];                                   // tile kb of the step: 16 bytes per lane, tiles 512 bytes apart
-#pragma unroll
-                for (int kb = 0; kb < 4; ++kb) {
-                    a[kb] = __ldg(pa + (kt * 4 + kb) * 32);
-                    b[kb] = __ldg(pb + (kt * 4 + kb) * 32);
-                }
-                const uint32_t slot = it & 1u;
-                bool have = mbar_wait(sf_empty0 + 8 * slot, ((it >> 1) & 1u) ^ 1u);
-                if (!have && lane == 0) atomicExch(error, 6);
-                have = __all_sync(0xFFFFFFFFu, have);
-                if (!have) { ok = false; break; }
-                tc_fence_after();
-                tmem_store16(lane_base + slot * 32u, a[0], a[1], a[2], a[3]);
-                tmem_store16(lane_base + slot * 32u + 16u, b[0], b[1], b[2], b[3]);
-                tmem_store_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(sf_full0 + 8 * slot);
+        const uint32_t lane_base = tmem + kSfBase + ((uint32_t)((warp & 3) * 32) << 16);
+        int32_t t = blockIdx.x, kt = 0;                                   // the step whose tiles are loaded next
+        const uint4 *pa = nullptr, *pb = nullptr;
+        auto load_next = [&](uint4 (&a)[4], uint4 (&b)[4]) {               // false when there is no further step
+            if (t >= num_tiles) return false;
+            if (kt == 0) {
+                int32_t tile_m, tile_n;
+                tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
+                pa = reinterpret_cast<const uint4*>(sfa + (size_t)tile_m * ktiles * 512) + lane;
+                pb = reinterpret_cast<const uint4*>(sfb + (size_t)tile_n * ktiles * 512) + lane;
             }
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {                               // tile kb of the step: 16 bytes per lane, tiles 512 bytes apart
+                a[kb] = __ldg(pa + (kt * 4 + kb) * 32);
+                b[kb] = __ldg(pb + (kt * 4 + kb) * 32);
+            }
+            if (++kt == k_iters) { kt = 0; t += gridDim.x; }
+            return true;
+        };
+        uint4 a[4], b[4], an[4], bn[4];
+        bool more = load_next(a, b);
+        for (uint32_t it = 0; more; ++it) {
+            more = load_next(an, bn);
+            const uint32_t slot = it % kSfSlots;
+            bool have = mbar_wait(sf_empty0 + 8 * slot, ((it / kSfSlots) & 1u) ^ 1u);
+            if (!have && lane == 0) atomicExch(error, 6);
+            have = __all_sync(0xFFFFFFFFu, have);
+            if (!have) break;
+            tc_fence_after();
+            tmem_store16(lane_base + slot * 32u, a[0], a[1], a[2], a[3]);
+            tmem_store16(lane_base + slot * 32u + 16u, b[0], b[1], b[2], b[3]);
+            tmem_store_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sf_full0 + 8 * slot);
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) { a[kb] = an[kb]; b[kb] = bn[kb]; }
         }
     } else {
         // ---- epilogue: warp w owns the accumulator lanes (rows of the tile) 32 (w % 4) .. 32 (w % 4) + 31
         const int quarter = warp & 3;
+        float* staging = reinterpret_cast<float*>(gemm_smem_raw + (bars - raw) + 512) + (warp - 2) * 32 * kStagePitch;
         const float scale = __fmul_rn(__ldg(alpha_a), __ldg(alpha_b));
         const float c1 = __uint_as_float(0x3F5B6DB7u);                 // fp32(6/7)
         const float c2 = __fdiv_rn(36.0f, 49.0f);
@@ -403,7 +421,9 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
             have = __all_sync(0xFFFFFFFFu, have);
             if (!have) break;
             tc_fence_after();
-            float* out = c + ((size_t)tile_m * kTileM + quarter * 32 + lane) * (size_t)n_cols + (size_t)tile_n * kTileN;
+            // this thread's part of every store: row (lane / 8) of each group of four rows, 16 bytes at column 4 (lane % 8)
+            float* out = c + ((size_t)tile_m * kTileM + quarter * 32 + (lane >> 3)) * (size_t)n_cols + (size_t)tile_n * kTileN +
+                         4 * (lane & 7);
             const uint32_t lane_base = tmem + buf * kTileN + ((uint32_t)(quarter * 32) << 16);
             for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
                 uint32_t r0[32], r1[32], r2[32];
@@ -425,9 +445,18 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     if (planes == 3) acc = __fmaf_rn(c2, __uint_as_float(r2[jj]), __fmaf_rn(c1, __uint_as_float(r1[jj]), acc));
                     v[jj] = __fmul_rn(acc, scale);
                 }
+                // A thread holds 32 columns of ONE row; stored as they are, every store instruction of the warp would
+                // touch 32 different rows.  Through shared memory each instruction writes four rows of 128 contiguous bytes.
 #pragma unroll
                 for (int jj = 0; jj < 32; jj += 4)
-                    *reinterpret_cast<float4*>(out + chunk * 32 + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+                    *reinterpret_cast<float4*>(staging + lane * kStagePitch + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 x = *reinterpret_cast<const float4*>(staging + (4 * i + (lane >> 3)) * kStagePitch + 4 * (lane & 7));
+                    *reinterpret_cast<float4*>(out + (size_t)(4 * i) * n_cols + chunk * 32) = x;
+                }
+                __syncwarp();
             }
         }
     }
