@@ -289,6 +289,16 @@ ABS_API void abs_profile_events(void* quantize_begin, void* quantize_end);
  * low byte as an integer-valued float and out is float: value of E4M3 byte / FP element code. */
 ABS_API abs_status_t abs_selftest_convert(int kind, const float* in_f32, int64_t n, void* out, void* stream);
 
+/* Self-test hook for the bounded waits of abs_matmul: the same call, but in every block the loads of pipeline step
+ * number `stall_step` (counted from 0 over the block's tiles) are announced and never issued, so the block's waits run
+ * out after their limit (one second each, concurrently), the error word is set, the block frees its tensor memory and
+ * returns.  Nothing faults and nothing waits without a bound; abs_matmul_check then reports ABS_ERR_CUDA and the next
+ * abs_matmul call works normally.  c_f32 is left incomplete. */
+ABS_API abs_status_t abs_selftest_matmul_stall(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
+                                               const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m,
+                                               int64_t n, int64_t k, float* c_f32, void* workspace, size_t workspace_bytes,
+                                               void* stream, int32_t stall_step);
+
 #ifdef __cplusplus
 }
 #endif

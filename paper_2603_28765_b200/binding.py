@@ -36,7 +36,7 @@ EXPORTS = [
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
     "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled", "abs_quantize_dequantize",
-    "abs_matmul_workspace_bytes", "abs_matmul", "abs_matmul_check",
+    "abs_matmul_workspace_bytes", "abs_matmul", "abs_matmul_check", "abs_selftest_matmul_stall",
 ]
 
 
@@ -110,6 +110,8 @@ def lib():
             L.abs_matmul.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
             L.abs_matmul_check.restype = C.c_int
             L.abs_matmul_check.argtypes = [vp, vp]
+            L.abs_selftest_matmul_stall.restype = C.c_int
+            L.abs_selftest_matmul_stall.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp, C.c_int32]
             L.abs_profile_events.restype = None
             L.abs_profile_events.argtypes = [vp, vp]
             L.abs_selftest_convert.restype = C.c_int

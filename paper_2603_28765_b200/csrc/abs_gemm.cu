@@ -262,7 +262,7 @@ template <int PLANES>
 __global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
                 const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t tiles_m,
-                int32_t tiles_n, int32_t k_iters, int* __restrict__ error) {
+                int32_t tiles_n, int32_t k_iters, int* __restrict__ error, int32_t stall_step) {
     constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
@@ -308,6 +308,7 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     if (!mbar_wait(empty0 + 8 * s, ((it / kStages) & 1u) ^ 1u)) { atomicExch(error, 1); ok = false; break; }
                     const uint32_t st = base + s * kStageBytes, bar = full0 + 8 * s;
                     mbar_expect_tx(bar, bytes);
+                    if ((int32_t)it == stall_step) continue;      // self-test only: the bytes announced never arrive
                     for (int p = 0; p < planes; ++p) {
                         tma_load_2d(st + p * kPlaneBytes, &maps.a[p], kt * (kStageK / 2), tile_m * kTileM, bar);
                         tma_load_2d(st + (PLANES + p) * kPlaneBytes, &maps.b[p], kt * (kStageK / 2), tile_n * kTileN, bar);
@@ -554,9 +555,9 @@ size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k
     return gemm_layout(m, n, k).total;
 }
 
-abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
-                        const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
-                        void* workspace, size_t workspace_bytes, void* stream) {
+static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
+                                const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
+                                void* workspace, size_t workspace_bytes, void* stream, int32_t stall_step) {
     const absq::CallRange range("abs_matmul");
     if (fmt != ABS_FMT_IF4 && fmt != ABS_FMT_NVFP4) return ABS_ERR_FMT;
     if (!gemm_shape_ok(fmt, m, n, k)) return ABS_ERR_SHAPE;
@@ -620,12 +621,27 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
     const cudaError_t e =
         has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 320, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int*)ws)
+                             (int*)ws, stall_step)
                 : launch_pdl(if4_gemm_kernel<1>, pgrid, 320, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int*)ws);
+                             (int*)ws, stall_step);
     if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
+}
+
+abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
+                        const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_f32, workspace, workspace_bytes, stream, -1);
+}
+
+abs_status_t abs_selftest_matmul_stall(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
+                                       const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n,
+                                       int64_t k, float* c_f32, void* workspace, size_t workspace_bytes, void* stream,
+                                       int32_t stall_step) {
+    if (stall_step < 0) return ABS_ERR_SHAPE;
+    return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_f32, workspace, workspace_bytes, stream,
+                       stall_step);
 }
 
 abs_status_t abs_matmul_check(const void* workspace, void* stream) {

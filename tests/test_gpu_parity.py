@@ -1052,3 +1052,29 @@ def test_linear_layer_on_the_tensor_cores(B, oracle):
     # and the emulated layer (BF16 GEMMs on dequantized operands) gives the same products up to its BF16 roundings
     y_e = linear.forward(xd, wd).double().cpu().numpy()
     assert np.linalg.norm(y - y_e) / np.linalg.norm(y) < 1e-2
+
+
+def test_matmul_wait_limit_is_reported_and_the_next_call_works(B, oracle):
+    """Every wait inside the product kernel is bounded (one second).  The self-test entry announces the loads of one
+    pipeline step and never issues them: no fault and no unbounded wait, the blocks give up, set the error word, free
+    their tensor memory and return; abs_matmul_check reports it, and the next ordinary call on the same workspace
+    gives the right result again."""
+    import time
+    m, n, k = 256, 256, 1024
+    a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+    qa, qb = B.abs_quantize(1, to_dev(a)), B.abs_quantize(1, to_dev(b))
+    L = B.lib()
+    need = L.abs_matmul_workspace_bytes(1, m, n, k)
+    ws = torch.empty(need + 1024, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 1024
+    good = B.abs_matmul(1, qa, qb, m, n, k, workspace=ws, check=True).clone()
+    out = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    args = (1, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), qb[0].data_ptr(), qb[1].data_ptr(), qb[2].data_ptr(),
+            m, n, k, out.data_ptr(), ws.data_ptr() + off, need, None)
+    t0 = time.time()
+    assert L.abs_selftest_matmul_stall(*args, 2) == 0                      # the launch itself succeeds
+    assert L.abs_matmul_check(ws.data_ptr() + off, None) == 6              # ABS_ERR_CUDA: a wait ran out
+    assert time.time() - t0 < 20.0
+    assert L.abs_selftest_matmul_stall(*args, -1) == 2                     # not a way to make an ordinary call
+    again = B.abs_matmul(1, qa, qb, m, n, k, workspace=ws, check=True)
+    assert torch.equal(again, good)
