@@ -243,7 +243,7 @@ ABS_API float abs_alpha_from_amax(abs_fmt_t fmt, float amax);
  *   b_codes, b_scales  B likewise: [n, k]
  *   c_f32              out, [m, n] float, row-major
  *   workspace          device memory, 1024-byte aligned, at least abs_matmul_workspace_bytes(fmt, m, n, k) bytes
- * m and n must be multiples of 128, k a multiple of 256 (ABS_ERR_SHAPE otherwise; abs_matmul_workspace_bytes
+ * m is any positive number of rows; n must be a multiple of 128, k a multiple of 256 (ABS_ERR_SHAPE otherwise; abs_matmul_workspace_bytes
  * returns 0).  Asynchronous like the other calls.  Every wait inside the kernel is bounded; if one runs out (it
  * never should) the kernel stops and leaves a non-zero word at the start of the workspace, which
  * abs_matmul_check(workspace, stream) reads back (it synchronises the stream): ABS_OK, or ABS_ERR_CUDA.

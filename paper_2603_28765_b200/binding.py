@@ -262,7 +262,7 @@ def abs_matmul(fmt: int, qa, qb, m: int, n: int, k: int, out=None, workspace=Non
     L = lib()
     need = L.abs_matmul_workspace_bytes(fmt, m, n, k)
     if need == 0:
-        raise AbsError(2, "abs_matmul: m, n multiples of 128 and k a multiple of 256; IF4 or NVFP4")
+        raise AbsError(2, "abs_matmul: n a multiple of 128 and k a multiple of 256; IF4 or NVFP4")
     if workspace is None:
         workspace = torch.empty(need + 1024, dtype=torch.uint8, device=qa[0].device)
     off = (-workspace.data_ptr()) % 1024

@@ -70,8 +70,9 @@ struct SplitOperand {
     const uint8_t* scales;         // [rows, k / 16] row-major
     uint4 *plane_f, *plane_h, *plane_l;
     uint8_t* sf_tiled;             // magnitudes of the scales in the 128x4-tile layout
+    int64_t rows;
     int64_t pairs;                 // rows * k / 32: pairs of groups (16 bytes of codes)
-    int64_t sf_items;              // rows / 128 * ktiles / 4 * 32: one item = 4 rows x 16 scales
+    int64_t sf_items;              // ceil(rows / 128) * ktiles / 4 * 32: one item = 4 rows x 16 scales
     uint32_t gpr, ktiles;          // groups per row (a multiple of 16), gpr / 4
 };
 
@@ -110,8 +111,8 @@ __global__ void __launch_bounds__(256) if4_split_kernel(const SplitOperand a, co
         uint4 r[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const int64_t row = rb * 128 + q * 32 + lane;
-            r[q] = __ldg(reinterpret_cast<const uint4*>(o.scales + row * o.gpr) + kq);
+            const int64_t row = rb * 128 + q * 32 + lane;       // rows beyond the operand (last row block) get zero scales
+            r[q] = row < o.rows ? __ldg(reinterpret_cast<const uint4*>(o.scales + row * o.gpr) + kq) : make_uint4(0u, 0u, 0u, 0u);
         }
         uint4* out = reinterpret_cast<uint4*>(o.sf_tiled + ((size_t)rb * o.ktiles + (size_t)kq * 4u) * 512u) + lane;
         constexpr uint32_t kMag = 0x7F7F7F7Fu;
@@ -262,7 +263,7 @@ template <int PLANES>
 __global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
                 const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t tiles_m,
-                int32_t tiles_n, int32_t k_iters, int* __restrict__ error, int32_t stall_step) {
+                int32_t tiles_n, int32_t k_iters, int32_t m_rows, int* __restrict__ error, int32_t stall_step) {
     constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
@@ -423,8 +424,8 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
             if (!have) break;
             tc_fence_after();
             // this thread's part of every store: row (lane / 8) of each group of four rows, 16 bytes at column 4 (lane % 8)
-            float* out = c + ((size_t)tile_m * kTileM + quarter * 32 + (lane >> 3)) * (size_t)n_cols + (size_t)tile_n * kTileN +
-                         4 * (lane & 7);
+            const int32_t row0 = tile_m * kTileM + quarter * 32 + (lane >> 3);
+            float* out = c + (size_t)row0 * (size_t)n_cols + (size_t)tile_n * kTileN + 4 * (lane & 7);
             const uint32_t lane_base = tmem + buf * kTileN + ((uint32_t)(quarter * 32) << 16);
             for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
                 uint32_t r0[32], r1[32], r2[32];
@@ -455,7 +456,8 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const float4 x = *reinterpret_cast<const float4*>(staging + (4 * i + (lane >> 3)) * kStagePitch + 4 * (lane & 7));
-                    *reinterpret_cast<float4*>(out + (size_t)(4 * i) * n_cols + chunk * 32) = x;
+                    if (row0 + 4 * i < m_rows)                          // the last row block may be partial
+                        *reinterpret_cast<float4*>(out + (size_t)(4 * i) * n_cols + chunk * 32) = x;
                 }
                 __syncwarp();
             }
@@ -531,7 +533,7 @@ GemmLayout gemm_layout(int64_t m, int64_t n, int64_t k) {
     GemmLayout L;
     L.plane_a = round1k((size_t)m * k / 2);
     L.plane_b = round1k((size_t)n * k / 2);
-    L.sf_a = round1k((size_t)m * k / 16);
+    L.sf_a = round1k((size_t)((m + kTileM - 1) / kTileM * kTileM) * k / 16);
     L.sf_b = round1k((size_t)n * k / 16);
     L.off_a = 1024;
     L.off_b = L.off_a + 3 * L.plane_a;
@@ -542,7 +544,7 @@ GemmLayout gemm_layout(int64_t m, int64_t n, int64_t k) {
 }
 
 bool gemm_shape_ok(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k) {
-    return (fmt == ABS_FMT_IF4 || fmt == ABS_FMT_NVFP4) && m > 0 && n > 0 && k > 0 && m % kTileM == 0 && n % kTileN == 0 &&
+    return (fmt == ABS_FMT_IF4 || fmt == ABS_FMT_NVFP4) && m > 0 && n > 0 && k > 0 && n % kTileN == 0 &&
            k % kStageK == 0 && m < ((int64_t)1 << 30) && n < ((int64_t)1 << 30) && k < ((int64_t)1 << 30);
 }
 
@@ -589,8 +591,9 @@ static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* 
         so[op].plane_h = (uint4*)(ws + off + plane);
         so[op].plane_l = (uint4*)(ws + off + 2 * plane);
         so[op].sf_tiled = ws + (op ? L.off_sfb : L.off_sfa);
+        so[op].rows = rows;
         so[op].pairs = rows * (k / 32);
-        so[op].sf_items = rows / 128 * (int64_t)(ktiles / 4u) * 32;
+        so[op].sf_items = (rows + 127) / 128 * (int64_t)(ktiles / 4u) * 32;
         so[op].gpr = gpr;
         so[op].ktiles = ktiles;
     }
@@ -615,16 +618,16 @@ static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* 
             attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
     });
     if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
-    const int32_t tiles_m = (int32_t)(m / kTileM), tiles_n = (int32_t)(n / kTileN);
+    const int32_t tiles_m = (int32_t)((m + kTileM - 1) / kTileM), tiles_n = (int32_t)(n / kTileN);
     const int64_t num_tiles = (int64_t)tiles_m * tiles_n;
     const dim3 pgrid((unsigned)(num_tiles < sm_count[dev] ? num_tiles : sm_count[dev]));
     const cudaError_t e =
         has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 320, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int*)ws, stall_step)
+                             (int32_t)m, (int*)ws, stall_step)
                 : launch_pdl(if4_gemm_kernel<1>, pgrid, 320, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
                              (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int*)ws, stall_step);
+                             (int32_t)m, (int*)ws, stall_step);
     if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }

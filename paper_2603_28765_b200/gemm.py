@@ -10,7 +10,7 @@ Both take operands quantized along K: A as [M, K], B as [N, K] (codes, scales, a
                      factor 1, 6/7 or 36/49 (none, one, both groups stored as integers) in FP32 on the
                      scale path.  This is the library's own tensor-core kernel (``abs_matmul``: block-scaled
                      FP4 MMAs on the codes themselves, three accumulators, factors in the FP32 epilogue)
-                     whenever M and N are multiples of 128 and K of 256.
+                     whenever N is a multiple of 128 and K of 256 (any M).
 ``matmul_mac_split`` the same arithmetic for any shape, and the cross-check of the kernel above, from parts
                      that are exact in BF16: the library's split dequantize produces, for each operand, the
                      FP-group part and the raw integer-group part -- each a 4-bit code times an E4M3 scale,
@@ -46,7 +46,7 @@ def matmul_emulated(qa, qb, m: int, n: int, k: int):
 
 def matmul_mac(qa, qb, m: int, n: int, k: int):
     """Sec. 5.2 MAC arithmetic: the library's tcgen05 kernel where the shape allows, else the BF16 split."""
-    if m % 128 == 0 and n % 128 == 0 and k % 256 == 0:
+    if n % 128 == 0 and k % 256 == 0:
         return B.abs_matmul(FMT, qa, qb, m, n, k)
     return matmul_mac_split(qa, qb, m, n, k)
 

@@ -71,7 +71,7 @@ def _opts(*, hadamard: bool = False, stochastic: bool = False, sign_mask: int = 
 
 def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4):
     """Y = q(X) q(W)^T as float32 [tokens, d_out]: both operands quantized along d_in, one ``abs_matmul``.
-    tokens and d_out must be multiples of 128, d_in of 256."""
+    d_out must be a multiple of 128, d_in of 256 (any number of tokens)."""
     tokens, d_in = x.shape
     d_out = w.shape[0]
     return B.abs_matmul(fmt, B.abs_quantize(fmt, x), B.abs_quantize(fmt, w), tokens, d_out, d_in)

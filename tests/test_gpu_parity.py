@@ -853,7 +853,7 @@ def test_tensor_core_matmul_matches_mac_reference(B, oracle, fmt):
     mixed and INT x INT group pairs, factors 1, 6/7, 36/49 in the FP32 epilogue) against the float64 reference of the
     MAC arithmetic of Sec. 5.2.  Every code product is exact; the difference is the FP32 accumulation of the tensor
     core over K terms, so the tolerance is that of an FP32 sum (2e-5 of the largest |C| is ample up to K = 4096)."""
-    for (m, n, k) in ((128, 128, 256), (256, 384, 1024), (128, 256, 4096), (640, 128, 512)):
+    for (m, n, k) in ((128, 128, 256), (256, 384, 1024), (128, 256, 4096), (640, 128, 512), (1, 128, 256), (100, 256, 512), (333, 128, 1024)):
         a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
         qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
         oa, ob = oracle.quantize(fmt, a, threads=THREADS), oracle.quantize(fmt, b, threads=THREADS)
@@ -863,9 +863,15 @@ def test_tensor_core_matmul_matches_mac_reference(B, oracle, fmt):
         assert err < 2e-5, (fmt, m, n, k, err)
         if fmt == 1:
             assert 0.05 < float((oa[1] >> 7).mean()) < 0.95     # both kinds of groups take part
+    # a partial last row block: nothing is written below row m
+    m, n, k = 100, 128, 256
+    qa, qb = B.abs_quantize(fmt, to_dev(I.generate("cfg2", m, k))), B.abs_quantize(fmt, to_dev(I.generate("cfg3a", n, k, seed=9)))
+    guard = torch.full((128, n), 7.0, dtype=torch.float32, device="cuda")
+    B.abs_matmul(fmt, qa, qb, m, n, k, out=guard, check=True)
+    assert bool((guard[m:] == 7.0).all()) and not bool((guard[:m] == 7.0).all())
     # shapes the kernel does not take, and other formats
     L = B.lib()
-    assert L.abs_matmul_workspace_bytes(fmt, 100, 128, 256) == 0 and L.abs_matmul_workspace_bytes(fmt, 128, 128, 128) == 0
+    assert L.abs_matmul_workspace_bytes(fmt, 128, 100, 256) == 0 and L.abs_matmul_workspace_bytes(fmt, 128, 128, 128) == 0
     assert L.abs_matmul_workspace_bytes(2, 128, 128, 256) == 0
     ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
     out = torch.empty((128, 128), dtype=torch.float32, device="cuda")
