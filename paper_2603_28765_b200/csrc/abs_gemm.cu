@@ -13,15 +13,14 @@
 // (3 x 128 columns) and meet only in the epilogue.  Every product and partial sum is exact in the tensor core's
 // FP32 accumulation up to its rounding of the running sum, which is what the float64 reference is compared to.
 //
-// Kernel: persistent, one block per SM over the 128 x 128 tiles of C.  One thread feeds the pipeline with TMA
-// (cp.async.bulk.tensor.2d, 128-byte swizzle, each load for this CTA alone; the scale tiles with plain bulk copies)
-// and runs ahead into the next tile, one thread copies the scales to tensor memory (tcgen05.cp) and issues the MMAs,
-// four warps read the accumulators back (tcgen05.ld) and write C.  Every mbarrier wait is bounded in time: when a
-// wait runs out the block raises an error word, stops issuing, frees its tensor memory and returns.
+// Kernel: persistent, one block of ten warps per SM over the 128 x 128 tiles of C.  One thread feeds the pipeline with
+// TMA (cp.async.bulk.tensor.2d, 128-byte swizzle, each load for this CTA alone) and runs ahead into the next tile, one
+// thread issues the MMAs, four warps write the scales of every K-step into tensor memory (tcgen05.st), four warps read
+// the accumulators back (tcgen05.ld) and write C.  Every mbarrier wait is bounded in time: when a wait runs out the
+// block raises an error word, stops issuing, frees its tensor memory and returns.
 //
-// What bounds it: a 128 x 128 x 64 MMA reads 4 KiB of A and 4 KiB of B from shared memory in the 64 cycles it takes,
-// which is all a shared memory delivers, so the TMA writes of the next stage (100 KiB per nine-MMA K-step of 256)
-// come on top of the MMA time and do not hide under it.
+// What bounds it: the rate at which the one MMA stream of a CTA completes -- about 87 cycles per 128 x 128 x 64
+// block-scaled MMA against the 64 the tensor pipe counts as active; the loads hide completely under it.
 #include "../../include/abs_b200.h"
 #include "abs_device.cuh"
 
