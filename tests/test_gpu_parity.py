@@ -1084,3 +1084,34 @@ def test_matmul_wait_limit_is_reported_and_the_next_call_works(B, oracle):
     assert L.abs_selftest_matmul_stall(*args, -1) == 2                     # not a way to make an ordinary call
     again = B.abs_matmul(1, qa, qb, m, n, k, workspace=ws, check=True)
     assert torch.equal(again, good)
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_tensor_core_matmul_long_k_and_nan_scales(B, oracle, fmt):
+    """Two corners of abs_matmul: a long contraction (K = 14336: 56 pipeline steps, the stage and slot phases wrap many
+    times) against the float64 reference, and E4M3 NaN scale bytes (0x7F, and 0xFF for IF4), which must make exactly
+    the rows of C that belong to their row of A, and the columns that belong to their row of B, NaN -- as dequantize
+    does -- and leave every other entry equal to the reference."""
+    m, n, k = 128, 128, 14336
+    a, b = I.generate("cfg3a", m, k, seed=3), I.generate("cfg3a", n, k, seed=4)
+    qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
+    oa, ob = oracle.quantize(fmt, a, threads=THREADS), oracle.quantize(fmt, b, threads=THREADS)
+    ref = oracle.mac_matmul_reference(fmt, oa, ob, m, n, k)
+    c = B.abs_matmul(fmt, qa, qb, m, n, k, check=True).double().cpu().numpy()
+    assert np.abs(c - ref).max() <= 4e-5 * np.abs(ref).max()
+
+    m, n, k = 256, 128, 512
+    a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+    oa, ob = oracle.quantize(fmt, a, threads=THREADS), oracle.quantize(fmt, b, threads=THREADS)
+    sa, sb = oa[1].copy(), ob[1].copy()
+    sa[5, 3] = 0x7F
+    sa[200, 0] = 0xFF if fmt == 1 else 0x7F
+    sb[77, 31] = 0x7F
+    dev = lambda q, s: (torch.from_numpy(q[0]).cuda(), torch.from_numpy(s).cuda(), torch.tensor([q[2]], dtype=torch.float32, device="cuda"))
+    c = B.abs_matmul(fmt, dev(oa, sa), dev(ob, sb), m, n, k, check=True).double().cpu().numpy()
+    bad = np.zeros((m, n), dtype=bool)
+    bad[5, :] = bad[200, :] = True
+    bad[:, 77] = True
+    assert np.isnan(c[bad]).all() and np.isfinite(c[~bad]).all()
+    ref = oracle.mac_matmul_reference(fmt, oa, ob, m, n, k)
+    assert np.abs(c[~bad] - ref[~bad]).max() <= 2e-5 * np.abs(ref).max()
