@@ -1115,3 +1115,9 @@ def test_tensor_core_matmul_long_k_and_nan_scales(B, oracle, fmt):
     assert np.isnan(c[bad]).all() and np.isfinite(c[~bad]).all()
     ref = oracle.mac_matmul_reference(fmt, oa, ob, m, n, k)
     assert np.abs(c[~bad] - ref[~bad]).max() <= 2e-5 * np.abs(ref).max()
+    # an all-zero operand (every scale byte zero) gives an all-zero product, not NaN
+    z = np.zeros((m, k), dtype=np.uint16)
+    qz = B.abs_quantize(fmt, to_dev(z))
+    assert int(qz[1].max().item()) == 0
+    cz = B.abs_matmul(fmt, qz, B.abs_quantize(fmt, to_dev(b)), m, n, k, check=True)
+    assert bool((cz == 0).all())
