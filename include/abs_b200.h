@@ -252,6 +252,11 @@ ABS_API size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, i
 ABS_API abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
                                 const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n,
                                 int64_t k, float* c_f32, void* workspace, size_t workspace_bytes, void* stream);
+/* The same product written as bf16 [m, n]: each entry is the FP32 result of abs_matmul rounded to nearest even, so
+ * that it can go straight into the next abs_quantize call. */
+ABS_API abs_status_t abs_matmul_bf16(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
+                                     const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n,
+                                     int64_t k, void* c_bf16, void* workspace, size_t workspace_bytes, void* stream);
 ABS_API abs_status_t abs_matmul_check(const void* workspace, void* stream);
 
 /* Host-buffer variants: `*_host` pointers are HOST memory (pinned memory makes the copies

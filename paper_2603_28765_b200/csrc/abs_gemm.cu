@@ -25,6 +25,7 @@
 #include "abs_device.cuh"
 
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <mutex>
 
@@ -203,6 +204,12 @@ __device__ __forceinline__ void tmem_load32(uint32_t addr, uint32_t (&r)[32]) {
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(addr) : "memory");
 }
+// Two FP32 values rounded to nearest even bf16, the first in the low half.
+__device__ __forceinline__ uint32_t bf16x2_bits(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ void tmem_load_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // 32 lanes x 16 columns of 32 bits: thread t of the warp writes columns c .. c+15 of lane (warp % 4) * 32 + t.
 __device__ __forceinline__ void tmem_store16(uint32_t addr, const uint4& a, const uint4& b, const uint4& c, const uint4& d) {
@@ -258,10 +265,11 @@ __device__ __forceinline__ void tile_of(int32_t t, int32_t tiles_m, int32_t tile
 // acc_full / acc_empty barriers; NVFP4, with one accumulator of 128 columns, alternates between two of them so that a
 // tile's epilogue overlaps the next tile's MMAs, IF4 (3 x 128 columns) has room for one set and overlaps the epilogue
 // only with the next tile's loads.
-template <int PLANES>
+// OUT_BF16: C is written as bf16 (round to nearest even of the same FP32 value), else as FP32.
+template <int PLANES, bool OUT_BF16>
 __global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
-                const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, float* __restrict__ c, int32_t tiles_m,
+                const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, void* __restrict__ c_out, int32_t tiles_m,
                 int32_t tiles_n, int32_t k_iters, int32_t m_rows, int* __restrict__ error, int32_t stall_step) {
     constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
@@ -423,8 +431,12 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
             if (!have) break;
             tc_fence_after();
             // this thread's part of every store: row (lane / 8) of each group of four rows, 16 bytes at column 4 (lane % 8)
-            const int32_t row0 = tile_m * kTileM + quarter * 32 + (lane >> 3);
-            float* out = c + (size_t)row0 * (size_t)n_cols + (size_t)tile_n * kTileN + 4 * (lane & 7);
+            // this thread's part of every store.  FP32: row (lane / 8) of each group of four rows, 16 bytes at column
+            // 4 (lane % 8); bf16: row (lane / 4) of each group of eight rows, 16 bytes at column 8 (lane % 4)
+            const int32_t row0 = tile_m * kTileM + quarter * 32 + (OUT_BF16 ? (lane >> 2) : (lane >> 3));
+            float* out = reinterpret_cast<float*>(c_out) + (size_t)row0 * (size_t)n_cols + (size_t)tile_n * kTileN + 4 * (lane & 7);
+            __nv_bfloat16* out16 = reinterpret_cast<__nv_bfloat16*>(c_out) + (size_t)row0 * (size_t)n_cols + (size_t)tile_n * kTileN +
+                                   8 * (lane & 3);
             const uint32_t lane_base = tmem + buf * kTileN + ((uint32_t)(quarter * 32) << 16);
             for (int chunk = 0; chunk < kTileN / 32; ++chunk) {
                 uint32_t r0[32], r1[32], r2[32];
@@ -448,15 +460,34 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                 }
                 // A thread holds 32 columns of ONE row; stored as they are, every store instruction of the warp would
                 // touch 32 different rows.  Through shared memory each instruction writes four rows of 128 contiguous bytes.
+                if constexpr (!OUT_BF16) {
 #pragma unroll
-                for (int jj = 0; jj < 32; jj += 4)
-                    *reinterpret_cast<float4*>(staging + lane * kStagePitch + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
-                __syncwarp();
+                    for (int jj = 0; jj < 32; jj += 4)
+                        *reinterpret_cast<float4*>(staging + lane * kStagePitch + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+                    __syncwarp();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float4 x = *reinterpret_cast<const float4*>(staging + (4 * i + (lane >> 3)) * kStagePitch + 4 * (lane & 7));
-                    if (row0 + 4 * i < m_rows)                          // the last row block may be partial
-                        *reinterpret_cast<float4*>(out + (size_t)(4 * i) * n_cols + chunk * 32) = x;
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 x = *reinterpret_cast<const float4*>(staging + (4 * i + (lane >> 3)) * kStagePitch + 4 * (lane & 7));
+                        if (row0 + 4 * i < m_rows)                      // the last row block may be partial
+                            *reinterpret_cast<float4*>(out + (size_t)(4 * i) * n_cols + chunk * 32) = x;
+                    }
+                } else {
+                    // 32 bf16 = 64 bytes per row, rows 20 words apart; a store instruction writes eight rows of 64 bytes
+                    uint32_t* stg = reinterpret_cast<uint32_t*>(staging);
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 8) {
+                        uint4 pk;
+                        pk.x = bf16x2_bits(v[jj], v[jj + 1]); pk.y = bf16x2_bits(v[jj + 2], v[jj + 3]);
+                        pk.z = bf16x2_bits(v[jj + 4], v[jj + 5]); pk.w = bf16x2_bits(v[jj + 6], v[jj + 7]);
+                        *reinterpret_cast<uint4*>(stg + lane * 20 + jj / 2) = pk;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 x = *reinterpret_cast<const uint4*>(stg + (8 * i + (lane >> 2)) * 20 + 4 * (lane & 3));
+                        if (row0 + 8 * i < m_rows)
+                            *reinterpret_cast<uint4*>(out16 + (size_t)(8 * i) * n_cols + chunk * 32) = x;
+                    }
                 }
                 __syncwarp();
             }
@@ -557,8 +588,8 @@ size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k
 }
 
 static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
-                                const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
-                                void* workspace, size_t workspace_bytes, void* stream, int32_t stall_step) {
+                                const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, void* c_f32,
+                                void* workspace, size_t workspace_bytes, void* stream, int32_t stall_step, bool out_bf16 = false) {
     const absq::CallRange range("abs_matmul");
     if (fmt != ABS_FMT_IF4 && fmt != ABS_FMT_NVFP4) return ABS_ERR_FMT;
     if (!gemm_shape_ok(fmt, m, n, k)) return ABS_ERR_SHAPE;
@@ -612,21 +643,28 @@ static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* 
     std::call_once(attr_once[dev], [dev]() {
         if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count[dev] < 1)
             sm_count[dev] = 1;
-        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
+        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
         if (attr_err[dev] == cudaSuccess)
-            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
+            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
+        if (attr_err[dev] == cudaSuccess)
+            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
+        if (attr_err[dev] == cudaSuccess)
+            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
     });
     if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
     const int32_t tiles_m = (int32_t)((m + kTileM - 1) / kTileM), tiles_n = (int32_t)(n / kTileN);
     const int64_t num_tiles = (int64_t)tiles_m * tiles_n;
     const dim3 pgrid((unsigned)(num_tiles < sm_count[dev] ? num_tiles : sm_count[dev]));
-    const cudaError_t e =
-        has_int ? launch_pdl(if4_gemm_kernel<3>, pgrid, 320, kGemmSmemBytes<3>, s, maps, (const uint8_t*)(ws + L.off_sfa),
-                             (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int32_t)m, (int*)ws, stall_step)
-                : launch_pdl(if4_gemm_kernel<1>, pgrid, 320, kGemmSmemBytes<1>, s, maps, (const uint8_t*)(ws + L.off_sfa),
-                             (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),
-                             (int32_t)m, (int*)ws, stall_step);
+    cudaError_t e;
+#define ABS_LAUNCH_GEMM(P, O)                                                                                           \
+    e = launch_pdl(if4_gemm_kernel<P, O>, pgrid, 320, kGemmSmemBytes<P>, s, maps, (const uint8_t*)(ws + L.off_sfa),      \
+                   (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),   \
+                   (int32_t)m, (int*)ws, stall_step)
+    if (has_int && out_bf16) ABS_LAUNCH_GEMM(3, true);
+    else if (has_int) ABS_LAUNCH_GEMM(3, false);
+    else if (out_bf16) ABS_LAUNCH_GEMM(1, true);
+    else ABS_LAUNCH_GEMM(1, false);
+#undef ABS_LAUNCH_GEMM
     if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
 }
@@ -635,6 +673,13 @@ abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales
                         const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, float* c_f32,
                         void* workspace, size_t workspace_bytes, void* stream) {
     return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_f32, workspace, workspace_bytes, stream, -1);
+}
+
+abs_status_t abs_matmul_bf16(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
+                             const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, void* c_bf16,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_bf16, workspace, workspace_bytes, stream, -1,
+                       true);
 }
 
 abs_status_t abs_selftest_matmul_stall(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,

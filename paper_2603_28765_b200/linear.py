@@ -69,12 +69,13 @@ def _opts(*, hadamard: bool = False, stochastic: bool = False, sign_mask: int = 
     return B.make_opts(flags, sign_mask, seed) if flags else None
 
 
-def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4):
-    """Y = q(X) q(W)^T as float32 [tokens, d_out]: both operands quantized along d_in, one ``abs_matmul``.
-    d_out must be a multiple of 128, d_in of 256 (any number of tokens)."""
+def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4, *, bf16: bool = False):
+    """Y = q(X) q(W)^T as float32 [tokens, d_out] (bfloat16 with ``bf16``, ready to be the next layer's input): both
+    operands quantized along d_in, one ``abs_matmul``.  d_out must be a multiple of 128, d_in of 256 (any number of
+    tokens)."""
     tokens, d_in = x.shape
     d_out = w.shape[0]
-    return B.abs_matmul(fmt, B.abs_quantize(fmt, x), B.abs_quantize(fmt, w), tokens, d_out, d_in)
+    return B.abs_matmul(fmt, B.abs_quantize(fmt, x), B.abs_quantize(fmt, w), tokens, d_out, d_in, bf16=bf16)
 
 
 def backward_tc(x, w, dy, fmt: int = B.ABS_FMT_IF4, *, sign_mask: int = 0x5A3C, seed: int = 0):

@@ -1121,3 +1121,17 @@ def test_tensor_core_matmul_long_k_and_nan_scales(B, oracle, fmt):
     assert int(qz[1].max().item()) == 0
     cz = B.abs_matmul(fmt, qz, B.abs_quantize(fmt, to_dev(b)), m, n, k, check=True)
     assert bool((cz == 0).all())
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_tensor_core_matmul_bf16_output_is_the_rounded_fp32_output(B, oracle, fmt):
+    """abs_matmul_bf16 writes the FP32 result of abs_matmul rounded to nearest even: bit for bit the bf16 conversion of
+    the FP32 output, on full and partial row blocks, and nothing below row m."""
+    for (m, n, k) in ((256, 384, 1024), (100, 128, 256), (1152, 256, 512)):
+        a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+        qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
+        c32 = B.abs_matmul(fmt, qa, qb, m, n, k, check=True)
+        guard = torch.full((m + 28, n), 3.0, dtype=torch.bfloat16, device="cuda")
+        B.abs_matmul(fmt, qa, qb, m, n, k, out=guard, check=True, bf16=True)
+        assert torch.equal(guard[:m], c32.to(torch.bfloat16)), (fmt, m, n, k)
+        assert bool((guard[m:] == 3.0).all())
