@@ -36,7 +36,8 @@ EXPORTS = [
     "abs_dequantize", "abs_dequantize_ex", "abs_amax", "abs_alpha_from_amax", "abs_host_workspace_bytes",
     "abs_quantize_host", "abs_dequantize_host", "abs_selftest_convert", "abs_profile_events",
     "abs_quantize_noalloc", "abs_quantize_transposed", "abs_scales_bytes_swizzled", "abs_quantize_dequantize",
-    "abs_matmul_workspace_bytes", "abs_matmul", "abs_matmul_bf16", "abs_matmul_check", "abs_selftest_matmul_stall",
+    "abs_matmul_workspace_bytes", "abs_matmul", "abs_matmul_bf16", "abs_matmul_bf16_scaled", "abs_matmul_check",
+    "abs_selftest_matmul_stall",
 ]
 
 
@@ -110,6 +111,8 @@ def lib():
             L.abs_matmul.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
             L.abs_matmul_bf16.restype = C.c_int
             L.abs_matmul_bf16.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+            L.abs_matmul_bf16_scaled.restype = C.c_int
+            L.abs_matmul_bf16_scaled.argtypes = [C.c_int, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, C.c_int, vp, vp, sz, vp]
             L.abs_matmul_check.restype = C.c_int
             L.abs_matmul_check.argtypes = [vp, vp]
             L.abs_selftest_matmul_stall.restype = C.c_int
@@ -257,10 +260,12 @@ def abs_dequantize(fmt: int, codes, scales, tensor_scale, rows: int, cols: int, 
 
 
 def abs_matmul(fmt: int, qa, qb, m: int, n: int, k: int, out=None, workspace=None, stream=None, check: bool = False,
-               bf16: bool = False):
+               bf16: bool = False, next_fmt: int | None = None, next_alpha=None):
     """C = A B^T on the tensor cores for two quantized operands ``qa`` = (codes, scales, alpha) of A [m, k] and
     ``qb`` of B [n, k] (row-major scales), with the MAC arithmetic of Sec. 5.2.  Returns C as float32 [m, n], or with
-    ``bf16`` as bfloat16 (the same values rounded to nearest even).  ``check`` synchronises and raises if a wait inside
+    ``bf16`` as bfloat16 (the same values rounded to nearest even).  With ``next_fmt`` (bf16 output only) the kernel also
+    leaves the tensor scale that ``abs_quantize(next_fmt, C)`` would compute in ``next_alpha`` (a CUDA float32[1],
+    allocated when not given) and the call returns (C, next_alpha).  ``check`` synchronises and raises if a wait inside
     the kernel ran out."""
     import torch
     L = lib()
@@ -275,6 +280,17 @@ def abs_matmul(fmt: int, qa, qb, m: int, n: int, k: int, out=None, workspace=Non
     assert out.dtype == (torch.bfloat16 if bf16 else torch.float32)
     with torch.cuda.device(qa[0].device):
         sp = _stream_ptr(stream)
+        if next_fmt is not None:
+            assert bf16
+            if next_alpha is None:
+                next_alpha = torch.zeros(1, dtype=torch.float32, device=qa[0].device)
+            rc = L.abs_matmul_bf16_scaled(fmt, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), qb[0].data_ptr(),
+                                          qb[1].data_ptr(), qb[2].data_ptr(), m, n, k, out.data_ptr(), next_fmt,
+                                          next_alpha.data_ptr(), workspace.data_ptr() + off, workspace.numel() - off, sp)
+            _check(rc, "abs_matmul_bf16_scaled")
+            if check:
+                _check(L.abs_matmul_check(workspace.data_ptr() + off, sp), "abs_matmul (a wait inside the kernel ran out)")
+            return out, next_alpha
         rc = (L.abs_matmul_bf16 if bf16 else L.abs_matmul)(fmt, qa[0].data_ptr(), qa[1].data_ptr(), qa[2].data_ptr(), qb[0].data_ptr(), qb[1].data_ptr(),
                           qb[2].data_ptr(), m, n, k, out.data_ptr(), workspace.data_ptr() + off, workspace.numel() - off, sp)
         _check(rc, "abs_matmul")

@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(256) if4_split_kernel(const SplitOperand a, co
     pdl_launch_dependents();
     pdl_wait();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x, first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (first == 0) *error = 0;
+    if (first == 0) { error[0] = 0; error[1] = 0; error[2] = 0; }     // error word, output maximum, ticket
     const int64_t code_items = has_int ? a.pairs + b.pairs : 0;
     for (int64_t i = first; i < code_items; i += stride) {
         const SplitOperand& o = i < a.pairs ? a : b;
@@ -270,7 +270,8 @@ template <int PLANES, bool OUT_BF16>
 __global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
                 const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, void* __restrict__ c_out, int32_t tiles_m,
-                int32_t tiles_n, int32_t k_iters, int32_t m_rows, int* __restrict__ error, int32_t stall_step) {
+                int32_t tiles_n, int32_t k_iters, int32_t m_rows, int* __restrict__ error, int32_t stall_step,
+                float* __restrict__ next_alpha, float next_denom) {
     constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
@@ -421,6 +422,8 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
         const float c1 = __uint_as_float(0x3F5B6DB7u);                 // fp32(6/7)
         const float c2 = __fdiv_rn(36.0f, 49.0f);
         uint32_t j = 0;
+        uint32_t out_max = 0u;                  // bf16 output with next_alpha: largest |C| bit pattern this thread has written
+        bool all_tiles = true;
         for (int32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++j) {
             int32_t tile_m, tile_n;
             tile_of(t, tiles_m, tiles_n, tile_m, tile_n);
@@ -428,9 +431,9 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
             bool have = mbar_wait(acc_full0 + 8 * buf, (j / kAccBufs) & 1u);
             if (!have && lane == 0) atomicExch(error, 3);
             have = __all_sync(0xFFFFFFFFu, have);
-            if (!have) break;
+            if (!have) { all_tiles = false; break; }
             tc_fence_after();
-            // this thread's part of every store: row (lane / 8) of each group of four rows, 16 bytes at column 4 (lane % 8)
+            const bool own_row_valid = tile_m * kTileM + quarter * 32 + lane < m_rows;   // the row whose values this thread holds
             // this thread's part of every store.  FP32: row (lane / 8) of each group of four rows, 16 bytes at column
             // 4 (lane % 8); bf16: row (lane / 4) of each group of eight rows, 16 bytes at column 8 (lane % 4)
             const int32_t row0 = tile_m * kTileM + quarter * 32 + (OUT_BF16 ? (lane >> 2) : (lane >> 3));
@@ -480,6 +483,11 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                         pk.x = bf16x2_bits(v[jj], v[jj + 1]); pk.y = bf16x2_bits(v[jj + 2], v[jj + 3]);
                         pk.z = bf16x2_bits(v[jj + 4], v[jj + 5]); pk.w = bf16x2_bits(v[jj + 6], v[jj + 7]);
                         *reinterpret_cast<uint4*>(stg + lane * 20 + jj / 2) = pk;
+                        if (next_alpha != nullptr && own_row_valid) {
+                            const uint32_t w4[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) out_max = max(out_max, max(w4[q] & 0x7FFFu, (w4[q] >> 16) & 0x7FFFu));
+                        }
                     }
                     __syncwarp();
 #pragma unroll
@@ -490,6 +498,20 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     }
                 }
                 __syncwarp();
+            }
+        }
+        // The global maximum of |C| as written (bf16), for the next quantizer's tensor scale (Eq. 1): every epilogue
+        // warp publishes its maximum with an atomic and takes a ticket; the last of all warps converts and writes alpha.
+        if (OUT_BF16 && next_alpha != nullptr && all_tiles) {
+            const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, out_max);
+            if (lane == 0) {
+                atomicMax(reinterpret_cast<unsigned int*>(error) + 1, wmax);
+                __threadfence();
+                const int ticket = atomicAdd(error + 2, 1);
+                if (ticket == (int)gridDim.x * 4 - 1) {
+                    const float A = __uint_as_float(atomicMax(reinterpret_cast<unsigned int*>(error) + 1, 0u) << 16);
+                    *next_alpha = (A == 0.0f) ? 1.0f : __fdiv_rn(A, next_denom);
+                }
             }
         }
     }
@@ -589,7 +611,8 @@ size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k
 
 static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha, const void* b_codes,
                                 const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k, void* c_f32,
-                                void* workspace, size_t workspace_bytes, void* stream, int32_t stall_step, bool out_bf16 = false) {
+                                void* workspace, size_t workspace_bytes, void* stream, int32_t stall_step, bool out_bf16 = false,
+                                float* next_alpha = nullptr, float next_denom = 0.0f) {
     const absq::CallRange range("abs_matmul");
     if (fmt != ABS_FMT_IF4 && fmt != ABS_FMT_NVFP4) return ABS_ERR_FMT;
     if (!gemm_shape_ok(fmt, m, n, k)) return ABS_ERR_SHAPE;
@@ -659,7 +682,7 @@ static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* 
 #define ABS_LAUNCH_GEMM(P, O)                                                                                           \
     e = launch_pdl(if4_gemm_kernel<P, O>, pgrid, 320, kGemmSmemBytes<P>, s, maps, (const uint8_t*)(ws + L.off_sfa),      \
                    (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),   \
-                   (int32_t)m, (int*)ws, stall_step)
+                   (int32_t)m, (int*)ws, stall_step, next_alpha, next_denom)
     if (has_int && out_bf16) ABS_LAUNCH_GEMM(3, true);
     else if (has_int) ABS_LAUNCH_GEMM(3, false);
     else if (out_bf16) ABS_LAUNCH_GEMM(1, true);
@@ -680,6 +703,23 @@ abs_status_t abs_matmul_bf16(abs_fmt_t fmt, const void* a_codes, const void* a_s
                              void* workspace, size_t workspace_bytes, void* stream) {
     return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_bf16, workspace, workspace_bytes, stream, -1,
                        true);
+}
+
+abs_status_t abs_matmul_bf16_scaled(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
+                                    const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n, int64_t k,
+                                    void* c_bf16, abs_fmt_t next_fmt, float* next_alpha, void* workspace, size_t workspace_bytes,
+                                    void* stream) {
+    if (!next_alpha) return ABS_ERR_NULL;
+    float m_fp;
+    switch (next_fmt) {
+        case ABS_FMT_NVFP4: case ABS_FMT_IF4: case ABS_FMT_IF4_BS8: case ABS_FMT_NVFP4_BS8: m_fp = 6.0f; break;
+        case ABS_FMT_IF3: case ABS_FMT_IF3_BS8: m_fp = 4.0f; break;
+        case ABS_FMT_IF6_E2M3: m_fp = 7.5f; break;
+        case ABS_FMT_IF6_E3M2: m_fp = 28.0f; break;
+        default: return ABS_ERR_FMT;
+    }
+    return matmul_impl(fmt, a_codes, a_scales, a_alpha, b_codes, b_scales, b_alpha, m, n, k, c_bf16, workspace, workspace_bytes, stream, -1,
+                       true, next_alpha, m_fp * 448.0f);
 }
 
 abs_status_t abs_selftest_matmul_stall(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,

@@ -69,13 +69,23 @@ def _opts(*, hadamard: bool = False, stochastic: bool = False, sign_mask: int = 
     return B.make_opts(flags, sign_mask, seed) if flags else None
 
 
-def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4, *, bf16: bool = False):
+def forward_tc(x, w, fmt: int = B.ABS_FMT_IF4, *, bf16: bool = False, next_fmt: int | None = None):
     """Y = q(X) q(W)^T as float32 [tokens, d_out] (bfloat16 with ``bf16``, ready to be the next layer's input): both
-    operands quantized along d_in, one ``abs_matmul``.  d_out must be a multiple of 128, d_in of 256 (any number of
-    tokens)."""
+    operands quantized along d_in, one ``abs_matmul``.  With ``next_fmt`` (implies bf16) the product kernel also leaves
+    the tensor scale of Y for that format, and the call returns (Y, alpha): ``quantize_with(next_fmt, Y, alpha)`` then
+    quantizes Y without a pass for its maximum.  d_out must be a multiple of 128, d_in of 256 (any number of tokens)."""
     tokens, d_in = x.shape
     d_out = w.shape[0]
-    return B.abs_matmul(fmt, B.abs_quantize(fmt, x), B.abs_quantize(fmt, w), tokens, d_out, d_in, bf16=bf16)
+    qx, qw = B.abs_quantize(fmt, x), B.abs_quantize(fmt, w)
+    if next_fmt is not None:
+        return B.abs_matmul(fmt, qx, qw, tokens, d_out, d_in, bf16=True, next_fmt=next_fmt)
+    return B.abs_matmul(fmt, qx, qw, tokens, d_out, d_in, bf16=bf16)
+
+
+def quantize_with(fmt: int, x, alpha):
+    """abs_quantize of ``x`` with a tensor scale that is already known (a CUDA float32[1], e.g. from ``forward_tc`` with
+    ``next_fmt``): the group-quantize kernel alone.  Returns (codes, scales, alpha)."""
+    return B.abs_quantize(fmt, x, tensor_scale=alpha, opts=B.make_opts(B.ABS_F_ALPHA_GIVEN))
 
 
 def backward_tc(x, w, dy, fmt: int = B.ABS_FMT_IF4, *, sign_mask: int = 0x5A3C, seed: int = 0):

@@ -1135,3 +1135,25 @@ def test_tensor_core_matmul_bf16_output_is_the_rounded_fp32_output(B, oracle, fm
         B.abs_matmul(fmt, qa, qb, m, n, k, out=guard, check=True, bf16=True)
         assert torch.equal(guard[:m], c32.to(torch.bfloat16)), (fmt, m, n, k)
         assert bool((guard[m:] == 3.0).all())
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+def test_matmul_leaves_the_tensor_scale_of_its_output(B, oracle, fmt):
+    """abs_matmul_bf16_scaled: the epilogue's running maximum of |C| gives the alpha of Eq. 1 for the next quantizer.
+    It must be the very float abs_quantize computes with its own pass over C (for several next formats), on full and
+    partial row blocks, so that quantizing C with ABS_F_ALPHA_GIVEN and that alpha gives the same bytes."""
+    for (m, n, k) in ((256, 384, 1024), (100, 128, 256), (2048, 2048, 512)):
+        a, b = I.generate("cfg2", m, k), I.generate("cfg3a", n, k, seed=9)
+        qa, qb = B.abs_quantize(fmt, to_dev(a)), B.abs_quantize(fmt, to_dev(b))
+        for next_fmt in (1, 2, 3):
+            c, alpha = B.abs_matmul(fmt, qa, qb, m, n, k, bf16=True, next_fmt=next_fmt, check=True)
+            codes, scales, alpha_own = B.abs_quantize(next_fmt, c)
+            assert float(alpha.item()) == float(alpha_own.item()), (fmt, m, n, k, next_fmt)
+            og = B.make_opts(B.ABS_F_ALPHA_GIVEN)
+            codes2, scales2, _ = B.abs_quantize(next_fmt, c, tensor_scale=alpha.clone(), opts=og)
+            assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+    # an all-zero product: alpha 1, as the quantizer's own pass gives
+    z = to_dev(np.zeros((128, 256), dtype=np.uint16))
+    c, alpha = B.abs_matmul(fmt, B.abs_quantize(fmt, z), B.abs_quantize(fmt, to_dev(I.generate("cfg3a", 128, 256, seed=9))),
+                            128, 128, 256, bf16=True, next_fmt=1, check=True)
+    assert float(alpha.item()) == 1.0 and bool((c == 0).all())
