@@ -260,7 +260,8 @@ ABS_API abs_status_t abs_matmul_bf16(abs_fmt_t fmt, const void* a_codes, const v
 /* abs_matmul_bf16 that also prepares the next quantization of its output: the epilogue keeps the largest |C| it writes
  * and the kernel leaves  next_alpha = max|C| / (M_FP(next_fmt) * 448)  (Eq. 1; 1 for an all-zero C) in the device float
  * next_alpha -- the value abs_quantize(next_fmt, C, ...) would compute with its own pass over C.  The next call can then
- * be abs_quantize_ex with ABS_F_ALPHA_GIVEN and tensor_scale_f32 = next_alpha: same bytes, one pass over C less. */
+ * be abs_quantize_ex with ABS_F_ALPHA_GIVEN and tensor_scale_f32 = next_alpha: same bytes, one pass over C less.
+ * next_alpha is left unwritten when a wait inside the kernel ran out (abs_matmul_check then reports it). */
 ABS_API abs_status_t abs_matmul_bf16_scaled(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
                                             const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m,
                                             int64_t n, int64_t k, void* c_bf16, abs_fmt_t next_fmt, float* next_alpha,
