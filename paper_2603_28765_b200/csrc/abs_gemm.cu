@@ -32,18 +32,20 @@
 namespace absq {
 
 constexpr int kTileM = 128, kTileN = 128;
-constexpr int kStageK = 256;                       // elements of K per pipeline stage: 128 bytes of packed codes per row
+constexpr int kStageK = 256;                       // elements of K of one TMA box: 128 bytes of packed codes per row
 constexpr int kMmaK = 64;                          // K of one tcgen05.mma kind::mxf4nvf4
-constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one plane of one operand in one stage
-// A stage holds PLANES planes of A and PLANES of B (the scales do not pass through shared memory).  IF4 (three
-// planes, 96 KiB) has room for two stages; plain NVFP4 (one plane, 32 KiB) is bound by load latency and takes six.
-template <int PLANES> constexpr int kStageBytes = 2 * PLANES * kPlaneBytes;
-template <int PLANES> constexpr int kStages = PLANES == 3 ? 2 : 6;
+constexpr int kPlaneBytes = kTileM * kStageK / 2;  // 16 KiB: one box (128 rows x 128 bytes) of one plane of one operand
+// A pipeline stage (one K-step) holds KBOXES boxes of each of the PLANES planes of A and of B (the scales do not pass
+// through shared memory).  IF4 (three planes, one box: K = 256, 96 KiB) has room for two stages.  Plain NVFP4 issues one
+// MMA per K-block, so the hand-overs of a step weigh more: its steps are two boxes long where K allows (K = 512, 64 KiB,
+// three stages), else one box (32 KiB, six stages).
+template <int PLANES, int KBOXES> constexpr int kStageBytes = 2 * PLANES * KBOXES * kPlaneBytes;
+template <int PLANES, int KBOXES> constexpr int kStages = PLANES == 3 ? 2 : (KBOXES == 2 ? 3 : 6);
 // Epilogue staging: each of the four epilogue warps turns its 32 rows x 32 columns of a chunk through shared memory
 // (rows 36 floats apart: 16-byte aligned and free of bank conflicts for 128-bit accesses both ways).
 constexpr int kStagePitch = 36, kStagingBytes = 4 * 32 * kStagePitch * 4;
-template <int PLANES> constexpr int kGemmSmemBytes =
-    kStages<PLANES> * kStageBytes<PLANES> + 1024 /* alignment slack */ + 512 /* barriers */ + kStagingBytes;
+template <int PLANES, int KBOXES> constexpr int kGemmSmemBytes =
+    kStages<PLANES, KBOXES> * kStageBytes<PLANES, KBOXES> + 1024 /* alignment slack */ + 512 /* barriers */ + kStagingBytes;
 constexpr uint64_t kWaitLimitNs = 1000000000ull;   // one second: how long an mbarrier wait polls before the block gives up
 
 // ----------------------------------------------------------------------------- operand split
@@ -266,13 +268,14 @@ __device__ __forceinline__ void tile_of(int32_t t, int32_t tiles_m, int32_t tile
 // tile's epilogue overlaps the next tile's MMAs, IF4 (3 x 128 columns) has room for one set and overlaps the epilogue
 // only with the next tile's loads.
 // OUT_BF16: C is written as bf16 (round to nearest even of the same FP32 value), else as FP32.
-template <int PLANES, bool OUT_BF16>
+template <int PLANES, bool OUT_BF16, int KBOXES = 1>
 __global__ void __launch_bounds__(320, 1)
 if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict__ sfa, const uint8_t* __restrict__ sfb,
                 const float* __restrict__ alpha_a, const float* __restrict__ alpha_b, void* __restrict__ c_out, int32_t tiles_m,
                 int32_t tiles_n, int32_t k_iters, int32_t m_rows, int* __restrict__ error, int32_t stall_step,
                 float* __restrict__ next_alpha, float next_denom) {
-    constexpr int planes = PLANES, kStages = absq::kStages<PLANES>, kStageBytes = absq::kStageBytes<PLANES>;
+    constexpr int planes = PLANES, kStages = absq::kStages<PLANES, KBOXES>, kStageBytes = absq::kStageBytes<PLANES, KBOXES>;
+    constexpr int kStepBlocks = KBOXES * (kStageK / kMmaK);          // MMA K-blocks (and scale tiles per operand) of one step
     constexpr int kAccBufs = PLANES == 1 ? 2 : 1;
     extern __shared__ uint8_t gemm_smem_raw[];
     const uint32_t raw = smem_u32(gemm_smem_raw);
@@ -280,7 +283,8 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     // Scale slots in tensor memory: 32 columns each (16 of A scales, 16 of B scales).  IF4 has room for two behind its
     // three accumulators; NVFP4, whose K-steps are only four MMAs long, takes eight behind its two accumulators so
     // that the scale warps can run several steps ahead of the MMAs.
-    constexpr uint32_t kSfSlots = PLANES == 1 ? 8 : 2, kSfBase = PLANES == 1 ? 2 * kTileN : 3 * kTileN;
+    constexpr uint32_t kSlotCols = 8u * kStepBlocks;                  // 4 columns per K-block and operand
+    constexpr uint32_t kSfSlots = PLANES == 1 ? 256u / kSlotCols : 2u, kSfBase = PLANES == 1 ? 2 * kTileN : 3 * kTileN;
     // barriers: full[], empty[] (stages), acc_full[2], acc_empty[2], sf_full[], sf_empty[] (slots); then the tmem address word
     const uint32_t bars = base + kStages * kStageBytes;
     uint32_t* tmem_word = reinterpret_cast<uint32_t*>(gemm_smem_raw + (bars - raw) + 320);
@@ -306,7 +310,7 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     if (warp == 0) {
         if (lane == 0) {
             // ---- producer: TMA loads of the operand planes
-            const uint32_t bytes = (uint32_t)planes * 2u * kPlaneBytes;
+            const uint32_t bytes = (uint32_t)planes * 2u * KBOXES * kPlaneBytes;
             uint32_t it = 0;
             bool ok = true;
             for (int32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -318,10 +322,12 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     const uint32_t st = base + s * kStageBytes, bar = full0 + 8 * s;
                     mbar_expect_tx(bar, bytes);
                     if ((int32_t)it == stall_step) continue;      // self-test only: the bytes announced never arrive
-                    for (int p = 0; p < planes; ++p) {
-                        tma_load_2d(st + p * kPlaneBytes, &maps.a[p], kt * (kStageK / 2), tile_m * kTileM, bar);
-                        tma_load_2d(st + (PLANES + p) * kPlaneBytes, &maps.b[p], kt * (kStageK / 2), tile_n * kTileN, bar);
-                    }
+                    for (int p = 0; p < planes; ++p)
+                        for (int box = 0; box < KBOXES; ++box) {
+                            const int32_t x = (kt * KBOXES + box) * (kStageK / 2);
+                            tma_load_2d(st + (p * KBOXES + box) * kPlaneBytes, &maps.a[p], x, tile_m * kTileM, bar);
+                            tma_load_2d(st + ((PLANES + p) * KBOXES + box) * kPlaneBytes, &maps.b[p], x, tile_n * kTileN, bar);
+                        }
                 }
             }
         }
@@ -341,16 +347,21 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                     if (!mbar_wait(sf_full0 + 8 * slot, (it / kSfSlots) & 1u)) { atomicExch(error, 5); ok = false; break; }
                     tc_fence_after();
                     const uint32_t st = base + s * kStageBytes;
-                    const uint32_t tsfa = tmem + kSfBase + slot * 32u, tsfb = tsfa + 16;
+                    const uint32_t tsfa = tmem + kSfBase + slot * kSlotCols, tsfb = tsfa + kSlotCols / 2;
                     // the MMAs of a step, one accumulator after the other (K order inside an accumulator is free)
-                    auto desc_a = [&](int p, int kb) { return operand_desc(st + p * kPlaneBytes + kb * (kMmaK / 2)); };
-                    auto desc_b = [&](int p, int kb) { return operand_desc(st + (PLANES + p) * kPlaneBytes + kb * (kMmaK / 2)); };
+                    // K-block kb of a step lies in box kb / 4 of its plane, 32 bytes per K-block inside the box's 128-byte rows
+                    auto desc_a = [&](int p, int kb) {
+                        return operand_desc(st + (p * KBOXES + (kb >> 2)) * kPlaneBytes + (kb & 3) * (kMmaK / 2));
+                    };
+                    auto desc_b = [&](int p, int kb) {
+                        return operand_desc(st + ((PLANES + p) * KBOXES + (kb >> 2)) * kPlaneBytes + (kb & 3) * (kMmaK / 2));
+                    };
 #pragma unroll
-                    for (int kb = 0; kb < kStageK / kMmaK; ++kb)
+                    for (int kb = 0; kb < kStepBlocks; ++kb)
                         tc_mma_nvf4(acc, desc_a(0, kb), desc_b(0, kb), kInstrDesc, !(kt == 0 && kb == 0), tsfa + 4 * kb, tsfb + 4 * kb);   // F F
                     if constexpr (PLANES == 3) {
 #pragma unroll
-                        for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                        for (int kb = 0; kb < kStepBlocks; ++kb) {
                             const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
                             tc_mma_nvf4<kFill>(acc + kTileN, desc_a(0, kb), desc_b(1, kb), kInstrDesc, !(kt == 0 && kb == 0), fa, fb);   // F H
                             tc_mma_nvf4<kLastUse>(acc + kTileN, desc_a(0, kb), desc_b(2, kb), kInstrDesc, true, fa, fb);                 // F L
@@ -358,7 +369,7 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                             tc_mma_nvf4(acc + kTileN, desc_a(2, kb), desc_b(0, kb), kInstrDesc, true, fa, fb);                           // L F
                         }
 #pragma unroll
-                        for (int kb = 0; kb < kStageK / kMmaK; ++kb) {
+                        for (int kb = 0; kb < kStepBlocks; ++kb) {
                             const uint32_t fa = tsfa + 4 * kb, fb = tsfb + 4 * kb;
                             tc_mma_nvf4<kFill>(acc + 2 * kTileN, desc_a(1, kb), desc_b(1, kb), kInstrDesc, !(kt == 0 && kb == 0), fa, fb);  // H H
                             tc_mma_nvf4<kLastUse>(acc + 2 * kTileN, desc_a(1, kb), desc_b(2, kb), kInstrDesc, true, fa, fb);              // H L
@@ -375,11 +386,11 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
     } else if (warp >= 6) {
         // ---- scales: this warp's copy of every K-step's scale tiles, global memory -> registers -> tensor memory
         // The loads of step it + 1 are in flight while step it waits for its slot and is written.
-        const int32_t ktiles = k_iters * (kStageK / kMmaK);
+        const int32_t ktiles = k_iters * kStepBlocks;
         const uint32_t lane_base = tmem + kSfBase + ((uint32_t)((warp & 3) * 32) << 16);
         int32_t t = blockIdx.x, kt = 0;                                   // the step whose tiles are loaded next
         const uint4 *pa = nullptr, *pb = nullptr;
-        auto load_next = [&](uint4 (&a)[4], uint4 (&b)[4]) {               // false when there is no further step
+        auto load_next = [&](uint4 (&a)[kStepBlocks], uint4 (&b)[kStepBlocks]) {   // false when there is no further step
             if (t >= num_tiles) return false;
             if (kt == 0) {
                 int32_t tile_m, tile_n;
@@ -388,31 +399,41 @@ if4_gemm_kernel(const __grid_constant__ GemmMaps maps, const uint8_t* __restrict
                 pb = reinterpret_cast<const uint4*>(sfb + (size_t)tile_n * ktiles * 512) + lane;
             }
 #pragma unroll
-            for (int kb = 0; kb < 4; ++kb) {                               // tile kb of the step: 16 bytes per lane, tiles 512 bytes apart
-                a[kb] = __ldg(pa + (kt * 4 + kb) * 32);
-                b[kb] = __ldg(pb + (kt * 4 + kb) * 32);
+            for (int kb = 0; kb < kStepBlocks; ++kb) {                     // tile kb of the step: 16 bytes per lane, tiles 512 bytes apart
+                a[kb] = __ldg(pa + (kt * kStepBlocks + kb) * 32);
+                b[kb] = __ldg(pb + (kt * kStepBlocks + kb) * 32);
             }
             if (++kt == k_iters) { kt = 0; t += gridDim.x; }
             return true;
         };
-        uint4 a[4], b[4], an[4], bn[4];
+        // One step of lookahead in registers where a step is one box long; with two-box steps the four scale slots
+        // already let these warps run three steps ahead of the MMAs.
+        constexpr bool kLookahead = KBOXES == 1;
+        uint4 a[kStepBlocks], b[kStepBlocks], an[kLookahead ? kStepBlocks : 1], bn[kLookahead ? kStepBlocks : 1];
         bool more = load_next(a, b);
         for (uint32_t it = 0; more; ++it) {
-            more = load_next(an, bn);
+            if constexpr (kLookahead) more = load_next(an, bn);
             const uint32_t slot = it % kSfSlots;
             bool have = mbar_wait(sf_empty0 + 8 * slot, ((it / kSfSlots) & 1u) ^ 1u);
             if (!have && lane == 0) atomicExch(error, 6);
             have = __all_sync(0xFFFFFFFFu, have);
             if (!have) break;
             tc_fence_after();
-            tmem_store16(lane_base + slot * 32u, a[0], a[1], a[2], a[3]);
-            tmem_store16(lane_base + slot * 32u + 16u, b[0], b[1], b[2], b[3]);
+#pragma unroll
+            for (int g = 0; g < KBOXES; ++g) {
+                tmem_store16(lane_base + slot * kSlotCols + 16u * g, a[4 * g], a[4 * g + 1], a[4 * g + 2], a[4 * g + 3]);
+                tmem_store16(lane_base + slot * kSlotCols + kSlotCols / 2 + 16u * g, b[4 * g], b[4 * g + 1], b[4 * g + 2], b[4 * g + 3]);
+            }
             tmem_store_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(sf_full0 + 8 * slot);
+            if constexpr (kLookahead) {
 #pragma unroll
-            for (int kb = 0; kb < 4; ++kb) { a[kb] = an[kb]; b[kb] = bn[kb]; }
+                for (int kb = 0; kb < kStepBlocks; ++kb) { a[kb] = an[kb]; b[kb] = bn[kb]; }
+            } else {
+                more = load_next(a, b);
+            }
         }
     } else {
         // ---- epilogue: warp w owns the accumulator lanes (rows of the tile) 32 (w % 4) .. 32 (w % 4) + 31
@@ -666,27 +687,32 @@ static abs_status_t matmul_impl(abs_fmt_t fmt, const void* a_codes, const void* 
     std::call_once(attr_once[dev], [dev]() {
         if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count[dev] < 1)
             sm_count[dev] = 1;
-        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
-        if (attr_err[dev] == cudaSuccess)
-            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
-        if (attr_err[dev] == cudaSuccess)
-            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<3>);
-        if (attr_err[dev] == cudaSuccess)
-            attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes<1>);
+        attr_err[dev] = cudaSuccess;
+#define ABS_GEMM_ATTR(P, O, B)                                                                                         \
+    if (attr_err[dev] == cudaSuccess)                                                                                   \
+        attr_err[dev] = cudaFuncSetAttribute(if4_gemm_kernel<P, O, B>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                             kGemmSmemBytes<P, B>)
+        ABS_GEMM_ATTR(3, false, 1); ABS_GEMM_ATTR(3, true, 1);
+        ABS_GEMM_ATTR(1, false, 1); ABS_GEMM_ATTR(1, true, 1);
+        ABS_GEMM_ATTR(1, false, 2); ABS_GEMM_ATTR(1, true, 2);
+#undef ABS_GEMM_ATTR
     });
     if (attr_err[dev] != cudaSuccess) return ABS_ERR_CUDA;
     const int32_t tiles_m = (int32_t)((m + kTileM - 1) / kTileM), tiles_n = (int32_t)(n / kTileN);
     const int64_t num_tiles = (int64_t)tiles_m * tiles_n;
     const dim3 pgrid((unsigned)(num_tiles < sm_count[dev] ? num_tiles : sm_count[dev]));
     cudaError_t e;
-#define ABS_LAUNCH_GEMM(P, O)                                                                                           \
-    e = launch_pdl(if4_gemm_kernel<P, O>, pgrid, 320, kGemmSmemBytes<P>, s, maps, (const uint8_t*)(ws + L.off_sfa),      \
-                   (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n, (int32_t)(k / kStageK),   \
-                   (int32_t)m, (int*)ws, stall_step, next_alpha, next_denom)
-    if (has_int && out_bf16) ABS_LAUNCH_GEMM(3, true);
-    else if (has_int) ABS_LAUNCH_GEMM(3, false);
-    else if (out_bf16) ABS_LAUNCH_GEMM(1, true);
-    else ABS_LAUNCH_GEMM(1, false);
+#define ABS_LAUNCH_GEMM(P, O, B)                                                                                        \
+    e = launch_pdl(if4_gemm_kernel<P, O, B>, pgrid, 320, kGemmSmemBytes<P, B>, s, maps, (const uint8_t*)(ws + L.off_sfa), \
+                   (const uint8_t*)(ws + L.off_sfb), a_alpha, b_alpha, c_f32, tiles_m, tiles_n,                           \
+                   (int32_t)(k / (kStageK * B)), (int32_t)m, (int*)ws, stall_step, next_alpha, next_denom)
+    const bool long_steps = !has_int && k % (2 * kStageK) == 0;      // NVFP4: K-steps of 512 where K allows
+    if (has_int && out_bf16) ABS_LAUNCH_GEMM(3, true, 1);
+    else if (has_int) ABS_LAUNCH_GEMM(3, false, 1);
+    else if (long_steps && out_bf16) ABS_LAUNCH_GEMM(1, true, 2);
+    else if (long_steps) ABS_LAUNCH_GEMM(1, false, 2);
+    else if (out_bf16) ABS_LAUNCH_GEMM(1, true, 1);
+    else ABS_LAUNCH_GEMM(1, false, 1);
 #undef ABS_LAUNCH_GEMM
     if (e != cudaSuccess) return ABS_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ABS_OK : ABS_ERR_CUDA;
