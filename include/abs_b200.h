@@ -247,7 +247,9 @@ ABS_API float abs_alpha_from_amax(abs_fmt_t fmt, float amax);
  * returns 0).  Asynchronous like the other calls.  Every wait inside the kernel is bounded; if one runs out (it
  * never should) the kernel stops and leaves a non-zero word at the start of the workspace, which
  * abs_matmul_check(workspace, stream) reads back (it synchronises the stream): ABS_OK, or ABS_ERR_CUDA.
- * Single GPU: the tensor maps cover the caller's workspace on the current device only. */
+ * The workspace belongs to one call at a time: calls that share it must be ordered on one stream (concurrent calls on
+ * different streams take a workspace each).  Its contents mean nothing between calls.
+ * Single GPU: the tensor maps cover the caller's workspace and operands on the current device only. */
 ABS_API size_t abs_matmul_workspace_bytes(abs_fmt_t fmt, int64_t m, int64_t n, int64_t k);
 ABS_API abs_status_t abs_matmul(abs_fmt_t fmt, const void* a_codes, const void* a_scales, const float* a_alpha,
                                 const void* b_codes, const void* b_scales, const float* b_alpha, int64_t m, int64_t n,
